@@ -1,0 +1,202 @@
+"""Seeded synthetic inputs shaped like the paper's MSA workloads.
+
+This module only draws random tensors and chooses sample positions. It holds none of
+the method's arithmetic, so both the CUDA path's tests and the CPU oracle's tests may
+use it without sharing any computation.
+
+Recipe (every tensor): draw fp32 N(0,1), multiply by 1/sqrt(last_dim) of that tensor,
+optionally add the planted shift, round to bf16.  Draw order: Q, K, V, Q_idx, K_idx,
+then the planted-block choice and its directions.  Large tensors are drawn in row
+chunks of ``CHUNK_ROWS`` so that the fp32 temporary stays small; the chunking is part
+of the recipe (same seed + same device type => same bits).
+"""
+
+from __future__ import annotations
+
+from dataclasses import dataclass, replace
+from typing import Dict, Tuple
+
+import numpy as np
+import torch
+
+CHUNK_ROWS = 65536
+
+
+@dataclass(frozen=True)
+class MSAConfig:
+    """Shape of one workload, in the paper's notation (Section 2 and Section 3.1).
+
+    T = N (sequence length), n_q_heads = H_q, n_kv_heads = H_kv, head_dim = d_h,
+    idx_dim = d_idx, block_size = B_k, top_k = k.  ``seq_lens`` is used by decode
+    workloads only (one cached sequence per entry, one new query token each).
+    """
+
+    name: str
+    mode: str  # "prefill" | "decode"
+    T: int
+    n_q_heads: int
+    n_kv_heads: int
+    block_size: int
+    top_k: int
+    head_dim: int = 128
+    idx_dim: int = 64
+    seed: int = 0
+    planted_frac: float = 0.0
+    planted_shift: float = 0.0
+    seq_lens: Tuple[int, ...] = ()
+
+    @property
+    def group(self) -> int:
+        return self.n_q_heads // self.n_kv_heads
+
+    @property
+    def n_blocks(self) -> int:
+        return -(-self.T // self.block_size)
+
+    def scaled(self, **kw) -> "MSAConfig":
+        return replace(self, **kw)
+
+
+CONFIGS: Dict[str, MSAConfig] = {
+    "c1": MSAConfig("c1", "prefill", 2048, 8, 1, 64, 8, seed=0),
+    "c2": MSAConfig("c2", "prefill", 32768, 64, 8, 64, 32, seed=1),
+    "c3": MSAConfig("c3", "prefill", 131072, 64, 8, 128, 64, seed=2,
+                    planted_frac=0.05, planted_shift=2.0),
+    "c4": MSAConfig("c4", "prefill", 1048576, 64, 8, 128, 64, seed=3),
+    "c5": MSAConfig("c5", "decode", 1048576, 64, 8, 128, 64, seed=4,
+                    seq_lens=(131072,) * 16 + (1048576,) * 16),
+}
+
+
+def _gen(device, seed: int) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    return g
+
+
+def _draw(gen: torch.Generator, rows: int, inner: Tuple[int, ...], std: float,
+          device, shift_rows: torch.Tensor | None = None,
+          shift_vec: torch.Tensor | None = None) -> torch.Tensor:
+    """rows x inner bf16 tensor ~ N(0, std^2), drawn in chunks of CHUNK_ROWS rows.
+
+    ``shift_rows`` (bool [rows]) and ``shift_vec`` (fp32, broadcastable to inner) add a
+    constant vector to the marked rows before the bf16 rounding.
+    """
+    out = torch.empty((rows,) + inner, dtype=torch.bfloat16, device=device)
+    for r0 in range(0, rows, CHUNK_ROWS):
+        r1 = min(rows, r0 + CHUNK_ROWS)
+        x = torch.randn((r1 - r0,) + inner, generator=gen, device=device,
+                        dtype=torch.float32)
+        x.mul_(std)
+        if shift_rows is not None:
+            m = shift_rows[r0:r1].to(torch.float32)
+            x.add_(m.view((-1,) + (1,) * len(inner)) * shift_vec)
+        out[r0:r1] = x.to(torch.bfloat16)
+    return out
+
+
+def _planted(cfg: MSAConfig, gen: torch.Generator, n_tokens: int, device):
+    """Marks the tokens of round(frac*B) random blocks; returns (mask, u_idx, u_main)."""
+    n_blocks = -(-n_tokens // cfg.block_size)
+    n_plant = int(round(cfg.planted_frac * n_blocks))
+    perm = torch.randperm(n_blocks, generator=gen, device=device)
+    chosen = perm[:n_plant]
+    u_idx = torch.randn(cfg.idx_dim, generator=gen, device=device, dtype=torch.float32)
+    u_idx = u_idx / u_idx.norm()
+    u_main = torch.randn(cfg.head_dim, generator=gen, device=device, dtype=torch.float32)
+    u_main = u_main / u_main.norm()
+    block_mask = torch.zeros(n_blocks, dtype=torch.bool, device=device)
+    block_mask[chosen] = True
+    tok_mask = block_mask.repeat_interleave(cfg.block_size)[:n_tokens]
+    return tok_mask, u_idx * cfg.planted_shift, u_main * cfg.planted_shift, chosen
+
+
+def make_prefill_inputs(cfg: MSAConfig, device="cpu", sharp: bool = False):
+    """Q [T,H_q,d_h], K,V [T,H_kv,d_h], Q_idx [T,H_kv,d_idx], K_idx [T,d_idx], all bf16.
+
+    ``sharp=True`` drops the 1/sqrt(d) scaling (logits ~ N(0,1) instead of ~N(0,1e-4)),
+    which makes softmax weights non-uniform and the outputs O(1e-1): a variant used by
+    the parity tests because the default recipe gives outputs of magnitude ~1e-3.
+    """
+    device = torch.device(device)
+    gen = _gen(device, cfg.seed)
+    T, d, di = cfg.T, cfg.head_dim, cfg.idx_dim
+    s_main = 1.0 if sharp else d ** -0.5
+    s_idx = 1.0 if sharp else di ** -0.5
+    tok_mask = sh_idx = sh_main = None
+    if cfg.planted_frac > 0.0:
+        # The planted choice is drawn from its own generator so that it does not
+        # depend on how many values the tensors consumed.
+        pg = _gen(device, cfg.seed + 1000003)
+        tok_mask, sh_idx, sh_main, _ = _planted(cfg, pg, T, device)
+    q = _draw(gen, T, (cfg.n_q_heads, d), s_main, device)
+    k = _draw(gen, T, (cfg.n_kv_heads, d), s_main, device, tok_mask, sh_main)
+    v = _draw(gen, T, (cfg.n_kv_heads, d), s_main, device)
+    q_idx = _draw(gen, T, (cfg.n_kv_heads, di), s_idx, device)
+    k_idx = _draw(gen, T, (di,), s_idx, device, tok_mask, sh_idx)
+    return {"q": q, "k": k, "v": v, "q_idx": q_idx, "k_idx": k_idx}
+
+
+def make_decode_inputs(cfg: MSAConfig, device="cpu", sharp: bool = False):
+    """One new query token per cached sequence.
+
+    Caches are packed token-major: ``k_cache``/``v_cache`` [sum(L),H_kv,d_h] and
+    ``k_idx_cache`` [sum(L),d_idx]; sequence s occupies rows
+    ``seq_offsets[s] .. seq_offsets[s]+seq_lens[s]`` (the new token's K/V/K_idx are
+    already appended at its last row).  ``q`` [batch,H_q,d_h], ``q_idx`` [batch,H_kv,d_idx].
+    """
+    device = torch.device(device)
+    gen = _gen(device, cfg.seed)
+    lens = list(cfg.seq_lens)
+    batch, total = len(lens), int(sum(lens))
+    d, di = cfg.head_dim, cfg.idx_dim
+    s_main = 1.0 if sharp else d ** -0.5
+    s_idx = 1.0 if sharp else di ** -0.5
+    q = _draw(gen, batch, (cfg.n_q_heads, d), s_main, device)
+    k_cache = _draw(gen, total, (cfg.n_kv_heads, d), s_main, device)
+    v_cache = _draw(gen, total, (cfg.n_kv_heads, d), s_main, device)
+    q_idx = _draw(gen, batch, (cfg.n_kv_heads, di), s_idx, device)
+    k_idx_cache = _draw(gen, total, (di,), s_idx, device)
+    offs = np.concatenate([[0], np.cumsum(lens)[:-1]]).astype(np.int64)
+    return {
+        "q": q, "q_idx": q_idx, "k_cache": k_cache, "v_cache": v_cache,
+        "k_idx_cache": k_idx_cache,
+        "seq_offsets": torch.from_numpy(offs).to(device),
+        "seq_lens": torch.tensor(lens, dtype=torch.int32, device=device),
+    }
+
+
+def sample_positions(T: int, block_size: int, top_k: int, n: int, seed: int) -> np.ndarray:
+    """Stratified, sorted, unique sample of at least min(n, T) query positions in [0, T).
+
+    Always holds: the whole first block, the positions around the first block edge and
+    around the point where the number of visible blocks reaches k, both sides of a few
+    random block boundaries, the last positions; the rest uniform at random.
+    """
+    rng = np.random.default_rng(seed)
+    pos = set(range(min(block_size, T)))
+    for p in (block_size - 1, block_size, top_k * block_size - 1, top_k * block_size,
+              top_k * block_size + 1, T - 1, T - 2, (T - 1) // block_size * block_size,
+              (T - 1) // block_size * block_size - 1):
+        if 0 <= p < T:
+            pos.add(int(p))
+    n_blocks = -(-T // block_size)
+    for b in rng.integers(1, max(2, n_blocks), size=8):
+        for p in (int(b) * block_size - 1, int(b) * block_size):
+            if 0 <= p < T:
+                pos.add(p)
+    target = min(n, T)
+    while len(pos) < target:
+        pos.update(int(p) for p in rng.integers(0, T, size=target - len(pos)))
+    return np.array(sorted(pos), dtype=np.int64)
+
+
+def to_bits(t: torch.Tensor) -> np.ndarray:
+    """bf16 tensor (any device) -> contiguous numpy uint16 array of its bit patterns."""
+    assert t.dtype == torch.bfloat16
+    return t.detach().contiguous().cpu().view(torch.uint16).numpy()
+
+
+def bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    """uint16 bf16 bit patterns -> exact float32 values."""
+    return (bits.astype(np.uint32) << 16).view(np.float32)

@@ -1,0 +1,366 @@
+"""Pins the CPU oracle to things other than itself (no GPU needed).
+
+Each test checks an oracle function against what the paper or the mathematics fixes:
+invariants, special cases that reduce to a library routine, or brute force written here
+independently in NumPy on tiny inputs.
+"""
+
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2606_13392_b200.inputs import (MSAConfig, bits_to_f32, make_prefill_inputs,
+                                          to_bits)
+
+
+def tiny(T=40, Hq=4, Hkv=2, Bk=4, k=3, d=8, di=4, seed=0, sharp=True):
+    cfg = MSAConfig("tiny", "prefill", T, Hq, Hkv, Bk, k, head_dim=d, idx_dim=di, seed=seed)
+    t = make_prefill_inputs(cfg, "cpu", sharp=sharp)
+    return cfg, {n: to_bits(x) for n, x in t.items()}
+
+
+def f64(bits):
+    return bits_to_f32(bits).astype(np.float64)
+
+
+# ---------------------------------------------------------------- brute force (P4)
+def brute_scores(q_idx, k_idx, i, r, Bk):
+    """Eq. 6 by enumeration: returns dict block -> max score over visible tokens."""
+    qi, ki = f64(q_idx), f64(k_idx)
+    out = {}
+    for j in range(i + 1):
+        s = float(np.dot(qi[i, r], ki[j])) / np.sqrt(qi.shape[-1])
+        b = j // Bk
+        out[b] = max(out.get(b, -np.inf), s)
+    return out
+
+
+def brute_select(block_scores, i, Bk, k):
+    """Eq. 7 + local block by full sort of (score desc, index asc)."""
+    loc = i // Bk
+    earlier = sorted((b for b in block_scores if b < loc),
+                     key=lambda b: (-block_scores[b], b))
+    return sorted(earlier[:max(0, k - 1)] + [loc])
+
+
+def brute_attn(q, K, V, i, h, r, blocks, Bk):
+    """Eq. 8 by explicit token-set enumeration."""
+    qf, Kf, Vf = f64(q), f64(K), f64(V)
+    toks = [j for j in range(i + 1) if j // Bk in blocks]
+    z = np.array([np.dot(qf[i, h], Kf[j, r]) for j in toks]) / np.sqrt(qf.shape[-1])
+    w = np.exp(z - z.max())
+    w /= w.sum()
+    o = sum(wj * Vf[j, r] for wj, j in zip(w, toks))
+    lse = z.max() + np.log(np.exp(z - z.max()).sum())
+    return o, lse, toks
+
+
+@pytest.mark.parametrize("T,Hq,Hkv,Bk,k", [
+    (37, 2, 1, 4, 1), (37, 2, 2, 4, 2), (64, 4, 2, 8, 3), (23, 2, 1, 2, 3), (50, 4, 2, 4, 3),
+])
+def test_brute_force_tiny(T, Hq, Hkv, Bk, k):
+    cfg, x = tiny(T=T, Hq=Hq, Hkv=Hkv, Bk=Bk, k=k, seed=T + k)
+    pos = np.arange(T)
+    M, I, O, LSE = oracle.msa_forward(x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"],
+                                      pos, Bk, k)
+    G = Hq // Hkv
+    for i in range(T):
+        for r in range(Hkv):
+            bs = brute_scores(x["q_idx"], x["k_idx"], i, r, Bk)
+            for b in range(cfg.n_blocks):
+                want = bs.get(b, -np.inf)
+                assert M[i, r, b] == pytest.approx(want, rel=1e-12, abs=1e-14)
+            sel = brute_select(bs, i, Bk, k)
+            got = [b for b in I[i, r] if b >= 0]
+            assert got == sel
+            assert list(I[i, r, len(sel):]) == [-1] * (k - len(sel))
+            for h in range(r * G, (r + 1) * G):
+                o, lse, _ = brute_attn(x["q"], x["k"], x["v"], i, h, r, set(sel), Bk)
+                np.testing.assert_allclose(O[i, h], o, rtol=1e-11, atol=1e-13)
+                assert LSE[i, h] == pytest.approx(lse, rel=1e-12)
+
+
+# ---------------------------------------------------------------- P1, P9: selection rules
+def test_local_block_forced_and_inf_formulation():
+    cfg, x = tiny(T=200, Hq=4, Hkv=2, Bk=8, k=5, seed=3)
+    pos = np.arange(cfg.T)
+    M = oracle.index_scores(x["q_idx"], x["k_idx"], pos, cfg.block_size)
+    I = oracle.topk_select(M, pos, cfg.T, cfg.block_size, cfg.top_k)
+    for i in pos:
+        loc = i // cfg.block_size
+        for r in range(cfg.n_kv_heads):
+            got = [b for b in I[i, r] if b >= 0]
+            assert loc in got and got == sorted(got) and len(set(got)) == len(got)
+            assert len(got) == min(cfg.top_k, loc + 1)
+            assert max(got) == loc  # nothing beyond the local block
+            # Equivalent statement: give the local block +inf and take a plain top-k
+            # (stable sort by descending score keeps the lower index first among ties).
+            row = M[i, r].copy()
+            row[loc] = np.inf
+            order = np.argsort(-row, kind="stable")[:min(cfg.top_k, loc + 1)]
+            assert sorted(order.tolist()) == got
+            if loc < cfg.top_k:
+                assert got == list(range(loc + 1))
+
+
+def test_selection_invariances():
+    cfg, x = tiny(T=160, Hq=2, Hkv=2, Bk=4, k=6, seed=5)
+    pos = np.arange(cfg.T)
+    M = oracle.index_scores(x["q_idx"], x["k_idx"], pos, cfg.block_size)
+    I = oracle.topk_select(M, pos, cfg.T, cfg.block_size, cfg.top_k)
+    # exact (power-of-two) positive scaling and a per-row shift do not change the set
+    I2 = oracle.topk_select(M * 4.0, pos, cfg.T, cfg.block_size, cfg.top_k)
+    assert np.array_equal(I, I2)
+    shift = np.random.default_rng(0).integers(-8, 8, size=M.shape[:2] + (1,)).astype(np.float64)
+    with np.errstate(invalid="ignore"):
+        Ms = np.where(np.isfinite(M), np.round(M * 2 ** 20) / 2 ** 20 + shift, M)
+        I_a = oracle.topk_select(np.where(np.isfinite(M), np.round(M * 2 ** 20) / 2 ** 20, M),
+                                 pos, cfg.T, cfg.block_size, cfg.top_k)
+    I_b = oracle.topk_select(Ms, pos, cfg.T, cfg.block_size, cfg.top_k)
+    assert np.array_equal(I_a, I_b)
+
+
+def test_tie_break_lower_index_wins():
+    # 6 earlier blocks with equal scores: the lowest indices are taken.
+    B, k, Bk = 8, 4, 2
+    M = np.full((1, 1, B), -np.inf)
+    M[0, 0, :7] = 1.0
+    M[0, 0, 6] = 0.5  # local block's own score is irrelevant
+    pos = np.array([6 * Bk + 1])
+    I = oracle.topk_select(M, pos, B * Bk, Bk, k)
+    assert I[0, 0].tolist() == [0, 1, 2, 6]
+    M[0, 0, 4] = 2.0
+    I = oracle.topk_select(M, pos, B * Bk, Bk, k)
+    assert I[0, 0].tolist() == [0, 1, 4, 6]
+
+
+# ---------------------------------------------------------------- P2: exp-free == top-k of softmax
+def test_exp_free_equals_topk_of_softmax():
+    cfg, x = tiny(T=256, Hq=2, Hkv=2, Bk=4, k=9, seed=7)
+    pos = np.arange(cfg.T)
+    M = oracle.index_scores(x["q_idx"], x["k_idx"], pos, cfg.block_size)
+    I = oracle.topk_select(M, pos, cfg.T, cfg.block_size, cfg.top_k)
+    for i in pos[::3]:
+        loc = i // cfg.block_size
+        if loc == 0:
+            continue
+        for r in range(cfg.n_kv_heads):
+            row = M[i, r, :loc]
+            p = np.exp(row - row.max())
+            p /= p.sum()  # softmax over the rankable blocks, in double
+            sel = np.array([b for b in I[i, r] if 0 <= b < loc], dtype=int)
+            unsel = np.setdiff1d(np.arange(loc), sel)
+            assert len(sel) == min(cfg.top_k - 1, loc)
+            if len(unsel) and len(sel):
+                assert p[sel].min() >= p[unsel].max()
+
+
+# ---------------------------------------------------------------- P11: torch.topk agrees
+def test_matches_torch_topk_away_from_ties():
+    cfg, x = tiny(T=512, Hq=2, Hkv=1, Bk=4, k=8, seed=11)
+    pos = np.arange(cfg.T)
+    M = oracle.index_scores(x["q_idx"], x["k_idx"], pos, cfg.block_size)
+    I = oracle.topk_select(M, pos, cfg.T, cfg.block_size, cfg.top_k)
+    checked = 0
+    for i in pos:
+        loc = i // cfg.block_size
+        if loc < cfg.top_k:
+            continue
+        row = torch.from_numpy(M[i, 0, :loc])
+        vals, idx = torch.topk(row, cfg.top_k - 1)
+        srt = torch.sort(row, descending=True).values
+        if srt[cfg.top_k - 2] == srt[cfg.top_k - 1]:
+            continue  # boundary tie: torch's choice is unspecified
+        assert sorted(idx.tolist() + [loc]) == I[i, 0].tolist()
+        checked += 1
+    assert checked > 300
+
+
+# ---------------------------------------------------------------- P8: stage 1 vs library matmul
+def test_index_scores_match_matmul_reshape_max():
+    cfg, x = tiny(T=96, Hq=4, Hkv=2, Bk=8, k=3, di=16, seed=13)
+    pos = np.arange(cfg.T)
+    M = oracle.index_scores(x["q_idx"], x["k_idx"], pos, cfg.block_size)
+    qi, ki = f64(x["q_idx"]), f64(x["k_idx"])
+    S = np.einsum("irc,jc->irj", qi, ki) / np.sqrt(cfg.idx_dim)  # [T,Hkv,T]
+    causal = np.arange(cfg.T)[None, :] <= np.arange(cfg.T)[:, None]
+    S = np.where(causal[:, None, :], S, -np.inf)
+    want = S.reshape(cfg.T, cfg.n_kv_heads, cfg.n_blocks, cfg.block_size).max(-1)
+    np.testing.assert_allclose(M, want, rtol=1e-12, atol=1e-14)
+    # invisible blocks are exactly -inf, visible ones finite
+    for i in range(cfg.T):
+        loc = i // cfg.block_size
+        assert np.all(np.isfinite(M[i, :, :loc + 1]))
+        assert np.all(np.isneginf(M[i, :, loc + 1:]))
+
+
+def test_index_scores_ragged_last_block():
+    cfg, x = tiny(T=45, Hq=2, Hkv=1, Bk=8, k=2, di=8, seed=17)
+    pos = np.array([44, 40, 39, 7, 0])
+    M = oracle.index_scores(x["q_idx"][pos], x["k_idx"], pos, cfg.block_size)
+    assert M.shape == (5, 1, 6)
+    qi, ki = f64(x["q_idx"]), f64(x["k_idx"])
+    for a, i in enumerate(pos):
+        s = (ki[: i + 1] @ qi[i, 0]) / np.sqrt(cfg.idx_dim)
+        for b in range(6):
+            seg = s[b * 8: (b + 1) * 8]
+            want = seg.max() if len(seg) else -np.inf
+            assert M[a, 0, b] == pytest.approx(want, rel=1e-12, abs=1e-14)
+
+
+# ---------------------------------------------------------------- P3: k >= B  ==> dense causal GQA
+def test_all_blocks_selected_equals_dense_and_sdpa():
+    cfg, x = tiny(T=70, Hq=6, Hkv=2, Bk=8, k=9, d=16, di=8, seed=19, sharp=True)
+    assert cfg.top_k >= cfg.n_blocks
+    pos = np.arange(cfg.T)
+    _, I, O, LSE = oracle.msa_forward(x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"],
+                                      pos, cfg.block_size, cfg.top_k)
+    Od, LSEd = oracle.dense_attn(x["q"], x["k"], x["v"], pos)
+    np.testing.assert_allclose(O, Od, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(LSE, LSEd, rtol=1e-12)
+    # library routine: torch SDPA, causal, KV heads repeated per group (adjacent heads)
+    G = cfg.group
+    q = torch.from_numpy(f64(x["q"])).permute(1, 0, 2)[None]  # [1,Hq,T,d]
+    k = torch.from_numpy(f64(x["k"])).permute(1, 0, 2).repeat_interleave(G, 0)[None]
+    v = torch.from_numpy(f64(x["v"])).permute(1, 0, 2).repeat_interleave(G, 0)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True)
+    ref = ref[0].permute(1, 0, 2).numpy()
+    np.testing.assert_allclose(O, ref, rtol=1e-9, atol=1e-12)
+
+
+def test_dense_attn_matches_numpy_definition():
+    cfg, x = tiny(T=33, Hq=4, Hkv=2, Bk=4, k=2, d=8, seed=23)
+    pos = np.array([0, 1, 17, 32])
+    Od, LSEd = oracle.dense_attn(x["q"][pos], x["k"], x["v"], pos)
+    qf, Kf, Vf = f64(x["q"]), f64(x["k"]), f64(x["v"])
+    for a, t in enumerate(pos):
+        for h in range(4):
+            r = h // 2
+            z = Kf[: t + 1, r] @ qf[t, h] / np.sqrt(8)
+            al = np.exp(z) / np.exp(z).sum()
+            np.testing.assert_allclose(Od[a, h], al @ Vf[: t + 1, r], rtol=1e-12, atol=1e-14)
+            assert LSEd[a, h] == pytest.approx(np.log(np.exp(z).sum()), rel=1e-12)
+
+
+# ---------------------------------------------------------------- P6: token budget
+def test_token_budget():
+    cfg, x = tiny(T=130, Hq=2, Hkv=1, Bk=8, k=4, seed=29)
+    pos = np.arange(cfg.T)
+    M = oracle.index_scores(x["q_idx"], x["k_idx"], pos, cfg.block_size)
+    I = oracle.topk_select(M, pos, cfg.T, cfg.block_size, cfg.top_k)
+    for i in pos:
+        sel = [b for b in I[i, 0] if b >= 0]
+        n_tok = sum(min((b + 1) * 8, i + 1) - b * 8 for b in sel)
+        assert n_tok <= cfg.top_k * cfg.block_size
+        full = (i // 8 >= cfg.top_k - 1) and (i % 8 == 7)
+        assert (n_tok == cfg.top_k * cfg.block_size) == full
+
+
+# ---------------------------------------------------------------- P7: combine identity
+def test_combine_identity_any_partition():
+    cfg, x = tiny(T=90, Hq=4, Hkv=2, Bk=8, k=5, d=8, seed=31)
+    i = 85
+    pos = np.array([i])
+    qrow = x["q"][pos]
+    M = oracle.index_scores(x["q_idx"][pos], x["k_idx"], pos, cfg.block_size)
+    I = oracle.topk_select(M, pos, cfg.T, cfg.block_size, cfg.top_k)
+    O, LSE = oracle.sparse_attn(qrow, x["k"], x["v"], I, pos, cfg.block_size)
+    sel = [int(b) for b in I[0, 0] if b >= 0]
+    assert len(sel) == 5
+    for parts in ([[0], [1], [2], [3], [4]], [[0, 1, 2, 3, 4]], [[0, 3], [1], [2, 4]],
+                  [[4], [0, 1, 2, 3]]):
+        for h in range(cfg.n_q_heads):
+            r = h // cfg.group
+            blocks = [int(b) for b in I[0, r] if b >= 0]
+            Op, Lp = [], []
+            for part in parts:
+                Ipart = np.full((1, cfg.n_kv_heads, cfg.top_k), -1, dtype=np.int32)
+                Ipart[0, r, :len(part)] = sorted(blocks[t] for t in part)
+                o, l = oracle.sparse_attn(qrow, x["k"], x["v"], Ipart, pos, cfg.block_size)
+                Op.append(o[0, h])
+                Lp.append(l[0, h])
+            o_c, lse_c = oracle.combine(np.stack(Op), np.array(Lp))
+            np.testing.assert_allclose(o_c, O[0, h], rtol=1e-12, atol=1e-14)
+            assert lse_c == pytest.approx(LSE[0, h], rel=1e-12)
+
+
+def test_combine_closed_form_two_parts():
+    # two parts with LSE ln(1) and ln(3): weights 1/4 and 3/4
+    o, lse = oracle.combine(np.array([[4.0, 0.0], [0.0, 8.0]]), np.log(np.array([1.0, 3.0])))
+    np.testing.assert_allclose(o, [1.0, 6.0], rtol=1e-14)
+    assert lse == pytest.approx(np.log(4.0), rel=1e-14)
+    # an empty part (LSE = -inf) is ignored
+    o, lse = oracle.combine(np.array([[4.0, 0.0], [7.0, 7.0]]), np.array([0.0, -np.inf]))
+    np.testing.assert_allclose(o, [4.0, 0.0])
+    assert lse == 0.0
+
+
+# ---------------------------------------------------------------- P10: decode == last prefill row; causality
+def test_decode_is_last_row_and_future_tokens_do_not_matter():
+    cfg, x = tiny(T=77, Hq=4, Hkv=2, Bk=8, k=4, seed=37)
+    pos = np.arange(cfg.T)
+    M, I, O, LSE = oracle.msa_forward(x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"],
+                                      pos, cfg.block_size, cfg.top_k)
+    for L in (1, 8, 9, 40, 77):
+        p = np.array([L - 1])
+        Md, Id, Od, Ld = oracle.msa_forward(x["q"][p], x["k"][:L], x["v"][:L],
+                                            x["q_idx"][p], x["k_idx"][:L], p,
+                                            cfg.block_size, cfg.top_k)
+        nb = -(-L // cfg.block_size)
+        np.testing.assert_array_equal(Md[0], M[L - 1][:, :nb])
+        np.testing.assert_array_equal(Id[0], I[L - 1])
+        np.testing.assert_array_equal(Od[0], O[L - 1])
+        np.testing.assert_array_equal(Ld[0], LSE[L - 1])
+
+
+# ---------------------------------------------------------------- P12: softmax sanity
+def test_output_in_convex_hull_and_lse_finite():
+    cfg, x = tiny(T=120, Hq=4, Hkv=2, Bk=8, k=3, d=8, seed=41)
+    pos = np.arange(cfg.T)
+    _, I, O, LSE = oracle.msa_forward(x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"],
+                                      pos, cfg.block_size, cfg.top_k)
+    Vf = f64(x["v"])
+    assert np.all(np.isfinite(LSE)) and np.all(np.isfinite(O))
+    for i in pos[::7]:
+        for h in range(cfg.n_q_heads):
+            r = h // cfg.group
+            toks = [j for j in range(i + 1) if j // 8 in set(I[i, r].tolist())]
+            lo, hi = Vf[toks, r].min(0), Vf[toks, r].max(0)
+            assert np.all(O[i, h] >= lo - 1e-12) and np.all(O[i, h] <= hi + 1e-12)
+    # a query at position 0 sees one token: output is exactly that value row, LSE = z
+    np.testing.assert_allclose(O[0, 0], Vf[0, 0], rtol=1e-15)
+
+
+def test_group_sharing_uses_adjacent_heads():
+    # Make KV head 1's values distinct constants: heads 2,3 (group 1) must output them.
+    cfg, x = tiny(T=24, Hq=4, Hkv=2, Bk=4, k=2, d=8, seed=43)
+    v = torch.zeros(24, 2, 8, dtype=torch.bfloat16)
+    v[:, 0] = 1.0
+    v[:, 1] = -2.0
+    pos = np.arange(24)
+    _, _, O, _ = oracle.msa_forward(x["q"], x["k"], to_bits(v), x["q_idx"], x["k_idx"], pos, 4, 2)
+    np.testing.assert_allclose(O[:, 0:2], 1.0, rtol=1e-14)
+    np.testing.assert_allclose(O[:, 2:4], -2.0, rtol=1e-14)
+
+
+# ---------------------------------------------------------------- P5: printed FLOPs ratio
+def test_flops_model_printed_ratio():
+    path = os.path.join(os.path.dirname(__file__), "golden", "flops_reduction_1m.txt")
+    vals = {}
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        key, val = line.split()
+        vals[key] = float(val)
+    N = int(vals["N"])
+    ratio = oracle.flops_gqa(N, int(vals["H_q"]), int(vals["d_h"])) / oracle.flops_msa(
+        N, int(vals["H_q"]), int(vals["H_kv"]), int(vals["d_h"]), int(vals["d_idx"]),
+        int(vals["k"]), int(vals["B_k"]))
+    assert round(ratio, 1) == vals["ratio"]
+    # closed forms of the two terms
+    assert oracle.flops_gqa(10, 3, 5) == 2 * 3 * 5 * 100
+    assert oracle.flops_msa(10, 4, 2, 5, 7, 3, 2) == 2 * 7 * 100 + 4 * 4 * 5 * 10 * 3 * 2
