@@ -1,0 +1,236 @@
+/*
+ * msa.h - C ABI of the B200 (sm_100a) forward hot path of MiniMax Sparse Attention.
+ *
+ * The path is Algorithm 1, lines 3-5 of the paper:
+ *   line 3  BlockMaxPool : index scoring + causal block max        (Eq. 6)  msa_index_scores
+ *   line 4  TopK         : exp-free Top-k, local block forced in   (Eq. 7)  msa_topk_select
+ *   line 5  TopKAttn     : block-sparse GQA softmax attention      (Eq. 8)  msa_sparse_attn_prefill
+ *                                                                           msa_sparse_attn_decode
+ *
+ * Conventions common to every call
+ *   - Every pointer is a DEVICE pointer unless its name ends in "_host".  The caller owns
+ *     every buffer, including workspaces; the library allocates no device memory, never
+ *     frees, and never synchronises the stream unless a call says so.
+ *   - bf16 tensors are passed as `const void*`; all tensors are dense, token-major, last
+ *     dimension contiguous:  Q [T,H_q,d_h], K,V [T,H_kv,d_h], Q_idx [T,H_kv,d_idx],
+ *     K_idx [T,d_idx] (one index key head shared by all groups, Eq. 5).  Bases must be
+ *     16-byte aligned.
+ *   - Indices are 0-based: token j is in block j / B_k (Eq. 4); query head h is in GQA
+ *     group r = h / G, G = H_q / H_kv (Section 2.1); B = ceil(kv_len / B_k).
+ *   - A "query range" is rows [q_begin, q_begin + q_count) of one sequence of kv_len
+ *     tokens; q_begin + q_count <= kv_len; row pointers point at row q_begin.
+ *   - Calls return MSA_OK after enqueuing their work on `stream`.  Argument, shape,
+ *     alignment and workspace errors are returned before anything is launched.  CUDA
+ *     launch errors map to MSA_ERR_CUDA.  Device-side anomalies (a bounded wait that ran
+ *     out, a block index out of range) never trap: they set a status word that
+ *     msa_check_async_status() reads.
+ *   - Fast kernels are specialised for d_h = 128, d_idx = 64, B_k in {64,128},
+ *     G in {8,16}; other shapes (d_h, d_idx multiples of 8, d_h <= 256, d_idx <= 128)
+ *     run on generic kernels.  k is limited to 1..128.
+ */
+#ifndef MSA_H_
+#define MSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MSA_OK = 0,
+    MSA_ERR_INVALID_ARG = 1, /* null pointer, negative size, misaligned base, bad range   */
+    MSA_ERR_UNSUPPORTED = 2, /* shape outside what the kernels implement                   */
+    MSA_ERR_WORKSPACE = 3,   /* workspace smaller than the *_workspace_bytes() minimum     */
+    MSA_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed                        */
+    MSA_ERR_TIMEOUT = 5,     /* a device-side bounded wait ran out (see async status)      */
+    MSA_ERR_BAD_INDEX = 6    /* a block index outside [-1, B) was met on the device        */
+} msa_status_t;
+
+/* Shape of one MSA layer, in the paper's notation (Sections 2 and 3.1). */
+typedef struct {
+    int32_t n_q_heads;   /* H_q                                                   */
+    int32_t n_kv_heads;  /* H_kv (= number of GQA groups = index query heads)     */
+    int32_t head_dim;    /* d_h                                                   */
+    int32_t idx_dim;     /* d_idx                                                 */
+    int32_t block_size;  /* B_k                                                   */
+    int32_t top_k;       /* k, blocks per (query, group) including the local one  */
+    float softmax_scale; /* 0 => 1/sqrt(d_h)   (Eq. 1, Eq. 8)                     */
+    float index_scale;   /* 0 => 1/sqrt(d_idx) (Eq. 6)                            */
+} msa_shape_t;
+
+typedef void* msa_stream_t; /* a cudaStream_t */
+
+const char* msa_status_string(msa_status_t s);
+
+/*
+ * Reads and clears the device-side status word (synchronises the device).  Returns
+ * MSA_OK, MSA_ERR_TIMEOUT or MSA_ERR_BAD_INDEX; *detail (optional, host) receives a code
+ * naming the kernel and the wait or index that failed.
+ */
+msa_status_t msa_check_async_status(int32_t* detail_host);
+
+/* ------------------------------------------------------------------------------------
+ * Stage 1 - Eq. 6 (Algorithm 1, line 3; Section 6 appendix remark that inference needs
+ * only the block-wise maximum of Q_idx K_idx^T).
+ *   scores[q, r, b] = index_scale * max_{j in block b, j <= q_begin+q} <Q_idx[q,r,:], K_idx[j,:]>
+ *   scores[q, r, b] = -inf for blocks with no visible token (b > (q_begin+q)/B_k).
+ * q_idx  [q_count,H_kv,d_idx] bf16 (rows of the range), k_idx [kv_len,d_idx] bf16,
+ * scores [q_count,H_kv,ld_scores] fp32, ld_scores >= B and a multiple of 4; columns
+ * b in [0,B) of every row are written, columns [B, ld_scores) are left untouched.
+ */
+msa_status_t msa_index_scores(const msa_shape_t* shape, const void* q_idx, const void* k_idx,
+                              int64_t q_begin, int64_t q_count, int64_t kv_len,
+                              float* scores, int64_t ld_scores, msa_stream_t stream);
+
+/*
+ * Stage 1 for batched decode: sequence s has its K_idx rows at
+ * k_idx_cache[seq_offsets[s] .. seq_offsets[s]+seq_lens[s]) and one query (its last
+ * token, position seq_lens[s]-1, already appended to the cache).
+ * q_idx [batch,H_kv,d_idx]; seq_offsets int64 [batch] (in tokens); seq_lens int32 [batch];
+ * scores [batch,H_kv,ld_scores]: columns [0, ceil(seq_lens[s]/B_k)) are written with the
+ * Eq. 6 values, columns up to ceil(max_seq_len/B_k) with -inf.
+ */
+msa_status_t msa_index_scores_decode(const msa_shape_t* shape, const void* q_idx,
+                                     const void* k_idx_cache, const int64_t* seq_offsets,
+                                     const int32_t* seq_lens, int32_t batch,
+                                     int64_t max_seq_len, float* scores, int64_t ld_scores,
+                                     msa_stream_t stream);
+
+/* ------------------------------------------------------------------------------------
+ * Stage 2 - Eq. 7 with the Local Block rule (Section 3.2) and exp-free ranking
+ * (Section 4.1): for row (q, r), loc = (q_begin+q)/B_k is always selected and the
+ * other min(k-1, loc) entries are the earlier blocks with the largest raw scores
+ * (ties: lower block index wins).
+ * block_idx [q_count,H_kv,k] int32: ascending block indices, padded with -1 when fewer
+ * than k blocks are visible.  Only columns [0, loc] of a scores row are read.
+ */
+msa_status_t msa_topk_select(const msa_shape_t* shape, const float* scores, int64_t ld_scores,
+                             int64_t q_begin, int64_t q_count, int64_t kv_len,
+                             int32_t* block_idx, msa_stream_t stream);
+
+/* Stage 2 for batched decode: row (s, r) ranks blocks of sequence s, loc = (seq_lens[s]-1)/B_k. */
+msa_status_t msa_topk_select_decode(const msa_shape_t* shape, const float* scores,
+                                    int64_t ld_scores, const int32_t* seq_lens, int32_t batch,
+                                    int32_t* block_idx, msa_stream_t stream);
+
+/* ------------------------------------------------------------------------------------
+ * Stage 3, prefill - Eq. 8 (Algorithm 1, line 5): for each query of the range and each
+ * head h of group r, softmax attention over the causally visible tokens of the blocks
+ * block_idx[q, r, :] (entries < 0 are skipped), using KV head r.
+ *   out [q_count,H_q,d_h] bf16;  lse [q_count,H_q] fp32 or NULL:
+ *   lse = log sum_j exp(softmax_scale * <q, k_j>) over the attended tokens (natural log).
+ * The specialised path gathers, per (KV block, KV head), the queries that selected it
+ * (KV-outer order, Section 4.2), writes locally normalised partials to the workspace
+ * and merges them with the LSE-weighted combine of Section 4.2.  The workspace bounds
+ * how many queries are in flight at once; a larger workspace means fewer passes.
+ * A block index outside [-1, loc] is skipped and reported through the async status.
+ */
+msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, const void* k,
+                                     const void* v, const int32_t* block_idx,
+                                     int64_t q_begin, int64_t q_count, int64_t kv_len,
+                                     void* out, float* lse, void* workspace,
+                                     size_t workspace_bytes, msa_stream_t stream);
+
+/* Minimum and preferred workspace for msa_sparse_attn_prefill (bytes; either may be NULL). */
+msa_status_t msa_sparse_attn_prefill_workspace_bytes(const msa_shape_t* shape, int64_t q_count,
+                                                     int64_t kv_len, size_t* min_bytes,
+                                                     size_t* preferred_bytes);
+
+/* ------------------------------------------------------------------------------------
+ * Stage 3, decode - Eq. 8 for one query per cached sequence (position seq_lens[s]-1).
+ * q [batch,H_q,d_h]; k_cache, v_cache [cache_tokens,H_kv,d_h] bf16 packed token-major,
+ * sequence s at rows seq_offsets[s]..; block_idx [batch,H_kv,k]; out [batch,H_q,d_h]
+ * bf16; lse [batch,H_q] fp32 or NULL.  The selected blocks of each (sequence, KV head)
+ * are split over several CTAs; partials are merged with the Section 4.2 combine.
+ */
+msa_status_t msa_sparse_attn_decode(const msa_shape_t* shape, const void* q, const void* k_cache,
+                                    const void* v_cache, int64_t cache_tokens,
+                                    const int64_t* seq_offsets, const int32_t* seq_lens,
+                                    int32_t batch, const int32_t* block_idx, void* out,
+                                    float* lse, void* workspace, size_t workspace_bytes,
+                                    msa_stream_t stream);
+
+msa_status_t msa_sparse_attn_decode_workspace_bytes(const msa_shape_t* shape, int32_t batch,
+                                                    size_t* min_bytes);
+
+/* ------------------------------------------------------------------------------------
+ * Whole path, prefill (Algorithm 1, lines 3-5) for one sequence of T tokens: runs stage 1
+ * and 2 over query chunks sized to the workspace, then stage 3.  block_idx [T,H_kv,k] is
+ * an output (required); lse may be NULL.  workspace >= msa_prefill_forward_workspace_bytes.
+ */
+msa_status_t msa_prefill_forward(const msa_shape_t* shape, const void* q, const void* k,
+                                 const void* v, const void* q_idx, const void* k_idx, int64_t T,
+                                 void* out, float* lse, int32_t* block_idx, void* workspace,
+                                 size_t workspace_bytes, msa_stream_t stream);
+
+msa_status_t msa_prefill_forward_workspace_bytes(const msa_shape_t* shape, int64_t T,
+                                                 size_t* min_bytes, size_t* preferred_bytes);
+
+/*
+ * Same, from HOST buffers: copies q, k, v, q_idx, k_idx host->device into the staging
+ * area at the front of `workspace`, runs msa_prefill_forward, copies `out` (and lse,
+ * block_idx when non-NULL) back, and synchronises `stream` before returning.  Host
+ * buffers should be page-locked for the copies to run at full rate.
+ * workspace >= msa_prefill_forward_host_workspace_bytes.
+ */
+msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_host,
+                                      const void* k_host, const void* v_host,
+                                      const void* q_idx_host, const void* k_idx_host, int64_t T,
+                                      void* out_host, float* lse_host, int32_t* block_idx_host,
+                                      void* workspace, size_t workspace_bytes,
+                                      msa_stream_t stream);
+
+msa_status_t msa_prefill_forward_host_workspace_bytes(const msa_shape_t* shape, int64_t T,
+                                                      size_t* min_bytes,
+                                                      size_t* preferred_bytes);
+
+/*
+ * Whole path, decode step (stages 1-3 for one new token per sequence).  scores
+ * [batch,H_kv,ld_scores] and block_idx [batch,H_kv,k] are outputs kept for the caller.
+ */
+msa_status_t msa_decode_forward(const msa_shape_t* shape, const void* q, const void* q_idx,
+                                const void* k_cache, const void* v_cache,
+                                const void* k_idx_cache, int64_t cache_tokens,
+                                const int64_t* seq_offsets, const int32_t* seq_lens,
+                                int32_t batch, int64_t max_seq_len, float* scores,
+                                int64_t ld_scores, int32_t* block_idx, void* out, float* lse,
+                                void* workspace, size_t workspace_bytes, msa_stream_t stream);
+
+/*
+ * Same with the step's inputs and result in HOST memory: q_host [batch,H_q,d_h] and
+ * q_idx_host [batch,H_kv,d_idx] are copied in, out_host [batch,H_q,d_h] is copied back;
+ * the caches stay resident on the device.  q_dev/q_idx_dev/out_dev are device staging
+ * buffers of the same sizes.  Synchronises `stream` before returning.
+ */
+msa_status_t msa_decode_forward_host(const msa_shape_t* shape, const void* q_host,
+                                     const void* q_idx_host, void* q_dev, void* q_idx_dev,
+                                     const void* k_cache, const void* v_cache,
+                                     const void* k_idx_cache, int64_t cache_tokens,
+                                     const int64_t* seq_offsets, const int32_t* seq_lens,
+                                     int32_t batch, int64_t max_seq_len, float* scores,
+                                     int64_t ld_scores, int32_t* block_idx, void* out_dev,
+                                     void* out_host, void* workspace, size_t workspace_bytes,
+                                     msa_stream_t stream);
+
+/* Number of kernel launches the library has enqueued since the process started. */
+int64_t msa_launch_count(void);
+
+/*
+ * Optional per-stage timing for benchmarks (the paper has no counterpart).  Between
+ * msa_profile_begin() and msa_profile_end() every kernel launch of the library is
+ * bracketed by CUDA events on its stream; msa_profile_end() synchronises the device and
+ * returns, per stage, the summed device time in milliseconds and the number of launches
+ * (arrays of 8: 0 index scoring, 1 top-k, 2 reverse index/schedule, 3 prefill attention,
+ * 4 combine, 5 decode index scoring, 6 decode attention, 7 decode combine).  The first
+ * msa_profile_begin() creates the event pool (8192 launches); MSA_ERR_UNSUPPORTED from
+ * msa_profile_end() means the pool ran out and the sums are partial.  Not thread-safe.
+ */
+msa_status_t msa_profile_begin(void);
+msa_status_t msa_profile_end(float* stage_ms_host, int64_t* stage_launches_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MSA_H_ */

@@ -1,0 +1,80 @@
+"""Convenience layer over the binding: allocates outputs/workspaces with torch and calls the
+C ABI.  No arithmetic happens here."""
+
+from __future__ import annotations
+
+from typing import Dict, Optional
+
+import torch
+
+from . import binding as B
+from .inputs import MSAConfig
+
+
+def prefill_forward(cfg: MSAConfig, x: Dict[str, torch.Tensor], workspace: Optional[torch.Tensor] = None,
+                    want_lse: bool = True, workspace_bytes: Optional[int] = None):
+    """Algorithm 1 lines 3-5 on device tensors q,k,v,q_idx,k_idx -> (out, lse, block_idx)."""
+    shape = B.shape_of(cfg)
+    T = x["q"].shape[0]
+    dev = x["q"].device
+    out = torch.empty_like(x["q"])
+    lse = torch.empty((T, cfg.n_q_heads), dtype=torch.float32, device=dev) if want_lse else None
+    block_idx = torch.empty((T, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32, device=dev)
+    if workspace is None:
+        mn, pf = B.msa_prefill_forward_workspace_bytes(shape, T)
+        workspace = B.alloc_workspace(pf if workspace_bytes is None else max(mn, workspace_bytes), dev)
+    B.msa_prefill_forward(shape, x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"], T, out, lse,
+                          block_idx, workspace)
+    return out, lse, block_idx
+
+
+def index_scores(cfg: MSAConfig, q_idx: torch.Tensor, k_idx: torch.Tensor, q_begin: int, q_count: int,
+                 kv_len: Optional[int] = None) -> torch.Tensor:
+    """Eq. 6 for rows [q_begin, q_begin+q_count); q_idx holds the whole sequence's rows."""
+    shape = B.shape_of(cfg)
+    kv_len = k_idx.shape[0] if kv_len is None else kv_len
+    ld = B.score_ld(kv_len, cfg.block_size)
+    scores = torch.full((q_count, cfg.n_kv_heads, ld), float("nan"), dtype=torch.float32,
+                        device=q_idx.device)
+    B.msa_index_scores(shape, q_idx[q_begin:q_begin + q_count], k_idx, q_begin, q_count, kv_len,
+                       scores, ld)
+    return scores
+
+
+def topk_select(cfg: MSAConfig, scores: torch.Tensor, q_begin: int, kv_len: int) -> torch.Tensor:
+    shape = B.shape_of(cfg)
+    q_count, _, ld = scores.shape
+    block_idx = torch.empty((q_count, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32,
+                            device=scores.device)
+    B.msa_topk_select(shape, scores, ld, q_begin, q_count, kv_len, block_idx)
+    return block_idx
+
+
+def sparse_attn_prefill(cfg: MSAConfig, q, k, v, block_idx, q_begin: int = 0,
+                        workspace_bytes: Optional[int] = None):
+    shape = B.shape_of(cfg)
+    q_count, kv_len = q.shape[0], k.shape[0]
+    out = torch.empty_like(q)
+    lse = torch.empty((q_count, cfg.n_q_heads), dtype=torch.float32, device=q.device)
+    mn, pf = B.msa_sparse_attn_prefill_workspace_bytes(shape, q_count, kv_len)
+    ws = B.alloc_workspace(pf if workspace_bytes is None else max(mn, workspace_bytes), q.device)
+    B.msa_sparse_attn_prefill(shape, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, ws)
+    return out, lse
+
+
+def decode_forward(cfg: MSAConfig, x: Dict[str, torch.Tensor]):
+    """One decode step for a batch of cached sequences -> (out, lse, block_idx, scores)."""
+    shape = B.shape_of(cfg)
+    batch = x["q"].shape[0]
+    dev = x["q"].device
+    max_len = int(max(cfg.seq_lens))
+    ld = B.score_ld(max_len, cfg.block_size)
+    scores = torch.empty((batch, cfg.n_kv_heads, ld), dtype=torch.float32, device=dev)
+    block_idx = torch.empty((batch, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32, device=dev)
+    out = torch.empty_like(x["q"])
+    lse = torch.empty((batch, cfg.n_q_heads), dtype=torch.float32, device=dev)
+    ws = B.alloc_workspace(B.msa_sparse_attn_decode_workspace_bytes(shape, batch), dev)
+    B.msa_decode_forward(shape, x["q"], x["q_idx"], x["k_cache"], x["v_cache"], x["k_idx_cache"],
+                         x["k_cache"].shape[0], x["seq_offsets"], x["seq_lens"], batch, max_len,
+                         scores, ld, block_idx, out, lse, ws)
+    return out, lse, block_idx, scores

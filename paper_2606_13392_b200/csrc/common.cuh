@@ -1,0 +1,72 @@
+// Shared device/host helpers of the MSA CUDA library (not used by the CPU oracle).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/msa.h"
+
+namespace msa {
+
+constexpr int kMaxKvHeadsGeneric = 16;
+constexpr int kWarp = 32;
+
+// Device status word: 0 = ok, otherwise (code << 24) | detail.  Kernels receive its
+// address as an argument; the first non-zero value wins.
+enum AsyncCode : int { kAsyncOk = 0, kAsyncTimeout = 1, kAsyncBadIndex = 2 };
+
+__device__ __forceinline__ void report_async(int* status, int code, int detail) {
+    atomicCAS(status, 0, (code << 24) | (detail & 0xFFFFFF));
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
+    return __uint_as_float(((uint32_t)b) << 16);
+}
+
+// Two packed bf16 (low half first) -> two floats.
+__device__ __forceinline__ float2 bf16x2_to_float2(uint32_t u) {
+    return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+int* async_status_ptr();  // device address of the status word of the current device
+
+// Stages of the path, for launch counting and the optional per-stage timing.
+enum Stage : int {
+    kStageIndex = 0,      // Eq. 6, prefill
+    kStageTopk = 1,       // Eq. 7
+    kStageSchedule = 2,   // reverse index + work list (KV-outer prefill)
+    kStageAttn = 3,       // Eq. 8, prefill partials
+    kStageCombine = 4,    // LSE-weighted merge
+    kStageIndexDecode = 5,
+    kStageAttnDecode = 6,
+    kStageCombineDecode = 7,
+    kNumStages = 8
+};
+
+// Wraps one kernel launch: counts it and, while profiling is on, brackets it with CUDA
+// events on the launching stream.
+class StageScope {
+public:
+    StageScope(int stage, cudaStream_t st);
+    ~StageScope();
+private:
+    int slot_;
+    cudaStream_t st_;
+};
+
+}  // namespace msa

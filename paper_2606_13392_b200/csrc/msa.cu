@@ -1,0 +1,510 @@
+// C ABI of the MSA forward path (see include/msa.h): argument validation, workspace
+// planning and kernel dispatch.  All arithmetic is in the kernels included below.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+#include "generic.cuh"
+#include "topk.cuh"
+
+namespace msa {
+
+static std::atomic<int64_t> g_launches{0};
+
+// Optional per-stage timing: a fixed pool of event pairs, created by msa_profile_begin().
+constexpr int kProfSlots = 8192;
+static bool g_prof_on = false;
+static int g_prof_used = 0;
+static cudaEvent_t g_prof_ev[kProfSlots][2];
+static int g_prof_stage[kProfSlots];
+static bool g_prof_created = false;
+
+StageScope::StageScope(int stage, cudaStream_t st) : slot_(-1), st_(st) {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (g_prof_on && g_prof_used < kProfSlots) {
+        slot_ = g_prof_used++;
+        g_prof_stage[slot_] = stage;
+        cudaEventRecord(g_prof_ev[slot_][0], st_);
+    }
+}
+StageScope::~StageScope() {
+    if (slot_ >= 0) cudaEventRecord(g_prof_ev[slot_][1], st_);
+}
+
+__device__ int g_async_status = 0;
+
+int* async_status_ptr() {
+    // One address per device; looked up on each call (cheap, no allocation).
+    int* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_async_status) != cudaSuccess) return nullptr;
+    return p;
+}
+
+struct Resolved {
+    int H_q, H_kv, G, d, d_idx, B_k, k;
+    float softmax_scale, index_scale;
+};
+
+static msa_status_t resolve(const msa_shape_t* s, Resolved& r) {
+    if (s == nullptr) return MSA_ERR_INVALID_ARG;
+    if (s->n_q_heads <= 0 || s->n_kv_heads <= 0 || s->head_dim <= 0 || s->idx_dim <= 0 ||
+        s->block_size <= 0 || s->top_k <= 0)
+        return MSA_ERR_INVALID_ARG;
+    if (s->n_q_heads % s->n_kv_heads != 0) return MSA_ERR_INVALID_ARG;
+    r.H_q = s->n_q_heads; r.H_kv = s->n_kv_heads; r.G = r.H_q / r.H_kv;
+    r.d = s->head_dim; r.d_idx = s->idx_dim; r.B_k = s->block_size; r.k = s->top_k;
+    if (r.k > 128) return MSA_ERR_UNSUPPORTED;
+    if (r.d % 8 != 0 || r.d > 256 || r.d_idx % 8 != 0 || r.d_idx > 128) return MSA_ERR_UNSUPPORTED;
+    if (r.H_kv > kMaxKvHeadsGeneric || r.G > 32) return MSA_ERR_UNSUPPORTED;
+    if (!(s->softmax_scale >= 0.f) || !(s->index_scale >= 0.f)) return MSA_ERR_INVALID_ARG;
+    r.softmax_scale = s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf((float)r.d);
+    r.index_scale = s->index_scale > 0.f ? s->index_scale : 1.0f / sqrtf((float)r.d_idx);
+    return MSA_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static msa_status_t check_range(int64_t q_begin, int64_t q_count, int64_t kv_len) {
+    if (q_begin < 0 || q_count < 0 || kv_len < 0 || q_begin + q_count > kv_len)
+        return MSA_ERR_INVALID_ARG;
+    return MSA_OK;
+}
+
+static msa_status_t launch_status() {
+    return cudaPeekAtLastError() == cudaSuccess ? MSA_OK : MSA_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------- stage 1
+static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const void* k_idx,
+                                     const RowMap& rows, int64_t n_rows, float* scores,
+                                     int64_t ld_scores, cudaStream_t st) {
+    if (n_rows == 0 || rows.n_cols == 0) return MSA_OK;
+    constexpr int WARPS = 8;
+    const int64_t n_chunks = ceil_div64(rows.n_cols, WARPS);
+    const int64_t grid = n_rows * n_chunks;
+    if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
+    const size_t smem = sizeof(float) * (size_t)r.H_kv * r.d_idx;
+    {
+        StageScope sc(rows.seq_lens ? kStageIndexDecode : kStageIndex, st);
+        index_scores_generic_kernel<WARPS><<<(unsigned)grid, WARPS * 32, smem, st>>>(
+            (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx, rows, n_chunks, r.H_kv, r.d_idx,
+            r.B_k, r.index_scale, scores, ld_scores);
+    }
+    return launch_status();
+}
+
+// ---------------------------------------------------------------------- stage 2
+static msa_status_t run_topk(const Resolved& r, const float* scores, int64_t ld_scores,
+                             const RowMap& rows, int64_t n_q, int32_t* block_idx,
+                             cudaStream_t st) {
+    const int64_t n_rows = n_q * r.H_kv;
+    if (n_rows == 0) return MSA_OK;
+    const int64_t grid = ceil_div64(n_rows, kTopkWarps);
+    if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
+    const dim3 g((unsigned)grid), b(kTopkWarps * 32);
+    StageScope sc(kStageTopk, st);
+    if (r.k <= 32)
+        topk_select_kernel<1><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx);
+    else if (r.k <= 64)
+        topk_select_kernel<2><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx);
+    else
+        topk_select_kernel<4><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx);
+    return launch_status();
+}
+
+// ---------------------------------------------------------------------- stage 3 (generic)
+static msa_status_t run_attn_generic(const Resolved& r, const void* q, const void* k, const void* v,
+                                     const int32_t* block_idx, const RowMap& rows, int64_t n_q,
+                                     void* out, float* lse, cudaStream_t st) {
+    if (n_q == 0) return MSA_OK;
+    const int64_t grid = n_q * r.H_kv;
+    if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
+    int* status = async_status_ptr();
+    if (status == nullptr) return MSA_ERR_CUDA;
+    const size_t smem = sizeof(float) * (size_t)r.G * r.d;
+    {
+        StageScope sc(rows.seq_lens ? kStageAttnDecode : kStageAttn, st);
+        sparse_attn_generic_kernel<<<(unsigned)grid, r.G * 32, smem, st>>>(
+            (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, block_idx, rows,
+            r.H_q, r.H_kv, r.d, r.B_k, r.k, r.softmax_scale, (__nv_bfloat16*)out, lse, status);
+    }
+    return launch_status();
+}
+
+static RowMap prefill_rows(int64_t q_begin, int64_t kv_len, int B_k) {
+    RowMap m;
+    m.q_begin = q_begin; m.kv_len = kv_len; m.seq_offsets = nullptr; m.seq_lens = nullptr;
+    m.n_cols = ceil_div64(kv_len, B_k);
+    return m;
+}
+
+static RowMap decode_rows(const int64_t* seq_offsets, const int32_t* seq_lens, int64_t max_len,
+                          int B_k) {
+    RowMap m;
+    m.q_begin = 0; m.kv_len = 0; m.seq_offsets = seq_offsets; m.seq_lens = seq_lens;
+    m.n_cols = ceil_div64(max_len, B_k);
+    return m;
+}
+
+constexpr size_t kAlign = 256;
+static size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+}  // namespace msa
+
+using namespace msa;
+
+extern "C" {
+
+const char* msa_status_string(msa_status_t s) {
+    switch (s) {
+        case MSA_OK: return "ok";
+        case MSA_ERR_INVALID_ARG: return "invalid argument";
+        case MSA_ERR_UNSUPPORTED: return "unsupported shape";
+        case MSA_ERR_WORKSPACE: return "workspace too small";
+        case MSA_ERR_CUDA: return "CUDA error";
+        case MSA_ERR_TIMEOUT: return "device-side wait timed out";
+        case MSA_ERR_BAD_INDEX: return "block index out of range";
+    }
+    return "unknown status";
+}
+
+int64_t msa_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+msa_status_t msa_profile_begin(void) {
+    if (!g_prof_created) {
+        for (int i = 0; i < kProfSlots; ++i)
+            for (int j = 0; j < 2; ++j)
+                if (cudaEventCreate(&g_prof_ev[i][j]) != cudaSuccess) return MSA_ERR_CUDA;
+        g_prof_created = true;
+    }
+    g_prof_used = 0;
+    g_prof_on = true;
+    return MSA_OK;
+}
+
+msa_status_t msa_profile_end(float* stage_ms_host, int64_t* stage_launches_host) {
+    g_prof_on = false;
+    if (cudaDeviceSynchronize() != cudaSuccess) return MSA_ERR_CUDA;
+    for (int i = 0; i < kNumStages; ++i) {
+        if (stage_ms_host) stage_ms_host[i] = 0.f;
+        if (stage_launches_host) stage_launches_host[i] = 0;
+    }
+    for (int i = 0; i < g_prof_used; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, g_prof_ev[i][0], g_prof_ev[i][1]) != cudaSuccess) return MSA_ERR_CUDA;
+        if (stage_ms_host) stage_ms_host[g_prof_stage[i]] += ms;
+        if (stage_launches_host) stage_launches_host[g_prof_stage[i]] += 1;
+    }
+    const bool overflow = g_prof_used >= kProfSlots;
+    g_prof_used = 0;
+    return overflow ? MSA_ERR_UNSUPPORTED : MSA_OK;
+}
+
+msa_status_t msa_check_async_status(int32_t* detail_host) {
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_async_status, sizeof(int)) != cudaSuccess) return MSA_ERR_CUDA;
+    if (v != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_async_status, &zero, sizeof(int)) != cudaSuccess) return MSA_ERR_CUDA;
+    }
+    if (detail_host) *detail_host = v & 0xFFFFFF;
+    const int code = v >> 24;
+    if (code == kAsyncTimeout) return MSA_ERR_TIMEOUT;
+    if (code == kAsyncBadIndex) return MSA_ERR_BAD_INDEX;
+    return MSA_OK;
+}
+
+msa_status_t msa_index_scores(const msa_shape_t* shape, const void* q_idx, const void* k_idx,
+                              int64_t q_begin, int64_t q_count, int64_t kv_len, float* scores,
+                              int64_t ld_scores, msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if ((s = check_range(q_begin, q_count, kv_len)) != MSA_OK) return s;
+    if (q_count == 0) return MSA_OK;
+    if (!q_idx || !k_idx || !scores || !aligned16(q_idx) || !aligned16(k_idx) || !aligned16(scores))
+        return MSA_ERR_INVALID_ARG;
+    const int64_t B = ceil_div64(kv_len, r.B_k);
+    if (ld_scores < B || ld_scores % 4 != 0) return MSA_ERR_INVALID_ARG;
+    return run_index_scores(r, q_idx, k_idx, prefill_rows(q_begin, kv_len, r.B_k), q_count, scores,
+                            ld_scores, (cudaStream_t)stream);
+}
+
+msa_status_t msa_index_scores_decode(const msa_shape_t* shape, const void* q_idx,
+                                     const void* k_idx_cache, const int64_t* seq_offsets,
+                                     const int32_t* seq_lens, int32_t batch, int64_t max_seq_len,
+                                     float* scores, int64_t ld_scores, msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if (batch < 0 || max_seq_len < 0) return MSA_ERR_INVALID_ARG;
+    if (batch == 0) return MSA_OK;
+    if (!q_idx || !k_idx_cache || !seq_offsets || !seq_lens || !scores || !aligned16(q_idx) ||
+        !aligned16(k_idx_cache) || !aligned16(scores))
+        return MSA_ERR_INVALID_ARG;
+    if (ld_scores < ceil_div64(max_seq_len, r.B_k) || ld_scores % 4 != 0) return MSA_ERR_INVALID_ARG;
+    return run_index_scores(r, q_idx, k_idx_cache, decode_rows(seq_offsets, seq_lens, max_seq_len, r.B_k),
+                            batch, scores, ld_scores, (cudaStream_t)stream);
+}
+
+msa_status_t msa_topk_select(const msa_shape_t* shape, const float* scores, int64_t ld_scores,
+                             int64_t q_begin, int64_t q_count, int64_t kv_len, int32_t* block_idx,
+                             msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if ((s = check_range(q_begin, q_count, kv_len)) != MSA_OK) return s;
+    if (q_count == 0) return MSA_OK;
+    if (!scores || !block_idx || !aligned16(scores)) return MSA_ERR_INVALID_ARG;
+    if (ld_scores < ceil_div64(kv_len, r.B_k) || ld_scores % 4 != 0) return MSA_ERR_INVALID_ARG;
+    return run_topk(r, scores, ld_scores, prefill_rows(q_begin, kv_len, r.B_k), q_count, block_idx,
+                    (cudaStream_t)stream);
+}
+
+msa_status_t msa_topk_select_decode(const msa_shape_t* shape, const float* scores, int64_t ld_scores,
+                                    const int32_t* seq_lens, int32_t batch, int32_t* block_idx,
+                                    msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if (batch < 0) return MSA_ERR_INVALID_ARG;
+    if (batch == 0) return MSA_OK;
+    if (!scores || !block_idx || !seq_lens || !aligned16(scores) || ld_scores % 4 != 0 || ld_scores <= 0)
+        return MSA_ERR_INVALID_ARG;
+    RowMap rows = decode_rows(nullptr, seq_lens, 0, r.B_k);  // offsets are not needed for ranking
+    return run_topk(r, scores, ld_scores, rows, batch, block_idx, (cudaStream_t)stream);
+}
+
+msa_status_t msa_sparse_attn_prefill_workspace_bytes(const msa_shape_t* shape, int64_t q_count,
+                                                     int64_t kv_len, size_t* min_bytes,
+                                                     size_t* preferred_bytes) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if (q_count < 0 || kv_len < 0) return MSA_ERR_INVALID_ARG;
+    if (min_bytes) *min_bytes = kAlign;
+    if (preferred_bytes) *preferred_bytes = kAlign;
+    return MSA_OK;
+}
+
+msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, const void* k,
+                                     const void* v, const int32_t* block_idx, int64_t q_begin,
+                                     int64_t q_count, int64_t kv_len, void* out, float* lse,
+                                     void* workspace, size_t workspace_bytes, msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if ((s = check_range(q_begin, q_count, kv_len)) != MSA_OK) return s;
+    if (q_count == 0) return MSA_OK;
+    if (!q || !k || !v || !block_idx || !out || !aligned16(q) || !aligned16(k) || !aligned16(v) ||
+        !aligned16(out))
+        return MSA_ERR_INVALID_ARG;
+    size_t need = 0;
+    msa_sparse_attn_prefill_workspace_bytes(shape, q_count, kv_len, &need, nullptr);
+    if (workspace == nullptr || workspace_bytes < need) return MSA_ERR_WORKSPACE;
+    return run_attn_generic(r, q, k, v, block_idx, prefill_rows(q_begin, kv_len, r.B_k), q_count, out,
+                            lse, (cudaStream_t)stream);
+}
+
+msa_status_t msa_sparse_attn_decode_workspace_bytes(const msa_shape_t* shape, int32_t batch,
+                                                    size_t* min_bytes) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if (batch < 0) return MSA_ERR_INVALID_ARG;
+    if (min_bytes) *min_bytes = kAlign;
+    return MSA_OK;
+}
+
+msa_status_t msa_sparse_attn_decode(const msa_shape_t* shape, const void* q, const void* k_cache,
+                                    const void* v_cache, int64_t cache_tokens,
+                                    const int64_t* seq_offsets, const int32_t* seq_lens,
+                                    int32_t batch, const int32_t* block_idx, void* out, float* lse,
+                                    void* workspace, size_t workspace_bytes, msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if (batch < 0 || cache_tokens < 0) return MSA_ERR_INVALID_ARG;
+    if (batch == 0) return MSA_OK;
+    if (!q || !k_cache || !v_cache || !seq_offsets || !seq_lens || !block_idx || !out ||
+        !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out))
+        return MSA_ERR_INVALID_ARG;
+    size_t need = 0;
+    msa_sparse_attn_decode_workspace_bytes(shape, batch, &need);
+    if (workspace == nullptr || workspace_bytes < need) return MSA_ERR_WORKSPACE;
+    return run_attn_generic(r, q, k_cache, v_cache, block_idx, decode_rows(seq_offsets, seq_lens, 0, r.B_k),
+                            batch, out, lse, (cudaStream_t)stream);
+}
+
+// ---------------------------------------------------------------------- whole path
+static int64_t score_ld(int64_t T, int B_k) { return (ceil_div64(T, B_k) + 3) / 4 * 4; }
+
+static int64_t pick_score_chunk(const Resolved& r, int64_t T, size_t bytes_for_scores) {
+    const size_t row_bytes = sizeof(float) * (size_t)r.H_kv * (size_t)score_ld(T, r.B_k);
+    int64_t rows = (int64_t)(bytes_for_scores / row_bytes);
+    if (rows > T) rows = T;
+    if (rows >= 128) rows = rows / 128 * 128;
+    return rows;
+}
+
+msa_status_t msa_prefill_forward_workspace_bytes(const msa_shape_t* shape, int64_t T,
+                                                 size_t* min_bytes, size_t* preferred_bytes) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if (T < 0) return MSA_ERR_INVALID_ARG;
+    size_t a_min = 0, a_pref = 0;
+    msa_sparse_attn_prefill_workspace_bytes(shape, T, T, &a_min, &a_pref);
+    const size_t row_bytes = sizeof(float) * (size_t)r.H_kv * (size_t)score_ld(T, r.B_k);
+    const int64_t rows_min = T < 128 ? T : 128;
+    const int64_t rows_pref = T < 32768 ? T : 32768;
+    const size_t s_min = align_up(row_bytes * (size_t)rows_min);
+    const size_t s_pref = align_up(row_bytes * (size_t)rows_pref);
+    // stages 1-2 finish before stage 3 starts, so the two regions overlap
+    if (min_bytes) *min_bytes = (s_min > a_min ? s_min : a_min) + kAlign;
+    if (preferred_bytes) *preferred_bytes = (s_pref > a_pref ? s_pref : a_pref) + kAlign;
+    return MSA_OK;
+}
+
+msa_status_t msa_prefill_forward(const msa_shape_t* shape, const void* q, const void* k,
+                                 const void* v, const void* q_idx, const void* k_idx, int64_t T,
+                                 void* out, float* lse, int32_t* block_idx, void* workspace,
+                                 size_t workspace_bytes, msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if (T < 0) return MSA_ERR_INVALID_ARG;
+    if (T == 0) return MSA_OK;
+    if (!q || !k || !v || !q_idx || !k_idx || !out || !block_idx) return MSA_ERR_INVALID_ARG;
+    size_t need = 0;
+    msa_prefill_forward_workspace_bytes(shape, T, &need, nullptr);
+    if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
+    const int64_t ld = score_ld(T, r.B_k);
+    const int64_t chunk = pick_score_chunk(r, T, workspace_bytes);
+    if (chunk <= 0) return MSA_ERR_WORKSPACE;
+    float* scores = static_cast<float*>(workspace);
+    for (int64_t q0 = 0; q0 < T; q0 += chunk) {
+        const int64_t qc = (T - q0) < chunk ? (T - q0) : chunk;
+        const char* qi = static_cast<const char*>(q_idx) + (size_t)q0 * r.H_kv * r.d_idx * 2;
+        // Only keys up to the chunk's last query are visible, so score that prefix.
+        const int64_t kv_vis = q0 + qc;
+        s = msa_index_scores(shape, qi, k_idx, q0, qc, kv_vis, scores, ld, stream);
+        if (s != MSA_OK) return s;
+        s = msa_topk_select(shape, scores, ld, q0, qc, kv_vis, block_idx + (size_t)q0 * r.H_kv * r.k, stream);
+        if (s != MSA_OK) return s;
+    }
+    return msa_sparse_attn_prefill(shape, q, k, v, block_idx, 0, T, T, out, lse, workspace,
+                                   workspace_bytes, stream);
+}
+
+static size_t host_staging_bytes(const Resolved& r, int64_t T, size_t off[8]) {
+    size_t o = 0;
+    off[0] = o; o += align_up((size_t)T * r.H_q * r.d * 2);      // q
+    off[1] = o; o += align_up((size_t)T * r.H_kv * r.d * 2);     // k
+    off[2] = o; o += align_up((size_t)T * r.H_kv * r.d * 2);     // v
+    off[3] = o; o += align_up((size_t)T * r.H_kv * r.d_idx * 2); // q_idx
+    off[4] = o; o += align_up((size_t)T * r.d_idx * 2);          // k_idx
+    off[5] = o; o += align_up((size_t)T * r.H_q * r.d * 2);      // out
+    off[6] = o; o += align_up((size_t)T * r.H_q * 4);            // lse
+    off[7] = o; o += align_up((size_t)T * r.H_kv * r.k * 4);     // block_idx
+    return o;
+}
+
+msa_status_t msa_prefill_forward_host_workspace_bytes(const msa_shape_t* shape, int64_t T,
+                                                      size_t* min_bytes, size_t* preferred_bytes) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    size_t mn = 0, pf = 0, off[8];
+    if ((s = msa_prefill_forward_workspace_bytes(shape, T, &mn, &pf)) != MSA_OK) return s;
+    const size_t stage = host_staging_bytes(r, T, off);
+    if (min_bytes) *min_bytes = stage + mn;
+    if (preferred_bytes) *preferred_bytes = stage + pf;
+    return MSA_OK;
+}
+
+msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_host,
+                                      const void* k_host, const void* v_host,
+                                      const void* q_idx_host, const void* k_idx_host, int64_t T,
+                                      void* out_host, float* lse_host, int32_t* block_idx_host,
+                                      void* workspace, size_t workspace_bytes, msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if (T < 0) return MSA_ERR_INVALID_ARG;
+    if (T == 0) return MSA_OK;
+    if (!q_host || !k_host || !v_host || !q_idx_host || !k_idx_host || !out_host)
+        return MSA_ERR_INVALID_ARG;
+    size_t need = 0, off[8];
+    if ((s = msa_prefill_forward_host_workspace_bytes(shape, T, &need, nullptr)) != MSA_OK) return s;
+    if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
+    const size_t stage = host_staging_bytes(r, T, off);
+    char* w = static_cast<char*>(workspace);
+    cudaStream_t st = (cudaStream_t)stream;
+    const void* src[5] = {q_host, k_host, v_host, q_idx_host, k_idx_host};
+    const size_t nbytes[5] = {(size_t)T * r.H_q * r.d * 2, (size_t)T * r.H_kv * r.d * 2,
+                              (size_t)T * r.H_kv * r.d * 2, (size_t)T * r.H_kv * r.d_idx * 2,
+                              (size_t)T * r.d_idx * 2};
+    for (int i = 0; i < 5; ++i)
+        if (cudaMemcpyAsync(w + off[i], src[i], nbytes[i], cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return MSA_ERR_CUDA;
+    s = msa_prefill_forward(shape, w + off[0], w + off[1], w + off[2], w + off[3], w + off[4], T,
+                            w + off[5], lse_host ? (float*)(w + off[6]) : nullptr,
+                            (int32_t*)(w + off[7]), w + stage, workspace_bytes - stage, stream);
+    if (s != MSA_OK) return s;
+    if (cudaMemcpyAsync(out_host, w + off[5], (size_t)T * r.H_q * r.d * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return MSA_ERR_CUDA;
+    if (lse_host &&
+        cudaMemcpyAsync(lse_host, w + off[6], (size_t)T * r.H_q * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return MSA_ERR_CUDA;
+    if (block_idx_host &&
+        cudaMemcpyAsync(block_idx_host, w + off[7], (size_t)T * r.H_kv * r.k * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return MSA_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? MSA_OK : MSA_ERR_CUDA;
+}
+
+msa_status_t msa_decode_forward(const msa_shape_t* shape, const void* q, const void* q_idx,
+                                const void* k_cache, const void* v_cache, const void* k_idx_cache,
+                                int64_t cache_tokens, const int64_t* seq_offsets,
+                                const int32_t* seq_lens, int32_t batch, int64_t max_seq_len,
+                                float* scores, int64_t ld_scores, int32_t* block_idx, void* out,
+                                float* lse, void* workspace, size_t workspace_bytes,
+                                msa_stream_t stream) {
+    msa_status_t s = msa_index_scores_decode(shape, q_idx, k_idx_cache, seq_offsets, seq_lens, batch,
+                                             max_seq_len, scores, ld_scores, stream);
+    if (s != MSA_OK) return s;
+    s = msa_topk_select_decode(shape, scores, ld_scores, seq_lens, batch, block_idx, stream);
+    if (s != MSA_OK) return s;
+    return msa_sparse_attn_decode(shape, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens,
+                                  batch, block_idx, out, lse, workspace, workspace_bytes, stream);
+}
+
+msa_status_t msa_decode_forward_host(const msa_shape_t* shape, const void* q_host,
+                                     const void* q_idx_host, void* q_dev, void* q_idx_dev,
+                                     const void* k_cache, const void* v_cache,
+                                     const void* k_idx_cache, int64_t cache_tokens,
+                                     const int64_t* seq_offsets, const int32_t* seq_lens,
+                                     int32_t batch, int64_t max_seq_len, float* scores,
+                                     int64_t ld_scores, int32_t* block_idx, void* out_dev,
+                                     void* out_host, void* workspace, size_t workspace_bytes,
+                                     msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if (batch < 0) return MSA_ERR_INVALID_ARG;
+    if (batch == 0) return MSA_OK;
+    if (!q_host || !q_idx_host || !q_dev || !q_idx_dev || !out_dev || !out_host) return MSA_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t qb = (size_t)batch * r.H_q * r.d * 2, qib = (size_t)batch * r.H_kv * r.d_idx * 2;
+    if (cudaMemcpyAsync(q_dev, q_host, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return MSA_ERR_CUDA;
+    if (cudaMemcpyAsync(q_idx_dev, q_idx_host, qib, cudaMemcpyHostToDevice, st) != cudaSuccess) return MSA_ERR_CUDA;
+    s = msa_decode_forward(shape, q_dev, q_idx_dev, k_cache, v_cache, k_idx_cache, cache_tokens,
+                           seq_offsets, seq_lens, batch, max_seq_len, scores, ld_scores, block_idx,
+                           out_dev, nullptr, workspace, workspace_bytes, stream);
+    if (s != MSA_OK) return s;
+    if (cudaMemcpyAsync(out_host, out_dev, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MSA_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? MSA_OK : MSA_ERR_CUDA;
+}
+
+}  // extern "C"

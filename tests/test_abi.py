@@ -1,0 +1,96 @@
+"""C-ABI checks that need no GPU: the library loads, exports every declared symbol, and
+rejects bad arguments before launching anything."""
+
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2606_13392_b200 import binding as B
+from paper_2606_13392_b200.build import build_library
+from paper_2606_13392_b200.inputs import CONFIGS
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build_library()
+    return B.lib()
+
+
+def declared_symbols():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in os.listdir(inc):
+        if f.endswith(".h"):
+            text = open(os.path.join(inc, f)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names.update(re.findall(r"\b(msa_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_symbols()
+    assert "msa_index_scores" in names and "msa_topk_select" in names
+    assert "msa_sparse_attn_prefill" in names and "msa_sparse_attn_decode" in names
+    for n in names:
+        assert hasattr(lib, n), "library does not export %s" % n
+    assert set(B.EXPORTS) <= set(names)
+
+
+def test_status_strings(lib):
+    assert B.status_string(0) == "ok"
+    assert "workspace" in B.status_string(3)
+    assert B.status_string(99) == "unknown status"
+
+
+def test_argument_validation_without_launch(lib):
+    shape = B.shape_of(CONFIGS["c1"])
+    null = ctypes.c_void_p(0)
+    i64 = ctypes.c_int64
+    # range outside the sequence
+    assert lib.msa_index_scores(ctypes.byref(shape), null, null, i64(10), i64(10), i64(15), null,
+                                i64(4), null) == 1
+    # null pointers with a non-empty range
+    assert lib.msa_index_scores(ctypes.byref(shape), null, null, i64(0), i64(1), i64(1), null,
+                                i64(4), null) == 1
+    # an empty range is a valid no-op
+    assert lib.msa_index_scores(ctypes.byref(shape), null, null, i64(0), i64(0), i64(0), null,
+                                i64(4), null) == 0
+    assert lib.msa_topk_select(ctypes.byref(shape), null, i64(4), i64(0), i64(0), i64(0), null, null) == 0
+    # bad shapes
+    bad = B.shape_of(CONFIGS["c1"].scaled(n_q_heads=7, n_kv_heads=2))
+    assert lib.msa_topk_select(ctypes.byref(bad), null, i64(4), i64(0), i64(0), i64(0), null, null) == 1
+    bad = B.shape_of(CONFIGS["c1"].scaled(top_k=100000))
+    assert lib.msa_topk_select(ctypes.byref(bad), null, i64(4), i64(0), i64(0), i64(0), null, null) == 2
+    bad = B.shape_of(CONFIGS["c1"].scaled(head_dim=100))
+    assert lib.msa_topk_select(ctypes.byref(bad), null, i64(4), i64(0), i64(0), i64(0), null, null) == 2
+    assert lib.msa_index_scores(None, null, null, i64(0), i64(0), i64(0), null, i64(4), null) == 1
+
+
+def test_workspace_queries(lib):
+    for name in ("c1", "c2", "c3", "c4"):
+        cfg = CONFIGS[name]
+        shape = B.shape_of(cfg)
+        mn, pf = B.msa_prefill_forward_workspace_bytes(shape, cfg.T)
+        assert 0 < mn <= pf
+        hmn, hpf = B.msa_prefill_forward_host_workspace_bytes(shape, cfg.T)
+        assert hmn > mn and hpf >= hmn
+        amn, apf = B.msa_sparse_attn_prefill_workspace_bytes(shape, cfg.T, cfg.T)
+        assert 0 < amn <= apf <= pf
+    assert B.msa_sparse_attn_decode_workspace_bytes(B.shape_of(CONFIGS["c5"]), 32) > 0
+    # a workspace below the minimum is refused before any launch
+    shape = B.shape_of(CONFIGS["c2"])
+    one = ctypes.c_void_p(256)  # non-null, never dereferenced on this path
+    code = lib.msa_prefill_forward(ctypes.byref(shape), one, one, one, one, one, ctypes.c_int64(32768),
+                                   one, None, one, one, ctypes.c_size_t(16), None)
+    assert code == 3
+
+
+def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "missing.so"))
+    with pytest.raises(RuntimeError, match="missing"):
+        B.lib()

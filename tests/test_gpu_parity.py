@@ -1,0 +1,223 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Sizes here are ones the oracle finishes in seconds; full-size
+configurations are covered on sampled query positions in test_gpu_full_configs.py."""
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2606_13392_b200 import api
+from paper_2606_13392_b200 import binding as B
+from paper_2606_13392_b200.inputs import (CONFIGS, MSAConfig, make_decode_inputs,
+                                          make_prefill_inputs, sample_positions, to_bits)
+from parity_utils import check_attn, check_scores, check_selection
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _bits(x):
+    return {n: to_bits(t) for n, t in x.items() if t.dtype == torch.bfloat16}
+
+
+def _assert_clean():
+    code, detail = B.check_async_status()
+    assert code == 0, "device status %d detail %d" % (code, detail)
+
+
+def run_prefill_case(cfg: MSAConfig, sharp: bool, n_sample: int, ws_bytes=None):
+    x = make_prefill_inputs(cfg, DEV, sharp=sharp)
+    xb = _bits(x)
+    T = cfg.T
+    pos = np.arange(T) if n_sample >= T else sample_positions(T, cfg.block_size, cfg.top_k, n_sample, 7)
+
+    # --- whole path on the GPU
+    out, lse, I = api.prefill_forward(cfg, x, workspace_bytes=ws_bytes)
+    torch.cuda.synchronize()
+    _assert_clean()
+
+    # --- stage 1 at the sampled rows (one call per run of consecutive positions)
+    M_gpu = np.empty((len(pos), cfg.n_kv_heads, cfg.n_blocks), dtype=np.float32)
+    runs = np.split(np.arange(len(pos)), np.where(np.diff(pos) != 1)[0] + 1)
+    for run in runs:
+        q0, qc = int(pos[run[0]]), len(run)
+        s = api.index_scores(cfg, x["q_idx"], x["k_idx"], q0, qc)
+        M_gpu[run] = s[:, :, :cfg.n_blocks].cpu().numpy()
+    M_ref = oracle.index_scores(xb["q_idx"][pos], xb["k_idx"], pos, cfg.block_size)
+    score_err = check_scores(M_gpu, M_ref, pos, cfg.block_size)
+
+    # --- stage 2: the GPU's own pipeline against the oracle's selection
+    I_ref = oracle.topk_select(M_ref, pos, T, cfg.block_size, cfg.top_k)
+    I_gpu = I.cpu().numpy()[pos]
+    exact, n_rows = check_selection(I_gpu, I_ref, M_ref, pos, cfg.block_size, cfg.top_k)
+
+    # --- stage 3: oracle attention on the GPU's index lists
+    O_ref, LSE_ref = oracle.sparse_attn(xb["q"][pos], xb["k"], xb["v"], I_gpu, pos, cfg.block_size)
+    o = out.float().cpu().numpy()[pos]
+    stats = check_attn(o, lse.cpu().numpy()[pos], O_ref, LSE_ref, cfg.name)
+    stats.update(score_err=score_err, exact_sets=exact, rows=n_rows)
+    return stats
+
+
+@pytest.mark.parametrize("sharp", [False, True])
+def test_c1_full(sharp):
+    stats = run_prefill_case(CONFIGS["c1"], sharp, n_sample=10 ** 9)
+    assert stats["exact_sets"] >= 0.999
+    print("c1", sharp, stats)
+
+
+@pytest.mark.parametrize("sharp", [False, True])
+def test_c2_shape_reduced_length(sharp):
+    cfg = CONFIGS["c2"].scaled(name="c2-4k", T=4096 + 37)  # ragged last block
+    stats = run_prefill_case(cfg, sharp, n_sample=384)
+    assert stats["exact_sets"] >= 0.999
+    print("c2-4k", sharp, stats)
+
+
+@pytest.mark.parametrize("sharp", [False, True])
+def test_c3_shape_reduced_length(sharp):
+    cfg = CONFIGS["c3"].scaled(name="c3-12k", T=12288 + 5)
+    stats = run_prefill_case(cfg, sharp, n_sample=256)
+    assert stats["exact_sets"] >= 0.999
+    print("c3-12k", sharp, stats)
+
+
+def test_c3_shape_small_workspace_many_passes():
+    # Same numbers must come out when the workspace forces many query ranges / score chunks.
+    cfg = CONFIGS["c3"].scaled(name="c3-6k", T=6144 + 77)
+    x = make_prefill_inputs(cfg, DEV, sharp=True)
+    shape = B.shape_of(cfg)
+    mn, pf = B.msa_prefill_forward_workspace_bytes(shape, cfg.T)
+    o1, l1, i1 = api.prefill_forward(cfg, x, workspace_bytes=pf)
+    o2, l2, i2 = api.prefill_forward(cfg, x, workspace_bytes=mn)
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert torch.equal(i1, i2)
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
+
+
+@pytest.mark.parametrize("T,Hq,Hkv,Bk,k,d,di", [
+    (1, 8, 1, 64, 8, 128, 64),        # a single token
+    (63, 8, 1, 64, 8, 128, 64),       # less than one block
+    (65, 16, 2, 64, 4, 128, 64),      # one token into the second block
+    (300, 4, 2, 8, 3, 32, 16),        # tiny blocks, generic shapes
+    (257, 6, 3, 16, 5, 64, 32),       # G = 2, H_kv = 3
+    (1000, 16, 1, 32, 40, 128, 64),   # k larger than the number of blocks: dense causal
+    (777, 32, 2, 128, 2, 128, 64),    # G = 16, k = 2 (local + one)
+    (500, 8, 1, 64, 1, 128, 64),      # k = 1: local block only
+])
+def test_odd_shapes_full(T, Hq, Hkv, Bk, k, d, di):
+    cfg = MSAConfig("odd", "prefill", T, Hq, Hkv, Bk, k, head_dim=d, idx_dim=di, seed=T)
+    stats = run_prefill_case(cfg, True, n_sample=10 ** 9)
+    assert stats["exact_sets"] >= 0.995
+    if k >= cfg.n_blocks:  # every visible block selected: equals dense causal GQA (Eq. 1)
+        x = make_prefill_inputs(cfg, DEV, sharp=True)
+        xb = _bits(x)
+        out, lse, _ = api.prefill_forward(cfg, x)
+        Od, Ld = oracle.dense_attn(xb["q"], xb["k"], xb["v"], np.arange(T))
+        check_attn(out.float().cpu().numpy(), lse.cpu().numpy(), Od, Ld, "dense")
+
+
+def test_topk_bit_exact_on_arbitrary_scores():
+    # Stage 2 alone on fp32 scores with many exact ties: sets must equal the oracle's bit for
+    # bit (same values, same total order).
+    g = torch.Generator(device="cpu").manual_seed(5)
+    for (T, Bk, k, Hkv) in [(4096, 4, 64, 2), (3000, 2, 33, 1), (2048, 1, 128, 1), (5000, 8, 17, 3),
+                            (9000, 1, 64, 1)]:
+        cfg = MSAConfig("tk", "prefill", T, Hkv, Hkv, Bk, k)
+        nb = cfg.n_blocks
+        ld = B.score_ld(T, Bk)
+        # coarse values => plenty of ties; a few +/-0 and -inf-free rows
+        M = torch.randint(-50, 50, (T, Hkv, ld), generator=g).float() * 0.25
+        M[::7] = torch.randn((len(range(0, T, 7)), Hkv, ld), generator=g)
+        M[3::11] = -0.0
+        Md = M.to(DEV)
+        I = api.topk_select(cfg, Md, 0, T).cpu().numpy()
+        pos = np.arange(T)
+        I_ref = oracle.topk_select(M[:, :, :nb].double().numpy(), pos, T, Bk, k)
+        assert np.array_equal(I, I_ref), (T, Bk, k)
+
+
+def test_topk_row_offsets_and_ranges():
+    cfg = MSAConfig("tk2", "prefill", 6000, 2, 2, 4, 32)
+    ld = B.score_ld(cfg.T, cfg.block_size)
+    g = torch.Generator(device="cpu").manual_seed(9)
+    M = torch.randn((cfg.T, 2, ld), generator=g)
+    I_ref = oracle.topk_select(M[:, :, :cfg.n_blocks].double().numpy(), np.arange(cfg.T), cfg.T, 4, 32)
+    for q0, qc in [(0, 1), (5, 100), (4097, 1903), (5999, 1)]:
+        I = api.topk_select(cfg, M[q0:q0 + qc].contiguous().to(DEV), q0, cfg.T).cpu().numpy()
+        assert np.array_equal(I, I_ref[q0:q0 + qc])
+
+
+def run_decode_case(cfg: MSAConfig, sharp: bool):
+    x = make_decode_inputs(cfg, DEV, sharp=sharp)
+    out, lse, I, scores = api.decode_forward(cfg, x)
+    torch.cuda.synchronize()
+    _assert_clean()
+    offs = x["seq_offsets"].cpu().numpy()
+    res = []
+    for s, L in enumerate(cfg.seq_lens):
+        sl = slice(int(offs[s]), int(offs[s]) + L)
+        kb, vb = to_bits(x["k_cache"][sl]), to_bits(x["v_cache"][sl])
+        kib = to_bits(x["k_idx_cache"][sl])
+        pos = np.array([L - 1])
+        nb = -(-L // cfg.block_size)
+        M_ref = oracle.index_scores(to_bits(x["q_idx"][s:s + 1]), kib, pos, cfg.block_size)
+        M_gpu = scores[s:s + 1, :, :nb].cpu().numpy()
+        check_scores(M_gpu, M_ref, pos, cfg.block_size)
+        nb_max = -(-max(cfg.seq_lens) // cfg.block_size)
+        assert torch.isneginf(scores[s, :, nb:nb_max]).all()
+        I_ref = oracle.topk_select(M_ref, pos, L, cfg.block_size, cfg.top_k)
+        I_gpu = I[s:s + 1].cpu().numpy()
+        exact, _ = check_selection(I_gpu, I_ref, M_ref, pos, cfg.block_size, cfg.top_k)
+        O_ref, LSE_ref = oracle.sparse_attn(to_bits(x["q"][s:s + 1]), kb, vb, I_gpu, pos, cfg.block_size)
+        st = check_attn(out[s:s + 1].float().cpu().numpy(), lse[s:s + 1].cpu().numpy(), O_ref, LSE_ref,
+                        "decode seq %d" % s)
+        st["exact"] = exact
+        res.append(st)
+    return res
+
+
+@pytest.mark.parametrize("sharp", [False, True])
+def test_decode_small_batch_mixed_lengths(sharp):
+    cfg = CONFIGS["c5"].scaled(name="c5-small", seq_lens=(1, 127, 128, 129, 8192, 8200, 20000, 16384 + 64))
+    res = run_decode_case(cfg, sharp)
+    assert np.mean([r["exact"] for r in res]) >= 0.95
+
+
+def test_decode_generic_shape():
+    cfg = MSAConfig("dec-odd", "decode", 0, 6, 3, 16, 5, head_dim=64, idx_dim=32, seed=3,
+                    seq_lens=(5, 16, 17, 400, 1000))
+    run_decode_case(cfg, True)
+
+
+def test_decode_equals_last_prefill_row():
+    # The decode call on a cache of length L gives row L-1 of the prefill call (same kernels'
+    # arithmetic may differ in order, so compare within tolerance, and sets exactly).
+    cfg = CONFIGS["c3"].scaled(name="c3-9k", T=9000)
+    x = make_prefill_inputs(cfg, DEV, sharp=True)
+    out, lse, I = api.prefill_forward(cfg, x)
+    dcfg = cfg.scaled(mode="decode", seq_lens=(cfg.T,))
+    xd = {"q": x["q"][-1:].contiguous(), "q_idx": x["q_idx"][-1:].contiguous(), "k_cache": x["k"],
+          "v_cache": x["v"], "k_idx_cache": x["k_idx"],
+          "seq_offsets": torch.zeros(1, dtype=torch.int64, device=DEV),
+          "seq_lens": torch.tensor([cfg.T], dtype=torch.int32, device=DEV)}
+    od, ld_, Id, _ = api.decode_forward(dcfg, xd)
+    assert torch.equal(Id[0], I[-1])
+    assert torch.allclose(od[0].float(), out[-1].float(), atol=2e-2)
+    assert torch.allclose(ld_[0], lse[-1], atol=2e-3)
+
+
+def test_bad_block_index_is_reported_not_dereferenced():
+    cfg = CONFIGS["c1"]
+    x = make_prefill_inputs(cfg, DEV)
+    out, lse, I = api.prefill_forward(cfg, x)
+    bad = I.clone()
+    bad[100, 0, 0] = 10 ** 6   # far outside the sequence
+    bad[200, 0, 1] = -7        # not the padding value
+    o2, _ = api.sparse_attn_prefill(cfg, x["q"], x["k"], x["v"], bad)
+    code, _ = B.check_async_status()
+    assert code == 6  # MSA_ERR_BAD_INDEX
+    assert torch.isfinite(o2.float()).all()
+    assert B.check_async_status()[0] == 0  # cleared
