@@ -1,0 +1,445 @@
+#!/usr/bin/env python
+"""Benchmark of the MSA forward hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c4|c5|...] [--impl reference]
+
+One step = one pass of the whole path (index scoring -> Top-k -> block-sparse attention) over
+one synthetic workload resident in HBM.  Prints ONE JSON line (rank 0).  With N > 1 (torchrun)
+every rank runs its own independent sequence (the path needs no exchange): weak scaling.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2606_13392_b200.inputs import (CONFIGS, MSAConfig, make_decode_inputs,  # noqa: E402
+                                          make_prefill_inputs, to_bits)
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+# ----------------------------------------------------------------------------- algorithmic work
+def prefill_work(cfg: MSAConfig):
+    """Algorithmic FLOPs/bytes of one prefill pass (formulas: Section 3.3 and Section 4.2)."""
+    T, Bk, k = cfg.T, cfg.block_size, cfg.top_k
+    i = np.arange(T, dtype=np.int64)
+    loc = i // Bk
+    n_sel = np.minimum(k, loc + 1)
+    tokens = (n_sel - 1) * Bk + (i % Bk) + 1          # visible tokens of the selected blocks
+    pairs = int(n_sel.sum()) * cfg.n_kv_heads          # (query, group, block) pairs
+    gd2 = 2 * cfg.group * cfg.head_dim                 # bytes of one (query, group) bf16 row set
+    return {
+        "index_flops": float(cfg.n_kv_heads) * cfg.idx_dim * T * (T + 1),
+        "attn_flops": 4.0 * cfg.n_q_heads * cfg.head_dim * float(tokens.sum()),
+        "topk_bytes": 4.0 * cfg.n_kv_heads * float((loc + 1).sum()) + 4.0 * T * cfg.n_kv_heads * k,
+        # KV-outer with bf16 partials: K+V once, per pair Q gather + partial write, final O
+        "attn_bytes": 2.0 * 2 * T * cfg.n_kv_heads * cfg.head_dim + pairs * (2.0 * gd2 + 4 * cfg.group)
+                      + 2.0 * T * cfg.n_q_heads * cfg.head_dim,
+        # combine: reads every partial (+ its LSE) once, writes O and LSE
+        "combine_bytes": pairs * (gd2 + 4.0 * cfg.group) + T * cfg.n_q_heads * (2.0 * cfg.head_dim + 4),
+        "pairs": pairs,
+    }
+
+
+def decode_work(cfg: MSAConfig):
+    Bk, k = cfg.block_size, cfg.top_k
+    lens = np.array(cfg.seq_lens, dtype=np.int64)
+    loc = (lens - 1) // Bk
+    n_sel = np.minimum(k, loc + 1)
+    tokens = (n_sel - 1) * Bk + ((lens - 1) % Bk) + 1
+    return {
+        "index_bytes": 2.0 * cfg.idx_dim * float(lens.sum()),
+        "index_flops": 2.0 * cfg.n_kv_heads * cfg.idx_dim * float(lens.sum()),
+        "attn_bytes": 2.0 * 2 * cfg.n_kv_heads * cfg.head_dim * float(tokens.sum()),
+        "attn_flops": 4.0 * cfg.n_q_heads * cfg.head_dim * float(tokens.sum()),
+    }
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [t.strip() for t in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            # "under load": samples drawing more than half of the highest power seen
+            hi = max(pw)
+            load = [s for s, w in zip(sm, pw) if w >= 0.5 * hi] or sm
+            out.update(sm_mhz=statistics.median(load), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=hi)
+        return out
+
+
+# ----------------------------------------------------------------------------- oracle leg
+def oracle_sample_prefill(cfg: MSAConfig, x_bits, n: int, seed: int = 123):
+    """Times the CPU oracle (as it stands) on n uniformly drawn query positions."""
+    import oracle
+    rng = np.random.default_rng(seed)
+    pos = np.sort(rng.choice(cfg.T, size=min(n, cfg.T), replace=False)).astype(np.int64)
+    q, qi = x_bits["q"][pos], x_bits["q_idx"][pos]
+    t0 = time.perf_counter()
+    oracle.msa_forward(q, x_bits["k"], x_bits["v"], qi, x_bits["k_idx"], pos, cfg.block_size, cfg.top_k)
+    dt = time.perf_counter() - t0
+    return len(pos), dt
+
+
+def oracle_sample_decode(cfg: MSAConfig, xd, seqs):
+    import oracle
+    offs = xd["seq_offsets"].cpu().numpy()
+    prepared = []
+    for s in seqs:
+        L = cfg.seq_lens[s]
+        sl = slice(int(offs[s]), int(offs[s]) + L)
+        prepared.append((to_bits(xd["q"][s:s + 1]), to_bits(xd["k_cache"][sl]), to_bits(xd["v_cache"][sl]),
+                         to_bits(xd["q_idx"][s:s + 1]), to_bits(xd["k_idx_cache"][sl]), np.array([L - 1])))
+    t0 = time.perf_counter()
+    for (q, k, v, qi, ki, pos) in prepared:
+        oracle.msa_forward(q, k, v, qi, ki, pos, cfg.block_size, cfg.top_k)
+    return len(seqs), time.perf_counter() - t0
+
+
+def oracle_sample_size(cfg: MSAConfig) -> int:
+    """Query positions that take the oracle roughly 10-30 s on ~8-16 host cores."""
+    per_q = cfg.n_kv_heads * cfg.idx_dim * cfg.T / 2 + \
+        cfg.n_q_heads * cfg.head_dim * 2 * min(cfg.T / 2, cfg.top_k * cfg.block_size)
+    return int(max(16, min(cfg.T, 4.0e10 / per_q)))
+
+
+# ----------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c3")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cfg = CONFIGS[args.workload]
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(cfg, args)
+        return
+    run_ours(cfg, args, rank, local_rank, world)
+
+
+def base_line(cfg: MSAConfig, args, n_gpus: int):
+    metric = "msa_prefill_tokens_per_s" if cfg.mode == "prefill" else "msa_decode_tokens_per_s"
+    conf = {"workload": "%s: %s" % (cfg.name, describe(cfg)), "l2": "inputs larger than L2 (126 MB)",
+            "sharding": "one independent sequence per rank, no collective"}
+    return {"metric": metric, "unit": "tokens/s", "n_gpus": n_gpus, "steps": args.steps,
+            "warmup": args.warmup, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": conf}
+
+
+def describe(cfg: MSAConfig) -> str:
+    if cfg.mode == "prefill":
+        return ("prefill fwd, batch 1, T=%d causal, %d q heads / %d kv heads, d_h=%d, d_idx=%d, B_k=%d, k=%d"
+                % (cfg.T, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.idx_dim, cfg.block_size, cfg.top_k))
+    return ("decode, batch %d (lens %s), %d q heads / %d kv heads, d_h=%d, d_idx=%d, B_k=%d, k=%d"
+            % (len(cfg.seq_lens), sorted(set(cfg.seq_lens)), cfg.n_q_heads, cfg.n_kv_heads,
+               cfg.head_dim, cfg.idx_dim, cfg.block_size, cfg.top_k))
+
+
+def run_reference(cfg: MSAConfig, args):
+    import oracle
+    line = base_line(cfg, args, 1)
+    steps, warm = max(1, args.steps), args.warmup
+    if cfg.mode == "prefill":
+        x = make_prefill_inputs(cfg, "cpu")
+        xb = {n: to_bits(t) for n, t in x.items()}
+        n = max(8, oracle_sample_size(cfg) // (4 * (steps + min(warm, 1))))
+        for _ in range(min(warm, 1)):
+            oracle_sample_prefill(cfg, xb, n, 1)
+        tot_n, tot_t = 0, 0.0
+        for s in range(steps):
+            m, dt = oracle_sample_prefill(cfg, xb, n, 100 + s)
+            tot_n += m; tot_t += dt
+        sample = "%d uniformly drawn query positions per step, all heads" % n
+    else:
+        small = cfg.scaled(seq_lens=tuple(sorted(set(cfg.seq_lens))))
+        xd = make_decode_inputs(small, "cpu")
+        tot_n, tot_t = 0, 0.0
+        for s in range(steps):
+            m, dt = oracle_sample_decode(small, xd, list(range(len(small.seq_lens))))
+            tot_n += m; tot_t += dt
+        sample = "one sequence of each cache length per step"
+    val = tot_n / tot_t
+    line.update(impl="reference", value=val, ms_per_step=1e3 * tot_t / steps, dtype="f64",
+                cpu_baseline={"value": val, "unit": "tokens/s", "cores": oracle.n_threads(),
+                              "kind": "oracle", "sample": sample},
+                e2e={"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+def run_ours(cfg: MSAConfig, args, rank: int, local_rank: int, world: int):
+    import torch.distributed as dist
+    from paper_2606_13392_b200 import binding as B
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    shape = B.shape_of(cfg)
+    mycfg = cfg.scaled(seed=cfg.seed + 7919 * rank)
+    stream = torch.cuda.current_stream()
+
+    if cfg.mode == "prefill":
+        x = make_prefill_inputs(mycfg, dev)
+        T = cfg.T
+        out = torch.empty_like(x["q"])
+        lse = torch.empty((T, cfg.n_q_heads), dtype=torch.float32, device=dev)
+        block_idx = torch.empty((T, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32, device=dev)
+        mn, pf = B.msa_prefill_forward_workspace_bytes(shape, T)
+        ws = B.alloc_workspace(pf, dev)
+        units = T
+
+        def step():
+            B.msa_prefill_forward(shape, x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"], T, out, lse,
+                                  block_idx, ws)
+    else:
+        x = make_decode_inputs(mycfg, dev)
+        batch = len(cfg.seq_lens)
+        max_len = int(max(cfg.seq_lens))
+        ld = B.score_ld(max_len, cfg.block_size)
+        scores = torch.empty((batch, cfg.n_kv_heads, ld), dtype=torch.float32, device=dev)
+        block_idx = torch.empty((batch, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32, device=dev)
+        out = torch.empty_like(x["q"])
+        lse = torch.empty((batch, cfg.n_q_heads), dtype=torch.float32, device=dev)
+        ws = B.alloc_workspace(B.msa_sparse_attn_decode_workspace_bytes(shape, batch), dev)
+        units = batch
+        cache_tokens = x["k_cache"].shape[0]
+
+        def step():
+            B.msa_decode_forward(shape, x["q"], x["q_idx"], x["k_cache"], x["v_cache"], x["k_idx_cache"],
+                                 cache_tokens, x["seq_offsets"], x["seq_lens"], batch, max_len, scores,
+                                 ld, block_idx, out, lse, ws)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 0)):
+        step()
+    barrier()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    n_before = B.launch_count()
+    B.profile_begin()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    stages = B.profile_end()
+    launches = B.launch_count() - n_before
+    clocks = sampler.stop() if sampler else None
+    code, detail = B.check_async_status()
+    if code != 0:
+        raise RuntimeError("device status %d (detail %d) after the timed region" % (code, detail))
+
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * units / (ms_step * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    line = base_line(cfg, args, world)
+    line.update(value=value, ms_per_step=ms_step, gpu_launches=int(launches), clocks=clocks)
+
+    # ---- per-kernel figures and the roofline of the dominant kernel
+    hbm, tf_b, tf_s = peaks["hbm_gbs"], peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
+    src = "of " + peaks["_source"]
+    kern = {}
+    if cfg.mode == "prefill":
+        w = prefill_work(cfg)
+        spec = {"index_scores": ("tensor", w["index_flops"]), "topk_select": ("hbm", w["topk_bytes"]),
+                "attn_prefill": ("hbm", w["attn_bytes"]), "combine": ("hbm", w["combine_bytes"]),
+                "schedule": ("hbm", 0.0)}
+        extra = {"attn_prefill_tflops": None}
+    else:
+        w = decode_work(cfg)
+        spec = {"index_scores_decode": ("hbm", w["index_bytes"]), "attn_decode": ("hbm", w["attn_bytes"]),
+                "topk_select": ("hbm", 0.0), "combine_decode": ("hbm", 0.0)}
+        extra = {}
+    for name, (ms, n) in stages.items():
+        if n == 0:
+            continue
+        per_step_ms = ms / args.steps
+        ent = {"ms_per_step": per_step_ms, "launches_per_step": n / args.steps}
+        if name in spec and spec[name][1] > 0:
+            bound, work = spec[name]
+            if bound == "tensor":
+                ach = work / (per_step_ms * 1e-3) / 1e12
+                ent.update(bound="tensor", achieved=ach, unit="TFLOP/s", peak=tf_s, frac=ach / tf_s)
+            else:
+                ach = work / (per_step_ms * 1e-3) / 1e9
+                ent.update(bound="hbm", achieved=ach, unit="GB/s", peak=hbm, frac=ach / hbm)
+        kern[name] = ent
+    if cfg.mode == "prefill" and "attn_prefill" in kern:
+        a_ms = kern["attn_prefill"]["ms_per_step"] + kern.get("combine", {}).get("ms_per_step", 0.0)
+        kern["attn_prefill"]["tensor_tflops"] = w["attn_flops"] / (kern["attn_prefill"]["ms_per_step"] * 1e-3) / 1e12
+        kern["attn_prefill"]["tensor_frac_of_sustained_peak"] = kern["attn_prefill"]["tensor_tflops"] / tf_s
+        extra["attn_plus_combine_ms"] = a_ms
+    dom = max((n for n in kern if "bound" in kern[n]), key=lambda n: kern[n]["ms_per_step"], default=None)
+    if dom is not None:
+        d = kern[dom]
+        line["roofline"] = {"kernel": dom, "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"],
+                            "unit": d["unit"], "frac": d["frac"], "traffic": None,
+                            "peak_source": src + " (sustained bf16)" if d["bound"] == "tensor" else src}
+    line["kernels"] = kern
+    line["peaks"] = {"hbm_gbs": hbm, "bf16_tflops_burst": tf_b, "bf16_tflops_sustained": tf_s,
+                     "source": peaks["_source"]}
+    if cfg.mode == "prefill":
+        line["tflops_total"] = (w["index_flops"] + w["attn_flops"]) / (ms_step * 1e-3) / 1e12
+
+    # ---- end to end from host buffers (copies inside the timed region)
+    if not args.no_e2e:
+        line["e2e"] = run_e2e(cfg, shape, x, B, dev, min(args.steps, 3), world)
+
+    # ---- the oracle on this machine's host cores (bounded sample)
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        if cfg.mode == "prefill":
+            xb = {n: to_bits(tn) for n, tn in x.items()}
+            n = oracle_sample_size(cfg)
+            m, dt = oracle_sample_prefill(cfg, xb, n)
+            sample = "%d uniformly drawn query positions of the same inputs, all heads" % m
+        else:
+            seqs = [0, len(cfg.seq_lens) - 1]
+            m, dt = oracle_sample_decode(cfg, x, seqs)
+            sample = "sequences %s of the same batch (one of each cache length)" % seqs
+        line["cpu_baseline"] = {"value": m / dt, "unit": "tokens/s", "cores": oracle.n_threads(),
+                                "kind": "oracle", "sample": sample, "seconds": dt}
+    print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_e2e(cfg, shape, x, B, dev, steps, world):
+    stream = torch.cuda.current_stream()
+    if cfg.mode == "prefill":
+        T = cfg.T
+        host = {n: t.cpu().pin_memory() for n, t in x.items()}
+        out_h = torch.empty(x["q"].shape, dtype=torch.bfloat16).pin_memory()
+        mn, pf = B.msa_prefill_forward_host_workspace_bytes(shape, T)
+        ws = B.alloc_workspace(pf, dev)
+        h2d = sum(t.numel() * t.element_size() for t in host.values())
+        d2h = out_h.numel() * 2
+
+        def step():
+            B.msa_prefill_forward_host(shape, host["q"], host["k"], host["v"], host["q_idx"],
+                                       host["k_idx"], T, out_h, None, None, ws)
+        units = T
+    else:
+        batch = len(cfg.seq_lens)
+        max_len = int(max(cfg.seq_lens))
+        ld = B.score_ld(max_len, cfg.block_size)
+        qh, qih = x["q"].cpu().pin_memory(), x["q_idx"].cpu().pin_memory()
+        out_h = torch.empty(x["q"].shape, dtype=torch.bfloat16).pin_memory()
+        qd, qid, od = torch.empty_like(x["q"]), torch.empty_like(x["q_idx"]), torch.empty_like(x["q"])
+        scores = torch.empty((batch, cfg.n_kv_heads, ld), dtype=torch.float32, device=dev)
+        bi = torch.empty((batch, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32, device=dev)
+        ws = B.alloc_workspace(B.msa_sparse_attn_decode_workspace_bytes(shape, batch), dev)
+        h2d = qh.numel() * 2 + qih.numel() * 2
+        d2h = out_h.numel() * 2
+
+        def step():
+            B.msa_decode_forward_host(shape, qh, qih, qd, qid, x["k_cache"], x["v_cache"], x["k_idx_cache"],
+                                      x["k_cache"].shape[0], x["seq_offsets"], x["seq_lens"], batch, max_len,
+                                      scores, ld, bi, od, out_h, ws)
+        units = batch
+    step()  # warm-up (page-locks are already in place)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return {"value": world * units / (ms * 1e-3), "unit": "tokens/s", "ms_per_step": ms,
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps}
+
+
+if __name__ == "__main__":
+    main()
