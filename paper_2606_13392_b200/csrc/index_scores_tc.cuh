@@ -1,0 +1,184 @@
+// Eq. 6 on the 5th-gen tensor cores (d_idx = 64, B_k in {64,128}).
+//
+// One CTA per (tile of 128 queries, index head r).  It streams the visible prefix of K_idx in
+// tiles of 256 keys through a TMA ring, multiplies each against the resident 128x64 query
+// tile with tcgen05.mma (M=128, N=256, four K=16 steps) into one of two 256-column TMEM
+// accumulators, and eight epilogue warps reduce the finished accumulator to per-block row
+// maxima (TMEM lane = query row, so the maximum over a block's columns is thread-local)
+// while the next tile is being multiplied.  Only the tile that crosses the diagonal applies
+// the causal mask.  Blocks beyond a query's local block are filled with -inf at the end.
+#pragma once
+
+#include "tc_common.cuh"
+
+namespace msa {
+
+constexpr int kIdxStages = 4;
+constexpr int kIdxTileQ = 128;
+constexpr int kIdxTileK = 256;
+constexpr int kIdxThreads = 320;  // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
+
+struct IdxSmem {
+    alignas(1024) uint8_t a[kIdxTileQ * 128];                   // 128 query rows x 64 bf16
+    alignas(1024) uint8_t b[kIdxStages][kIdxTileK * 128];       // 256 key rows x 64 bf16 per stage
+    alignas(8) uint64_t full[kIdxStages];
+    uint64_t empty[kIdxStages];
+    uint64_t a_full;
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort;
+};
+
+template <int BK>
+__global__ void __launch_bounds__(kIdxThreads, 1)
+index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                       int64_t q_begin, int64_t q_count, int H_kv, float scale,
+                       float* __restrict__ scores, int64_t ld_scores, int64_t n_cols, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    IdxSmem& sm = *reinterpret_cast<IdxSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t n_qtiles = (q_count + kIdxTileQ - 1) / kIdxTileQ;
+    // Longest items first: the last query tile sees the most keys.
+    const int64_t qt = n_qtiles - 1 - (int64_t)(blockIdx.x / H_kv);
+    const int r = (int)(blockIdx.x % H_kv);
+    const int64_t q0 = qt * kIdxTileQ;
+    int64_t q_hi = q0 + kIdxTileQ - 1;
+    if (q_hi > q_count - 1) q_hi = q_count - 1;
+    const int n_tiles = (int)((q_begin + q_hi) / kIdxTileK) + 1;
+    volatile int* abort = &sm.abort;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kIdxStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
+        mbar_init(&sm.a_full, 1);
+        mbar_init(&sm.drain, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&sm.acc_full[b], 1); mbar_init(&sm.acc_empty[b], 8); }
+        sm.abort = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+    }
+    if (warp == 1) tmem_alloc(&sm.tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_arrive_expect_tx(&sm.a_full, kIdxTileQ * 128);
+            tma_load_3d(sm.a, &tm_q, 0, r, (int)q0, &sm.a_full);
+            for (int t = 0; t < n_tiles; ++t) {
+                const int s = t % kIdxStages;
+                if (!mbar_wait(&sm.empty[s], ((t / kIdxStages) & 1) ^ 1, abort)) {
+                    report_async(status, kAsyncTimeout, 0x101);
+                    break;
+                }
+                mbar_arrive_expect_tx(&sm.full[s], kIdxTileK * 128);
+                tma_load_2d(sm.b[s], &tm_k, 0, t * kIdxTileK, &sm.full[s]);
+            }
+            if (*abort != 0) spin_cycles(200000);  // let copies already in flight land
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(kIdxTileQ, kIdxTileK, false, false);
+            const uint64_t a_desc = make_smem_desc(smem_u32(sm.a), 16, 1024);
+            bool ok = mbar_wait(&sm.a_full, 0, abort);
+            if (!ok) report_async(status, kAsyncTimeout, 0x102);
+            for (int t = 0; ok && t < n_tiles; ++t) {
+                const int s = t % kIdxStages, buf = t & 1;
+                if (!mbar_wait(&sm.acc_empty[buf], ((t >> 1) & 1) ^ 1, abort)) {
+                    report_async(status, kAsyncTimeout, 0x103);
+                    break;
+                }
+                if (!mbar_wait(&sm.full[s], (t / kIdxStages) & 1, abort)) {
+                    report_async(status, kAsyncTimeout, 0x104);
+                    break;
+                }
+                tc_fence_after();
+                const uint64_t b_desc = make_smem_desc(smem_u32(sm.b[s]), 16, 1024);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per K step
+                    mma_bf16_ss(tmem + buf * kIdxTileK, a_desc + 2 * kk, b_desc + 2 * kk, idesc, kk > 0);
+                mma_commit(&sm.empty[s]);
+                mma_commit(&sm.acc_full[buf]);
+            }
+            if (*abort != 0) {  // unwinding: wait for the MMAs already issued before TMEM is freed
+                mma_commit(&sm.drain);
+                mbar_wait_quiet(&sm.drain, 0, 20000000);
+            }
+        }
+    } else {
+        const int ew = warp - 2;            // 0..7
+        const int quarter = warp & 3;       // TMEM lanes this warp may read
+        const int half = ew >> 2;           // which 128 columns of the 256-column tile
+        const int row = quarter * 32 + lane;
+        const int64_t q = q0 + row;
+        const int64_t pos = q_begin + q;
+        const bool valid_row = q < q_count;
+        const int64_t loc = pos / BK;
+        float* out_row = scores + (q * H_kv + r) * ld_scores;
+        for (int t = 0; t < n_tiles; ++t) {
+            const int buf = t & 1;
+            if (!mbar_wait(&sm.acc_full[buf], (t >> 1) & 1, abort)) {
+                report_async(status, kAsyncTimeout, 0x105);
+                break;
+            }
+            tc_fence_after();
+            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + buf * kIdxTileK + half * 128;
+            uint32_t v[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld_32x32(taddr + c * 32, v[c]);
+            tmem_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
+
+            const int64_t key0 = (int64_t)t * kIdxTileK + half * 128;
+            const bool need_mask = key0 + 127 > pos;
+            constexpr int NB = 128 / BK;  // blocks in this thread's 128 columns
+            float best[NB];
+#pragma unroll
+            for (int i = 0; i < NB; ++i) best[i] = -INFINITY;
+            if (!need_mask) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        best[(c * 32 + e) / BK] = fmaxf(best[(c * 32 + e) / BK], __uint_as_float(v[c][e]));
+            } else {
+                const int lim = (int)(pos - key0);  // columns 0..lim are visible (may be negative)
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const float x = (c * 32 + e <= lim) ? __uint_as_float(v[c][e]) : -INFINITY;
+                        best[(c * 32 + e) / BK] = fmaxf(best[(c * 32 + e) / BK], x);
+                    }
+            }
+            if (valid_row) {
+#pragma unroll
+                for (int i = 0; i < NB; ++i) {
+                    const int64_t b = key0 / BK + i;
+                    if (b <= loc) out_row[b] = best[i] * scale;
+                }
+            }
+        }
+        // Blocks with no visible token: -inf (Eq. 6).  Warp ew fills rows ew, ew+8, ...
+        for (int rr = ew; rr < kIdxTileQ; rr += 8) {
+            const int64_t qq = q0 + rr;
+            if (qq >= q_count) break;
+            float* orow = scores + (qq * H_kv + r) * ld_scores;
+            for (int64_t b = (q_begin + qq) / BK + 1 + lane; b < n_cols; b += 32) orow[b] = -INFINITY;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+}  // namespace msa

@@ -7,6 +7,7 @@
 #include "common.cuh"
 #include "generic.cuh"
 #include "topk.cuh"
+#include "index_scores_tc.cuh"
 
 namespace msa {
 
@@ -75,11 +76,84 @@ static msa_status_t launch_status() {
     return cudaPeekAtLastError() == cudaSuccess ? MSA_OK : MSA_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------------- tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    // Looked up through the runtime so that the library does not link against libcuda.
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &qres) ==
+                cudaSuccess && qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+bool encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                      const uint64_t* strides_bytes, const uint32_t* box) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t gdim[5], gstr[5];
+    cuuint32_t bx[5], es[5];
+    for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i];
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr, bx, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // ---------------------------------------------------------------------- stage 1
+template <int BK>
+static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
+                                    int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
+                                    int64_t n_cols, cudaStream_t st) {
+    CUtensorMap tm_q, tm_k;
+    const uint64_t qd[3] = {64, (uint64_t)r.H_kv, (uint64_t)q_count};
+    const uint64_t qs[2] = {128, (uint64_t)r.H_kv * 128};
+    const uint32_t qb[3] = {64, 1, kIdxTileQ};
+    const uint64_t kd[2] = {64, (uint64_t)kv_len};
+    const uint64_t ks[1] = {128};
+    const uint32_t kb[2] = {64, kIdxTileK};
+    if (!encode_tmap_bf16(&tm_q, q_idx, 3, qd, qs, qb) || !encode_tmap_bf16(&tm_k, k_idx, 2, kd, ks, kb))
+        return MSA_ERR_CUDA;
+    int* status = async_status_ptr();
+    if (status == nullptr) return MSA_ERR_CUDA;
+    const size_t smem = sizeof(IdxSmem) + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(index_scores_tc_kernel<BK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem) != cudaSuccess)
+            return MSA_ERR_CUDA;
+        attr_set = true;
+    }
+    const int64_t grid = ceil_div64(q_count, kIdxTileQ) * r.H_kv;
+    if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
+    {
+        StageScope sc(kStageIndex, st);
+        index_scores_tc_kernel<BK><<<(unsigned)grid, kIdxThreads, smem, st>>>(
+            tm_q, tm_k, q_begin, q_count, r.H_kv, r.index_scale, scores, ld_scores, n_cols, status);
+    }
+    return launch_status();
+}
+
 static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const void* k_idx,
                                      const RowMap& rows, int64_t n_rows, float* scores,
                                      int64_t ld_scores, cudaStream_t st) {
     if (n_rows == 0 || rows.n_cols == 0) return MSA_OK;
+    if (rows.seq_lens == nullptr && r.d_idx == 64 && (r.B_k == 64 || r.B_k == 128) &&
+        rows.kv_len < 2147483647LL && n_rows >= 32) {
+        if (r.B_k == 64)
+            return launch_index_tc<64>(r, q_idx, k_idx, rows.q_begin, n_rows, rows.kv_len, scores, ld_scores,
+                                       rows.n_cols, st);
+        return launch_index_tc<128>(r, q_idx, k_idx, rows.q_begin, n_rows, rows.kv_len, scores, ld_scores,
+                                    rows.n_cols, st);
+    }
     constexpr int WARPS = 8;
     const int64_t n_chunks = ceil_div64(rows.n_cols, WARPS);
     const int64_t grid = n_rows * n_chunks;
