@@ -1,0 +1,411 @@
+// Eq. 8 for prefill in KV-outer order (Section 4.2) on tcgen05/TMEM (d_h = 128,
+// B_k in {64,128}, G in {8,16}).
+//
+// For one range of queries:
+//   1. reverse index: count, per (KV block, KV head) tile, the queries that selected it;
+//      exclusive scan; scatter 32-bit handles (query << 8 | slot), slot = position of the
+//      block in the query's ascending list, so every partial has its own place and no
+//      atomics touch the outputs;
+//   2. attention: a tile's handles are cut into items of 128/G queries; an item stacks those
+//      queries' G heads into one 128-row operand (query concatenation), computes
+//      S = Q K_b^T into TMEM, a row softmax local to the item (one block = one S tile),
+//      P (bf16) to shared memory, O = P V_b into TMEM, and writes the locally normalised
+//      partial and its log-sum-exp to the workspace;
+//   3. combine: LSE-weighted merge of each query's partials (Section 4.2, two-phase forward).
+#pragma once
+
+#include "tc_common.cuh"
+
+namespace msa {
+
+constexpr int kAttnThreads = 192;  // warp 0: TMA + item walk, warp 1: MMA, warps 2-5: softmax/epilogue
+
+struct RangeParams {
+    int64_t q_begin;   // absolute position of the first query of the call
+    int64_t q_first;   // first query of this range, relative to the call
+    int32_t q_count;   // queries in this range
+    int32_t n_blocks;  // KV blocks visible to the range: ceil((q_begin+q_first+q_count)/B_k)
+    int32_t H_kv, top_k;
+};
+
+// ---------------------------------------------------------------- 1. reverse index
+// One thread per (query, group, slot) entry.  pass 0 counts, pass 1 scatters.
+template <int BK>
+__global__ void revidx_kernel(const int32_t* __restrict__ block_idx, RangeParams p, int pass,
+                              int32_t* __restrict__ cnt, const int32_t* __restrict__ tile_off,
+                              uint32_t* __restrict__ handles, int* status) {
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t n = (int64_t)p.q_count * p.H_kv * p.top_k;
+    if (e >= n) return;
+    const int s = (int)(e % p.top_k);
+    const int64_t qr = e / p.top_k;
+    const int r = (int)(qr % p.H_kv);
+    const int64_t ql = qr / p.H_kv;
+    const int64_t pos = p.q_begin + p.q_first + ql;
+    const int32_t b = block_idx[((p.q_first + ql) * p.H_kv + r) * (int64_t)p.top_k + s];
+    if (b < 0 || (int64_t)b > pos / BK) {
+        if (b != -1 && pass == 0) report_async(status, kAsyncBadIndex, 0x301);
+        return;
+    }
+    const int tile = b * p.H_kv + r;
+    const int at = atomicAdd(&cnt[tile], 1);
+    if (pass == 1) handles[tile_off[tile] + at] = ((uint32_t)ql << 8) | (uint32_t)s;
+}
+
+// Single-CTA exclusive scan of the tile counts -> pair offsets and item offsets; clears the
+// counters so that the scatter pass can reuse them as cursors.
+__global__ void __launch_bounds__(1024)
+revidx_scan_kernel(int32_t* __restrict__ cnt, int n_tiles, int qpi, int32_t* __restrict__ tile_off,
+                   int32_t* __restrict__ item_off) {
+    __shared__ int s_pairs[1024], s_items[1024];
+    const int t = threadIdx.x;
+    const int per = (n_tiles + 1023) / 1024;
+    const int lo = t * per, hi = min(n_tiles, lo + per);
+    int pairs = 0, items = 0;
+    for (int i = lo; i < hi; ++i) { pairs += cnt[i]; items += (cnt[i] + qpi - 1) / qpi; }
+    s_pairs[t] = pairs; s_items[t] = items;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {
+        const int a = t >= off ? s_pairs[t - off] : 0, b = t >= off ? s_items[t - off] : 0;
+        __syncthreads();
+        s_pairs[t] += a; s_items[t] += b;
+        __syncthreads();
+    }
+    int po = s_pairs[t] - pairs, io = s_items[t] - items;
+    for (int i = lo; i < hi; ++i) {
+        const int c = cnt[i];
+        tile_off[i] = po; item_off[i] = io;
+        po += c; io += (c + qpi - 1) / qpi;
+        cnt[i] = 0;
+    }
+    if (t == 1023) { tile_off[n_tiles] = s_pairs[1023]; item_off[n_tiles] = s_items[1023]; }
+}
+
+// ---------------------------------------------------------------- 2. attention
+template <int BK>
+struct AttnSmem {
+    alignas(1024) uint8_t q[2][128 * 128];   // [d half][row = query*G + head][64 bf16]; reused for P
+    alignas(1024) uint8_t k[2][BK * 128];    // [d half][key][64 bf16]
+    alignas(1024) uint8_t v[2][BK * 128];
+    alignas(8) uint64_t in_full, s_full, p_full, o_full, epi_done, drain;
+    uint32_t tmem_base;
+    int abort;
+    // per-item info, double-buffered by item parity
+    int32_t info_block[2], info_r[2], info_nq[2];
+    uint32_t info_handle[2][16];
+};
+
+template <int BK, int G>
+__global__ void __launch_bounds__(kAttnThreads, 2)
+attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                       const __grid_constant__ CUtensorMap tm_v, RangeParams p,
+                       const int32_t* __restrict__ tile_off, const int32_t* __restrict__ item_off,
+                       const uint32_t* __restrict__ handles, float scale_log2e,
+                       __nv_bfloat16* __restrict__ o_buf, float* __restrict__ lse_buf, int* status) {
+    constexpr int QPI = 128 / G;            // queries per item
+    constexpr int TMEM_COLS = 256;          // S: BK columns at 0, O: 128 columns at 128
+    constexpr uint32_t Q_BOX_BYTES = G * 128;
+    constexpr uint32_t KV_BYTES = 4 * BK * 128;
+    extern __shared__ uint8_t smem_raw[];
+    AttnSmem<BK>& sm =
+        *reinterpret_cast<AttnSmem<BK>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int* abort = &sm.abort;
+
+    const int n_tiles = p.n_blocks * p.H_kv;
+    const int total_items = item_off[n_tiles];
+    const int per_cta = (total_items + gridDim.x - 1) / gridDim.x;
+    const int it_lo = min(total_items, (int)blockIdx.x * per_cta);
+    const int it_hi = min(total_items, it_lo + per_cta);
+
+    if (threadIdx.x == 0) {
+        mbar_init(&sm.in_full, 1);
+        mbar_init(&sm.s_full, 1);
+        mbar_init(&sm.p_full, 4);
+        mbar_init(&sm.o_full, 1);
+        mbar_init(&sm.epi_done, 4);
+        mbar_init(&sm.drain, 1);
+        sm.abort = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+    }
+    if (warp == 1) tmem_alloc(&sm.tmem_base, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+    const uint32_t tmem_s = tmem, tmem_o = tmem + 128;
+
+    if (warp == 0) {
+        // ---------------- producer: walks the item list, gathers Q rows, loads K/V tiles
+        int tile = 0;
+        if (it_lo < it_hi) {  // last tile whose first item is <= it_lo (skips empty tiles)
+            int lo = 0, hi = n_tiles;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (item_off[mid] <= it_lo) lo = mid; else hi = mid;
+            }
+            tile = lo;
+        }
+        int loaded_tile = -1;
+        for (int it = it_lo; it < it_hi; ++it) {
+            const int n = it - it_lo;
+            while (item_off[tile + 1] <= it) ++tile;
+            const int b = tile / p.H_kv, r = tile % p.H_kv;
+            const int first = tile_off[tile] + (it - item_off[tile]) * QPI;
+            const int nq = min(QPI, tile_off[tile + 1] - first);
+            // Q/P and K/V buffers are free once the previous item's second MMA has finished.
+            if (n > 0 && !mbar_wait(&sm.o_full, (n - 1) & 1, abort)) {
+                if (lane == 0) report_async(status, kAsyncTimeout, 0x311);
+                break;
+            }
+            uint32_t h = 0;
+            if (lane < nq) h = handles[first + lane];
+            if (lane < QPI) sm.info_handle[n & 1][lane] = h;
+            if (lane == 0) {
+                sm.info_block[n & 1] = b; sm.info_r[n & 1] = r; sm.info_nq[n & 1] = nq;
+            }
+            __syncwarp();
+            const bool new_tile = tile != loaded_tile;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(&sm.in_full, nq * 2 * Q_BOX_BYTES + (new_tile ? KV_BYTES : 0u));
+                if (new_tile) {
+                    tma_load_3d(sm.k[0], &tm_k, 0, r, b * BK, &sm.in_full);
+                    tma_load_3d(sm.k[1], &tm_k, 64, r, b * BK, &sm.in_full);
+                    tma_load_3d(sm.v[0], &tm_v, 0, r, b * BK, &sm.in_full);
+                    tma_load_3d(sm.v[1], &tm_v, 64, r, b * BK, &sm.in_full);
+                }
+            }
+            __syncwarp();
+            // One 8-row (G-row) box per (query, d half): 2*QPI boxes, one per lane.
+            if (lane < 2 * QPI) {
+                const int qi = lane >> 1, dh = lane & 1;
+                const uint32_t hq = __shfl_sync((2 * QPI == 32) ? 0xffffffffu : ((1u << (2 * QPI)) - 1u), h, qi);
+                if (qi < nq)
+                    tma_load_3d(sm.q[dh] + qi * Q_BOX_BYTES, &tm_q, dh * 64, r * G,
+                                (int)(p.q_first + (hq >> 8)), &sm.in_full);
+            }
+            loaded_tile = tile;
+        }
+        if (*abort != 0) spin_cycles(200000);
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = make_idesc_bf16(128, BK, false, false);
+            constexpr uint32_t idesc_o = make_idesc_bf16(128, 128, false, true);
+            const uint64_t qd0 = make_smem_desc(smem_u32(sm.q[0]), 16, 1024);
+            const uint64_t qd1 = make_smem_desc(smem_u32(sm.q[1]), 16, 1024);
+            const uint64_t kd0 = make_smem_desc(smem_u32(sm.k[0]), 16, 1024);
+            const uint64_t kd1 = make_smem_desc(smem_u32(sm.k[1]), 16, 1024);
+            // V as the MN-major B operand: next 64 columns of d are BK*128 bytes away.
+            const uint64_t vd = make_smem_desc(smem_u32(sm.v[0]), BK * 128, 1024);
+            for (int it = it_lo; it < it_hi; ++it) {
+                const int n = it - it_lo;
+                if (!mbar_wait(&sm.in_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x321); break; }
+                if (n > 0 && !mbar_wait(&sm.epi_done, (n - 1) & 1, abort)) {
+                    report_async(status, kAsyncTimeout, 0x322);
+                    break;
+                }
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(tmem_s, qd0 + 2 * kk, kd0 + 2 * kk, idesc_s, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(tmem_s, qd1 + 2 * kk, kd1 + 2 * kk, idesc_s, true);
+                mma_commit(&sm.s_full);
+                if (!mbar_wait(&sm.p_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x323); break; }
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < BK / 16; ++kk) {
+                    // P: K-major, 64 keys per 128-byte row atom; V: 16 keys = 2048 bytes per step.
+                    const uint64_t pd = ((kk >> 2) ? qd1 : qd0) + 2 * (kk & 3);
+                    mma_bf16_ss(tmem_o, pd, vd + (uint64_t)(kk * 2048 / 16), idesc_o, kk > 0);
+                }
+                mma_commit(&sm.o_full);
+            }
+            if (*abort != 0) {
+                mma_commit(&sm.drain);
+                mbar_wait_quiet(&sm.drain, 0, 20000000);
+            }
+        }
+    } else {
+        // ---------------- softmax + epilogue: thread = row of the 128-row operand
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const int qi = row / G, g = row % G;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        for (int it = it_lo; it < it_hi; ++it) {
+            const int n = it - it_lo;
+            if (!mbar_wait(&sm.s_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x331); break; }
+            tc_fence_after();
+            const int b = sm.info_block[n & 1], r = sm.info_r[n & 1], nq = sm.info_nq[n & 1];
+            const uint32_t h = sm.info_handle[n & 1][qi];
+            const bool valid = qi < nq;
+            const int64_t ql = h >> 8;
+            const int slot = h & 0xFF;
+            const int64_t pos = p.q_begin + p.q_first + ql;
+            // visible columns of this block for this query: 0..lim
+            int64_t lim64 = pos - (int64_t)b * BK;
+            const int lim = valid ? (int)(lim64 > BK - 1 ? BK - 1 : lim64) : BK - 1;
+
+            uint32_t sv[BK / 32][32];
+#pragma unroll
+            for (int c = 0; c < BK / 32; ++c) tmem_ld_32x32(tmem_s + lane_base + c * 32, sv[c]);
+            tmem_wait_ld();
+            float mx = -INFINITY;
+            if (lim == BK - 1) {
+#pragma unroll
+                for (int c = 0; c < BK / 32; ++c)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(sv[c][e]));
+            } else {
+#pragma unroll
+                for (int c = 0; c < BK / 32; ++c)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        if (c * 32 + e > lim) sv[c][e] = 0xFF800000u;  // -inf
+                        mx = fmaxf(mx, __uint_as_float(sv[c][e]));
+                    }
+            }
+            const float mc = mx * scale_log2e;
+            float ell = 0.f;
+            // P row -> shared memory, K-major, 128-byte swizzle: 16-byte chunk j of row m goes to
+            // chunk (j ^ (m & 7)) of that row.
+#pragma unroll
+            for (int c = 0; c < BK / 32; ++c) {
+#pragma unroll
+                for (int j4 = 0; j4 < 4; ++j4) {
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        const float p0 = exp2f(fmaf(__uint_as_float(sv[c][j4 * 8 + 2 * w]), scale_log2e, -mc));
+                        const float p1 = exp2f(fmaf(__uint_as_float(sv[c][j4 * 8 + 2 * w + 1]), scale_log2e, -mc));
+                        ell += p0 + p1;
+                        const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+                        pk[w] = *reinterpret_cast<const uint32_t*>(&pb);
+                    }
+                    const int col = c * 32 + j4 * 8;          // first key of this 16-byte chunk
+                    const int half = col >> 6, j = (col & 63) >> 3;
+                    uint4* dst = reinterpret_cast<uint4*>(sm.q[half] + row * 128 + ((j ^ (row & 7)) << 4));
+                    *dst = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.p_full);
+
+            // ---- epilogue: O row / ell -> bf16 partial, LSE partial
+            if (!mbar_wait(&sm.o_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x332); break; }
+            tc_fence_after();
+            const float inv = 1.0f / ell;
+            const int64_t prow = (ql * p.H_kv + r) * (int64_t)p.top_k + slot;
+            __nv_bfloat16* orow = o_buf + (prow * G + g) * 128;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t ov[32];
+                tmem_ld_32x32(tmem_o + lane_base + c * 32, ov);
+                tmem_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int j4 = 0; j4 < 4; ++j4) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) {
+                            const __nv_bfloat162 ob = __floats2bfloat162_rn(
+                                __uint_as_float(ov[j4 * 8 + 2 * w]) * inv, __uint_as_float(ov[j4 * 8 + 2 * w + 1]) * inv);
+                            pk[w] = *reinterpret_cast<const uint32_t*>(&ob);
+                        }
+                        *reinterpret_cast<uint4*>(orow + c * 32 + j4 * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                }
+            }
+            if (valid) lse_buf[prow * G + g] = (mc + log2f(ell)) * 0.6931471805599453f;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.epi_done);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, TMEM_COLS);
+    }
+}
+
+// ---------------------------------------------------------------- 3. combine
+// One CTA per (query, KV head): thread t handles head t/16 and 8 consecutive d elements.
+//   a = max_s LSE_s, LSE = a + log sum_s exp(LSE_s - a), w_s = exp(LSE_s - LSE), O = sum_s w_s O_s.
+template <int BK, int G>
+__global__ void __launch_bounds__(G * 16)
+combine_kernel(const int32_t* __restrict__ block_idx, RangeParams p, const __nv_bfloat16* __restrict__ o_buf,
+               const float* __restrict__ lse_buf, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+    __shared__ float w_s[128][G];   // top_k <= 128
+    __shared__ int valid_s[128];
+    const int ql = blockIdx.x / p.H_kv, r = blockIdx.x % p.H_kv;
+    const int t = threadIdx.x;
+    const int64_t q = p.q_first + ql;
+    const int64_t loc = (p.q_begin + q) / BK;
+    const int32_t* sel = block_idx + (q * p.H_kv + r) * (int64_t)p.top_k;
+    const int64_t pbase = ((int64_t)ql * p.H_kv + r) * p.top_k;
+    for (int s = t; s < p.top_k; s += G * 16) {
+        const int32_t b = sel[s];
+        valid_s[s] = (b >= 0 && (int64_t)b <= loc) ? 1 : 0;
+    }
+    __syncthreads();
+    const int g = t >> 4, dc = (t & 15) * 8;
+    {   // 16 threads per head: thread j of a head owns slots j, j+16, ...
+        const int j = t & 15;
+        float lv[8];
+        float a = -INFINITY;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int s = j + 16 * u;
+            lv[u] = (s < p.top_k && valid_s[s]) ? lse_buf[(pbase + s) * G + g] : -INFINITY;
+            a = fmaxf(a, lv[u]);
+        }
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+        float sum = 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) sum += (lv[u] > -INFINITY) ? expf(lv[u] - a) : 0.f;
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        const float L = a + logf(sum);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int s = j + 16 * u;
+            if (s < p.top_k) w_s[s][g] = (lv[u] > -INFINITY) ? expf(lv[u] - L) : 0.f;
+        }
+        if (j == 0 && lse != nullptr) lse[q * (int64_t)(p.H_kv * G) + r * G + g] = L;
+    }
+    __syncthreads();
+    float acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    const __nv_bfloat16* src = o_buf + (pbase * G + g) * 128 + dc;
+#pragma unroll 4
+    for (int s = 0; s < p.top_k; ++s) {
+        if (!valid_s[s]) continue;
+        const uint4 x = __ldg(reinterpret_cast<const uint4*>(src + (int64_t)s * G * 128));
+        const float w = w_s[s][g];
+        const float2 a0 = bf16x2_to_float2(x.x), a1 = bf16x2_to_float2(x.y);
+        const float2 a2 = bf16x2_to_float2(x.z), a3 = bf16x2_to_float2(x.w);
+        acc[0] = fmaf(w, a0.x, acc[0]); acc[1] = fmaf(w, a0.y, acc[1]);
+        acc[2] = fmaf(w, a1.x, acc[2]); acc[3] = fmaf(w, a1.y, acc[3]);
+        acc[4] = fmaf(w, a2.x, acc[4]); acc[5] = fmaf(w, a2.y, acc[5]);
+        acc[6] = fmaf(w, a3.x, acc[6]); acc[7] = fmaf(w, a3.y, acc[7]);
+    }
+    uint32_t pk[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat162 ob = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+        pk[i] = *reinterpret_cast<const uint32_t*>(&ob);
+    }
+    *reinterpret_cast<uint4*>(out + (q * (int64_t)(p.H_kv * G) + r * G + g) * 128 + dc) =
+        make_uint4(pk[0], pk[1], pk[2], pk[3]);
+}
+
+}  // namespace msa

@@ -8,6 +8,7 @@
 #include "generic.cuh"
 #include "topk.cuh"
 #include "index_scores_tc.cuh"
+#include "attn_prefill_tc.cuh"
 
 namespace msa {
 
@@ -224,6 +225,133 @@ static RowMap decode_rows(const int64_t* seq_offsets, const int32_t* seq_lens, i
 constexpr size_t kAlign = 256;
 static size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
+// ---------------------------------------------------------------------- stage 3 (KV-outer, tcgen05)
+static bool attn_tc_supported(const Resolved& r) {
+    return r.d == 128 && (r.B_k == 64 || r.B_k == 128) && (r.G == 8 || r.G == 16);
+}
+
+// Workspace of the KV-outer path for ranges of R queries:
+//   [cnt | tile_off | item_off] int32 per (block, head) tile, handles, LSE_buf, O_buf.
+struct AttnPlan {
+    int64_t R;
+    size_t off_cnt, off_tile_off, off_item_off, off_handles, off_lse, off_obuf, total;
+};
+
+static size_t attn_per_query_bytes(const Resolved& r) {
+    return (size_t)r.H_q * r.k * r.d * 2 + (size_t)r.H_q * r.k * 4 + (size_t)r.H_kv * r.k * 4;
+}
+
+static AttnPlan attn_plan(const Resolved& r, int64_t kv_len, int64_t R) {
+    AttnPlan p;
+    p.R = R;
+    const size_t n_tiles = (size_t)ceil_div64(kv_len, r.B_k) * r.H_kv + 1;
+    size_t o = 0;
+    p.off_cnt = o; o += align_up(n_tiles * 4);
+    p.off_tile_off = o; o += align_up(n_tiles * 4);
+    p.off_item_off = o; o += align_up(n_tiles * 4);
+    p.off_handles = o; o += align_up((size_t)R * r.H_kv * r.k * 4);
+    p.off_lse = o; o += align_up((size_t)R * r.H_q * r.k * 4);
+    p.off_obuf = o; o += align_up((size_t)R * r.H_q * r.k * r.d * 2);
+    p.total = o;
+    return p;
+}
+
+static int64_t attn_range_for(const Resolved& r, int64_t q_count, int64_t kv_len, size_t ws_bytes) {
+    const size_t fixed = attn_plan(r, kv_len, 0).total + 4 * kAlign;
+    if (ws_bytes <= fixed) return 0;
+    int64_t R = (int64_t)((ws_bytes - fixed) / attn_per_query_bytes(r));
+    if (R > q_count) R = q_count;
+    if (R > (1 << 23)) R = 1 << 23;  // handles keep the query in 24 bits
+    if (R >= 128) R = R / 128 * 128;
+    return R;
+}
+
+static int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            n = 148;
+    }
+    return n;
+}
+
+template <int BK, int G>
+static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const void* k, const void* v,
+                                        const int32_t* block_idx, int64_t q_begin, int64_t q_count,
+                                        int64_t kv_len, void* out, float* lse, void* ws, size_t ws_bytes,
+                                        cudaStream_t st) {
+    const int64_t R = attn_range_for(r, q_count, kv_len, ws_bytes);
+    if (R <= 0) return MSA_ERR_WORKSPACE;
+    const AttnPlan pl = attn_plan(r, kv_len, R);
+    char* w = static_cast<char*>(ws);
+    int32_t* cnt = (int32_t*)(w + pl.off_cnt);
+    int32_t* tile_off = (int32_t*)(w + pl.off_tile_off);
+    int32_t* item_off = (int32_t*)(w + pl.off_item_off);
+    uint32_t* handles = (uint32_t*)(w + pl.off_handles);
+    float* lse_buf = (float*)(w + pl.off_lse);
+    __nv_bfloat16* o_buf = (__nv_bfloat16*)(w + pl.off_obuf);
+
+    CUtensorMap tm_q, tm_k, tm_v;
+    const uint64_t qd[3] = {128, (uint64_t)r.H_q, (uint64_t)q_count};
+    const uint64_t qs[2] = {256, (uint64_t)r.H_q * 256};
+    const uint32_t qb[3] = {64, (uint32_t)G, 1};
+    const uint64_t kd[3] = {128, (uint64_t)r.H_kv, (uint64_t)kv_len};
+    const uint64_t ks[2] = {256, (uint64_t)r.H_kv * 256};
+    const uint32_t kb[3] = {64, 1, (uint32_t)BK};
+    if (!encode_tmap_bf16(&tm_q, q, 3, qd, qs, qb) || !encode_tmap_bf16(&tm_k, k, 3, kd, ks, kb) ||
+        !encode_tmap_bf16(&tm_v, v, 3, kd, ks, kb))
+        return MSA_ERR_CUDA;
+    int* status = async_status_ptr();
+    if (status == nullptr) return MSA_ERR_CUDA;
+    const size_t smem = sizeof(AttnSmem<BK>) + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(attn_prefill_tc_kernel<BK, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem) != cudaSuccess)
+            return MSA_ERR_CUDA;
+        attr_set = true;
+    }
+    const float scale_log2e = r.softmax_scale * 1.4426950408889634f;
+    const int grid_attn = 2 * sm_count();
+    for (int64_t q_first = 0; q_first < q_count; q_first += R) {
+        RangeParams p;
+        p.q_begin = q_begin; p.q_first = q_first;
+        p.q_count = (int32_t)((q_count - q_first) < R ? (q_count - q_first) : R);
+        p.n_blocks = (int32_t)ceil_div64(q_begin + q_first + p.q_count, BK);
+        p.H_kv = r.H_kv; p.top_k = r.k;
+        const int n_tiles = p.n_blocks * r.H_kv;
+        const int64_t entries = (int64_t)p.q_count * r.H_kv * r.k;
+        const unsigned eg = (unsigned)ceil_div64(entries, 256);
+        if (cudaMemsetAsync(cnt, 0, (size_t)(n_tiles + 1) * 4, st) != cudaSuccess) return MSA_ERR_CUDA;
+        {
+            StageScope sc(kStageSchedule, st);
+            revidx_kernel<BK><<<eg, 256, 0, st>>>(block_idx, p, 0, cnt, tile_off, handles, status);
+        }
+        {
+            StageScope sc(kStageSchedule, st);
+            revidx_scan_kernel<<<1, 1024, 0, st>>>(cnt, n_tiles, 128 / G, tile_off, item_off);
+        }
+        {
+            StageScope sc(kStageSchedule, st);
+            revidx_kernel<BK><<<eg, 256, 0, st>>>(block_idx, p, 1, cnt, tile_off, handles, status);
+        }
+        {
+            StageScope sc(kStageAttn, st);
+            attn_prefill_tc_kernel<BK, G><<<grid_attn, kAttnThreads, smem, st>>>(
+                tm_q, tm_k, tm_v, p, tile_off, item_off, handles, scale_log2e, o_buf, lse_buf, status);
+        }
+        {
+            StageScope sc(kStageCombine, st);
+            combine_kernel<BK, G><<<(unsigned)(p.q_count * r.H_kv), G * 16, 0, st>>>(
+                block_idx, p, o_buf, lse_buf, (__nv_bfloat16*)out, lse);
+        }
+        if (cudaPeekAtLastError() != cudaSuccess) return MSA_ERR_CUDA;
+    }
+    return MSA_OK;
+}
+
 }  // namespace msa
 
 using namespace msa;
@@ -357,8 +485,18 @@ msa_status_t msa_sparse_attn_prefill_workspace_bytes(const msa_shape_t* shape, i
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
     if (q_count < 0 || kv_len < 0) return MSA_ERR_INVALID_ARG;
-    if (min_bytes) *min_bytes = kAlign;
-    if (preferred_bytes) *preferred_bytes = kAlign;
+    size_t mn = kAlign, pf = kAlign;
+    if (attn_tc_supported(r) && q_count > 0) {
+        // at least 256 queries in flight; preferred: partial buffers of up to 16 GiB
+        const int64_t r_min = q_count < 256 ? q_count : 256;
+        int64_t r_pref = (int64_t)((16ull << 30) / attn_per_query_bytes(r));
+        if (r_pref > q_count) r_pref = q_count;
+        if (r_pref < r_min) r_pref = r_min;
+        mn = attn_plan(r, kv_len, r_min).total + 8 * kAlign;
+        pf = attn_plan(r, kv_len, r_pref).total + 8 * kAlign;
+    }
+    if (min_bytes) *min_bytes = mn;
+    if (preferred_bytes) *preferred_bytes = pf;
     return MSA_OK;
 }
 
@@ -376,9 +514,19 @@ msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, co
         return MSA_ERR_INVALID_ARG;
     size_t need = 0;
     msa_sparse_attn_prefill_workspace_bytes(shape, q_count, kv_len, &need, nullptr);
-    if (workspace == nullptr || workspace_bytes < need) return MSA_ERR_WORKSPACE;
+    if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (attn_tc_supported(r) && kv_len < 2147483647LL) {
+        if (r.B_k == 64 && r.G == 8)
+            return run_attn_prefill_tc<64, 8>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
+        if (r.B_k == 64 && r.G == 16)
+            return run_attn_prefill_tc<64, 16>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
+        if (r.B_k == 128 && r.G == 8)
+            return run_attn_prefill_tc<128, 8>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
+        return run_attn_prefill_tc<128, 16>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
+    }
     return run_attn_generic(r, q, k, v, block_idx, prefill_rows(q_begin, kv_len, r.B_k), q_count, out,
-                            lse, (cudaStream_t)stream);
+                            lse, st);
 }
 
 msa_status_t msa_sparse_attn_decode_workspace_bytes(const msa_shape_t* shape, int32_t batch,
