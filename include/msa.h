@@ -133,6 +133,38 @@ msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, co
                                      void* out, float* lse, void* workspace,
                                      size_t workspace_bytes, msa_stream_t stream);
 
+/*
+ * Stage 3, prefill, for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a convenience of the library.)
+ *
+ * Some hosts of this library are not allowed to call cudaMalloc, or to ask their framework
+ * for a buffer, at the point where they need attention: a plug-in running inside an engine
+ * that owns all device memory, a callback that runs after the memory pool has been frozen,
+ * a real-time loop where an allocation may stall on the driver.  msa_sparse_attn_prefill
+ * needs a caller-provided workspace, so such callers cannot use it.  This variant takes the
+ * same inputs and outputs and no workspace: its scratch (reverse index, partial outputs,
+ * partial log-sum-exps) lives in one fixed array of MSA_STATIC_SCRATCH_BYTES inside the
+ * library's device image.  Every GPU that loads the library holds that array until the
+ * process exits.
+ *
+ * Limits and rules:
+ *   - The query range is processed in passes of as many queries as fit the fixed array.
+ *     If fewer than min(q_count, 16) queries fit (long sequences with many heads and a large
+ *     k), the call returns MSA_ERR_WORKSPACE and launches nothing; use the workspace form.
+ *   - The call allocates nothing: no cudaMalloc/cudaFree and no allocating library routine.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and sets a kernel attribute; make that first call outside any stream capture.
+ *   - All calls share the one array, and it keeps the previous call's contents; the call
+ *     clears the counters that must start at zero itself.  Two calls whose kernels overlap
+ *     on the GPU (different streams, or different host threads) race on it: serialise them.
+ *   - Results equal those of msa_sparse_attn_prefill on the same inputs.
+ */
+#define MSA_STATIC_SCRATCH_BYTES (64u << 20)
+msa_status_t msa_sparse_attn_prefill_static(const msa_shape_t* shape, const void* q, const void* k,
+                                            const void* v, const int32_t* block_idx,
+                                            int64_t q_begin, int64_t q_count, int64_t kv_len,
+                                            void* out, float* lse, msa_stream_t stream);
+
 /* Minimum and preferred workspace for msa_sparse_attn_prefill (bytes; either may be NULL). */
 msa_status_t msa_sparse_attn_prefill_workspace_bytes(const msa_shape_t* shape, int64_t q_count,
                                                      int64_t kv_len, size_t* min_bytes,

@@ -25,7 +25,8 @@ c_i64, c_i32, c_vp, c_sz = ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctyp
 EXPORTS = [
     "msa_status_string", "msa_check_async_status", "msa_index_scores", "msa_index_scores_decode",
     "msa_topk_select", "msa_topk_select_decode", "msa_sparse_attn_prefill",
-    "msa_sparse_attn_prefill_workspace_bytes", "msa_sparse_attn_decode",
+    "msa_sparse_attn_prefill_workspace_bytes", "msa_sparse_attn_prefill_static",
+    "msa_sparse_attn_decode",
     "msa_sparse_attn_decode_workspace_bytes", "msa_prefill_forward",
     "msa_prefill_forward_workspace_bytes", "msa_prefill_forward_host",
     "msa_prefill_forward_host_workspace_bytes", "msa_decode_forward", "msa_decode_forward_host",
@@ -171,6 +172,27 @@ def msa_sparse_attn_prefill(shape, q, k, v, block_idx, q_begin, q_count, kv_len,
                                          c_i64(kv_len), _dev(out), _dev(lse), _dev(workspace),
                                          c_sz(workspace.numel() * workspace.element_size()),
                                          _stream(stream)), "msa_sparse_attn_prefill")
+
+
+STATIC_SCRATCH_BYTES = 64 << 20
+
+
+def msa_sparse_attn_prefill_static(shape, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse,
+                                   stream=None):
+    """Stage 3 (prefill) for callers that may not allocate device memory.
+
+    Same inputs and outputs as :func:`msa_sparse_attn_prefill`, but no workspace argument:
+    the scratch is a fixed array of ``STATIC_SCRATCH_BYTES`` inside the library's device
+    image.  Meant for hosts that cannot call ``cudaMalloc`` or ask torch for a buffer at
+    that point (a plug-in inside an engine that owns all device memory, code running after
+    the memory pool was frozen).  Raises ``MsaError`` (workspace) when fewer than
+    ``min(q_count, 16)`` queries fit the array.  Calls that overlap on the GPU race on the
+    shared array; make the first call on a device outside any stream capture.
+    """
+    _check(lib().msa_sparse_attn_prefill_static(ctypes.byref(shape), _dev(q), _dev(k), _dev(v),
+                                                _dev(block_idx), c_i64(q_begin), c_i64(q_count),
+                                                c_i64(kv_len), _dev(out), _dev(lse),
+                                                _stream(stream)), "msa_sparse_attn_prefill_static")
 
 
 def msa_sparse_attn_decode_workspace_bytes(shape, batch) -> int:

@@ -529,6 +529,58 @@ msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, co
                             lse, st);
 }
 
+// Scratch of msa_sparse_attn_prefill_static: part of the library's device image, so no call
+// ever allocates it.  In host code this name is only a handle for cudaGetSymbolAddress; it
+// is not a device address and must never be passed to a kernel as is.
+static __device__ __align__(256) unsigned char g_static_scratch[MSA_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device, looked up once per device.
+static msa_status_t static_scratch_ptr(void** out) {
+    constexpr int kMaxDevices = 64;
+    static void* cached[kMaxDevices] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MSA_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return MSA_ERR_UNSUPPORTED;
+    if (cached[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return MSA_ERR_CUDA;
+        cached[dev] = p;
+    }
+    *out = cached[dev];
+    return MSA_OK;
+}
+
+msa_status_t msa_sparse_attn_prefill_static(const msa_shape_t* shape, const void* q, const void* k,
+                                            const void* v, const int32_t* block_idx, int64_t q_begin,
+                                            int64_t q_count, int64_t kv_len, void* out, float* lse,
+                                            msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if ((s = check_range(q_begin, q_count, kv_len)) != MSA_OK) return s;
+    if (q_count == 0) return MSA_OK;
+    if (!q || !k || !v || !block_idx || !out || !aligned16(q) || !aligned16(k) || !aligned16(v) ||
+        !aligned16(out))
+        return MSA_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!attn_tc_supported(r) || kv_len >= 2147483647LL)  // the generic kernel needs no scratch at all
+        return run_attn_generic(r, q, k, v, block_idx, prefill_rows(q_begin, kv_len, r.B_k), q_count, out,
+                                lse, st);
+    // Refuse sizes the fixed array cannot serve: fewer than min(q_count, 16) queries per pass.
+    const int64_t fit = attn_range_for(r, q_count, kv_len, (size_t)MSA_STATIC_SCRATCH_BYTES);
+    if (fit < (q_count < 16 ? q_count : 16)) return MSA_ERR_WORKSPACE;
+    void* scratch = nullptr;
+    if ((s = static_scratch_ptr(&scratch)) != MSA_OK) return s;
+    const size_t bytes = (size_t)MSA_STATIC_SCRATCH_BYTES;
+    if (r.B_k == 64 && r.G == 8)
+        return run_attn_prefill_tc<64, 8>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, scratch, bytes, st);
+    if (r.B_k == 64 && r.G == 16)
+        return run_attn_prefill_tc<64, 16>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, scratch, bytes, st);
+    if (r.B_k == 128 && r.G == 8)
+        return run_attn_prefill_tc<128, 8>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, scratch, bytes, st);
+    return run_attn_prefill_tc<128, 16>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, scratch, bytes, st);
+}
+
 msa_status_t msa_sparse_attn_decode_workspace_bytes(const msa_shape_t* shape, int32_t batch,
                                                     size_t* min_bytes) {
     Resolved r;
