@@ -1,0 +1,54 @@
+"""GPU parity at the full sizes of the five benchmark configurations, in the launch
+configuration bench.py times (the whole-path C-ABI calls with their preferred workspaces).
+The oracle cannot run these sizes in full, so the prefill configurations are checked on a
+stratified sample of query positions (all heads); the decode batch is checked in full."""
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2606_13392_b200.inputs import CONFIGS
+from test_gpu_parity import run_decode_case, run_prefill_case
+
+pytestmark = pytest.mark.gpu
+
+
+def _free():
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+
+
+def test_c2_full_size_sampled():
+    stats = run_prefill_case(CONFIGS["c2"], False, n_sample=320)
+    assert stats["exact_sets"] >= 0.999
+    print("c2", stats)
+    _free()
+
+
+def test_c3_full_size_sampled():
+    stats = run_prefill_case(CONFIGS["c3"], False, n_sample=256)
+    assert stats["exact_sets"] >= 0.999
+    print("c3", stats)
+    _free()
+
+
+def test_c3_full_size_sharp_sampled():
+    stats = run_prefill_case(CONFIGS["c3"], True, n_sample=192)
+    assert stats["exact_sets"] >= 0.999
+    print("c3 sharp", stats)
+    _free()
+
+
+def test_c4_full_size_sampled():
+    stats = run_prefill_case(CONFIGS["c4"], False, n_sample=160)
+    assert stats["exact_sets"] >= 0.995
+    print("c4", stats)
+    _free()
+
+
+def test_c5_decode_full_batch():
+    res = run_decode_case(CONFIGS["c5"], False)
+    assert len(res) == 32
+    assert np.mean([r["exact"] for r in res]) >= 0.99
+    print("c5", res[0], res[-1])
+    _free()

@@ -28,9 +28,12 @@ def _assert_clean():
 
 def run_prefill_case(cfg: MSAConfig, sharp: bool, n_sample: int, ws_bytes=None):
     x = make_prefill_inputs(cfg, DEV, sharp=sharp)
-    xb = _bits(x)
     T = cfg.T
     pos = np.arange(T) if n_sample >= T else sample_positions(T, cfg.block_size, cfg.top_k, n_sample, 7)
+    pos_t = torch.from_numpy(pos).to(DEV)
+    # the oracle needs every key/value row but only the sampled query rows
+    kb, vb, kib = to_bits(x["k"]), to_bits(x["v"]), to_bits(x["k_idx"])
+    qb, qib = to_bits(x["q"][pos_t]), to_bits(x["q_idx"][pos_t])
 
     # --- whole path on the GPU
     out, lse, I = api.prefill_forward(cfg, x, workspace_bytes=ws_bytes)
@@ -44,18 +47,18 @@ def run_prefill_case(cfg: MSAConfig, sharp: bool, n_sample: int, ws_bytes=None):
         q0, qc = int(pos[run[0]]), len(run)
         s = api.index_scores(cfg, x["q_idx"], x["k_idx"], q0, qc)
         M_gpu[run] = s[:, :, :cfg.n_blocks].cpu().numpy()
-    M_ref = oracle.index_scores(xb["q_idx"][pos], xb["k_idx"], pos, cfg.block_size)
+    M_ref = oracle.index_scores(qib, kib, pos, cfg.block_size)
     score_err = check_scores(M_gpu, M_ref, pos, cfg.block_size)
 
     # --- stage 2: the GPU's own pipeline against the oracle's selection
     I_ref = oracle.topk_select(M_ref, pos, T, cfg.block_size, cfg.top_k)
-    I_gpu = I.cpu().numpy()[pos]
+    I_gpu = I[pos_t].cpu().numpy()
     exact, n_rows = check_selection(I_gpu, I_ref, M_ref, pos, cfg.block_size, cfg.top_k)
 
     # --- stage 3: oracle attention on the GPU's index lists
-    O_ref, LSE_ref = oracle.sparse_attn(xb["q"][pos], xb["k"], xb["v"], I_gpu, pos, cfg.block_size)
-    o = out.float().cpu().numpy()[pos]
-    stats = check_attn(o, lse.cpu().numpy()[pos], O_ref, LSE_ref, cfg.name)
+    O_ref, LSE_ref = oracle.sparse_attn(qb, kb, vb, I_gpu, pos, cfg.block_size)
+    o = out[pos_t].float().cpu().numpy()
+    stats = check_attn(o, lse[pos_t].cpu().numpy(), O_ref, LSE_ref, cfg.name)
     stats.update(score_err=score_err, exact_sets=exact, rows=n_rows)
     return stats
 
