@@ -65,6 +65,12 @@ CONFIGS: Dict[str, MSAConfig] = {
     "c4": MSAConfig("c4", "prefill", 1048576, 64, 8, 128, 64, seed=3),
     "c5": MSAConfig("c5", "decode", 1048576, 64, 8, 128, 64, seed=4,
                     seq_lens=(131072,) * 16 + (1048576,) * 16),
+    # Reduced cases of the same shapes, small enough for multi-pass profiler captures
+    # (inputs still larger than L2).
+    "c3-16k": MSAConfig("c3-16k", "prefill", 16384, 64, 8, 128, 64, seed=2,
+                        planted_frac=0.05, planted_shift=2.0),
+    "c5-small": MSAConfig("c5-small", "decode", 131072, 64, 8, 128, 64, seed=4,
+                          seq_lens=(32768,) * 8 + (131072,) * 8),
 }
 
 
