@@ -84,10 +84,10 @@ revidx_scan_kernel(int32_t* __restrict__ cnt, int n_tiles, int qpi, int32_t* __r
 // ---------------------------------------------------------------- 2. attention
 template <int BK>
 struct AttnSmem {
-    alignas(1024) uint8_t q[2][128 * 128];   // [d half][row = query*G + head][64 bf16]; reused for P
+    alignas(1024) uint8_t q[2][128 * 128];   // [d half][row = query*G + head][64 bf16]
     alignas(1024) uint8_t k[2][BK * 128];    // [d half][key][64 bf16]
     alignas(1024) uint8_t v[2][BK * 128];
-    alignas(8) uint64_t in_full, s_full, p_full, o_full, epi_done, drain;
+    alignas(8) uint64_t in_full, s_full, p_full, o_full, drain;
     uint32_t tmem_base;
     int abort;
     // per-item info, double-buffered by item parity
@@ -95,6 +95,14 @@ struct AttnSmem {
     uint32_t info_handle[2][16];
 };
 
+// Per-CTA pipeline (two CTAs share an SM):
+//   producer : Q(n+1) boxes as soon as MMA1(n) has read Q(n) (s_full); K/V of a new tile once
+//              MMA2(n) has read V (o_full).
+//   MMA      : in_full(n) -> S = Q K^T -> s_full(n);  p_full(n) -> O = P V -> o_full(n).
+//              MMAs execute in issue order, so S(n+1) may be issued right behind O(n) although
+//              P(n) lives in the columns S(n+1) overwrites.
+//   softmax  : s_full(n) -> read S row, exp2, write P (bf16 pairs) over the S columns ->
+//              p_full(n); o_full(n) -> O row / ell -> partial; then item n+1.
 template <int BK, int G>
 __global__ void __launch_bounds__(kAttnThreads, 2)
 attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -103,7 +111,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                        const uint32_t* __restrict__ handles, float scale_log2e,
                        __nv_bfloat16* __restrict__ o_buf, float* __restrict__ lse_buf, int* status) {
     constexpr int QPI = 128 / G;            // queries per item
-    constexpr int TMEM_COLS = 256;          // S: BK columns at 0, O: 128 columns at 128
+    constexpr int TMEM_COLS = 256;          // S (then P): columns 0..BK-1, O: columns 128..255
     constexpr uint32_t Q_BOX_BYTES = G * 128;
     constexpr uint32_t KV_BYTES = 4 * BK * 128;
     extern __shared__ uint8_t smem_raw[];
@@ -123,7 +131,6 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         mbar_init(&sm.s_full, 1);
         mbar_init(&sm.p_full, 4);
         mbar_init(&sm.o_full, 1);
-        mbar_init(&sm.epi_done, 4);
         mbar_init(&sm.drain, 1);
         sm.abort = 0;
         fence_mbar_init();
@@ -156,30 +163,23 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             const int b = tile / p.H_kv, r = tile % p.H_kv;
             const int first = tile_off[tile] + (it - item_off[tile]) * QPI;
             const int nq = min(QPI, tile_off[tile + 1] - first);
-            // Q/P and K/V buffers are free once the previous item's second MMA has finished.
-            if (n > 0 && !mbar_wait(&sm.o_full, (n - 1) & 1, abort)) {
+            uint32_t h = 0;
+            if (lane < nq) h = handles[first + lane];
+            // The Q buffer is free once the previous item's first MMA has read it.
+            if (n > 0 && !mbar_wait(&sm.s_full, (n - 1) & 1, abort)) {
                 if (lane == 0) report_async(status, kAsyncTimeout, 0x311);
                 break;
             }
-            uint32_t h = 0;
-            if (lane < nq) h = handles[first + lane];
             if (lane < QPI) sm.info_handle[n & 1][lane] = h;
             if (lane == 0) {
                 sm.info_block[n & 1] = b; sm.info_r[n & 1] = r; sm.info_nq[n & 1] = nq;
             }
             __syncwarp();
             const bool new_tile = tile != loaded_tile;
-            if (lane == 0) {
+            if (lane == 0)
                 mbar_arrive_expect_tx(&sm.in_full, nq * 2 * Q_BOX_BYTES + (new_tile ? KV_BYTES : 0u));
-                if (new_tile) {
-                    tma_load_3d(sm.k[0], &tm_k, 0, r, b * BK, &sm.in_full);
-                    tma_load_3d(sm.k[1], &tm_k, 64, r, b * BK, &sm.in_full);
-                    tma_load_3d(sm.v[0], &tm_v, 0, r, b * BK, &sm.in_full);
-                    tma_load_3d(sm.v[1], &tm_v, 64, r, b * BK, &sm.in_full);
-                }
-            }
             __syncwarp();
-            // One 8-row (G-row) box per (query, d half): 2*QPI boxes, one per lane.
+            // One G-row box per (query, d half): 2*QPI boxes, one per lane.
             if (lane < 2 * QPI) {
                 const int qi = lane >> 1, dh = lane & 1;
                 const uint32_t hq = __shfl_sync((2 * QPI == 32) ? 0xffffffffu : ((1u << (2 * QPI)) - 1u), h, qi);
@@ -187,7 +187,20 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     tma_load_3d(sm.q[dh] + qi * Q_BOX_BYTES, &tm_q, dh * 64, r * G,
                                 (int)(p.q_first + (hq >> 8)), &sm.in_full);
             }
-            loaded_tile = tile;
+            if (new_tile) {
+                // K/V buffers are free once the previous item's second MMA has read V.
+                if (n > 0 && !mbar_wait(&sm.o_full, (n - 1) & 1, abort)) {
+                    if (lane == 0) report_async(status, kAsyncTimeout, 0x312);
+                    break;
+                }
+                if (lane == 0) {
+                    tma_load_3d(sm.k[0], &tm_k, 0, r, b * BK, &sm.in_full);
+                    tma_load_3d(sm.k[1], &tm_k, 64, r, b * BK, &sm.in_full);
+                    tma_load_3d(sm.v[0], &tm_v, 0, r, b * BK, &sm.in_full);
+                    tma_load_3d(sm.v[1], &tm_v, 64, r, b * BK, &sm.in_full);
+                }
+                loaded_tile = tile;
+            }
         }
         if (*abort != 0) spin_cycles(200000);
     } else if (warp == 1) {
@@ -204,10 +217,6 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             for (int it = it_lo; it < it_hi; ++it) {
                 const int n = it - it_lo;
                 if (!mbar_wait(&sm.in_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x321); break; }
-                if (n > 0 && !mbar_wait(&sm.epi_done, (n - 1) & 1, abort)) {
-                    report_async(status, kAsyncTimeout, 0x322);
-                    break;
-                }
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(tmem_s, qd0 + 2 * kk, kd0 + 2 * kk, idesc_s, kk > 0);
@@ -217,11 +226,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 if (!mbar_wait(&sm.p_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x323); break; }
                 tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < BK / 16; ++kk) {
-                    // P: K-major, 64 keys per 128-byte row atom; V: 16 keys = 2048 bytes per step.
-                    const uint64_t pd = ((kk >> 2) ? qd1 : qd0) + 2 * (kk & 3);
-                    mma_bf16_ss(tmem_o, pd, vd + (uint64_t)(kk * 2048 / 16), idesc_o, kk > 0);
-                }
+                for (int kk = 0; kk < BK / 16; ++kk)  // P: 8 packed columns per 16 keys; V: 2048 bytes per 16 keys
+                    mma_bf16_ts(tmem_o, tmem_s + kk * 8, vd + (uint64_t)(kk * 2048 / 16), idesc_o, kk > 0);
                 mma_commit(&sm.o_full);
             }
             if (*abort != 0) {
@@ -246,7 +252,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             const int slot = h & 0xFF;
             const int64_t pos = p.q_begin + p.q_first + ql;
             // visible columns of this block for this query: 0..lim
-            int64_t lim64 = pos - (int64_t)b * BK;
+            const int64_t lim64 = pos - (int64_t)b * BK;
             const int lim = valid ? (int)(lim64 > BK - 1 ? BK - 1 : lim64) : BK - 1;
 
             uint32_t sv[BK / 32][32];
@@ -270,28 +276,22 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             }
             const float mc = mx * scale_log2e;
             float ell = 0.f;
-            // P row -> shared memory, K-major, 128-byte swizzle: 16-byte chunk j of row m goes to
-            // chunk (j ^ (m & 7)) of that row.
+            // P row (bf16 pairs) back into the first BK/2 columns of the S region.
 #pragma unroll
-            for (int c = 0; c < BK / 32; ++c) {
+            for (int c2 = 0; c2 < BK / 64; ++c2) {
+                uint32_t pk[32];
 #pragma unroll
-                for (int j4 = 0; j4 < 4; ++j4) {
-                    uint32_t pk[4];
-#pragma unroll
-                    for (int w = 0; w < 4; ++w) {
-                        const float p0 = exp2f(fmaf(__uint_as_float(sv[c][j4 * 8 + 2 * w]), scale_log2e, -mc));
-                        const float p1 = exp2f(fmaf(__uint_as_float(sv[c][j4 * 8 + 2 * w + 1]), scale_log2e, -mc));
-                        ell += p0 + p1;
-                        const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-                        pk[w] = *reinterpret_cast<const uint32_t*>(&pb);
-                    }
-                    const int col = c * 32 + j4 * 8;          // first key of this 16-byte chunk
-                    const int half = col >> 6, j = (col & 63) >> 3;
-                    uint4* dst = reinterpret_cast<uint4*>(sm.q[half] + row * 128 + ((j ^ (row & 7)) << 4));
-                    *dst = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                for (int w = 0; w < 32; ++w) {
+                    const int col = c2 * 64 + 2 * w;
+                    const float p0 = ex2_approx(fmaf(__uint_as_float(sv[col >> 5][col & 31]), scale_log2e, -mc));
+                    const float p1 = ex2_approx(fmaf(__uint_as_float(sv[col >> 5][(col & 31) + 1]), scale_log2e, -mc));
+                    ell += p0 + p1;
+                    const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+                    pk[w] = *reinterpret_cast<const uint32_t*>(&pb);
                 }
+                tmem_st_32x32(tmem_s + lane_base + c2 * 32, pk);
             }
-            fence_proxy_async_smem();
+            tmem_wait_st();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.p_full);
@@ -301,30 +301,31 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tc_fence_after();
             const float inv = 1.0f / ell;
             const int64_t prow = (ql * p.H_kv + r) * (int64_t)p.top_k + slot;
-            __nv_bfloat16* orow = o_buf + (prow * G + g) * 128;
+            // Partial layout inside a (query, group, slot) region of G*256 bytes: [16-byte chunk of d][head],
+            // so the G lanes of one query write G*16 contiguous bytes per store instruction.
+            __nv_bfloat16* oreg = o_buf + prow * (G * 128) + g * 8;
+            uint32_t ov[4][32];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t ov[32];
-                tmem_ld_32x32(tmem_o + lane_base + c * 32, ov);
-                tmem_wait_ld();
-                if (valid) {
+            for (int c = 0; c < 4; ++c) tmem_ld_32x32(tmem_o + lane_base + c * 32, ov[c]);
+            tmem_wait_ld();
+            if (valid) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int j4 = 0; j4 < 4; ++j4) {
                         uint32_t pk[4];
 #pragma unroll
                         for (int w = 0; w < 4; ++w) {
                             const __nv_bfloat162 ob = __floats2bfloat162_rn(
-                                __uint_as_float(ov[j4 * 8 + 2 * w]) * inv, __uint_as_float(ov[j4 * 8 + 2 * w + 1]) * inv);
+                                __uint_as_float(ov[c][j4 * 8 + 2 * w]) * inv,
+                                __uint_as_float(ov[c][j4 * 8 + 2 * w + 1]) * inv);
                             pk[w] = *reinterpret_cast<const uint32_t*>(&ob);
                         }
-                        *reinterpret_cast<uint4*>(orow + c * 32 + j4 * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        *reinterpret_cast<uint4*>(oreg + (c * 4 + j4) * (G * 8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
-                }
             }
             if (valid) lse_buf[prow * G + g] = (mc + log2f(ell)) * 0.6931471805599453f;
             tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.epi_done);
         }
     }
     tc_fence_before();
@@ -336,7 +337,9 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 }
 
 // ---------------------------------------------------------------- 3. combine
-// One CTA per (query, KV head): thread t handles head t/16 and 8 consecutive d elements.
+// One CTA per (query, KV head), G*16 threads.  Partials are stored as [16-byte chunk of d][head]
+// inside each (query, group, slot) region, so thread t reads chunk t/G of head t%G and a warp
+// reads 512 contiguous bytes per slot.
 //   a = max_s LSE_s, LSE = a + log sum_s exp(LSE_s - a), w_s = exp(LSE_s - LSE), O = sum_s w_s O_s.
 template <int BK, int G>
 __global__ void __launch_bounds__(G * 16)
@@ -344,6 +347,7 @@ combine_kernel(const int32_t* __restrict__ block_idx, RangeParams p, const __nv_
                const float* __restrict__ lse_buf, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     __shared__ float w_s[128][G];   // top_k <= 128
     __shared__ int valid_s[128];
+    __shared__ uint4 o_s[G][16];    // final rows, [head][chunk], for a coalesced store
     const int ql = blockIdx.x / p.H_kv, r = blockIdx.x % p.H_kv;
     const int t = threadIdx.x;
     const int64_t q = p.q_first + ql;
@@ -355,9 +359,8 @@ combine_kernel(const int32_t* __restrict__ block_idx, RangeParams p, const __nv_
         valid_s[s] = (b >= 0 && (int64_t)b <= loc) ? 1 : 0;
     }
     __syncthreads();
-    const int g = t >> 4, dc = (t & 15) * 8;
-    {   // 16 threads per head: thread j of a head owns slots j, j+16, ...
-        const int j = t & 15;
+    {   // weights: 16 threads per head, thread j of a head owns slots j, j+16, ...
+        const int g = t >> 4, j = t & 15;
         float lv[8];
         float a = -INFINITY;
 #pragma unroll
@@ -382,14 +385,15 @@ combine_kernel(const int32_t* __restrict__ block_idx, RangeParams p, const __nv_
         if (j == 0 && lse != nullptr) lse[q * (int64_t)(p.H_kv * G) + r * G + g] = L;
     }
     __syncthreads();
+    const int g = t % G, ch = t / G;  // head, 16-byte chunk of d
     float acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-    const __nv_bfloat16* src = o_buf + (pbase * G + g) * 128 + dc;
-#pragma unroll 4
+    const uint4* src = reinterpret_cast<const uint4*>(o_buf + pbase * (G * 128)) + t;
+#pragma unroll 8
     for (int s = 0; s < p.top_k; ++s) {
         if (!valid_s[s]) continue;
-        const uint4 x = __ldg(reinterpret_cast<const uint4*>(src + (int64_t)s * G * 128));
+        const uint4 x = __ldg(src + (int64_t)s * (G * 16));
         const float w = w_s[s][g];
         const float2 a0 = bf16x2_to_float2(x.x), a1 = bf16x2_to_float2(x.y);
         const float2 a2 = bf16x2_to_float2(x.z), a3 = bf16x2_to_float2(x.w);
@@ -404,8 +408,10 @@ combine_kernel(const int32_t* __restrict__ block_idx, RangeParams p, const __nv_
         const __nv_bfloat162 ob = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
         pk[i] = *reinterpret_cast<const uint32_t*>(&ob);
     }
-    *reinterpret_cast<uint4*>(out + (q * (int64_t)(p.H_kv * G) + r * G + g) * 128 + dc) =
-        make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    o_s[g][ch] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    __syncthreads();
+    // out[q, r*G + head, :]: the G rows are contiguous, G*256 bytes = G*16 chunks in order
+    reinterpret_cast<uint4*>(out + (q * (int64_t)(p.H_kv * G) + r * G) * 128)[t] = o_s[t >> 4][t & 15];
 }
 
 }  // namespace msa
