@@ -29,31 +29,36 @@ struct RangeParams {
 };
 
 // ---------------------------------------------------------------- 1. reverse index
-// One thread per (query, group, slot) entry.  pass 0 counts, pass 1 scatters.
+// One warp per (query, group) row of the index list.  Pass 0 counts the queries of every
+// (block, head) tile and remembers each entry's arrival rank within its tile; pass 1 (after
+// the scan) writes the handle to tile_off[tile] + rank without touching the counters again.
 template <int BK>
-__global__ void revidx_kernel(const int32_t* __restrict__ block_idx, RangeParams p, int pass,
-                              int32_t* __restrict__ cnt, const int32_t* __restrict__ tile_off,
-                              uint32_t* __restrict__ handles, int* status) {
-    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t n = (int64_t)p.q_count * p.H_kv * p.top_k;
-    if (e >= n) return;
-    const int s = (int)(e % p.top_k);
-    const int64_t qr = e / p.top_k;
-    const int r = (int)(qr % p.H_kv);
-    const int64_t ql = qr / p.H_kv;
-    const int64_t pos = p.q_begin + p.q_first + ql;
-    const int32_t b = block_idx[((p.q_first + ql) * p.H_kv + r) * (int64_t)p.top_k + s];
-    if (b < 0 || (int64_t)b > pos / BK) {
-        if (b != -1 && pass == 0) report_async(status, kAsyncBadIndex, 0x301);
-        return;
+__global__ void __launch_bounds__(256)
+revidx_kernel(const int32_t* __restrict__ block_idx, RangeParams p, int pass, int32_t* __restrict__ cnt,
+              const int32_t* __restrict__ tile_off, uint32_t* __restrict__ rank,
+              uint32_t* __restrict__ handles, int* status) {
+    const int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= p.q_count * p.H_kv) return;
+    const int ql = row / p.H_kv, r = row - ql * p.H_kv;
+    const int64_t loc = (p.q_begin + p.q_first + ql) / BK;
+    const int32_t* sel = block_idx + ((p.q_first + ql) * (int64_t)p.H_kv + r) * p.top_k;
+    for (int s = lane; s < p.top_k; s += 32) {
+        const int32_t b = sel[s];
+        if (b < 0 || (int64_t)b > loc) {
+            if (b != -1 && pass == 0) report_async(status, kAsyncBadIndex, 0x301);
+            continue;
+        }
+        const int tile = b * p.H_kv + r;
+        const int64_t e = (int64_t)row * p.top_k + s;
+        if (pass == 0)
+            rank[e] = (uint32_t)atomicAdd(&cnt[tile], 1);
+        else
+            handles[tile_off[tile] + rank[e]] = ((uint32_t)ql << 8) | (uint32_t)s;
     }
-    const int tile = b * p.H_kv + r;
-    const int at = atomicAdd(&cnt[tile], 1);
-    if (pass == 1) handles[tile_off[tile] + at] = ((uint32_t)ql << 8) | (uint32_t)s;
 }
 
-// Single-CTA exclusive scan of the tile counts -> pair offsets and item offsets; clears the
-// counters so that the scatter pass can reuse them as cursors.
+// Single-CTA exclusive scan of the tile counts -> pair offsets and item offsets.
 __global__ void __launch_bounds__(1024)
 revidx_scan_kernel(int32_t* __restrict__ cnt, int n_tiles, int qpi, int32_t* __restrict__ tile_off,
                    int32_t* __restrict__ item_off) {
@@ -76,7 +81,6 @@ revidx_scan_kernel(int32_t* __restrict__ cnt, int n_tiles, int qpi, int32_t* __r
         const int c = cnt[i];
         tile_off[i] = po; item_off[i] = io;
         po += c; io += (c + qpi - 1) / qpi;
-        cnt[i] = 0;
     }
     if (t == 1023) { tile_off[n_tiles] = s_pairs[1023]; item_off[n_tiles] = s_items[1023]; }
 }

@@ -1,0 +1,390 @@
+// Decode path (one query per cached sequence): HBM-bound streaming kernels.
+//
+//   index_scores_decode_kernel : Eq. 6 for the last token of every sequence.  One warp per key
+//       block streams the block's K_idx rows straight from global memory into mma.sync
+//       B fragments (no shared memory) and keeps the per-group running maximum.
+//   attn_decode_kernel         : Eq. 8.  Persistent CTAs; a producer warp streams the selected
+//       K/V blocks through a TMA ring in shared memory, four consumer warps each own 32 keys
+//       of every block (S = Q K^T with mma.sync, online softmax in registers, O^T += V^T P^T).
+//   attn_decode_combine_kernel : merges the per-warp partials of a sequence (Section 4.2
+//       combine).
+#pragma once
+
+#include "tc_common.cuh"
+
+namespace msa {
+
+__device__ __forceinline__ void mma_m16n8k16_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                  uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t smem_addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(smem_addr));
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t smem_addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(smem_addr));
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// ------------------------------------------------------------------ stage 1, decode
+// d_idx = 64, H_kv <= 8, any B_k that is a multiple of 8.  A = Q_idx padded to 16 rows.
+// The contraction index is permuted identically in A and B so that a lane's B fragment for
+// two consecutive k-steps is one 16-byte load: within a 32-wide segment of d, lane quad
+// position t owns d[8t..8t+7]; k-step 0 uses d[8t..8t+3], k-step 1 uses d[8t+4..8t+7].
+constexpr int kIdxDecWarps = 8;
+
+template <int UNROLL>
+__global__ void __launch_bounds__(kIdxDecWarps * 32)
+index_scores_decode_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_bfloat16* __restrict__ k_idx,
+                           const int64_t* __restrict__ seq_offsets, const int32_t* __restrict__ seq_lens,
+                           int batch, int H_kv, int B_k, float scale, float* __restrict__ scores,
+                           int64_t ld_scores, int64_t n_cols) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, t = lane & 3;
+    // Global list of (sequence, block) work items, including the -inf tail blocks of short
+    // sequences; dealt to warps round-robin, so neighbouring warps stream neighbouring blocks.
+    const int64_t total = (int64_t)batch * n_cols;
+    const int64_t n_warps = (int64_t)gridDim.x * kIdxDecWarps;
+    int64_t it = (int64_t)blockIdx.x * kIdxDecWarps + warp;
+    const int64_t it_end = total;
+    int cur_seq = -1;
+    uint32_t qa[8];   // A fragments of the current sequence's query: [segment][k-step][lo/hi]
+    int64_t len = 0, base = 0;
+    for (; it < it_end; it += n_warps) {
+        const int s = (int)(it / n_cols);
+        const int64_t b = it - (int64_t)s * n_cols;
+        if (s != cur_seq) {
+            cur_seq = s;
+            len = seq_lens[s];
+            base = seq_offsets[s];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) qa[i] = 0u;
+            if (g < H_kv) {
+                const uint4* qrow = reinterpret_cast<const uint4*>(q_idx + ((int64_t)s * H_kv + g) * 64);
+#pragma unroll
+                for (int seg = 0; seg < 2; ++seg) {
+                    const uint4 v = __ldg(qrow + seg * 4 + t);
+                    qa[seg * 4 + 0] = v.x; qa[seg * 4 + 1] = v.y;  // k-step 0: a0a1, a4a5
+                    qa[seg * 4 + 2] = v.z; qa[seg * 4 + 3] = v.w;  // k-step 1
+                }
+            }
+        }
+        float* out = scores + ((int64_t)s * H_kv) * ld_scores + b;
+        const int64_t j0 = b * B_k;
+        if (j0 >= len) {  // block beyond this sequence: -inf (Eq. 6)
+            if (lane < H_kv) out[(int64_t)lane * ld_scores] = -INFINITY;
+            continue;
+        }
+        const int64_t pos = len - 1;
+        int n_vis = (int)((pos - j0 + 1) < B_k ? (pos - j0 + 1) : B_k);
+        const int n_nt = (n_vis + 7) >> 3;  // 8-key tiles that hold a visible key
+        float best0 = -INFINITY, best1 = -INFINITY;
+        const __nv_bfloat16* kb = k_idx + (base + j0) * 64;
+        for (int nt0 = 0; nt0 < n_nt; nt0 += UNROLL) {
+            uint4 kv[UNROLL][2];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int nt = nt0 + u;
+                // rows past the visible range are clamped (loaded but masked below)
+                int row = nt * 8 + g;
+                if (row > n_vis - 1) row = n_vis - 1;
+                const uint4* krow = reinterpret_cast<const uint4*>(kb + (int64_t)row * 64);
+                kv[u][0] = ldg_stream(krow + t);
+                kv[u][1] = ldg_stream(krow + 4 + t);
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int nt = nt0 + u;
+                if (nt < n_nt) {
+                    float c[4] = {0.f, 0.f, 0.f, 0.f};
+                    mma_m16n8k16_bf16(c, qa[0], 0u, qa[1], 0u, kv[u][0].x, kv[u][0].y);
+                    mma_m16n8k16_bf16(c, qa[2], 0u, qa[3], 0u, kv[u][0].z, kv[u][0].w);
+                    mma_m16n8k16_bf16(c, qa[4], 0u, qa[5], 0u, kv[u][1].x, kv[u][1].y);
+                    mma_m16n8k16_bf16(c, qa[6], 0u, qa[7], 0u, kv[u][1].z, kv[u][1].w);
+                    // c[0], c[1]: group g, keys nt*8 + 2t, +1
+                    const int key = nt * 8 + 2 * t;
+                    if (key < n_vis) best0 = fmaxf(best0, c[0]);
+                    if (key + 1 < n_vis) best1 = fmaxf(best1, c[1]);
+                }
+            }
+        }
+        float best = fmaxf(best0, best1);
+        best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, 1));
+        best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, 2));
+        if (t == 0 && g < H_kv) out[(int64_t)g * ld_scores] = best * scale;
+    }
+}
+
+// ------------------------------------------------------------------ stage 3, decode
+constexpr int kDecStages = 6;
+constexpr int kDecThreads = 160;      // warp 0: TMA producer, warps 1-4: consumers
+constexpr int kDecBlocksPerItem = 8;  // selected blocks streamed by one work item
+constexpr int kDecPartsPerItem = 4;   // one partial per consumer warp
+
+template <int BK>
+struct DecSmem {
+    alignas(1024) uint8_t tile[kDecStages][2][BK * 128];  // [stage][d half][key][64 bf16], 128-byte swizzle
+    alignas(8) uint64_t full[kDecStages];
+    uint64_t empty[kDecStages];
+    int abort;
+};
+
+struct DecParams {
+    const __nv_bfloat16* q;         // [batch, H_q, 128]
+    const int32_t* block_idx;       // [batch, H_kv, top_k]
+    const int64_t* seq_offsets;
+    const int32_t* seq_lens;
+    float* part_o;                  // [items*4, 8, 128]
+    float* part_ml;                 // [items*4, 2, 8]  (running max in log2 units, sum)
+    int batch, H_kv, top_k, n_split;
+    float scale_log2e;
+};
+
+// 16-byte chunk `chunk` (0..15 over d) of key row `key` inside a swizzled K or V tile.
+template <int BK>
+__device__ __forceinline__ uint32_t dec_tile_addr(uint32_t tile_base, int key, int chunk) {
+    return tile_base + (uint32_t)((chunk >> 3) * (BK * 128) + key * 128 + (((chunk & 7) ^ (key & 7)) << 4));
+}
+
+template <int BK>
+__global__ void __launch_bounds__(kDecThreads, 1)
+attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                   DecParams p, int* status) {
+    constexpr int KPW = BK / 4;    // keys per consumer warp
+    constexpr int NT = KPW / 8;    // 8-key score tiles per warp
+    constexpr int KS = KPW / 16;   // 16-key steps of the second product
+    constexpr uint32_t TILE_BYTES = 2 * BK * 128;
+    extern __shared__ uint8_t smem_raw[];
+    DecSmem<BK>& sm = *reinterpret_cast<DecSmem<BK>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int* abort = &sm.abort;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kDecStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 4); }
+        sm.abort = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+    }
+    __syncthreads();
+    const int n_items = p.batch * p.H_kv * p.n_split;
+    const int G = 8;
+    const int H_q = p.H_kv * G;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t sc = 0;  // tiles issued so far
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+                const int u = item / p.n_split, sp = item - u * p.n_split;
+                const int seq = u / p.H_kv, r = u - seq * p.H_kv;
+                const int64_t len = p.seq_lens[seq], base = p.seq_offsets[seq];
+                const int64_t loc = (len - 1) / BK;
+                const int32_t* sel = p.block_idx + (int64_t)u * p.top_k;
+                for (int e = sp * kDecBlocksPerItem; ok && e < min(p.top_k, (sp + 1) * kDecBlocksPerItem); ++e) {
+                    const int32_t b = sel[e];
+                    if (b < 0 || (int64_t)b > loc) {
+                        if (b != -1) report_async(status, kAsyncBadIndex, 0x401);
+                        continue;
+                    }
+                    const int tok = (int)(base + (int64_t)b * BK);
+                    for (int kv = 0; kv < 2; ++kv, ++sc) {
+                        const int st = sc % kDecStages;
+                        if (!mbar_wait(&sm.empty[st], ((sc / kDecStages) & 1) ^ 1, abort)) {
+                            report_async(status, kAsyncTimeout, 0x402);
+                            ok = false;
+                            break;
+                        }
+                        mbar_arrive_expect_tx(&sm.full[st], TILE_BYTES);
+                        const CUtensorMap* tm = kv == 0 ? &tm_k : &tm_v;
+                        tma_load_3d(sm.tile[st][0], tm, 0, r, tok, &sm.full[st]);
+                        tma_load_3d(sm.tile[st][1], tm, 64, r, tok, &sm.full[st]);
+                    }
+                }
+            }
+            if (*abort != 0) spin_cycles(200000);
+        }
+    } else {
+        const int w = warp - 1;
+        const int g = lane >> 2, t = lane & 3;
+        uint32_t sc = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+            const int u = item / p.n_split, sp = item - u * p.n_split;
+            const int seq = u / p.H_kv, r = u - seq * p.H_kv;
+            const int64_t len = p.seq_lens[seq];
+            const int64_t pos = len - 1, loc = pos / BK;
+            const int32_t* sel = p.block_idx + (int64_t)u * p.top_k;
+            // A fragments of Q (rows 0-7 = the 8 heads of the group, rows 8-15 = zero padding)
+            uint32_t qa[8][2];
+            {
+                const __nv_bfloat16* qrow = p.q + ((int64_t)seq * H_q + r * G + g) * 128;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    qa[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * t);
+                    qa[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * t);
+                }
+            }
+            float m_run = -INFINITY, l_part = 0.f;
+            float acc[8][4];
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
+
+            for (int e = sp * kDecBlocksPerItem; ok && e < min(p.top_k, (sp + 1) * kDecBlocksPerItem); ++e) {
+                const int32_t b = sel[e];
+                if (b < 0 || (int64_t)b > loc) continue;
+                // ---- K tile: S[head g][keys of this warp]
+                int st = sc % kDecStages;
+                if (!mbar_wait(&sm.full[st], (sc / kDecStages) & 1, abort)) {
+                    if (lane == 0) report_async(status, kAsyncTimeout, 0x411);
+                    ok = false;
+                    break;
+                }
+                uint32_t tb = smem_u32(sm.tile[st][0]);
+                float c[NT][4];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+                    const int key = w * KPW + nt * 8 + (lane & 7);
+#pragma unroll
+                    for (int kc = 0; kc < 4; ++kc) {
+                        uint32_t r4[4];
+                        ldmatrix_x4(r4, dec_tile_addr<BK>(tb, key, kc * 4 + (lane >> 3)));
+                        mma_m16n8k16_bf16(c[nt], qa[2 * kc][0], 0u, qa[2 * kc][1], 0u, r4[0], r4[1]);
+                        mma_m16n8k16_bf16(c[nt], qa[2 * kc + 1][0], 0u, qa[2 * kc + 1][1], 0u, r4[2], r4[3]);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.empty[st]);
+                ++sc;
+                // ---- online softmax for head g over this warp's keys (values in log2 units)
+                const int lim = (int)(pos - (int64_t)b * BK);  // keys 0..lim of the block are visible
+                float mx = -INFINITY;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int key = w * KPW + nt * 8 + 2 * t;
+                    c[nt][0] = key <= lim ? c[nt][0] * p.scale_log2e : -INFINITY;
+                    c[nt][1] = key + 1 <= lim ? c[nt][1] * p.scale_log2e : -INFINITY;
+                    mx = fmaxf(mx, fmaxf(c[nt][0], c[nt][1]));
+                }
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float m_new = fmaxf(m_run, mx);
+                const float m_use = m_new == -INFINITY ? 0.f : m_new;   // slice fully masked so far
+                const float corr = ex2_approx(m_run - m_use);            // 0 when m_run = -inf
+                uint32_t pb[KS][2];
+                float psum = 0.f;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const float p0 = ex2_approx(c[nt][0] - m_use), p1 = ex2_approx(c[nt][1] - m_use);
+                    psum += p0 + p1;
+                    const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                    pb[nt >> 1][nt & 1] = *reinterpret_cast<const uint32_t*>(&pk);
+                }
+                l_part = l_part * corr + psum;
+                m_run = m_new;
+                const float corr0 = __shfl_sync(0xffffffffu, corr, (2 * t) * 4);
+                const float corr1 = __shfl_sync(0xffffffffu, corr, (2 * t + 1) * 4);
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) {
+                    acc[mt][0] *= corr0; acc[mt][1] *= corr1; acc[mt][2] *= corr0; acc[mt][3] *= corr1;
+                }
+                // ---- V tile: O^T[d][head] += V^T[d][key] P^T[key][head]
+                st = sc % kDecStages;
+                if (!mbar_wait(&sm.full[st], (sc / kDecStages) & 1, abort)) {
+                    if (lane == 0) report_async(status, kAsyncTimeout, 0x412);
+                    ok = false;
+                    break;
+                }
+                tb = smem_u32(sm.tile[st][0]);
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) {
+#pragma unroll
+                    for (int ks = 0; ks < KS; ++ks) {
+                        const int i = lane >> 3;
+                        const int key = w * KPW + ks * 16 + (i >> 1) * 8 + (lane & 7);
+                        uint32_t r4[4];
+                        ldmatrix_x4_trans(r4, dec_tile_addr<BK>(tb, key, mt * 2 + (i & 1)));
+                        mma_m16n8k16_bf16(acc[mt], r4[0], r4[1], r4[2], r4[3], pb[ks][0], pb[ks][1]);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.empty[st]);
+                ++sc;
+            }
+            // ---- partial of this warp: O^T (unnormalised), running max, sum
+            float l = l_part;
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            const int64_t pidx = (int64_t)item * kDecPartsPerItem + w;
+            float* po = p.part_o + pidx * (8 * 128);
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+                const int d0 = mt * 16 + g;
+                po[(2 * t) * 128 + d0] = acc[mt][0];
+                po[(2 * t + 1) * 128 + d0] = acc[mt][1];
+                po[(2 * t) * 128 + d0 + 8] = acc[mt][2];
+                po[(2 * t + 1) * 128 + d0 + 8] = acc[mt][3];
+            }
+            if (t == 0) {
+                p.part_ml[pidx * 16 + g] = m_run;
+                p.part_ml[pidx * 16 + 8 + g] = l;
+            }
+        }
+    }
+}
+
+// One warp per (sequence, head): merges the n_split*4 partials of its (sequence, KV head).
+__global__ void __launch_bounds__(128)
+attn_decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, int batch, int H_kv,
+                           int n_split, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+    const int row = blockIdx.x * 4 + (threadIdx.x >> 5);  // (seq, head)
+    const int lane = threadIdx.x & 31;
+    const int H_q = H_kv * 8;
+    if (row >= batch * H_q) return;
+    const int seq = row / H_q, h = row - seq * H_q;
+    const int r = h >> 3, g = h & 7;
+    const int n_parts = n_split * kDecPartsPerItem;
+    const int64_t p0 = ((int64_t)seq * H_kv + r) * n_parts;
+    float M = -INFINITY;
+    for (int i = lane; i < n_parts; i += 32) M = fmaxf(M, part_ml[(p0 + i) * 16 + g]);
+    M = warp_max(M);
+    float L = 0.f;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int i = 0; i < n_parts; ++i) {
+        const float mi = part_ml[(p0 + i) * 16 + g];
+        if (mi == -INFINITY) continue;
+        const float wgt = exp2f(mi - M);
+        L += wgt * part_ml[(p0 + i) * 16 + 8 + g];
+        const float4 o = *reinterpret_cast<const float4*>(part_o + (p0 + i) * (8 * 128) + g * 128 + lane * 4);
+        acc[0] = fmaf(wgt, o.x, acc[0]); acc[1] = fmaf(wgt, o.y, acc[1]);
+        acc[2] = fmaf(wgt, o.z, acc[2]); acc[3] = fmaf(wgt, o.w, acc[3]);
+    }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    const __nv_bfloat162 o01 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv);
+    const __nv_bfloat162 o23 = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);
+    uint2 pk;
+    pk.x = *reinterpret_cast<const uint32_t*>(&o01);
+    pk.y = *reinterpret_cast<const uint32_t*>(&o23);
+    *reinterpret_cast<uint2*>(out + (int64_t)row * 128 + lane * 4) = pk;
+    if (lse != nullptr && lane == 0) lse[row] = (M + log2f(L)) * 0.6931471805599453f;
+}
+
+}  // namespace msa

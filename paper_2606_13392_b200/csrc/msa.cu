@@ -9,6 +9,7 @@
 #include "topk.cuh"
 #include "index_scores_tc.cuh"
 #include "attn_prefill_tc.cuh"
+#include "decode.cuh"
 
 namespace msa {
 
@@ -234,11 +235,11 @@ static bool attn_tc_supported(const Resolved& r) {
 //   [cnt | tile_off | item_off] int32 per (block, head) tile, handles, LSE_buf, O_buf.
 struct AttnPlan {
     int64_t R;
-    size_t off_cnt, off_tile_off, off_item_off, off_handles, off_lse, off_obuf, total;
+    size_t off_cnt, off_tile_off, off_item_off, off_handles, off_rank, off_lse, off_obuf, total;
 };
 
 static size_t attn_per_query_bytes(const Resolved& r) {
-    return (size_t)r.H_q * r.k * r.d * 2 + (size_t)r.H_q * r.k * 4 + (size_t)r.H_kv * r.k * 4;
+    return (size_t)r.H_q * r.k * r.d * 2 + (size_t)r.H_q * r.k * 4 + (size_t)r.H_kv * r.k * 8;
 }
 
 static AttnPlan attn_plan(const Resolved& r, int64_t kv_len, int64_t R) {
@@ -250,6 +251,7 @@ static AttnPlan attn_plan(const Resolved& r, int64_t kv_len, int64_t R) {
     p.off_tile_off = o; o += align_up(n_tiles * 4);
     p.off_item_off = o; o += align_up(n_tiles * 4);
     p.off_handles = o; o += align_up((size_t)R * r.H_kv * r.k * 4);
+    p.off_rank = o; o += align_up((size_t)R * r.H_kv * r.k * 4);
     p.off_lse = o; o += align_up((size_t)R * r.H_q * r.k * 4);
     p.off_obuf = o; o += align_up((size_t)R * r.H_q * r.k * r.d * 2);
     p.total = o;
@@ -290,6 +292,7 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
     int32_t* tile_off = (int32_t*)(w + pl.off_tile_off);
     int32_t* item_off = (int32_t*)(w + pl.off_item_off);
     uint32_t* handles = (uint32_t*)(w + pl.off_handles);
+    uint32_t* rank = (uint32_t*)(w + pl.off_rank);
     float* lse_buf = (float*)(w + pl.off_lse);
     __nv_bfloat16* o_buf = (__nv_bfloat16*)(w + pl.off_obuf);
 
@@ -322,12 +325,11 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
         p.n_blocks = (int32_t)ceil_div64(q_begin + q_first + p.q_count, BK);
         p.H_kv = r.H_kv; p.top_k = r.k;
         const int n_tiles = p.n_blocks * r.H_kv;
-        const int64_t entries = (int64_t)p.q_count * r.H_kv * r.k;
-        const unsigned eg = (unsigned)ceil_div64(entries, 256);
+        const unsigned eg = (unsigned)ceil_div64((int64_t)p.q_count * r.H_kv, 8);  // 8 warps (rows) per CTA
         if (cudaMemsetAsync(cnt, 0, (size_t)(n_tiles + 1) * 4, st) != cudaSuccess) return MSA_ERR_CUDA;
         {
             StageScope sc(kStageSchedule, st);
-            revidx_kernel<BK><<<eg, 256, 0, st>>>(block_idx, p, 0, cnt, tile_off, handles, status);
+            revidx_kernel<BK><<<eg, 256, 0, st>>>(block_idx, p, 0, cnt, tile_off, rank, handles, status);
         }
         {
             StageScope sc(kStageSchedule, st);
@@ -335,7 +337,7 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
         }
         {
             StageScope sc(kStageSchedule, st);
-            revidx_kernel<BK><<<eg, 256, 0, st>>>(block_idx, p, 1, cnt, tile_off, handles, status);
+            revidx_kernel<BK><<<eg, 256, 0, st>>>(block_idx, p, 1, cnt, tile_off, rank, handles, status);
         }
         {
             StageScope sc(kStageAttn, st);
@@ -350,6 +352,71 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
         if (cudaPeekAtLastError() != cudaSuccess) return MSA_ERR_CUDA;
     }
     return MSA_OK;
+}
+
+// ---------------------------------------------------------------------- decode path
+static bool index_decode_fast(const Resolved& r) { return r.d_idx == 64 && r.H_kv <= 8; }
+
+static msa_status_t run_index_decode(const Resolved& r, const void* q_idx, const void* k_idx_cache,
+                                     const int64_t* seq_offsets, const int32_t* seq_lens, int batch,
+                                     int64_t n_cols, float* scores, int64_t ld_scores, cudaStream_t st) {
+    const int grid = sm_count() * 4;
+    StageScope sc(kStageIndexDecode, st);
+    index_scores_decode_kernel<8><<<grid, kIdxDecWarps * 32, 0, st>>>(
+        (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx_cache, seq_offsets, seq_lens, batch, r.H_kv,
+        r.B_k, r.index_scale, scores, ld_scores, n_cols);
+    return launch_status();
+}
+
+static bool attn_decode_fast(const Resolved& r) { return r.d == 128 && r.G == 8 && (r.B_k == 64 || r.B_k == 128); }
+
+static int decode_n_split(const Resolved& r) { return (r.k + kDecBlocksPerItem - 1) / kDecBlocksPerItem; }
+
+static size_t decode_ws_bytes(const Resolved& r, int batch) {
+    const size_t parts = (size_t)batch * r.H_kv * decode_n_split(r) * kDecPartsPerItem;
+    return align_up(parts * 8 * 128 * 4) + align_up(parts * 16 * 4) + kAlign;
+}
+
+template <int BK>
+static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const void* k_cache, const void* v_cache,
+                                       int64_t cache_tokens, const int64_t* seq_offsets, const int32_t* seq_lens,
+                                       int batch, const int32_t* block_idx, void* out, float* lse, void* ws,
+                                       cudaStream_t st) {
+    CUtensorMap tm_k, tm_v;
+    const uint64_t kd[3] = {128, (uint64_t)r.H_kv, (uint64_t)cache_tokens};
+    const uint64_t ks[2] = {256, (uint64_t)r.H_kv * 256};
+    const uint32_t kb[3] = {64, 1, (uint32_t)BK};
+    if (!encode_tmap_bf16(&tm_k, k_cache, 3, kd, ks, kb) || !encode_tmap_bf16(&tm_v, v_cache, 3, kd, ks, kb))
+        return MSA_ERR_CUDA;
+    int* status = async_status_ptr();
+    if (status == nullptr) return MSA_ERR_CUDA;
+    const size_t smem = sizeof(DecSmem<BK>) + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(attn_decode_kernel<BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+            cudaSuccess)
+            return MSA_ERR_CUDA;
+        attr_set = true;
+    }
+    DecParams p;
+    p.q = (const __nv_bfloat16*)q; p.block_idx = block_idx; p.seq_offsets = seq_offsets; p.seq_lens = seq_lens;
+    p.batch = batch; p.H_kv = r.H_kv; p.top_k = r.k; p.n_split = decode_n_split(r);
+    p.scale_log2e = r.softmax_scale * 1.4426950408889634f;
+    const size_t parts = (size_t)batch * r.H_kv * p.n_split * kDecPartsPerItem;
+    p.part_o = (float*)ws;
+    p.part_ml = (float*)((char*)ws + align_up(parts * 8 * 128 * 4));
+    const int n_items = batch * r.H_kv * p.n_split;
+    const int grid = n_items < sm_count() ? n_items : sm_count();
+    {
+        StageScope sc(kStageAttnDecode, st);
+        attn_decode_kernel<BK><<<grid, kDecThreads, smem, st>>>(tm_k, tm_v, p, status);
+    }
+    {
+        StageScope sc(kStageCombineDecode, st);
+        attn_decode_combine_kernel<<<(batch * r.H_q + 3) / 4, 128, 0, st>>>(p.part_o, p.part_ml, batch, r.H_kv,
+                                                                             p.n_split, (__nv_bfloat16*)out, lse);
+    }
+    return launch_status();
 }
 
 }  // namespace msa
@@ -446,6 +513,9 @@ msa_status_t msa_index_scores_decode(const msa_shape_t* shape, const void* q_idx
         !aligned16(k_idx_cache) || !aligned16(scores))
         return MSA_ERR_INVALID_ARG;
     if (ld_scores < ceil_div64(max_seq_len, r.B_k) || ld_scores % 4 != 0) return MSA_ERR_INVALID_ARG;
+    if (index_decode_fast(r))
+        return run_index_decode(r, q_idx, k_idx_cache, seq_offsets, seq_lens, batch,
+                                ceil_div64(max_seq_len, r.B_k), scores, ld_scores, (cudaStream_t)stream);
     return run_index_scores(r, q_idx, k_idx_cache, decode_rows(seq_offsets, seq_lens, max_seq_len, r.B_k),
                             batch, scores, ld_scores, (cudaStream_t)stream);
 }
@@ -587,7 +657,7 @@ msa_status_t msa_sparse_attn_decode_workspace_bytes(const msa_shape_t* shape, in
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
     if (batch < 0) return MSA_ERR_INVALID_ARG;
-    if (min_bytes) *min_bytes = kAlign;
+    if (min_bytes) *min_bytes = attn_decode_fast(r) ? decode_ws_bytes(r, batch) : kAlign;
     return MSA_OK;
 }
 
@@ -606,7 +676,14 @@ msa_status_t msa_sparse_attn_decode(const msa_shape_t* shape, const void* q, con
         return MSA_ERR_INVALID_ARG;
     size_t need = 0;
     msa_sparse_attn_decode_workspace_bytes(shape, batch, &need);
-    if (workspace == nullptr || workspace_bytes < need) return MSA_ERR_WORKSPACE;
+    if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
+    if (attn_decode_fast(r) && cache_tokens < 2147483647LL) {
+        if (r.B_k == 64)
+            return run_attn_decode_tc<64>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch,
+                                          block_idx, out, lse, workspace, (cudaStream_t)stream);
+        return run_attn_decode_tc<128>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch,
+                                       block_idx, out, lse, workspace, (cudaStream_t)stream);
+    }
     return run_attn_generic(r, q, k_cache, v_cache, block_idx, decode_rows(seq_offsets, seq_lens, 0, r.B_k),
                             batch, out, lse, (cudaStream_t)stream);
 }

@@ -22,6 +22,12 @@ __device__ __forceinline__ uint64_t topk_key(float s, uint32_t block) {
     return ((uint64_t)u << 32) | (uint32_t)(~block);
 }
 
+// Score part of a key, back as a float (inverse of the order-preserving image).
+__device__ __forceinline__ float topk_key_score(uint64_t key) {
+    const uint32_t u = (uint32_t)(key >> 32);
+    return __uint_as_float((u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u);
+}
+
 __device__ __forceinline__ uint64_t shfl_xor_u64(uint64_t v, int m) {
     return __shfl_xor_sync(0xffffffffu, v, m);
 }
@@ -93,7 +99,7 @@ __global__ void __launch_bounds__(kTopkWarps * 32)
 topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap rows,
                    int64_t n_rows, int H_kv, int B_k, int top_k, int32_t* __restrict__ block_idx) {
     constexpr int KCAP = 32 * R;
-    constexpr int STG = KCAP < 64 ? 64 : KCAP;
+    constexpr int STG = 160;  // flush threshold (32) + one round of four pushes (4 x 32)
     __shared__ uint64_t stg_all[kTopkWarps][STG];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * kTopkWarps + warp;
@@ -115,7 +121,10 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
     uint64_t kept[R];
 #pragma unroll
     for (int s = 0; s < R; ++s) kept[s] = 0;  // 0 is below every real key
-    uint64_t tau = 0;
+    // The stream is filtered on the fp32 score alone (score >= score of the current (k-1)-th
+    // best, -inf while fewer than k-1 are kept); the 64-bit key is only built for survivors and
+    // the exact order, ties included, is settled in the merges.
+    float tau_f = -INFINITY;
     int cnt = 0;
 
     auto flush = [&]() {
@@ -131,41 +140,42 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
             merge_top<R>(kept, nw, lane);
         }
         cnt = 0;
-        tau = element_at<R>(kept, m - 1);
+        const uint64_t tau = element_at<R>(kept, m - 1);
+        tau_f = tau != 0 ? topk_key_score(tau) : -INFINITY;
         __syncwarp();
     };
-    auto push = [&](uint64_t key, bool pass) {
+    // Appends the passing lanes' keys to the staging buffer (no flush inside: the buffer has
+    // room for a whole round of four pushes beyond the flush threshold).
+    auto push = [&](float x, uint32_t block, bool pass) {
         const unsigned mask = __ballot_sync(0xffffffffu, pass);
-        if (mask != 0u) {
-            if (pass) stg[cnt + __popc(mask & lt_mask)] = key;
-            cnt += __popc(mask);
-            if (cnt > STG - 32) flush();
-        }
+        if (pass) stg[cnt + __popc(mask & lt_mask)] = topk_key(x, block);
+        cnt += __popc(mask);
     };
 
     const int64_t n4 = loc >> 2;
     const float4* srow4 = reinterpret_cast<const float4*>(srow);
+    float4 nxt = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (lane < n4) nxt = __ldg(srow4 + lane);
     for (int64_t v0 = 0; v0 < n4; v0 += 32) {
         const int64_t vi = v0 + lane;
         const bool in = vi < n4;
-        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (in) x = __ldg(srow4 + vi);
-        const uint32_t b0 = (uint32_t)(vi << 2);
-        const uint64_t k0 = topk_key(x.x, b0), k1 = topk_key(x.y, b0 + 1);
-        const uint64_t k2 = topk_key(x.z, b0 + 2), k3 = topk_key(x.w, b0 + 3);
-        const bool p0 = in && k0 > tau, p1 = in && k1 > tau, p2 = in && k2 > tau, p3 = in && k3 > tau;
+        const float4 x = nxt;
+        if (vi + 32 < n4) nxt = __ldg(srow4 + vi + 32);  // next round's load is in flight while this one is ranked
+        const bool p0 = in && x.x >= tau_f, p1 = in && x.y >= tau_f;
+        const bool p2 = in && x.z >= tau_f, p3 = in && x.w >= tau_f;
         if (__ballot_sync(0xffffffffu, p0 | p1 | p2 | p3) == 0u) continue;
-        // tau may rise between the pushes; a stale pass only costs a slot in the staging area
-        push(k0, p0);
-        push(k1, p1 && k1 > tau);
-        push(k2, p2 && k2 > tau);
-        push(k3, p3 && k3 > tau);
+        const uint32_t b0 = (uint32_t)(vi << 2);
+        push(x.x, b0, p0);
+        push(x.y, b0 + 1, p1);
+        push(x.z, b0 + 2, p2);
+        push(x.w, b0 + 3, p3);
+        if (cnt > 32) flush();
     }
     {
         const int64_t idx = (n4 << 2) + lane;  // scalar tail (< 4 elements)
         const bool in = idx < loc;
-        const uint64_t key = in ? topk_key(__ldg(srow + idx), (uint32_t)idx) : 0;
-        push(key, in && key > tau);
+        const float x = in ? __ldg(srow + idx) : 0.f;
+        push(x, (uint32_t)idx, in && x >= tau_f);
     }
     if (cnt > 0) flush();
 
