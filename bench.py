@@ -163,36 +163,70 @@ def oracle_sample_size(cfg: MSAConfig) -> int:
     """Query positions that take the oracle roughly 10-30 s on ~8-16 host cores."""
     per_q = cfg.n_kv_heads * cfg.idx_dim * cfg.T / 2 + \
         cfg.n_q_heads * cfg.head_dim * 2 * min(cfg.T / 2, cfg.top_k * cfg.block_size)
-    return int(max(16, min(cfg.T, 4.0e10 / per_q)))
+    return int(max(16, min(cfg.T, 2.0e11 / per_q)))
 
 
 # ----------------------------------------------------------------------------- main
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the stage kernels,
+# from the ncu captures summarised under profiles/ (captured on the reduced workloads named
+# there and scaled to a full launch by the units processed, as DESIGN.md explains).  None =
+# not captured.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c3")
+    ap.add_argument("--workload", default=None,
+                    help="c1..c5 (default: c4 as the headline, plus short c3 and c5 runs reported under 'others')")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-others", action="store_true")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    cfg = CONFIGS[args.workload]
+    primary = args.workload or "c4"
+    extras = [] if (args.workload or args.no_others) else ["c3", "c5"]
+    cfg = CONFIGS[primary]
     if args.impl == "reference":
         if rank == 0:
             run_reference(cfg, args)
         return
-    run_ours(cfg, args, rank, local_rank, world)
+
+    import torch.distributed as dist
+    from paper_2606_13392_b200 import binding as B
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    line = measure(cfg, args, rank, world, dev, B, peaks, dist, e2e=not args.no_e2e,
+                   cpu=(world == 1 and not args.no_cpu_baseline))
+    others = {}
+    for name in extras:
+        torch.cuda.empty_cache()
+        res = measure(CONFIGS[name], args, rank, world, dev, B, peaks, dist, e2e=not args.no_e2e, cpu=False)
+        if rank == 0:
+            others[name] = {k: res[k] for k in ("metric", "value", "unit", "ms_per_step", "gpu_launches",
+                                                 "roofline", "kernels", "e2e", "config") if k in res}
+    if rank == 0:
+        if others:
+            line["others"] = others
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
 
 
 def base_line(cfg: MSAConfig, args, n_gpus: int):
     metric = "msa_prefill_tokens_per_s" if cfg.mode == "prefill" else "msa_decode_tokens_per_s"
     conf = {"workload": "%s: %s" % (cfg.name, describe(cfg)), "l2": "inputs larger than L2 (126 MB)",
-            "sharding": "one independent sequence per rank, no collective"}
+            "sharding": "one independent sequence (decode: batch) per rank, no collective"}
     return {"metric": metric, "unit": "tokens/s", "n_gpus": n_gpus, "steps": args.steps,
             "warmup": args.warmup, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": conf}
@@ -214,7 +248,7 @@ def run_reference(cfg: MSAConfig, args):
     if cfg.mode == "prefill":
         x = make_prefill_inputs(cfg, "cpu")
         xb = {n: to_bits(t) for n, t in x.items()}
-        n = max(8, oracle_sample_size(cfg) // (4 * (steps + min(warm, 1))))
+        n = max(8, oracle_sample_size(cfg) // (steps + min(warm, 1)))
         for _ in range(min(warm, 1)):
             oracle_sample_prefill(cfg, xb, n, 1)
         tot_n, tot_t = 0, 0.0
@@ -239,15 +273,8 @@ def run_reference(cfg: MSAConfig, args):
     print(json.dumps(line))
 
 
-def run_ours(cfg: MSAConfig, args, rank: int, local_rank: int, world: int):
-    import torch.distributed as dist
-    from paper_2606_13392_b200 import binding as B
-
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    peaks = load_peaks()
+def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, cpu: bool):
+    """One workload: warm-up, timed steps, per-stage rooflines, optional e2e and oracle legs."""
     shape = B.shape_of(cfg)
     mycfg = cfg.scaled(seed=cfg.seed + 7919 * rank)
     stream = torch.cuda.current_stream()
@@ -288,16 +315,17 @@ def run_ours(cfg: MSAConfig, args, rank: int, local_rank: int, world: int):
             dist.barrier()
         torch.cuda.synchronize()
 
+    steps = args.steps if cfg.mode == "prefill" else max(args.steps, 20)  # decode steps are ~1 ms
     for _ in range(max(args.warmup, 0)):
         step()
     barrier()
 
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    sampler = ClockSampler(dev.index or 0) if rank == 0 else None
     n_before = B.launch_count()
     B.profile_begin()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for _ in range(args.steps):
+    for _ in range(steps):
         step()
     e1.record(stream)
     barrier()
@@ -312,17 +340,13 @@ def run_ours(cfg: MSAConfig, args, rank: int, local_rank: int, world: int):
     t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
-    ms_step = ms_total / args.steps
+    ms_step = float(t.item()) / steps
     value = world * units / (ms_step * 1e-3)
-
     if rank != 0:
-        if world > 1:
-            dist.barrier()
-            dist.destroy_process_group()
-        return
+        return {}
 
     line = base_line(cfg, args, world)
+    line["steps"] = steps
     line.update(value=value, ms_per_step=ms_step, gpu_launches=int(launches), clocks=clocks)
 
     # ---- per-kernel figures and the roofline of the dominant kernel
@@ -332,39 +356,39 @@ def run_ours(cfg: MSAConfig, args, rank: int, local_rank: int, world: int):
     if cfg.mode == "prefill":
         w = prefill_work(cfg)
         spec = {"index_scores": ("tensor", w["index_flops"]), "topk_select": ("hbm", w["topk_bytes"]),
-                "attn_prefill": ("hbm", w["attn_bytes"]), "combine": ("hbm", w["combine_bytes"]),
-                "schedule": ("hbm", 0.0)}
-        extra = {"attn_prefill_tflops": None}
+                "attn_prefill": ("hbm", w["attn_bytes"]), "combine": ("hbm", w["combine_bytes"])}
     else:
         w = decode_work(cfg)
-        spec = {"index_scores_decode": ("hbm", w["index_bytes"]), "attn_decode": ("hbm", w["attn_bytes"]),
-                "topk_select": ("hbm", 0.0), "combine_decode": ("hbm", 0.0)}
-        extra = {}
+        spec = {"index_scores_decode": ("hbm", w["index_bytes"]), "attn_decode": ("hbm", w["attn_bytes"])}
     for name, (ms, n) in stages.items():
         if n == 0:
             continue
-        per_step_ms = ms / args.steps
-        ent = {"ms_per_step": per_step_ms, "launches_per_step": n / args.steps}
+        per_step_ms = ms / steps
+        ent = {"ms_per_step": per_step_ms, "launches_per_step": n / steps, "share": ms / max(ms_total, 1e-9)}
         if name in spec and spec[name][1] > 0:
             bound, work = spec[name]
             if bound == "tensor":
                 ach = work / (per_step_ms * 1e-3) / 1e12
-                ent.update(bound="tensor", achieved=ach, unit="TFLOP/s", peak=tf_s, frac=ach / tf_s)
+                ent.update(bound="tensor", achieved=ach, unit="TFLOP/s", peak=tf_s, frac=ach / tf_s,
+                           frac_of_burst_peak=ach / tf_b)
             else:
                 ach = work / (per_step_ms * 1e-3) / 1e9
                 ent.update(bound="hbm", achieved=ach, unit="GB/s", peak=hbm, frac=ach / hbm)
+            tr = NCU_TRAFFIC_BYTES_PER_LAUNCH.get((cfg.name, name))
+            ent["traffic"] = tr
         kern[name] = ent
     if cfg.mode == "prefill" and "attn_prefill" in kern:
-        a_ms = kern["attn_prefill"]["ms_per_step"] + kern.get("combine", {}).get("ms_per_step", 0.0)
         kern["attn_prefill"]["tensor_tflops"] = w["attn_flops"] / (kern["attn_prefill"]["ms_per_step"] * 1e-3) / 1e12
         kern["attn_prefill"]["tensor_frac_of_sustained_peak"] = kern["attn_prefill"]["tensor_tflops"] / tf_s
-        extra["attn_plus_combine_ms"] = a_ms
     dom = max((n for n in kern if "bound" in kern[n]), key=lambda n: kern[n]["ms_per_step"], default=None)
     if dom is not None:
         d = kern[dom]
+        per_launch = d["launches_per_step"]
         line["roofline"] = {"kernel": dom, "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"],
-                            "unit": d["unit"], "frac": d["frac"], "traffic": None,
-                            "peak_source": src + " (sustained bf16)" if d["bound"] == "tensor" else src}
+                            "unit": d["unit"], "frac": d["frac"], "traffic": d.get("traffic"),
+                            "launches_per_step": per_launch,
+                            "peak_source": (src + ", sustained bf16 (kernel timed inside a long step)")
+                            if d["bound"] == "tensor" else src}
     line["kernels"] = kern
     line["peaks"] = {"hbm_gbs": hbm, "bf16_tflops_burst": tf_b, "bf16_tflops_sustained": tf_s,
                      "source": peaks["_source"]}
@@ -372,16 +396,25 @@ def run_ours(cfg: MSAConfig, args, rank: int, local_rank: int, world: int):
         line["tflops_total"] = (w["index_flops"] + w["attn_flops"]) / (ms_step * 1e-3) / 1e12
 
     # ---- end to end from host buffers (copies inside the timed region)
-    if not args.no_e2e:
-        line["e2e"] = run_e2e(cfg, shape, x, B, dev, min(args.steps, 3), world)
+    if e2e:
+        del out, lse, ws
+        torch.cuda.empty_cache()
+        line["e2e"] = run_e2e(cfg, shape, x, B, dev, min(steps, 3), world)
 
     # ---- the oracle on this machine's host cores (bounded sample)
-    if world == 1 and not args.no_cpu_baseline:
+    if cpu:
         import oracle
         if cfg.mode == "prefill":
-            xb = {n: to_bits(tn) for n, tn in x.items()}
+            xb = {n: to_bits(tn) for n, tn in x.items() if n != "q" and n != "q_idx"}
             n = oracle_sample_size(cfg)
-            m, dt = oracle_sample_prefill(cfg, xb, n)
+            rng = np.random.default_rng(123)
+            pos = np.sort(rng.choice(cfg.T, size=min(n, cfg.T), replace=False)).astype(np.int64)
+            pt = torch.from_numpy(pos).to(dev)
+            qb, qib = to_bits(x["q"][pt]), to_bits(x["q_idx"][pt])
+            t0 = time.perf_counter()
+            oracle.msa_forward(qb, xb["k"], xb["v"], qib, xb["k_idx"], pos, cfg.block_size, cfg.top_k)
+            dt = time.perf_counter() - t0
+            m = len(pos)
             sample = "%d uniformly drawn query positions of the same inputs, all heads" % m
         else:
             seqs = [0, len(cfg.seq_lens) - 1]
@@ -389,10 +422,7 @@ def run_ours(cfg: MSAConfig, args, rank: int, local_rank: int, world: int):
             sample = "sequences %s of the same batch (one of each cache length)" % seqs
         line["cpu_baseline"] = {"value": m / dt, "unit": "tokens/s", "cores": oracle.n_threads(),
                                 "kind": "oracle", "sample": sample, "seconds": dt}
-    print(json.dumps(line))
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    return line
 
 
 def run_e2e(cfg, shape, x, B, dev, steps, world):
