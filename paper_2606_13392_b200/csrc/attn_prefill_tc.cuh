@@ -263,23 +263,18 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
             for (int c = 0; c < BK / 32; ++c) tmem_ld_32x32(tmem_s + lane_base + c * 32, sv[c]);
             tmem_wait_ld();
-            float mx = -INFINITY;
-            if (lim == BK - 1) {
+            if (lim != BK - 1) {
 #pragma unroll
                 for (int c = 0; c < BK / 32; ++c)
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(sv[c][e]));
-            } else {
-#pragma unroll
-                for (int c = 0; c < BK / 32; ++c)
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) {
+                    for (int e = 0; e < 32; ++e)
                         if (c * 32 + e > lim) sv[c][e] = 0xFF800000u;  // -inf
-                        mx = fmaxf(mx, __uint_as_float(sv[c][e]));
-                    }
             }
+            float mx = tree_max32(sv[0]);
+#pragma unroll
+            for (int c = 1; c < BK / 32; ++c) mx = fmaxf(mx, tree_max32(sv[c]));
             const float mc = mx * scale_log2e;
-            float ell = 0.f;
+            float ell4[4] = {0.f, 0.f, 0.f, 0.f};
             // P row (bf16 pairs) back into the first BK/2 columns of the S region.
 #pragma unroll
             for (int c2 = 0; c2 < BK / 64; ++c2) {
@@ -289,12 +284,13 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     const int col = c2 * 64 + 2 * w;
                     const float p0 = ex2_approx(fmaf(__uint_as_float(sv[col >> 5][col & 31]), scale_log2e, -mc));
                     const float p1 = ex2_approx(fmaf(__uint_as_float(sv[col >> 5][(col & 31) + 1]), scale_log2e, -mc));
-                    ell += p0 + p1;
+                    ell4[w & 3] += p0 + p1;
                     const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
                     pk[w] = *reinterpret_cast<const uint32_t*>(&pb);
                 }
                 tmem_st_32x32(tmem_s + lane_base + c2 * 32, pk);
             }
+            const float ell = (ell4[0] + ell4[1]) + (ell4[2] + ell4[3]);
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();

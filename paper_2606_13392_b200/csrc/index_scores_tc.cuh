@@ -141,22 +141,16 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             float best[NB];
 #pragma unroll
             for (int i = 0; i < NB; ++i) best[i] = -INFINITY;
-            if (!need_mask) {
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        best[(c * 32 + e) / BK] = fmaxf(best[(c * 32 + e) / BK], __uint_as_float(v[c][e]));
-            } else {
+            if (need_mask) {
                 const int lim = (int)(pos - key0);  // columns 0..lim are visible (may be negative)
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const float x = (c * 32 + e <= lim) ? __uint_as_float(v[c][e]) : -INFINITY;
-                        best[(c * 32 + e) / BK] = fmaxf(best[(c * 32 + e) / BK], x);
-                    }
+                    for (int e = 0; e < 32; ++e)
+                        if (c * 32 + e > lim) v[c][e] = 0xFF800000u;  // -inf
             }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) best[(c * 32) / BK] = fmaxf(best[(c * 32) / BK], tree_max32(v[c]));
             if (valid_row) {
 #pragma unroll
                 for (int i = 0; i < NB; ++i) {
