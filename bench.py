@@ -231,6 +231,20 @@ def main():
         dist.destroy_process_group()
 
 
+def rank_seed(seed: int, rank: int) -> int:
+    """Every rank draws its own independent sequence: no data is shared between ranks."""
+    return seed + 7919 * rank
+
+
+def aggregate(ms_total_local: float, steps: int, units: int, world: int, device, dist):
+    """MAX over ranks of the timed duration -> (ms per step, whole-job units per second)."""
+    t = torch.tensor([ms_total_local], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / steps
+    return ms_step, world * units / (ms_step * 1e-3)
+
+
 def base_line(cfg: MSAConfig, args, n_gpus: int):
     metric = "msa_prefill_tokens_per_s" if cfg.mode == "prefill" else "msa_decode_tokens_per_s"
     conf = {"workload": "%s: %s" % (cfg.name, describe(cfg)), "l2": "inputs larger than L2 (126 MB)",
@@ -284,7 +298,7 @@ def run_reference(cfg: MSAConfig, args):
 def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, cpu: bool):
     """One workload: warm-up, timed steps, per-stage rooflines, optional e2e and oracle legs."""
     shape = B.shape_of(cfg)
-    mycfg = cfg.scaled(seed=cfg.seed + 7919 * rank)
+    mycfg = cfg.scaled(seed=rank_seed(cfg.seed, rank))
     stream = torch.cuda.current_stream()
 
     if cfg.mode == "prefill":
@@ -345,11 +359,7 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
     if code != 0:
         raise RuntimeError("device status %d (detail %d) after the timed region" % (code, detail))
 
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / steps
-    value = world * units / (ms_step * 1e-3)
+    ms_step, value = aggregate(ms_total, steps, units, world, dev, dist)
     if rank != 0:
         return {}
 
