@@ -151,6 +151,9 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
     if (warp == 0) {
         // ---------------- producer: walks the item list, gathers Q rows, loads K/V tiles
+        // Tile metadata lives in registers and is refreshed only when the walk crosses into the
+        // next tile; an item's handles follow the previous item's in memory (the handle array is
+        // laid out tile after tile), so the next item's handles are fetched one item ahead.
         int tile = 0;
         if (it_lo < it_hi) {  // last tile whose first item is <= it_lo (skips empty tiles)
             int lo = 0, hi = n_tiles;
@@ -160,15 +163,29 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             }
             tile = lo;
         }
+        int i_next = 0, p_end = 0, first = 0;
+        const int handles_end = tile_off[n_tiles];
+        if (it_lo < it_hi) {
+            i_next = item_off[tile + 1]; p_end = tile_off[tile + 1];
+            first = tile_off[tile] + (it_lo - item_off[tile]) * QPI;
+        }
+        uint32_t h_next = 0;
+        if (it_lo < it_hi && first + lane < handles_end) h_next = handles[first + lane];
         int loaded_tile = -1;
         for (int it = it_lo; it < it_hi; ++it) {
             const int n = it - it_lo;
-            while (item_off[tile + 1] <= it) ++tile;
+            while (i_next <= it) {  // crossed into the next non-empty tile
+                ++tile;
+                i_next = item_off[tile + 1];
+                p_end = tile_off[tile + 1];
+            }
             const int b = tile / p.H_kv, r = tile % p.H_kv;
-            const int first = tile_off[tile] + (it - item_off[tile]) * QPI;
-            const int nq = min(QPI, tile_off[tile + 1] - first);
-            uint32_t h = 0;
-            if (lane < nq) h = handles[first + lane];
+            const int nq = min(QPI, p_end - first);
+            const uint32_t h = lane < nq ? h_next : 0u;
+            {
+                const int nf = first + nq;  // the next item's handles start where this item's end
+                h_next = (it + 1 < it_hi && nf + lane < handles_end) ? handles[nf + lane] : 0u;
+            }
             // The Q buffer is free once the previous item's first MMA has read it.
             if (n > 0 && !mbar_wait(&sm.s_full, (n - 1) & 1, abort)) {
                 if (lane == 0) report_async(status, kAsyncTimeout, 0x311);
@@ -205,6 +222,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 }
                 loaded_tile = tile;
             }
+            first += nq;
         }
         if (*abort != 0) spin_cycles(200000);
     } else if (warp == 1) {
