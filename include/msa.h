@@ -202,9 +202,13 @@ msa_status_t msa_prefill_forward_workspace_bytes(const msa_shape_t* shape, int64
 
 /*
  * Same, from HOST buffers: copies q, k, v, q_idx, k_idx host->device into the staging
- * area at the front of `workspace`, runs msa_prefill_forward, copies `out` (and lse,
- * block_idx when non-NULL) back, and synchronises `stream` before returning.  Host
- * buffers should be page-locked for the copies to run at full rate.
+ * area at the front of `workspace`, runs the three stages, copies `out` (and lse,
+ * block_idx when non-NULL) back, and synchronises before returning.  The copies run on a
+ * second stream owned by the library (created on first use) and overlap the kernels: the
+ * index inputs are uploaded first so that stages 1-2 start while Q, K and V are still in
+ * flight, and each finished query range of the output is copied back while the next one is
+ * computed.  Host buffers should be page-locked for the copies to run at full rate and to
+ * overlap at all.
  * workspace >= msa_prefill_forward_host_workspace_bytes.
  */
 msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_host,

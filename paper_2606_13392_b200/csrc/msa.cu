@@ -3,6 +3,7 @@
 #include <atomic>
 #include <cstdio>
 #include <cstring>
+#include <cstdlib>
 
 #include "common.cuh"
 #include "generic.cuh"
@@ -279,6 +280,48 @@ static int sm_count() {
     return n;
 }
 
+// Copy-out hook used by msa_prefill_forward_host: after each query range is combined, its
+// rows of O (and LSE) are copied to host memory on a second stream while the next range runs.
+struct HostOutHook {
+    bool on = false;
+    cudaStream_t copy = nullptr;
+    char* out_host = nullptr;
+    float* lse_host = nullptr;
+    int64_t rows_copied = 0;
+};
+static HostOutHook g_out_hook;
+
+static cudaEvent_t next_sync_event() {
+    constexpr int kPool = 2048;
+    static cudaEvent_t pool[kPool];
+    static int created = 0, cursor = 0;
+    if (created < kPool && cursor == created) {
+        if (cudaEventCreateWithFlags(&pool[created], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        ++created;
+    }
+    cudaEvent_t e = pool[cursor];
+    cursor = (cursor + 1) % kPool;
+    return e;
+}
+
+static msa_status_t hook_copy_rows(const Resolved& r, const void* out, const float* lse, int64_t row0,
+                                   int64_t rows, cudaStream_t st) {
+    HostOutHook& h = g_out_hook;
+    cudaEvent_t e = next_sync_event();
+    if (e == nullptr || cudaEventRecord(e, st) != cudaSuccess || cudaStreamWaitEvent(h.copy, e, 0) != cudaSuccess)
+        return MSA_ERR_CUDA;
+    const size_t rb = (size_t)r.H_q * r.d * 2;
+    if (cudaMemcpyAsync(h.out_host + (size_t)row0 * rb, (const char*)out + (size_t)row0 * rb, (size_t)rows * rb,
+                        cudaMemcpyDeviceToHost, h.copy) != cudaSuccess)
+        return MSA_ERR_CUDA;
+    if (h.lse_host && lse &&
+        cudaMemcpyAsync(h.lse_host + row0 * r.H_q, lse + row0 * r.H_q, (size_t)rows * r.H_q * 4,
+                        cudaMemcpyDeviceToHost, h.copy) != cudaSuccess)
+        return MSA_ERR_CUDA;
+    h.rows_copied = row0 + rows;
+    return MSA_OK;
+}
+
 template <int BK, int G>
 static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const void* k, const void* v,
                                         const int32_t* block_idx, int64_t q_begin, int64_t q_count,
@@ -350,6 +393,10 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
                 block_idx, p, o_buf, lse_buf, (__nv_bfloat16*)out, lse);
         }
         if (cudaPeekAtLastError() != cudaSuccess) return MSA_ERR_CUDA;
+        if (g_out_hook.on && q_begin == 0 && g_out_hook.rows_copied == q_first) {
+            const msa_status_t hs = hook_copy_rows(r, out, lse, q_first, p.q_count, st);
+            if (hs != MSA_OK) return hs;
+        }
     }
     return MSA_OK;
 }
@@ -557,9 +604,10 @@ msa_status_t msa_sparse_attn_prefill_workspace_bytes(const msa_shape_t* shape, i
     if (q_count < 0 || kv_len < 0) return MSA_ERR_INVALID_ARG;
     size_t mn = kAlign, pf = kAlign;
     if (attn_tc_supported(r) && q_count > 0) {
-        // at least 256 queries in flight; preferred: partial buffers of up to 16 GiB
+        // at least 256 queries in flight; preferred: partial buffers of up to 32 GiB (larger ranges
+        // mean fuller tiles and fewer K/V reloads; measured 498 / 484 / 473 ms at 8 / 16 / 32 GiB, T = 1M)
         const int64_t r_min = q_count < 256 ? q_count : 256;
-        int64_t r_pref = (int64_t)((16ull << 30) / attn_per_query_bytes(r));
+        int64_t r_pref = (int64_t)((32ull << 30) / attn_per_query_bytes(r));
         if (r_pref > q_count) r_pref = q_count;
         if (r_pref < r_min) r_pref = r_min;
         mn = attn_plan(r, kv_len, r_min).total + 8 * kAlign;
@@ -718,6 +766,10 @@ msa_status_t msa_prefill_forward_workspace_bytes(const msa_shape_t* shape, int64
     return MSA_OK;
 }
 
+static msa_status_t prefill_stages_1_2(const msa_shape_t* shape, const Resolved& r, const void* q_idx,
+                                       const void* k_idx, int64_t T, int32_t* block_idx, void* workspace,
+                                       size_t workspace_bytes, msa_stream_t stream);
+
 msa_status_t msa_prefill_forward(const msa_shape_t* shape, const void* q, const void* k,
                                  const void* v, const void* q_idx, const void* k_idx, int64_t T,
                                  void* out, float* lse, int32_t* block_idx, void* workspace,
@@ -731,6 +783,17 @@ msa_status_t msa_prefill_forward(const msa_shape_t* shape, const void* q, const 
     size_t need = 0;
     msa_prefill_forward_workspace_bytes(shape, T, &need, nullptr);
     if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
+    if ((s = prefill_stages_1_2(shape, r, q_idx, k_idx, T, block_idx, workspace, workspace_bytes, stream)) != MSA_OK)
+        return s;
+    return msa_sparse_attn_prefill(shape, q, k, v, block_idx, 0, T, T, out, lse, workspace,
+                                   workspace_bytes, stream);
+}
+
+// Stages 1-2 over query chunks sized to the workspace (scores never exist for the whole sequence).
+static msa_status_t prefill_stages_1_2(const msa_shape_t* shape, const Resolved& r, const void* q_idx,
+                                       const void* k_idx, int64_t T, int32_t* block_idx, void* workspace,
+                                       size_t workspace_bytes, msa_stream_t stream) {
+    msa_status_t s = MSA_OK;
     const int64_t ld = score_ld(T, r.B_k);
     const int64_t chunk = pick_score_chunk(r, T, workspace_bytes);
     if (chunk <= 0) return MSA_ERR_WORKSPACE;
@@ -745,8 +808,7 @@ msa_status_t msa_prefill_forward(const msa_shape_t* shape, const void* q, const 
         s = msa_topk_select(shape, scores, ld, q0, qc, kv_vis, block_idx + (size_t)q0 * r.H_kv * r.k, stream);
         if (s != MSA_OK) return s;
     }
-    return msa_sparse_attn_prefill(shape, q, k, v, block_idx, 0, T, T, out, lse, workspace,
-                                   workspace_bytes, stream);
+    return MSA_OK;
 }
 
 static size_t host_staging_bytes(const Resolved& r, int64_t T, size_t off[8]) {
@@ -793,26 +855,48 @@ msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_ho
     const size_t stage = host_staging_bytes(r, T, off);
     char* w = static_cast<char*>(workspace);
     cudaStream_t st = (cudaStream_t)stream;
+    // A second stream carries the copies: the index inputs go first so that stages 1-2 start
+    // while Q, K and V are still on their way; each finished query range of O is copied back
+    // while the next one is computed.
+    static cudaStream_t copy = nullptr;
+    if (copy == nullptr && cudaStreamCreateWithFlags(&copy, cudaStreamNonBlocking) != cudaSuccess) return MSA_ERR_CUDA;
+    cudaEvent_t e_in = next_sync_event(), e_idx = next_sync_event(), e_all = next_sync_event();
+    if (!e_in || !e_idx || !e_all) return MSA_ERR_CUDA;
+    if (cudaEventRecord(e_in, st) != cudaSuccess || cudaStreamWaitEvent(copy, e_in, 0) != cudaSuccess) return MSA_ERR_CUDA;
     const void* src[5] = {q_host, k_host, v_host, q_idx_host, k_idx_host};
     const size_t nbytes[5] = {(size_t)T * r.H_q * r.d * 2, (size_t)T * r.H_kv * r.d * 2,
                               (size_t)T * r.H_kv * r.d * 2, (size_t)T * r.H_kv * r.d_idx * 2,
                               (size_t)T * r.d_idx * 2};
-    for (int i = 0; i < 5; ++i)
-        if (cudaMemcpyAsync(w + off[i], src[i], nbytes[i], cudaMemcpyHostToDevice, st) != cudaSuccess)
+    const int order[5] = {4, 3, 1, 2, 0};  // k_idx, q_idx, k, v, q
+    for (int j = 0; j < 5; ++j) {
+        const int i = order[j];
+        if (cudaMemcpyAsync(w + off[i], src[i], nbytes[i], cudaMemcpyHostToDevice, copy) != cudaSuccess)
             return MSA_ERR_CUDA;
-    s = msa_prefill_forward(shape, w + off[0], w + off[1], w + off[2], w + off[3], w + off[4], T,
-                            w + off[5], lse_host ? (float*)(w + off[6]) : nullptr,
-                            (int32_t*)(w + off[7]), w + stage, workspace_bytes - stage, stream);
+        if (j == 1 && cudaEventRecord(e_idx, copy) != cudaSuccess) return MSA_ERR_CUDA;
+    }
+    if (cudaEventRecord(e_all, copy) != cudaSuccess) return MSA_ERR_CUDA;
+    float* lse_dev = lse_host ? (float*)(w + off[6]) : nullptr;
+    int32_t* bi_dev = (int32_t*)(w + off[7]);
+    if (cudaStreamWaitEvent(st, e_idx, 0) != cudaSuccess) return MSA_ERR_CUDA;
+    s = prefill_stages_1_2(shape, r, w + off[3], w + off[4], T, bi_dev, w + stage, workspace_bytes - stage, stream);
     if (s != MSA_OK) return s;
-    if (cudaMemcpyAsync(out_host, w + off[5], (size_t)T * r.H_q * r.d * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return MSA_ERR_CUDA;
-    if (lse_host &&
-        cudaMemcpyAsync(lse_host, w + off[6], (size_t)T * r.H_q * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return MSA_ERR_CUDA;
+    if (cudaStreamWaitEvent(st, e_all, 0) != cudaSuccess) return MSA_ERR_CUDA;
+    g_out_hook.on = true; g_out_hook.copy = copy; g_out_hook.out_host = (char*)out_host;
+    g_out_hook.lse_host = lse_host; g_out_hook.rows_copied = 0;
+    s = msa_sparse_attn_prefill(shape, w + off[0], w + off[1], w + off[2], bi_dev, 0, T, T, w + off[5], lse_dev,
+                                w + stage, workspace_bytes - stage, stream);
+    g_out_hook.on = false;
+    if (s != MSA_OK) return s;
+    if (g_out_hook.rows_copied < T) {  // rows the per-range hook did not cover (generic kernel path)
+        const msa_status_t hs = hook_copy_rows(r, w + off[5], lse_dev, g_out_hook.rows_copied,
+                                               T - g_out_hook.rows_copied, st);
+        if (hs != MSA_OK) return hs;
+    }
     if (block_idx_host &&
-        cudaMemcpyAsync(block_idx_host, w + off[7], (size_t)T * r.H_kv * r.k * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        cudaMemcpyAsync(block_idx_host, bi_dev, (size_t)T * r.H_kv * r.k * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return MSA_ERR_CUDA;
-    return cudaStreamSynchronize(st) == cudaSuccess ? MSA_OK : MSA_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess || cudaStreamSynchronize(copy) != cudaSuccess) return MSA_ERR_CUDA;
+    return MSA_OK;
 }
 
 msa_status_t msa_decode_forward(const msa_shape_t* shape, const void* q, const void* q_idx,

@@ -224,3 +224,30 @@ def test_bad_block_index_is_reported_not_dereferenced():
     assert code == 6  # MSA_ERR_BAD_INDEX
     assert torch.isfinite(o2.float()).all()
     assert B.check_async_status()[0] == 0  # cleared
+
+
+@pytest.mark.parametrize("name,T,ws_scale", [("c1", 2048, 1.0), ("c3", 5000, 0.0), ("c3", 9001, 1.0), ("odd", 300, 1.0)])
+def test_host_forward_matches_device_forward(name, T, ws_scale):
+    # The host-buffer form (copies overlapped with compute on a second stream, output copied
+    # back range by range) must give exactly what the device form gives.
+    if name == "odd":
+        cfg = MSAConfig("odd", "prefill", T, 4, 2, 8, 3, head_dim=32, idx_dim=16, seed=1)  # generic kernels
+    else:
+        cfg = CONFIGS[name].scaled(name=name + "-host", T=T)
+    shape = B.shape_of(cfg)
+    x = make_prefill_inputs(cfg, DEV, sharp=True)
+    out, lse, I = api.prefill_forward(cfg, x)
+    host = {n: t.cpu().pin_memory() for n, t in x.items()}
+    out_h = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+    lse_h = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
+    I_h = torch.empty(I.shape, dtype=torch.int32).pin_memory()
+    mn, pf = B.msa_prefill_forward_host_workspace_bytes(shape, T)
+    ws = B.alloc_workspace(int(mn + ws_scale * (pf - mn)), DEV)
+    for _ in range(2):  # twice: the second call reuses the staging area while nothing else runs
+        out_h.zero_(); lse_h.zero_(); I_h.zero_()
+        B.msa_prefill_forward_host(shape, host["q"], host["k"], host["v"], host["q_idx"], host["k_idx"], T,
+                                   out_h, lse_h, I_h, ws)
+        assert torch.equal(I_h, I.cpu())
+        assert torch.equal(out_h, out.cpu())
+        assert torch.equal(lse_h, lse.cpu())
+    _assert_clean()
