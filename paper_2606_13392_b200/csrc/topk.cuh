@@ -7,10 +7,12 @@
 //           (k-1)-th best; survivors are turned into order-preserving 32-bit keys, compacted
 //           into a shared staging buffer with a ballot, and merged 32 at a time into the
 //           sorted kept set (registers, bitonic networks on 32-bit keys).
-//   pass 2  walks the row again in index order and takes every block whose key beats the
-//           threshold plus, among the blocks that tie with it, the first ones in index order
-//           until k-1 are taken.  Walking in index order makes the output list ascending with
-//           no final sort; the local block is appended by construction (never ranked).
+//   pass 2  takes every block whose key beats the threshold plus, among the blocks that tie
+//           with it, the first ones in index order until k-1 are taken.  It reads the log of
+//           pass-1 survivors (shared memory, in block order), which contains every selected
+//           block; only rows with more survivors than the log holds are walked a second time.
+//           Index order makes the output list ascending with no final sort; the local block
+//           is appended by construction (never ranked).
 #pragma once
 
 #include "common.cuh"
@@ -96,14 +98,16 @@ __device__ __forceinline__ int warp_excl_scan(int v, int lane) {
     return x - v;
 }
 
-constexpr int kTopkWarps = 8;
+constexpr int kTopkWarps = 4;
 constexpr int kTopkStage = 160;  // flush threshold (32) + one round of four pushes (4 x 32)
+constexpr int kTopkLog = 768;    // survivors remembered per row for the index pass
 
 template <int R>
 __global__ void __launch_bounds__(kTopkWarps * 32)
 topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap rows,
                    int64_t n_rows, int H_kv, int B_k, int top_k, int32_t* __restrict__ block_idx) {
     __shared__ uint32_t stg_all[kTopkWarps][kTopkStage];
+    __shared__ uint2 log_all[kTopkWarps][kTopkLog];   // (key, block) of every survivor, in index order
     __shared__ int32_t out_all[kTopkWarps][32 * R];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * kTopkWarps + warp;
@@ -124,17 +128,19 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
     }
     const float* srow = scores + row * ld_scores;
     uint32_t* stg = stg_all[warp];
+    uint2* logb = log_all[warp];
     int32_t* outb = out_all[warp];
     const unsigned lt_mask = (1u << lane) - 1u;
-    const int64_t n4 = loc >> 2;
-    const float4* srow4 = reinterpret_cast<const float4*>(srow);
 
     // ------------------------------------------------------------------ pass 1: threshold value
+    // A round covers 128 consecutive blocks as four coalesced 32-wide loads, so that compacting
+    // the loads one after the other keeps the survivors in block order.
     uint32_t kept[R];
 #pragma unroll
     for (int s = 0; s < R; ++s) kept[s] = 0;  // 0 is below every real key
     float tau_f = -INFINITY;                   // score of the current m-th best (strict filter)
-    int cnt = 0;
+    int cnt = 0, n_log = 0;
+    bool log_ok = true;
 
     auto flush = [&](bool all) {
         __syncwarp();
@@ -157,36 +163,53 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         tau_f = tau != 0u ? topk_key_score(tau) : -INFINITY;
         __syncwarp();
     };
-    auto push = [&](float x, bool pass) {
-        const unsigned mask = __ballot_sync(0xffffffffu, pass);
-        if (pass) stg[cnt + __popc(mask & lt_mask)] = topk_key(x);
-        cnt += __popc(mask);
-    };
 
     {
-        float4 nxt = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (lane < n4) nxt = __ldg(srow4 + lane);
-        for (int64_t v0 = 0; v0 < n4; v0 += 32) {
-            const int64_t vi = v0 + lane;
-            const bool in = vi < n4;
-            const float4 x = nxt;
-            if (vi + 32 < n4) nxt = __ldg(srow4 + vi + 32);  // next round's load is in flight meanwhile
+        const int n = (int)loc;  // candidates are blocks [0, n); n < 2^31
+        float nxt[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int i = c * 32 + lane;
+            nxt[c] = i < n ? __ldg(srow + i) : -INFINITY;
+        }
+        for (int i0 = 0; i0 < n; i0 += 128) {
+            float x[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) x[c] = nxt[c];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {  // next round's loads are in flight while this one is ranked
+                const int i = i0 + 128 + c * 32 + lane;
+                nxt[c] = i < n ? __ldg(srow + i) : -INFINITY;
+            }
             // While fewer than m keys are kept everything passes; afterwards only strictly better
-            // scores can change the m-th best value.
-            const bool warm = tau_f == -INFINITY;
-            const bool p0 = in && (warm || x.x > tau_f), p1 = in && (warm || x.y > tau_f);
-            const bool p2 = in && (warm || x.z > tau_f), p3 = in && (warm || x.w > tau_f);
-            if (__ballot_sync(0xffffffffu, p0 | p1 | p2 | p3) == 0u) continue;
-            push(x.x, p0);
-            push(x.y, p1);
-            push(x.z, p2);
-            push(x.w, p3);
+            // scores can change the m-th best value.  (Out-of-range lanes hold -inf.)
+            unsigned mk[4];
+            if (tau_f == -INFINITY) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) mk[c] = __ballot_sync(0xffffffffu, i0 + c * 32 + lane < n);
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) mk[c] = __ballot_sync(0xffffffffu, x[c] > tau_f);
+            }
+            if ((mk[0] | mk[1] | mk[2] | mk[3]) == 0u) continue;
+            // survivors keep block order: component 0's lanes first, then component 1's, ...
+            const int n0 = __popc(mk[0]), n1 = __popc(mk[1]), n2 = __popc(mk[2]), n3 = __popc(mk[3]);
+            const int tot = n0 + n1 + n2 + n3;
+            if (log_ok && n_log + tot > kTopkLog) log_ok = false;
+            const int off[4] = {0, n0, n0 + n1, n0 + n1 + n2};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if (mk[c] & (1u << lane)) {
+                    const int rnk = off[c] + __popc(mk[c] & lt_mask);
+                    const uint32_t key = topk_key(x[c]);
+                    stg[cnt + rnk] = key;
+                    if (log_ok) logb[n_log + rnk] = make_uint2(key, (uint32_t)(i0 + c * 32 + lane));
+                }
+            }
+            cnt += tot;
+            n_log += tot;
             if (cnt >= 32) flush(false);
         }
-        const int64_t idx = (n4 << 2) + lane;  // scalar tail (< 4 elements)
-        const bool in = idx < loc;
-        const float x = in ? __ldg(srow + idx) : 0.f;
-        push(x, in && (tau_f == -INFINITY || x > tau_f));
         flush(true);
     }
     const uint32_t tau = element_at<R>(kept, m - 1);  // key of the m-th best score (loc > m, so it exists)
@@ -196,50 +219,39 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
     const int need_ties = m - n_gt;                    // blocks equal to the threshold still to take
 
     // ------------------------------------------------------------------ pass 2: indices, ascending
+    // Every selected block survived the filter when it was seen (its score beat the threshold
+    // of that moment), so the log holds them all, in block order; ties with the final threshold
+    // are taken first come, first served.  Only a row with more survivors than the log holds
+    // is walked a second time.
     int out_cnt = 0, ties_seen = 0;
-    for (int64_t v0 = 0; v0 < n4 + 1 && out_cnt < m; v0 += 32) {
-        const int64_t vi = v0 + lane;
-        float xs[4] = {0.f, 0.f, 0.f, 0.f};
-        int n_in = 0;  // valid components of this lane
-        if (vi < n4) {
-            const float4 x = __ldg(srow4 + vi);
-            xs[0] = x.x; xs[1] = x.y; xs[2] = x.z; xs[3] = x.w;
-            n_in = 4;
-        } else if (vi == n4) {  // the < 4 tail elements
-            n_in = (int)(loc - (n4 << 2));
-#pragma unroll
-            for (int c = 0; c < 3; ++c)
-                if (c < n_in) xs[c] = __ldg(srow + (n4 << 2) + c);
+    auto take_in_order = [&](uint32_t key, uint32_t blk, bool in) {
+        const bool gt = in && key > tau, eq = in && key == tau;
+        const unsigned eqm = __ballot_sync(0xffffffffu, eq);
+        bool take = gt;
+        if (eqm != 0u) {
+            take = take || (eq && (ties_seen + __popc(eqm & lt_mask)) < need_ties);
+            ties_seen += __popc(eqm);
         }
-        unsigned gt = 0, eq = 0;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const uint32_t key = topk_key(xs[c]);
-            if (c < n_in && key > tau) gt |= 1u << c;
-            if (c < n_in && key == tau) eq |= 1u << c;
+        const unsigned tm = __ballot_sync(0xffffffffu, take);
+        if (take) {
+            const int w = out_cnt + __popc(tm & lt_mask);
+            if (w < m) outb[w] = (int32_t)blk;
         }
-        if (__ballot_sync(0xffffffffu, (gt | eq) != 0u) == 0u) continue;
-        unsigned take = gt;
-        if (__ballot_sync(0xffffffffu, eq != 0u) != 0u) {  // ties: first ones in index order
-            const int ne = __popc(eq);
-            int rank = ties_seen + warp_excl_scan(ne, lane);
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (eq & (1u << c)) {
-                    if (rank < need_ties) take |= 1u << c;
-                    ++rank;
-                }
-            ties_seen = __shfl_sync(0xffffffffu, rank, 31);  // lane 31 ends at the running total
+        out_cnt += __popc(tm);
+    };
+    if (log_ok) {
+        for (int e0 = 0; e0 < n_log && out_cnt < m; e0 += 32) {
+            const int e = e0 + lane;
+            uint2 kv = make_uint2(0u, 0u);
+            if (e < n_log) kv = logb[e];
+            take_in_order(kv.x, kv.y, e < n_log);
         }
-        const int nt = __popc(take);
-        int w = out_cnt + warp_excl_scan(nt, lane);
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            if (take & (1u << c)) {
-                if (w < m) outb[w] = (int32_t)((vi << 2) + c);
-                ++w;
-            }
-        out_cnt = __shfl_sync(0xffffffffu, w, 31);
+    } else {
+        for (int64_t i0 = 0; i0 < loc && out_cnt < m; i0 += 32) {
+            const int64_t i = i0 + lane;
+            const float x = i < loc ? __ldg(srow + i) : 0.f;
+            take_in_order(topk_key(x), (uint32_t)i, i < loc);
+        }
     }
     __syncwarp();
     for (int e = lane; e < top_k; e += 32) orow[e] = e < m ? outb[e] : (e == m ? (int32_t)loc : -1);
