@@ -1,25 +1,29 @@
 // Eq. 6 on the 5th-gen tensor cores (d_idx = 64, B_k in {64,128}).
 //
-// One CTA per (tile of 128 queries, index head r).  It streams the visible prefix of K_idx in
-// tiles of 256 keys through a TMA ring, multiplies each against the resident 128x64 query
-// tile with tcgen05.mma (M=128, N=256, four K=16 steps) into one of two 256-column TMEM
-// accumulators, and eight epilogue warps reduce the finished accumulator to per-block row
-// maxima (TMEM lane = query row, so the maximum over a block's columns is thread-local)
-// while the next tile is being multiplied.  Only the tile that crosses the diagonal applies
-// the causal mask.  Blocks beyond a query's local block are filled with -inf at the end.
+// One CTA per (tile of 128 queries, NH consecutive index heads).  It streams the visible
+// prefix of K_idx in tiles of 256 keys through a TMA ring and multiplies every key tile
+// against the NH resident 128x64 query tiles, one after the other, with tcgen05.mma (M=128,
+// N=256, four K=16 steps), alternating between two 256-column TMEM accumulators; eight
+// epilogue warps reduce a finished accumulator to per-block row maxima (TMEM lane = query
+// row, so the maximum over a block's columns is thread-local) while the next head's product
+// runs.  Sharing one key tile among NH heads matters: with one head per CTA every 512 MMA
+// cycles need a fresh 32 KB tile from L2, about 9 TB/s over the chip, and the kernel is
+// L2-bound at 60 % tensor duty.  Only the tile that crosses the diagonal applies the causal
+// mask.  Blocks beyond a query's local block are filled with -inf at the end.
 #pragma once
 
 #include "tc_common.cuh"
 
 namespace msa {
 
-constexpr int kIdxStages = 4;
+constexpr int kIdxStages = 3;
 constexpr int kIdxTileQ = 128;
 constexpr int kIdxTileK = 256;
 constexpr int kIdxThreads = 320;  // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
 
+template <int NH>
 struct IdxSmem {
-    alignas(1024) uint8_t a[kIdxTileQ * 128];                   // 128 query rows x 64 bf16
+    alignas(1024) uint8_t a[NH][kIdxTileQ * 128];               // per head: 128 query rows x 64 bf16
     alignas(1024) uint8_t b[kIdxStages][kIdxTileK * 128];       // 256 key rows x 64 bf16 per stage
     alignas(8) uint64_t full[kIdxStages];
     uint64_t empty[kIdxStages];
@@ -31,18 +35,20 @@ struct IdxSmem {
     int abort;
 };
 
-template <int BK>
+template <int BK, int NH>
 __global__ void __launch_bounds__(kIdxThreads, 1)
 index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        int64_t q_begin, int64_t q_count, int H_kv, float scale,
                        float* __restrict__ scores, int64_t ld_scores, int64_t n_cols, int* status) {
     extern __shared__ uint8_t smem_raw[];
-    IdxSmem& sm = *reinterpret_cast<IdxSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    IdxSmem<NH>& sm =
+        *reinterpret_cast<IdxSmem<NH>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t n_qtiles = (q_count + kIdxTileQ - 1) / kIdxTileQ;
     // Longest items first: the last query tile sees the most keys.
-    const int64_t qt = n_qtiles - 1 - (int64_t)(blockIdx.x / H_kv);
-    const int r = (int)(blockIdx.x % H_kv);
+    const int n_hg = H_kv / NH;  // head groups
+    const int64_t qt = n_qtiles - 1 - (int64_t)(blockIdx.x / n_hg);
+    const int r0 = (int)(blockIdx.x % n_hg) * NH;
     const int64_t q0 = qt * kIdxTileQ;
     int64_t q_hi = q0 + kIdxTileQ - 1;
     if (q_hi > q_count - 1) q_hi = q_count - 1;
@@ -67,8 +73,8 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
     if (warp == 0) {
         if (lane == 0) {
-            mbar_arrive_expect_tx(&sm.a_full, kIdxTileQ * 128);
-            tma_load_3d(sm.a, &tm_q, 0, r, (int)q0, &sm.a_full);
+            mbar_arrive_expect_tx(&sm.a_full, NH * kIdxTileQ * 128);
+            for (int h = 0; h < NH; ++h) tma_load_3d(sm.a[h], &tm_q, 0, r0 + h, (int)q0, &sm.a_full);
             for (int t = 0; t < n_tiles; ++t) {
                 const int s = t % kIdxStages;
                 if (!mbar_wait(&sm.empty[s], ((t / kIdxStages) & 1) ^ 1, abort)) {
@@ -83,26 +89,30 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_bf16(kIdxTileQ, kIdxTileK, false, false);
-            const uint64_t a_desc = make_smem_desc(smem_u32(sm.a), 16, 1024);
             bool ok = mbar_wait(&sm.a_full, 0, abort);
             if (!ok) report_async(status, kAsyncTimeout, 0x102);
             for (int t = 0; ok && t < n_tiles; ++t) {
-                const int s = t % kIdxStages, buf = t & 1;
-                if (!mbar_wait(&sm.acc_empty[buf], ((t >> 1) & 1) ^ 1, abort)) {
-                    report_async(status, kAsyncTimeout, 0x103);
-                    break;
-                }
+                const int s = t % kIdxStages;
                 if (!mbar_wait(&sm.full[s], (t / kIdxStages) & 1, abort)) {
                     report_async(status, kAsyncTimeout, 0x104);
                     break;
                 }
-                tc_fence_after();
                 const uint64_t b_desc = make_smem_desc(smem_u32(sm.b[s]), 16, 1024);
+                for (int h = 0; h < NH; ++h) {
+                    const int u = t * NH + h, buf = u & 1;  // accumulators alternate over (tile, head)
+                    if (!mbar_wait(&sm.acc_empty[buf], ((u >> 1) & 1) ^ 1, abort)) {
+                        report_async(status, kAsyncTimeout, 0x103);
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint64_t a_desc = make_smem_desc(smem_u32(sm.a[h]), 16, 1024);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per K step
-                    mma_bf16_ss(tmem + buf * kIdxTileK, a_desc + 2 * kk, b_desc + 2 * kk, idesc, kk > 0);
+                    for (int kk = 0; kk < 4; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per K step
+                        mma_bf16_ss(tmem + buf * kIdxTileK, a_desc + 2 * kk, b_desc + 2 * kk, idesc, kk > 0);
+                    mma_commit(&sm.acc_full[buf]);
+                }
                 mma_commit(&sm.empty[s]);
-                mma_commit(&sm.acc_full[buf]);
             }
             if (*abort != 0) {  // unwinding: wait for the MMAs already issued before TMEM is freed
                 mma_commit(&sm.drain);
@@ -118,44 +128,48 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const int64_t pos = q_begin + q;
         const bool valid_row = q < q_count;
         const int64_t loc = pos / BK;
-        float* out_row = scores + (q * H_kv + r) * ld_scores;
-        for (int t = 0; t < n_tiles; ++t) {
-            const int buf = t & 1;
-            if (!mbar_wait(&sm.acc_full[buf], (t >> 1) & 1, abort)) {
-                report_async(status, kAsyncTimeout, 0x105);
-                break;
-            }
-            tc_fence_after();
-            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + buf * kIdxTileK + half * 128;
-            uint32_t v[4][32];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld_32x32(taddr + c * 32, v[c]);
-            tmem_wait_ld();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
-
+        bool live = true;
+        for (int t = 0; live && t < n_tiles; ++t) {
             const int64_t key0 = (int64_t)t * kIdxTileK + half * 128;
             const bool need_mask = key0 + 127 > pos;
-            constexpr int NB = 128 / BK;  // blocks in this thread's 128 columns
-            float best[NB];
+            const int lim = (int)(pos - key0);  // columns 0..lim are visible (may be negative)
+            for (int h = 0; h < NH; ++h) {
+                const int u = t * NH + h, buf = u & 1;
+                if (!mbar_wait(&sm.acc_full[buf], (u >> 1) & 1, abort)) {
+                    report_async(status, kAsyncTimeout, 0x105);
+                    live = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + buf * kIdxTileK + half * 128;
+                uint32_t v[4][32];
 #pragma unroll
-            for (int i = 0; i < NB; ++i) best[i] = -INFINITY;
-            if (need_mask) {
-                const int lim = (int)(pos - key0);  // columns 0..lim are visible (may be negative)
+                for (int c = 0; c < 4; ++c) tmem_ld_32x32(taddr + c * 32, v[c]);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
+
+                constexpr int NB = 128 / BK;  // blocks in this thread's 128 columns
+                float best[NB];
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int i = 0; i < NB; ++i) best[i] = -INFINITY;
+                if (need_mask) {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (c * 32 + e > lim) v[c][e] = 0xFF800000u;  // -inf
-            }
+                    for (int c = 0; c < 4; ++c)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) best[(c * 32) / BK] = fmaxf(best[(c * 32) / BK], tree_max32(v[c]));
-            if (valid_row) {
+                        for (int e = 0; e < 32; ++e)
+                            if (c * 32 + e > lim) v[c][e] = 0xFF800000u;  // -inf
+                }
 #pragma unroll
-                for (int i = 0; i < NB; ++i) {
-                    const int64_t b = key0 / BK + i;
-                    if (b <= loc) out_row[b] = best[i] * scale;
+                for (int c = 0; c < 4; ++c) best[(c * 32) / BK] = fmaxf(best[(c * 32) / BK], tree_max32(v[c]));
+                if (valid_row) {
+                    float* out_row = scores + (q * H_kv + r0 + h) * ld_scores;
+#pragma unroll
+                    for (int i = 0; i < NB; ++i) {
+                        const int64_t b = key0 / BK + i;
+                        if (b <= loc) out_row[b] = best[i] * scale;
+                    }
                 }
             }
         }
@@ -163,8 +177,10 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int rr = ew; rr < kIdxTileQ; rr += 8) {
             const int64_t qq = q0 + rr;
             if (qq >= q_count) break;
-            float* orow = scores + (qq * H_kv + r) * ld_scores;
-            for (int64_t b = (q_begin + qq) / BK + 1 + lane; b < n_cols; b += 32) orow[b] = -INFINITY;
+            for (int h = 0; h < NH; ++h) {
+                float* orow = scores + (qq * H_kv + r0 + h) * ld_scores;
+                for (int64_t b = (q_begin + qq) / BK + 1 + lane; b < n_cols; b += 32) orow[b] = -INFINITY;
+            }
         }
     }
     tc_fence_before();

@@ -75,6 +75,8 @@ static msa_status_t check_range(int64_t q_begin, int64_t q_count, int64_t kv_len
     return MSA_OK;
 }
 
+static int sm_count();
+
 static msa_status_t launch_status() {
     return cudaPeekAtLastError() == cudaSuccess ? MSA_OK : MSA_ERR_CUDA;
 }
@@ -112,7 +114,7 @@ bool encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64
 }
 
 // ---------------------------------------------------------------------- stage 1
-template <int BK>
+template <int BK, int NH>
 static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                     int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
                                     int64_t n_cols, cudaStream_t st) {
@@ -127,22 +129,38 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
         return MSA_ERR_CUDA;
     int* status = async_status_ptr();
     if (status == nullptr) return MSA_ERR_CUDA;
-    const size_t smem = sizeof(IdxSmem) + 1024;
+    const size_t smem = sizeof(IdxSmem<NH>) + 1024;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(index_scores_tc_kernel<BK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(index_scores_tc_kernel<BK, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem) != cudaSuccess)
             return MSA_ERR_CUDA;
         attr_set = true;
     }
-    const int64_t grid = ceil_div64(q_count, kIdxTileQ) * r.H_kv;
+    const int64_t grid = ceil_div64(q_count, kIdxTileQ) * (r.H_kv / NH);
     if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
     {
         StageScope sc(kStageIndex, st);
-        index_scores_tc_kernel<BK><<<(unsigned)grid, kIdxThreads, smem, st>>>(
+        index_scores_tc_kernel<BK, NH><<<(unsigned)grid, kIdxThreads, smem, st>>>(
             tm_q, tm_k, q_begin, q_count, r.H_kv, r.index_scale, scores, ld_scores, n_cols, status);
     }
     return launch_status();
+}
+
+// Heads sharing one key tile per CTA: the most (8, 4, 2, 1) that divide H_kv and still leave
+// at least two CTAs per SM, so that short chunks keep the machine full.
+template <int BK>
+static msa_status_t launch_index_tc_bk(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
+                                       int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
+                                       int64_t n_cols, cudaStream_t st) {
+    const int64_t n_qtiles = ceil_div64(q_count, kIdxTileQ);
+    int nh = 1;
+    for (int cand = 8; cand > 1; cand >>= 1)
+        if (r.H_kv % cand == 0 && n_qtiles * (r.H_kv / cand) >= 2 * sm_count()) { nh = cand; break; }
+    if (nh == 8) return launch_index_tc<BK, 8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    if (nh == 4) return launch_index_tc<BK, 4>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    if (nh == 2) return launch_index_tc<BK, 2>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    return launch_index_tc<BK, 1>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
 }
 
 static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const void* k_idx,
@@ -152,10 +170,10 @@ static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const
     if (rows.seq_lens == nullptr && r.d_idx == 64 && (r.B_k == 64 || r.B_k == 128) &&
         rows.kv_len < 2147483647LL && n_rows >= 32) {
         if (r.B_k == 64)
-            return launch_index_tc<64>(r, q_idx, k_idx, rows.q_begin, n_rows, rows.kv_len, scores, ld_scores,
+            return launch_index_tc_bk<64>(r, q_idx, k_idx, rows.q_begin, n_rows, rows.kv_len, scores, ld_scores,
+                                          rows.n_cols, st);
+        return launch_index_tc_bk<128>(r, q_idx, k_idx, rows.q_begin, n_rows, rows.kv_len, scores, ld_scores,
                                        rows.n_cols, st);
-        return launch_index_tc<128>(r, q_idx, k_idx, rows.q_begin, n_rows, rows.kv_len, scores, ld_scores,
-                                    rows.n_cols, st);
     }
     constexpr int WARPS = 8;
     const int64_t n_chunks = ceil_div64(rows.n_cols, WARPS);
