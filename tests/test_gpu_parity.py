@@ -251,3 +251,31 @@ def test_host_forward_matches_device_forward(name, T, ws_scale):
         assert torch.equal(out_h, out.cpu())
         assert torch.equal(lse_h, lse.cpu())
     _assert_clean()
+
+
+def test_sink_block_selected_by_every_query():
+    # Real workloads have an attention sink: one early block that nearly every query selects
+    # (Section 4.2, "pre-scheduled tile chunking").  Block 0's tile then holds every query of a
+    # range, thousands of times the average: the item list must spread it over all CTAs and the
+    # results must not change.
+    cfg = CONFIGS["c3"].scaled(name="c3-sink", T=16384 + 300)
+    x = make_prefill_inputs(cfg, DEV, sharp=True)
+    u = torch.zeros(cfg.idx_dim, device=DEV)
+    u[0] = 1.0
+    x["k_idx"][: cfg.block_size] = (x["k_idx"][: cfg.block_size].float() + 40.0 * u).to(torch.bfloat16)
+    x["q_idx"] = (x["q_idx"].float() + 6.0 * u).to(torch.bfloat16)
+    T = cfg.T
+    pos = sample_positions(T, cfg.block_size, cfg.top_k, 200, 3)
+    pos_t = torch.from_numpy(pos).to(DEV)
+    out, lse, I = api.prefill_forward(cfg, x)
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert bool((I[cfg.block_size:, :, 0] == 0).all()), "block 0 must be in every list"
+    kb, vb, kib = to_bits(x["k"]), to_bits(x["v"]), to_bits(x["k_idx"])
+    M_ref = oracle.index_scores(to_bits(x["q_idx"][pos_t]), kib, pos, cfg.block_size)
+    I_ref = oracle.topk_select(M_ref, pos, T, cfg.block_size, cfg.top_k)
+    I_gpu = I[pos_t].cpu().numpy()
+    exact, _ = check_selection(I_gpu, I_ref, M_ref, pos, cfg.block_size, cfg.top_k, eps=1e-4)
+    assert exact >= 0.995
+    O_ref, LSE_ref = oracle.sparse_attn(to_bits(x["q"][pos_t]), kb, vb, I_gpu, pos, cfg.block_size)
+    check_attn(out[pos_t].float().cpu().numpy(), lse[pos_t].cpu().numpy(), O_ref, LSE_ref, "sink")
