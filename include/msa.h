@@ -24,9 +24,9 @@
  *     launch errors map to MSA_ERR_CUDA.  Device-side anomalies (a bounded wait that ran
  *     out, a block index out of range) never trap: they set a status word that
  *     msa_check_async_status() reads.
- *   - Fast kernels are specialised for d_h = 128, d_idx = 64, B_k in {64,128},
- *     G in {8,16}; other shapes (d_h, d_idx multiples of 8, d_h <= 256, d_idx <= 128)
- *     run on generic kernels.  k is limited to 1..128.
+ *   - Fast kernels are specialised for d_h = 128, d_idx in {64,128}, B_k in {64,128},
+ *     G in {8,16} (decode index scoring: H_kv <= 8); other shapes (d_h, d_idx multiples
+ *     of 8, d_h <= 256, d_idx <= 128) run on generic kernels.  k is limited to 1..128.
  */
 #ifndef MSA_H_
 #define MSA_H_

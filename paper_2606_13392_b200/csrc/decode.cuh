@@ -43,13 +43,13 @@ __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
 }
 
 // ------------------------------------------------------------------ stage 1, decode
-// d_idx = 64, H_kv <= 8, any B_k that is a multiple of 8.  A = Q_idx padded to 16 rows.
+// d_idx = 32*NSEG (64 or 128), H_kv <= 8, any B_k.  A = Q_idx padded to 16 rows.
 // The contraction index is permuted identically in A and B so that a lane's B fragment for
 // two consecutive k-steps is one 16-byte load: within a 32-wide segment of d, lane quad
 // position t owns d[8t..8t+7]; k-step 0 uses d[8t..8t+3], k-step 1 uses d[8t+4..8t+7].
 constexpr int kIdxDecWarps = 8;
 
-template <int UNROLL>
+template <int UNROLL, int NSEG>
 __global__ void __launch_bounds__(kIdxDecWarps * 32)
 index_scores_decode_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_bfloat16* __restrict__ k_idx,
                            const int64_t* __restrict__ seq_offsets, const int32_t* __restrict__ seq_lens,
@@ -64,7 +64,8 @@ index_scores_decode_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_b
     int64_t it = (int64_t)blockIdx.x * kIdxDecWarps + warp;
     const int64_t it_end = total;
     int cur_seq = -1;
-    uint32_t qa[8];   // A fragments of the current sequence's query: [segment][k-step][lo/hi]
+    constexpr int D = 32 * NSEG;
+    uint32_t qa[4 * NSEG];  // A fragments of the current sequence's query: [segment][k-step][lo/hi]
     int64_t len = 0, base = 0;
     for (; it < it_end; it += n_warps) {
         const int s = (int)(it / n_cols);
@@ -74,11 +75,11 @@ index_scores_decode_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_b
             len = seq_lens[s];
             base = seq_offsets[s];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) qa[i] = 0u;
+            for (int i = 0; i < 4 * NSEG; ++i) qa[i] = 0u;
             if (g < H_kv) {
-                const uint4* qrow = reinterpret_cast<const uint4*>(q_idx + ((int64_t)s * H_kv + g) * 64);
+                const uint4* qrow = reinterpret_cast<const uint4*>(q_idx + ((int64_t)s * H_kv + g) * D);
 #pragma unroll
-                for (int seg = 0; seg < 2; ++seg) {
+                for (int seg = 0; seg < NSEG; ++seg) {
                     const uint4 v = __ldg(qrow + seg * 4 + t);
                     qa[seg * 4 + 0] = v.x; qa[seg * 4 + 1] = v.y;  // k-step 0: a0a1, a4a5
                     qa[seg * 4 + 2] = v.z; qa[seg * 4 + 3] = v.w;  // k-step 1
@@ -95,28 +96,29 @@ index_scores_decode_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_b
         int n_vis = (int)((pos - j0 + 1) < B_k ? (pos - j0 + 1) : B_k);
         const int n_nt = (n_vis + 7) >> 3;  // 8-key tiles that hold a visible key
         float best0 = -INFINITY, best1 = -INFINITY;
-        const __nv_bfloat16* kb = k_idx + (base + j0) * 64;
+        const __nv_bfloat16* kb = k_idx + (base + j0) * D;
         for (int nt0 = 0; nt0 < n_nt; nt0 += UNROLL) {
-            uint4 kv[UNROLL][2];
+            uint4 kv[UNROLL][NSEG];
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const int nt = nt0 + u;
                 // rows past the visible range are clamped (loaded but masked below)
                 int row = nt * 8 + g;
                 if (row > n_vis - 1) row = n_vis - 1;
-                const uint4* krow = reinterpret_cast<const uint4*>(kb + (int64_t)row * 64);
-                kv[u][0] = ldg_stream(krow + t);
-                kv[u][1] = ldg_stream(krow + 4 + t);
+                const uint4* krow = reinterpret_cast<const uint4*>(kb + (int64_t)row * D);
+#pragma unroll
+                for (int seg = 0; seg < NSEG; ++seg) kv[u][seg] = ldg_stream(krow + seg * 4 + t);
             }
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const int nt = nt0 + u;
                 if (nt < n_nt) {
                     float c[4] = {0.f, 0.f, 0.f, 0.f};
-                    mma_m16n8k16_bf16(c, qa[0], 0u, qa[1], 0u, kv[u][0].x, kv[u][0].y);
-                    mma_m16n8k16_bf16(c, qa[2], 0u, qa[3], 0u, kv[u][0].z, kv[u][0].w);
-                    mma_m16n8k16_bf16(c, qa[4], 0u, qa[5], 0u, kv[u][1].x, kv[u][1].y);
-                    mma_m16n8k16_bf16(c, qa[6], 0u, qa[7], 0u, kv[u][1].z, kv[u][1].w);
+#pragma unroll
+                    for (int seg = 0; seg < NSEG; ++seg) {
+                        mma_m16n8k16_bf16(c, qa[seg * 4], 0u, qa[seg * 4 + 1], 0u, kv[u][seg].x, kv[u][seg].y);
+                        mma_m16n8k16_bf16(c, qa[seg * 4 + 2], 0u, qa[seg * 4 + 3], 0u, kv[u][seg].z, kv[u][seg].w);
+                    }
                     // c[0], c[1]: group g, keys nt*8 + 2t, +1
                     const int key = nt * 8 + 2 * t;
                     if (key < n_vis) best0 = fmaxf(best0, c[0]);
@@ -150,8 +152,8 @@ struct DecParams {
     const int32_t* block_idx;       // [batch, H_kv, top_k]
     const int64_t* seq_offsets;
     const int32_t* seq_lens;
-    float* part_o;                  // [items*4, 8, 128]
-    float* part_ml;                 // [items*4, 2, 8]  (running max in log2 units, sum)
+    float* part_o;                  // [items*4, G, 128]
+    float* part_ml;                 // [items*4, 2, G]  (running max in log2 units, sum)
     int batch, H_kv, top_k, n_split;
     float scale_log2e;
 };
@@ -162,7 +164,7 @@ __device__ __forceinline__ uint32_t dec_tile_addr(uint32_t tile_base, int key, i
     return tile_base + (uint32_t)((chunk >> 3) * (BK * 128) + key * 128 + (((chunk & 7) ^ (key & 7)) << 4));
 }
 
-template <int BK>
+template <int BK, int G>
 __global__ void __launch_bounds__(kDecThreads, 1)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    DecParams p, int* status) {
@@ -183,7 +185,7 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
     }
     __syncthreads();
     const int n_items = p.batch * p.H_kv * p.n_split;
-    const int G = 8;
+    constexpr int HG = G / 8;  // half-groups of 8 heads: rows 0-7 and 8-15 of the 16-row MMA
     const int H_q = p.H_kv * G;
 
     if (warp == 0) {
@@ -230,27 +232,35 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
             const int64_t len = p.seq_lens[seq];
             const int64_t pos = len - 1, loc = pos / BK;
             const int32_t* sel = p.block_idx + (int64_t)u * p.top_k;
-            // A fragments of Q (rows 0-7 = the 8 heads of the group, rows 8-15 = zero padding)
-            uint32_t qa[8][2];
-            {
-                const __nv_bfloat16* qrow = p.q + ((int64_t)seq * H_q + r * G + g) * 128;
+            // A fragments of Q: rows 0-7 = heads 0-7 of the group, rows 8-15 = heads 8-15 (G = 16)
+            // or zero padding (G = 8)
+            uint32_t qa[8][4];
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) qa[ks][0] = qa[ks][1] = qa[ks][2] = qa[ks][3] = 0u;
+#pragma unroll
+            for (int hg = 0; hg < HG; ++hg) {
+                const __nv_bfloat16* qrow = p.q + ((int64_t)seq * H_q + r * G + hg * 8 + g) * 128;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    qa[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * t);
-                    qa[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * t);
+                    qa[ks][hg] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * t);
+                    qa[ks][2 + hg] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * t);
                 }
             }
-            float m_run = -INFINITY, l_part = 0.f;
-            float acc[8][4];
+            float m_run[HG], l_part[HG];
+            float acc[HG][8][4];
 #pragma unroll
-            for (int mt = 0; mt < 8; ++mt)
+            for (int hg = 0; hg < HG; ++hg) {
+                m_run[hg] = -INFINITY; l_part[hg] = 0.f;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
+                for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[hg][mt][i] = 0.f;
+            }
 
             for (int e = sp * kDecBlocksPerItem; ok && e < min(p.top_k, (sp + 1) * kDecBlocksPerItem); ++e) {
                 const int32_t b = sel[e];
                 if (b < 0 || (int64_t)b > loc) continue;
-                // ---- K tile: S[head g][keys of this warp]
+                // ---- K tile: S[head][keys of this warp]; c[.][0,1] = head g, c[.][2,3] = head 8+g
                 int st = sc % kDecStages;
                 if (!mbar_wait(&sm.full[st], (sc / kDecStages) & 1, abort)) {
                     if (lane == 0) report_async(status, kAsyncTimeout, 0x411);
@@ -267,44 +277,50 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                     for (int kc = 0; kc < 4; ++kc) {
                         uint32_t r4[4];
                         ldmatrix_x4(r4, dec_tile_addr<BK>(tb, key, kc * 4 + (lane >> 3)));
-                        mma_m16n8k16_bf16(c[nt], qa[2 * kc][0], 0u, qa[2 * kc][1], 0u, r4[0], r4[1]);
-                        mma_m16n8k16_bf16(c[nt], qa[2 * kc + 1][0], 0u, qa[2 * kc + 1][1], 0u, r4[2], r4[3]);
+                        mma_m16n8k16_bf16(c[nt], qa[2 * kc][0], qa[2 * kc][1], qa[2 * kc][2], qa[2 * kc][3], r4[0], r4[1]);
+                        mma_m16n8k16_bf16(c[nt], qa[2 * kc + 1][0], qa[2 * kc + 1][1], qa[2 * kc + 1][2],
+                                          qa[2 * kc + 1][3], r4[2], r4[3]);
                     }
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm.empty[st]);
                 ++sc;
-                // ---- online softmax for head g over this warp's keys (values in log2 units)
+                // ---- online softmax per head over this warp's keys (values in log2 units)
                 const int lim = (int)(pos - (int64_t)b * BK);  // keys 0..lim of the block are visible
-                float mx = -INFINITY;
+                uint32_t pb[HG][KS][2];
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const int key = w * KPW + nt * 8 + 2 * t;
-                    c[nt][0] = key <= lim ? c[nt][0] * p.scale_log2e : -INFINITY;
-                    c[nt][1] = key + 1 <= lim ? c[nt][1] * p.scale_log2e : -INFINITY;
-                    mx = fmaxf(mx, fmaxf(c[nt][0], c[nt][1]));
-                }
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float m_new = fmaxf(m_run, mx);
-                const float m_use = m_new == -INFINITY ? 0.f : m_new;   // slice fully masked so far
-                const float corr = ex2_approx(m_run - m_use);            // 0 when m_run = -inf
-                uint32_t pb[KS][2];
-                float psum = 0.f;
+                for (int hg = 0; hg < HG; ++hg) {
+                    float mx = -INFINITY;
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const float p0 = ex2_approx(c[nt][0] - m_use), p1 = ex2_approx(c[nt][1] - m_use);
-                    psum += p0 + p1;
-                    const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                    pb[nt >> 1][nt & 1] = *reinterpret_cast<const uint32_t*>(&pk);
-                }
-                l_part = l_part * corr + psum;
-                m_run = m_new;
-                const float corr0 = __shfl_sync(0xffffffffu, corr, (2 * t) * 4);
-                const float corr1 = __shfl_sync(0xffffffffu, corr, (2 * t + 1) * 4);
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const int key = w * KPW + nt * 8 + 2 * t;
+                        c[nt][2 * hg] = key <= lim ? c[nt][2 * hg] * p.scale_log2e : -INFINITY;
+                        c[nt][2 * hg + 1] = key + 1 <= lim ? c[nt][2 * hg + 1] * p.scale_log2e : -INFINITY;
+                        mx = fmaxf(mx, fmaxf(c[nt][2 * hg], c[nt][2 * hg + 1]));
+                    }
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                    const float m_new = fmaxf(m_run[hg], mx);
+                    const float m_use = m_new == -INFINITY ? 0.f : m_new;   // slice fully masked so far
+                    const float corr = ex2_approx(m_run[hg] - m_use);        // 0 when m_run = -inf
+                    float psum = 0.f;
 #pragma unroll
-                for (int mt = 0; mt < 8; ++mt) {
-                    acc[mt][0] *= corr0; acc[mt][1] *= corr1; acc[mt][2] *= corr0; acc[mt][3] *= corr1;
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const float p0 = ex2_approx(c[nt][2 * hg] - m_use), p1 = ex2_approx(c[nt][2 * hg + 1] - m_use);
+                        psum += p0 + p1;
+                        const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                        pb[hg][nt >> 1][nt & 1] = *reinterpret_cast<const uint32_t*>(&pk);
+                    }
+                    l_part[hg] = l_part[hg] * corr + psum;
+                    m_run[hg] = m_new;
+                    // O^T columns of this lane are heads 2t, 2t+1 of the half-group: fetch their factors
+                    const float corr0 = __shfl_sync(0xffffffffu, corr, (2 * t) * 4);
+                    const float corr1 = __shfl_sync(0xffffffffu, corr, (2 * t + 1) * 4);
+#pragma unroll
+                    for (int mt = 0; mt < 8; ++mt) {
+                        acc[hg][mt][0] *= corr0; acc[hg][mt][1] *= corr1;
+                        acc[hg][mt][2] *= corr0; acc[hg][mt][3] *= corr1;
+                    }
                 }
                 // ---- V tile: O^T[d][head] += V^T[d][key] P^T[key][head]
                 st = sc % kDecStages;
@@ -322,7 +338,9 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         const int key = w * KPW + ks * 16 + (i >> 1) * 8 + (lane & 7);
                         uint32_t r4[4];
                         ldmatrix_x4_trans(r4, dec_tile_addr<BK>(tb, key, mt * 2 + (i & 1)));
-                        mma_m16n8k16_bf16(acc[mt], r4[0], r4[1], r4[2], r4[3], pb[ks][0], pb[ks][1]);
+#pragma unroll
+                        for (int hg = 0; hg < HG; ++hg)
+                            mma_m16n8k16_bf16(acc[hg][mt], r4[0], r4[1], r4[2], r4[3], pb[hg][ks][0], pb[hg][ks][1]);
                     }
                 }
                 __syncwarp();
@@ -330,22 +348,25 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                 ++sc;
             }
             // ---- partial of this warp: O^T (unnormalised), running max, sum
-            float l = l_part;
-            l += __shfl_xor_sync(0xffffffffu, l, 1);
-            l += __shfl_xor_sync(0xffffffffu, l, 2);
             const int64_t pidx = (int64_t)item * kDecPartsPerItem + w;
-            float* po = p.part_o + pidx * (8 * 128);
+            float* po = p.part_o + pidx * (G * 128);
 #pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-                const int d0 = mt * 16 + g;
-                po[(2 * t) * 128 + d0] = acc[mt][0];
-                po[(2 * t + 1) * 128 + d0] = acc[mt][1];
-                po[(2 * t) * 128 + d0 + 8] = acc[mt][2];
-                po[(2 * t + 1) * 128 + d0 + 8] = acc[mt][3];
-            }
-            if (t == 0) {
-                p.part_ml[pidx * 16 + g] = m_run;
-                p.part_ml[pidx * 16 + 8 + g] = l;
+            for (int hg = 0; hg < HG; ++hg) {
+                float l = l_part[hg];
+                l += __shfl_xor_sync(0xffffffffu, l, 1);
+                l += __shfl_xor_sync(0xffffffffu, l, 2);
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) {
+                    const int d0 = mt * 16 + g;
+                    po[(hg * 8 + 2 * t) * 128 + d0] = acc[hg][mt][0];
+                    po[(hg * 8 + 2 * t + 1) * 128 + d0] = acc[hg][mt][1];
+                    po[(hg * 8 + 2 * t) * 128 + d0 + 8] = acc[hg][mt][2];
+                    po[(hg * 8 + 2 * t + 1) * 128 + d0 + 8] = acc[hg][mt][3];
+                }
+                if (t == 0) {
+                    p.part_ml[pidx * (2 * G) + hg * 8 + g] = m_run[hg];
+                    p.part_ml[pidx * (2 * G) + G + hg * 8 + g] = l;
+                }
             }
         }
     }
@@ -354,26 +375,26 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
 // One warp per (sequence, head): merges the n_split*4 partials of its (sequence, KV head).
 __global__ void __launch_bounds__(128)
 attn_decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, int batch, int H_kv,
-                           int n_split, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+                           int G, int n_split, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     const int row = blockIdx.x * 4 + (threadIdx.x >> 5);  // (seq, head)
     const int lane = threadIdx.x & 31;
-    const int H_q = H_kv * 8;
+    const int H_q = H_kv * G;
     if (row >= batch * H_q) return;
     const int seq = row / H_q, h = row - seq * H_q;
-    const int r = h >> 3, g = h & 7;
+    const int r = h / G, g = h - r * G;
     const int n_parts = n_split * kDecPartsPerItem;
     const int64_t p0 = ((int64_t)seq * H_kv + r) * n_parts;
     float M = -INFINITY;
-    for (int i = lane; i < n_parts; i += 32) M = fmaxf(M, part_ml[(p0 + i) * 16 + g]);
+    for (int i = lane; i < n_parts; i += 32) M = fmaxf(M, part_ml[(p0 + i) * (2 * G) + g]);
     M = warp_max(M);
     float L = 0.f;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     for (int i = 0; i < n_parts; ++i) {
-        const float mi = part_ml[(p0 + i) * 16 + g];
+        const float mi = part_ml[(p0 + i) * (2 * G) + g];
         if (mi == -INFINITY) continue;
         const float wgt = exp2f(mi - M);
-        L += wgt * part_ml[(p0 + i) * 16 + 8 + g];
-        const float4 o = *reinterpret_cast<const float4*>(part_o + (p0 + i) * (8 * 128) + g * 128 + lane * 4);
+        L += wgt * part_ml[(p0 + i) * (2 * G) + G + g];
+        const float4 o = *reinterpret_cast<const float4*>(part_o + ((p0 + i) * G + g) * 128 + lane * 4);
         acc[0] = fmaf(wgt, o.x, acc[0]); acc[1] = fmaf(wgt, o.y, acc[1]);
         acc[2] = fmaf(wgt, o.z, acc[2]); acc[3] = fmaf(wgt, o.w, acc[3]);
     }

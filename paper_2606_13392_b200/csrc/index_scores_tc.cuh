@@ -1,4 +1,4 @@
-// Eq. 6 on the 5th-gen tensor cores (d_idx = 64, B_k in {64,128}).
+// Eq. 6 on the 5th-gen tensor cores (d_idx in {64,128}, B_k in {64,128}).
 //
 // One CTA per (tile of 128 queries, NH consecutive index heads).  It streams the visible
 // prefix of K_idx in tiles of 256 keys through a TMA ring and multiplies every key tile
@@ -16,17 +16,17 @@
 
 namespace msa {
 
-constexpr int kIdxStages = 3;
 constexpr int kIdxTileQ = 128;
 constexpr int kIdxTileK = 256;
 constexpr int kIdxThreads = 320;  // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
 
-template <int NH>
+// NH heads per CTA, DI = d_idx / 64 swizzle atoms along the contraction, ST key-tile stages.
+template <int NH, int DI, int ST>
 struct IdxSmem {
-    alignas(1024) uint8_t a[NH][kIdxTileQ * 128];               // per head: 128 query rows x 64 bf16
-    alignas(1024) uint8_t b[kIdxStages][kIdxTileK * 128];       // 256 key rows x 64 bf16 per stage
-    alignas(8) uint64_t full[kIdxStages];
-    uint64_t empty[kIdxStages];
+    alignas(1024) uint8_t a[NH][DI][kIdxTileQ * 128];           // per head and atom: 128 query rows x 64 bf16
+    alignas(1024) uint8_t b[ST][DI][kIdxTileK * 128];           // per stage and atom: 256 key rows x 64 bf16
+    alignas(8) uint64_t full[ST];
+    uint64_t empty[ST];
     uint64_t a_full;
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
@@ -35,14 +35,14 @@ struct IdxSmem {
     int abort;
 };
 
-template <int BK, int NH>
+template <int BK, int NH, int DI, int ST>
 __global__ void __launch_bounds__(kIdxThreads, 1)
 index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        int64_t q_begin, int64_t q_count, int H_kv, float scale,
                        float* __restrict__ scores, int64_t ld_scores, int64_t n_cols, int* status) {
     extern __shared__ uint8_t smem_raw[];
-    IdxSmem<NH>& sm =
-        *reinterpret_cast<IdxSmem<NH>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    IdxSmem<NH, DI, ST>& sm =
+        *reinterpret_cast<IdxSmem<NH, DI, ST>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t n_qtiles = (q_count + kIdxTileQ - 1) / kIdxTileQ;
     // Longest items first: the last query tile sees the most keys.
@@ -56,7 +56,7 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     volatile int* abort = &sm.abort;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kIdxStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
+        for (int s = 0; s < ST; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
         mbar_init(&sm.a_full, 1);
         mbar_init(&sm.drain, 1);
         for (int b = 0; b < 2; ++b) { mbar_init(&sm.acc_full[b], 1); mbar_init(&sm.acc_empty[b], 8); }
@@ -73,16 +73,17 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
     if (warp == 0) {
         if (lane == 0) {
-            mbar_arrive_expect_tx(&sm.a_full, NH * kIdxTileQ * 128);
-            for (int h = 0; h < NH; ++h) tma_load_3d(sm.a[h], &tm_q, 0, r0 + h, (int)q0, &sm.a_full);
+            mbar_arrive_expect_tx(&sm.a_full, NH * DI * kIdxTileQ * 128);
+            for (int h = 0; h < NH; ++h)
+                for (int a = 0; a < DI; ++a) tma_load_3d(sm.a[h][a], &tm_q, a * 64, r0 + h, (int)q0, &sm.a_full);
             for (int t = 0; t < n_tiles; ++t) {
-                const int s = t % kIdxStages;
-                if (!mbar_wait(&sm.empty[s], ((t / kIdxStages) & 1) ^ 1, abort)) {
+                const int s = t % ST;
+                if (!mbar_wait(&sm.empty[s], ((t / ST) & 1) ^ 1, abort)) {
                     report_async(status, kAsyncTimeout, 0x101);
                     break;
                 }
-                mbar_arrive_expect_tx(&sm.full[s], kIdxTileK * 128);
-                tma_load_2d(sm.b[s], &tm_k, 0, t * kIdxTileK, &sm.full[s]);
+                mbar_arrive_expect_tx(&sm.full[s], DI * kIdxTileK * 128);
+                for (int a = 0; a < DI; ++a) tma_load_2d(sm.b[s][a], &tm_k, a * 64, t * kIdxTileK, &sm.full[s]);
             }
             if (*abort != 0) spin_cycles(200000);  // let copies already in flight land
         }
@@ -92,12 +93,11 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             bool ok = mbar_wait(&sm.a_full, 0, abort);
             if (!ok) report_async(status, kAsyncTimeout, 0x102);
             for (int t = 0; ok && t < n_tiles; ++t) {
-                const int s = t % kIdxStages;
-                if (!mbar_wait(&sm.full[s], (t / kIdxStages) & 1, abort)) {
+                const int s = t % ST;
+                if (!mbar_wait(&sm.full[s], (t / ST) & 1, abort)) {
                     report_async(status, kAsyncTimeout, 0x104);
                     break;
                 }
-                const uint64_t b_desc = make_smem_desc(smem_u32(sm.b[s]), 16, 1024);
                 for (int h = 0; h < NH; ++h) {
                     const int u = t * NH + h, buf = u & 1;  // accumulators alternate over (tile, head)
                     if (!mbar_wait(&sm.acc_empty[buf], ((u >> 1) & 1) ^ 1, abort)) {
@@ -106,10 +106,14 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         break;
                     }
                     tc_fence_after();
-                    const uint64_t a_desc = make_smem_desc(smem_u32(sm.a[h]), 16, 1024);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per K step
-                        mma_bf16_ss(tmem + buf * kIdxTileK, a_desc + 2 * kk, b_desc + 2 * kk, idesc, kk > 0);
+                    for (int a = 0; a < DI; ++a) {
+                        const uint64_t a_desc = make_smem_desc(smem_u32(sm.a[h][a]), 16, 1024);
+                        const uint64_t b_desc = make_smem_desc(smem_u32(sm.b[s][a]), 16, 1024);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per K step
+                            mma_bf16_ss(tmem + buf * kIdxTileK, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (a | kk) > 0);
+                    }
                     mma_commit(&sm.acc_full[buf]);
                 }
                 mma_commit(&sm.empty[s]);

@@ -114,25 +114,29 @@ bool encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64
 }
 
 // ---------------------------------------------------------------------- stage 1
-template <int BK, int NH>
+template <int BK, int NH, int DI>
 static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                     int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
                                     int64_t n_cols, cudaStream_t st) {
+    // key-tile stages: what fits beside the NH*DI query atoms in 227 KB of shared memory (at most 3)
+    constexpr int ST = (NH * DI * 16 + 3 * DI * 32 <= 224) ? 3 : 2;
+    static_assert(NH * DI * 16 + ST * DI * 32 <= 224, "shared memory budget");
     CUtensorMap tm_q, tm_k;
-    const uint64_t qd[3] = {64, (uint64_t)r.H_kv, (uint64_t)q_count};
-    const uint64_t qs[2] = {128, (uint64_t)r.H_kv * 128};
+    const uint64_t row_b = (uint64_t)DI * 128;  // bytes of one index vector
+    const uint64_t qd[3] = {(uint64_t)DI * 64, (uint64_t)r.H_kv, (uint64_t)q_count};
+    const uint64_t qs[2] = {row_b, (uint64_t)r.H_kv * row_b};
     const uint32_t qb[3] = {64, 1, kIdxTileQ};
-    const uint64_t kd[2] = {64, (uint64_t)kv_len};
-    const uint64_t ks[1] = {128};
+    const uint64_t kd[2] = {(uint64_t)DI * 64, (uint64_t)kv_len};
+    const uint64_t ks[1] = {row_b};
     const uint32_t kb[2] = {64, kIdxTileK};
     if (!encode_tmap_bf16(&tm_q, q_idx, 3, qd, qs, qb) || !encode_tmap_bf16(&tm_k, k_idx, 2, kd, ks, kb))
         return MSA_ERR_CUDA;
     int* status = async_status_ptr();
     if (status == nullptr) return MSA_ERR_CUDA;
-    const size_t smem = sizeof(IdxSmem<NH>) + 1024;
+    const size_t smem = sizeof(IdxSmem<NH, DI, ST>) + 1024;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(index_scores_tc_kernel<BK, NH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(index_scores_tc_kernel<BK, NH, DI, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem) != cudaSuccess)
             return MSA_ERR_CUDA;
         attr_set = true;
@@ -141,39 +145,44 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
     if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
     {
         StageScope sc(kStageIndex, st);
-        index_scores_tc_kernel<BK, NH><<<(unsigned)grid, kIdxThreads, smem, st>>>(
+        index_scores_tc_kernel<BK, NH, DI, ST><<<(unsigned)grid, kIdxThreads, smem, st>>>(
             tm_q, tm_k, q_begin, q_count, r.H_kv, r.index_scale, scores, ld_scores, n_cols, status);
     }
     return launch_status();
 }
 
-// Heads sharing one key tile per CTA: the most (8, 4, 2, 1) that divide H_kv and still leave
-// at least two CTAs per SM, so that short chunks keep the machine full.
-template <int BK>
+// Heads sharing one key tile per CTA: the most (8, 4, 2, 1; at most 2 when d_idx = 128, for
+// shared memory) that divide H_kv and still leave at least two CTAs per SM, so that short
+// chunks keep the machine full.
+template <int BK, int DI>
 static msa_status_t launch_index_tc_bk(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                        int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
                                        int64_t n_cols, cudaStream_t st) {
     const int64_t n_qtiles = ceil_div64(q_count, kIdxTileQ);
     int nh = 1;
-    for (int cand = 8; cand > 1; cand >>= 1)
+    for (int cand = (DI == 1 ? 8 : 2); cand > 1; cand >>= 1)
         if (r.H_kv % cand == 0 && n_qtiles * (r.H_kv / cand) >= 2 * sm_count()) { nh = cand; break; }
-    if (nh == 8) return launch_index_tc<BK, 8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
-    if (nh == 4) return launch_index_tc<BK, 4>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
-    if (nh == 2) return launch_index_tc<BK, 2>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
-    return launch_index_tc<BK, 1>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    if constexpr (DI == 1) {
+        if (nh == 8) return launch_index_tc<BK, 8, DI>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+        if (nh == 4) return launch_index_tc<BK, 4, DI>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    }
+    if (nh == 2) return launch_index_tc<BK, 2, DI>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    return launch_index_tc<BK, 1, DI>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
 }
 
 static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const void* k_idx,
                                      const RowMap& rows, int64_t n_rows, float* scores,
                                      int64_t ld_scores, cudaStream_t st) {
     if (n_rows == 0 || rows.n_cols == 0) return MSA_OK;
-    if (rows.seq_lens == nullptr && r.d_idx == 64 && (r.B_k == 64 || r.B_k == 128) &&
+    if (rows.seq_lens == nullptr && (r.d_idx == 64 || r.d_idx == 128) && (r.B_k == 64 || r.B_k == 128) &&
         rows.kv_len < 2147483647LL && n_rows >= 32) {
-        if (r.B_k == 64)
-            return launch_index_tc_bk<64>(r, q_idx, k_idx, rows.q_begin, n_rows, rows.kv_len, scores, ld_scores,
-                                          rows.n_cols, st);
-        return launch_index_tc_bk<128>(r, q_idx, k_idx, rows.q_begin, n_rows, rows.kv_len, scores, ld_scores,
-                                       rows.n_cols, st);
+        const int64_t qb = rows.q_begin, kl = rows.kv_len, nc = rows.n_cols;
+        if (r.d_idx == 64) {
+            if (r.B_k == 64) return launch_index_tc_bk<64, 1>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
+            return launch_index_tc_bk<128, 1>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
+        }
+        if (r.B_k == 64) return launch_index_tc_bk<64, 2>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
+        return launch_index_tc_bk<128, 2>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
     }
     constexpr int WARPS = 8;
     const int64_t n_chunks = ceil_div64(rows.n_cols, WARPS);
@@ -420,29 +429,36 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
 }
 
 // ---------------------------------------------------------------------- decode path
-static bool index_decode_fast(const Resolved& r) { return r.d_idx == 64 && r.H_kv <= 8; }
+static bool index_decode_fast(const Resolved& r) { return (r.d_idx == 64 || r.d_idx == 128) && r.H_kv <= 8; }
 
 static msa_status_t run_index_decode(const Resolved& r, const void* q_idx, const void* k_idx_cache,
                                      const int64_t* seq_offsets, const int32_t* seq_lens, int batch,
                                      int64_t n_cols, float* scores, int64_t ld_scores, cudaStream_t st) {
     const int grid = sm_count() * 4;
     StageScope sc(kStageIndexDecode, st);
-    index_scores_decode_kernel<8><<<grid, kIdxDecWarps * 32, 0, st>>>(
-        (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx_cache, seq_offsets, seq_lens, batch, r.H_kv,
-        r.B_k, r.index_scale, scores, ld_scores, n_cols);
+    if (r.d_idx == 64)
+        index_scores_decode_kernel<8, 2><<<grid, kIdxDecWarps * 32, 0, st>>>(
+            (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx_cache, seq_offsets, seq_lens, batch, r.H_kv,
+            r.B_k, r.index_scale, scores, ld_scores, n_cols);
+    else
+        index_scores_decode_kernel<4, 4><<<grid, kIdxDecWarps * 32, 0, st>>>(
+            (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx_cache, seq_offsets, seq_lens, batch, r.H_kv,
+            r.B_k, r.index_scale, scores, ld_scores, n_cols);
     return launch_status();
 }
 
-static bool attn_decode_fast(const Resolved& r) { return r.d == 128 && r.G == 8 && (r.B_k == 64 || r.B_k == 128); }
+static bool attn_decode_fast(const Resolved& r) {
+    return r.d == 128 && (r.G == 8 || r.G == 16) && (r.B_k == 64 || r.B_k == 128);
+}
 
 static int decode_n_split(const Resolved& r) { return (r.k + kDecBlocksPerItem - 1) / kDecBlocksPerItem; }
 
 static size_t decode_ws_bytes(const Resolved& r, int batch) {
     const size_t parts = (size_t)batch * r.H_kv * decode_n_split(r) * kDecPartsPerItem;
-    return align_up(parts * 8 * 128 * 4) + align_up(parts * 16 * 4) + kAlign;
+    return align_up(parts * r.G * 128 * 4) + align_up(parts * 2 * r.G * 4) + kAlign;
 }
 
-template <int BK>
+template <int BK, int G>
 static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const void* k_cache, const void* v_cache,
                                        int64_t cache_tokens, const int64_t* seq_offsets, const int32_t* seq_lens,
                                        int batch, const int32_t* block_idx, void* out, float* lse, void* ws,
@@ -458,7 +474,7 @@ static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const v
     const size_t smem = sizeof(DecSmem<BK>) + 1024;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(attn_decode_kernel<BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        if (cudaFuncSetAttribute(attn_decode_kernel<BK, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
             cudaSuccess)
             return MSA_ERR_CUDA;
         attr_set = true;
@@ -469,16 +485,16 @@ static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const v
     p.scale_log2e = r.softmax_scale * 1.4426950408889634f;
     const size_t parts = (size_t)batch * r.H_kv * p.n_split * kDecPartsPerItem;
     p.part_o = (float*)ws;
-    p.part_ml = (float*)((char*)ws + align_up(parts * 8 * 128 * 4));
+    p.part_ml = (float*)((char*)ws + align_up(parts * G * 128 * 4));
     const int n_items = batch * r.H_kv * p.n_split;
     const int grid = n_items < sm_count() ? n_items : sm_count();
     {
         StageScope sc(kStageAttnDecode, st);
-        attn_decode_kernel<BK><<<grid, kDecThreads, smem, st>>>(tm_k, tm_v, p, status);
+        attn_decode_kernel<BK, G><<<grid, kDecThreads, smem, st>>>(tm_k, tm_v, p, status);
     }
     {
         StageScope sc(kStageCombineDecode, st);
-        attn_decode_combine_kernel<<<(batch * r.H_q + 3) / 4, 128, 0, st>>>(p.part_o, p.part_ml, batch, r.H_kv,
+        attn_decode_combine_kernel<<<(batch * r.H_q + 3) / 4, 128, 0, st>>>(p.part_o, p.part_ml, batch, r.H_kv, G,
                                                                              p.n_split, (__nv_bfloat16*)out, lse);
     }
     return launch_status();
@@ -744,11 +760,14 @@ msa_status_t msa_sparse_attn_decode(const msa_shape_t* shape, const void* q, con
     msa_sparse_attn_decode_workspace_bytes(shape, batch, &need);
     if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
     if (attn_decode_fast(r) && cache_tokens < 2147483647LL) {
+        cudaStream_t st = (cudaStream_t)stream;
+        if (r.B_k == 64 && r.G == 8)
+            return run_attn_decode_tc<64, 8>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch, block_idx, out, lse, workspace, st);
         if (r.B_k == 64)
-            return run_attn_decode_tc<64>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch,
-                                          block_idx, out, lse, workspace, (cudaStream_t)stream);
-        return run_attn_decode_tc<128>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch,
-                                       block_idx, out, lse, workspace, (cudaStream_t)stream);
+            return run_attn_decode_tc<64, 16>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch, block_idx, out, lse, workspace, st);
+        if (r.G == 8)
+            return run_attn_decode_tc<128, 8>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch, block_idx, out, lse, workspace, st);
+        return run_attn_decode_tc<128, 16>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch, block_idx, out, lse, workspace, st);
     }
     return run_attn_generic(r, q, k_cache, v_cache, block_idx, decode_rows(seq_offsets, seq_lens, 0, r.B_k),
                             batch, out, lse, (cudaStream_t)stream);

@@ -65,6 +65,12 @@ CONFIGS: Dict[str, MSAConfig] = {
     "c4": MSAConfig("c4", "prefill", 1048576, 64, 8, 128, 64, seed=3),
     "c5": MSAConfig("c5", "decode", 1048576, 64, 8, 128, 64, seed=4,
                     seq_lens=(131072,) * 16 + (1048576,) * 16),
+    # The paper's own model regime (Section 5.3: 64 query heads, 4 KV heads, d_h = 128, B_k = 128,
+    # k = 16; d_idx = 128 reproduces its printed FLOPs ratio), as a second workload family.
+    "p128k": MSAConfig("p128k", "prefill", 131072, 64, 4, 128, 16, idx_dim=128, seed=6),
+    "p1m": MSAConfig("p1m", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=7),
+    "pdec": MSAConfig("pdec", "decode", 1048576, 64, 4, 128, 16, idx_dim=128, seed=8,
+                      seq_lens=(131072,) * 16 + (1048576,) * 16),
     # Reduced cases of the same shapes, small enough for multi-pass profiler captures
     # (inputs still larger than L2).
     "c3-16k": MSAConfig("c3-16k", "prefill", 16384, 64, 8, 128, 64, seed=2,

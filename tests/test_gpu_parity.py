@@ -279,3 +279,38 @@ def test_sink_block_selected_by_every_query():
     assert exact >= 0.995
     O_ref, LSE_ref = oracle.sparse_attn(to_bits(x["q"][pos_t]), kb, vb, I_gpu, pos, cfg.block_size)
     check_attn(out[pos_t].float().cpu().numpy(), lse[pos_t].cpu().numpy(), O_ref, LSE_ref, "sink")
+
+
+# The paper's own model regime (Section 5.3): 64 query heads / 4 KV heads (G = 16), d_h = 128,
+# B_k = 128, k = 16; d_idx = 128 is the value that reproduces its printed FLOPs ratio.
+PAPER_SHAPE = MSAConfig("paper-shape", "prefill", 20000 + 77, 64, 4, 128, 16, head_dim=128, idx_dim=128, seed=6)
+
+
+@pytest.mark.parametrize("sharp", [False, True])
+def test_paper_shape_prefill(sharp):
+    stats = run_prefill_case(PAPER_SHAPE, sharp, n_sample=256)
+    assert stats["exact_sets"] >= 0.999
+    print("paper-shape", sharp, stats)
+
+
+def test_paper_shape_small_chunks_and_b64():
+    # d_idx = 128 with B_k = 64 and a workspace that forces several score chunks and query ranges
+    cfg = PAPER_SHAPE.scaled(name="paper-b64", T=9000, block_size=64, top_k=24)
+    shape = B.shape_of(cfg)
+    mn, pf = B.msa_prefill_forward_workspace_bytes(shape, cfg.T)
+    stats = run_prefill_case(cfg, True, n_sample=200, ws_bytes=mn)
+    assert stats["exact_sets"] >= 0.999
+
+
+@pytest.mark.parametrize("sharp", [False, True])
+def test_paper_shape_decode(sharp):
+    cfg = PAPER_SHAPE.scaled(name="paper-decode", mode="decode", T=0,
+                             seq_lens=(1, 130, 4096, 5000, 30000, 16384 + 64))
+    res = run_decode_case(cfg, sharp)
+    assert np.mean([r["exact"] for r in res]) >= 0.95
+
+
+def test_decode_g16_b64():
+    cfg = MSAConfig("dec-g16", "decode", 0, 32, 2, 64, 12, head_dim=128, idx_dim=64, seed=8,
+                    seq_lens=(70, 640, 641, 7000))
+    run_decode_case(cfg, True)
