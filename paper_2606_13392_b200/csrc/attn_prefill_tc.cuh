@@ -28,6 +28,26 @@ struct RangeParams {
     int32_t H_kv, top_k;
 };
 
+// Tiles are numbered head after head: the whole grid works on one KV head at a time, so the
+// Q rows of (range, head) - gathered top_k times each - are the only hot lines in L2.
+__device__ __forceinline__ int tile_id(int b, int r, const RangeParams& p) {
+    return r * p.n_blocks + b;
+}
+__device__ __forceinline__ int n_phases(const RangeParams& p) { return p.H_kv; }
+// First partial row (slot 0) of (query ql of the range, KV head r): the partial buffers are
+// laid out [head][query][slot], so one head phase writes one contiguous part of them.
+__device__ __forceinline__ int64_t partial_base(int64_t ql, int r, const RangeParams& p) {
+    return ((int64_t)r * p.q_count + ql) * (int64_t)p.top_k;
+}
+// Items of phase ph dealt to this CTA: a contiguous share of the phase's item list.
+__device__ __forceinline__ void phase_items(const int32_t* __restrict__ item_off, const RangeParams& p, int ph,
+                                            int& lo, int& hi) {
+    const int a = item_off[ph * p.n_blocks], b = item_off[(ph + 1) * p.n_blocks];
+    const int per = (b - a + (int)gridDim.x - 1) / (int)gridDim.x;
+    lo = min(b, a + (int)blockIdx.x * per);
+    hi = min(b, lo + per);
+}
+
 // ---------------------------------------------------------------- 1. reverse index
 // One warp per (query, group) row of the index list.  Pass 0 counts the queries of every
 // (block, head) tile and remembers each entry's arrival rank within its tile; pass 1 (after
@@ -49,7 +69,7 @@ revidx_kernel(const int32_t* __restrict__ block_idx, RangeParams p, int pass, in
             if (b != -1 && pass == 0) report_async(status, kAsyncBadIndex, 0x301);
             continue;
         }
-        const int tile = b * p.H_kv + r;
+        const int tile = tile_id(b, r, p);
         const int64_t e = (int64_t)row * p.top_k + s;
         if (pass == 0)
             rank[e] = (uint32_t)atomicAdd(&cnt[tile], 1);
@@ -125,10 +145,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     volatile int* abort = &sm.abort;
 
     const int n_tiles = p.n_blocks * p.H_kv;
-    const int total_items = item_off[n_tiles];
-    const int per_cta = (total_items + gridDim.x - 1) / gridDim.x;
-    const int it_lo = min(total_items, (int)blockIdx.x * per_cta);
-    const int it_hi = min(total_items, it_lo + per_cta);
+    const int phases = n_phases(p);
 
     if (threadIdx.x == 0) {
         mbar_init(&sm.in_full, 1);
@@ -154,75 +171,77 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         // Tile metadata lives in registers and is refreshed only when the walk crosses into the
         // next tile; an item's handles follow the previous item's in memory (the handle array is
         // laid out tile after tile), so the next item's handles are fetched one item ahead.
-        int tile = 0;
-        if (it_lo < it_hi) {  // last tile whose first item is <= it_lo (skips empty tiles)
-            int lo = 0, hi = n_tiles;
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (item_off[mid] <= it_lo) lo = mid; else hi = mid;
-            }
-            tile = lo;
-        }
-        int i_next = 0, p_end = 0, first = 0;
         const int handles_end = tile_off[n_tiles];
-        if (it_lo < it_hi) {
-            i_next = item_off[tile + 1]; p_end = tile_off[tile + 1];
-            first = tile_off[tile] + (it_lo - item_off[tile]) * QPI;
-        }
-        uint32_t h_next = 0;
-        if (it_lo < it_hi && first + lane < handles_end) h_next = handles[first + lane];
-        int loaded_tile = -1;
-        for (int it = it_lo; it < it_hi; ++it) {
-            const int n = it - it_lo;
-            while (i_next <= it) {  // crossed into the next non-empty tile
-                ++tile;
-                i_next = item_off[tile + 1];
-                p_end = tile_off[tile + 1];
+        // Q rows are gathered top_k times each, K/V tiles and partials go by once.
+        const uint64_t pol_q = l2_policy_evict_last(), pol_kv = l2_policy_evict_first();
+        int loaded_tile = -1, n = 0;
+        bool ok = true;
+        for (int ph = 0; ph < phases && ok; ++ph) {
+            int it_lo, it_hi;
+            phase_items(item_off, p, ph, it_lo, it_hi);
+            if (it_lo >= it_hi) continue;
+            int tile;
+            {   // last tile of the phase whose first item is <= it_lo (skips empty tiles)
+                int lo = ph * p.n_blocks, hi = (ph + 1) * p.n_blocks;
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (item_off[mid] <= it_lo) lo = mid; else hi = mid;
+                }
+                tile = lo;
             }
-            const int b = tile / p.H_kv, r = tile % p.H_kv;
-            const int nq = min(QPI, p_end - first);
-            const uint32_t h = lane < nq ? h_next : 0u;
-            {
-                const int nf = first + nq;  // the next item's handles start where this item's end
-                h_next = (it + 1 < it_hi && nf + lane < handles_end) ? handles[nf + lane] : 0u;
-            }
-            // The Q buffer is free once the previous item's first MMA has read it.
-            if (n > 0 && !mbar_wait(&sm.s_full, (n - 1) & 1, abort)) {
-                if (lane == 0) report_async(status, kAsyncTimeout, 0x311);
-                break;
-            }
-            if (lane < QPI) sm.info_handle[n & 1][lane] = h;
-            if (lane == 0) {
-                sm.info_block[n & 1] = b; sm.info_r[n & 1] = r; sm.info_nq[n & 1] = nq;
-            }
-            __syncwarp();
-            const bool new_tile = tile != loaded_tile;
-            if (lane == 0)
-                mbar_arrive_expect_tx(&sm.in_full, nq * 2 * Q_BOX_BYTES + (new_tile ? KV_BYTES : 0u));
-            __syncwarp();
-            // One G-row box per (query, d half): 2*QPI boxes, one per lane.
-            if (lane < 2 * QPI) {
-                const int qi = lane >> 1, dh = lane & 1;
-                const uint32_t hq = __shfl_sync((2 * QPI == 32) ? 0xffffffffu : ((1u << (2 * QPI)) - 1u), h, qi);
-                if (qi < nq)
-                    tma_load_3d(sm.q[dh] + qi * Q_BOX_BYTES, &tm_q, dh * 64, r * G,
-                                (int)(p.q_first + (hq >> 8)), &sm.in_full);
-            }
-            if (new_tile) {
-                // K/V buffers are free once the previous item's second MMA has read V.
-                if (n > 0 && !mbar_wait(&sm.o_full, (n - 1) & 1, abort)) {
-                    if (lane == 0) report_async(status, kAsyncTimeout, 0x312);
+            int i_next = item_off[tile + 1], p_end = tile_off[tile + 1];
+            int first = tile_off[tile] + (it_lo - item_off[tile]) * QPI;
+            uint32_t h_next = first + lane < handles_end ? handles[first + lane] : 0u;
+            for (int it = it_lo; it < it_hi; ++it, ++n) {
+                while (i_next <= it) {  // crossed into the next non-empty tile
+                    ++tile;
+                    i_next = item_off[tile + 1];
+                    p_end = tile_off[tile + 1];
+                }
+                const int r = ph, b = tile - ph * p.n_blocks;
+                const int nq = min(QPI, p_end - first);
+                const uint32_t h = lane < nq ? h_next : 0u;
+                {
+                    const int nf = first + nq;  // the next item's handles start where this item's end
+                    h_next = (it + 1 < it_hi && nf + lane < handles_end) ? handles[nf + lane] : 0u;
+                }
+                // The Q buffer is free once the previous item's first MMA has read it.
+                if (n > 0 && !mbar_wait(&sm.s_full, (n - 1) & 1, abort)) {
+                    if (lane == 0) report_async(status, kAsyncTimeout, 0x311);
+                    ok = false;
                     break;
                 }
+                if (lane < QPI) sm.info_handle[n & 1][lane] = h;
                 if (lane == 0) {
-                    tma_load_3d(sm.k[0], &tm_k, 0, r, b * BK, &sm.in_full);
-                    tma_load_3d(sm.k[1], &tm_k, 64, r, b * BK, &sm.in_full);
-                    tma_load_3d(sm.v[0], &tm_v, 0, r, b * BK, &sm.in_full);
-                    tma_load_3d(sm.v[1], &tm_v, 64, r, b * BK, &sm.in_full);
+                    sm.info_block[n & 1] = b; sm.info_r[n & 1] = r; sm.info_nq[n & 1] = nq;
                 }
-                loaded_tile = tile;
+                __syncwarp();
+                const bool new_tile = tile != loaded_tile;
+                if (lane == 0)
+                    mbar_arrive_expect_tx(&sm.in_full, nq * 2 * Q_BOX_BYTES + (new_tile ? KV_BYTES : 0u));
+                __syncwarp();
+                // One box per query: its G heads x 128 d, one contiguous read of G*256 bytes, laid
+                // down as [8 heads][d half][8 heads][64 d] so that every 1 KB is one operand atom.
+                if (lane < nq)
+                    tma_load_5d_hint(&sm.q[0][0] + lane * (2 * Q_BOX_BYTES), &tm_q, 0, 0, 0, r * (G / 8),
+                                     (int)(p.q_first + (h >> 8)), &sm.in_full, pol_q);
+                if (new_tile) {
+                    // K/V buffers are free once the previous item's second MMA has read V.
+                    if (n > 0 && !mbar_wait(&sm.o_full, (n - 1) & 1, abort)) {
+                        if (lane == 0) report_async(status, kAsyncTimeout, 0x312);
+                        ok = false;
+                        break;
+                    }
+                    if (lane == 0) {
+                        tma_load_3d_hint(sm.k[0], &tm_k, 0, r, b * BK, &sm.in_full, pol_kv);
+                        tma_load_3d_hint(sm.k[1], &tm_k, 64, r, b * BK, &sm.in_full, pol_kv);
+                        tma_load_3d_hint(sm.v[0], &tm_v, 0, r, b * BK, &sm.in_full, pol_kv);
+                        tma_load_3d_hint(sm.v[1], &tm_v, 64, r, b * BK, &sm.in_full, pol_kv);
+                    }
+                    loaded_tile = tile;
+                }
+                first += nq;
             }
-            first += nq;
         }
         if (*abort != 0) spin_cycles(200000);
     } else if (warp == 1) {
@@ -230,14 +249,20 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (lane == 0) {
             constexpr uint32_t idesc_s = make_idesc_bf16(128, BK, false, false);
             constexpr uint32_t idesc_o = make_idesc_bf16(128, 128, false, true);
-            const uint64_t qd0 = make_smem_desc(smem_u32(sm.q[0]), 16, 1024);
-            const uint64_t qd1 = make_smem_desc(smem_u32(sm.q[1]), 16, 1024);
+            // Q atoms (8 rows x 64 d) of one d half are 2 KB apart; the other half sits 1 KB further.
+            const uint64_t qd0 = make_smem_desc(smem_u32(&sm.q[0][0]), 16, 2048);
+            const uint64_t qd1 = make_smem_desc(smem_u32(&sm.q[0][0]) + 1024, 16, 2048);
             const uint64_t kd0 = make_smem_desc(smem_u32(sm.k[0]), 16, 1024);
             const uint64_t kd1 = make_smem_desc(smem_u32(sm.k[1]), 16, 1024);
             // V as the MN-major B operand: next 64 columns of d are BK*128 bytes away.
             const uint64_t vd = make_smem_desc(smem_u32(sm.v[0]), BK * 128, 1024);
-            for (int it = it_lo; it < it_hi; ++it) {
-                const int n = it - it_lo;
+            int n_items = 0;
+            for (int ph = 0; ph < phases; ++ph) {
+                int lo, hi;
+                phase_items(item_off, p, ph, lo, hi);
+                n_items += max(hi - lo, 0);
+            }
+            for (int n = 0; n < n_items; ++n) {
                 if (!mbar_wait(&sm.in_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x321); break; }
                 tc_fence_after();
 #pragma unroll
@@ -263,8 +288,14 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const int row = quarter * 32 + lane;
         const int qi = row / G, g = row % G;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        for (int it = it_lo; it < it_hi; ++it) {
-            const int n = it - it_lo;
+        int n_items = 0;
+        for (int ph = 0; ph < phases; ++ph) {
+            int lo, hi;
+            phase_items(item_off, p, ph, lo, hi);
+            n_items += max(hi - lo, 0);
+        }
+        const uint64_t pol_o = l2_policy_evict_first();
+        for (int n = 0; n < n_items; ++n) {
             if (!mbar_wait(&sm.s_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x331); break; }
             tc_fence_after();
             const int b = sm.info_block[n & 1], r = sm.info_r[n & 1], nq = sm.info_nq[n & 1];
@@ -318,7 +349,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             if (!mbar_wait(&sm.o_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x332); break; }
             tc_fence_after();
             const float inv = 1.0f / ell;
-            const int64_t prow = (ql * p.H_kv + r) * (int64_t)p.top_k + slot;
+            const int64_t prow = partial_base(ql, r, p) + slot;
             // Partial layout inside a (query, group, slot) region of G*256 bytes: [16-byte chunk of d][head],
             // so the G lanes of one query write G*16 contiguous bytes per store instruction.
             __nv_bfloat16* oreg = o_buf + prow * (G * 128) + g * 8;
@@ -339,7 +370,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                                 __uint_as_float(ov[c][j4 * 8 + 2 * w + 1]) * inv);
                             pk[w] = *reinterpret_cast<const uint32_t*>(&ob);
                         }
-                        *reinterpret_cast<uint4*>(oreg + (c * 4 + j4) * (G * 8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        st_global_v4_hint(oreg + (c * 4 + j4) * (G * 8), pk[0], pk[1], pk[2], pk[3], pol_o);
                     }
             }
             if (valid) lse_buf[prow * G + g] = (mc + log2f(ell)) * 0.6931471805599453f;
@@ -371,7 +402,7 @@ combine_kernel(const int32_t* __restrict__ block_idx, RangeParams p, const __nv_
     const int64_t q = p.q_first + ql;
     const int64_t loc = (p.q_begin + q) / BK;
     const int32_t* sel = block_idx + (q * p.H_kv + r) * (int64_t)p.top_k;
-    const int64_t pbase = ((int64_t)ql * p.H_kv + r) * p.top_k;
+    const int64_t pbase = partial_base(ql, r, p);
     for (int s = t; s < p.top_k; s += G * 16) {
         const int32_t b = sel[s];
         valid_s[s] = (b >= 0 && (int64_t)b <= loc) ? 1 : 0;

@@ -76,6 +76,7 @@ static msa_status_t check_range(int64_t q_begin, int64_t q_count, int64_t kv_len
 }
 
 static int sm_count();
+static int current_device();
 
 static msa_status_t launch_status() {
     return cudaPeekAtLastError() == cudaSuccess ? MSA_OK : MSA_ERR_CUDA;
@@ -134,12 +135,13 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
     int* status = async_status_ptr();
     if (status == nullptr) return MSA_ERR_CUDA;
     const size_t smem = sizeof(IdxSmem<NH, DI, ST>) + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set_dev[64] = {false};  // the attribute is per device
+    const int dev_id = current_device();
+    if (!attr_set_dev[dev_id]) {
         if (cudaFuncSetAttribute(index_scores_tc_kernel<BK, NH, DI, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem) != cudaSuccess)
             return MSA_ERR_CUDA;
-        attr_set = true;
+        attr_set_dev[dev_id] = true;
     }
     const int64_t grid = ceil_div64(q_count, kIdxTileQ) * (r.H_kv / NH);
     if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
@@ -296,15 +298,18 @@ static int64_t attn_range_for(const Resolved& r, int64_t q_count, int64_t kv_len
     return R;
 }
 
+static int current_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+    return dev;
+}
+
 static int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            n = 148;
-    }
-    return n;
+    static int n[64] = {0};  // per device
+    const int dev = current_device();
+    if (n[dev] == 0 && cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        n[dev] = 148;
+    return n[dev];
 }
 
 // Copy-out hook used by msa_prefill_forward_host: after each query range is combined, its
@@ -367,24 +372,26 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
     __nv_bfloat16* o_buf = (__nv_bfloat16*)(w + pl.off_obuf);
 
     CUtensorMap tm_q, tm_k, tm_v;
-    const uint64_t qd[3] = {128, (uint64_t)r.H_q, (uint64_t)q_count};
-    const uint64_t qs[2] = {256, (uint64_t)r.H_q * 256};
-    const uint32_t qb[3] = {64, (uint32_t)G, 1};
+    // Q as (64 d, 8 heads, 2 d halves, H_q/8 head groups, query): one box is a query's G heads.
+    const uint64_t qd[5] = {64, 8, 2, (uint64_t)r.H_q / 8, (uint64_t)q_count};
+    const uint64_t qs[4] = {256, 128, 2048, (uint64_t)r.H_q * 256};
+    const uint32_t qb[5] = {64, 8, 2, (uint32_t)G / 8, 1};
     const uint64_t kd[3] = {128, (uint64_t)r.H_kv, (uint64_t)kv_len};
     const uint64_t ks[2] = {256, (uint64_t)r.H_kv * 256};
     const uint32_t kb[3] = {64, 1, (uint32_t)BK};
-    if (!encode_tmap_bf16(&tm_q, q, 3, qd, qs, qb) || !encode_tmap_bf16(&tm_k, k, 3, kd, ks, kb) ||
+    if (!encode_tmap_bf16(&tm_q, q, 5, qd, qs, qb) || !encode_tmap_bf16(&tm_k, k, 3, kd, ks, kb) ||
         !encode_tmap_bf16(&tm_v, v, 3, kd, ks, kb))
         return MSA_ERR_CUDA;
     int* status = async_status_ptr();
     if (status == nullptr) return MSA_ERR_CUDA;
     const size_t smem = sizeof(AttnSmem<BK>) + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set_dev[64] = {false};  // the attribute is per device
+    const int dev_id = current_device();
+    if (!attr_set_dev[dev_id]) {
         if (cudaFuncSetAttribute(attn_prefill_tc_kernel<BK, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem) != cudaSuccess)
             return MSA_ERR_CUDA;
-        attr_set = true;
+        attr_set_dev[dev_id] = true;
     }
     const float scale_log2e = r.softmax_scale * 1.4426950408889634f;
     const int grid_attn = 2 * sm_count();
@@ -472,12 +479,13 @@ static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const v
     int* status = async_status_ptr();
     if (status == nullptr) return MSA_ERR_CUDA;
     const size_t smem = sizeof(DecSmem<BK>) + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set_dev[64] = {false};  // the attribute is per device
+    const int dev_id = current_device();
+    if (!attr_set_dev[dev_id]) {
         if (cudaFuncSetAttribute(attn_decode_kernel<BK, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
             cudaSuccess)
             return MSA_ERR_CUDA;
-        attr_set = true;
+        attr_set_dev[dev_id] = true;
     }
     DecParams p;
     p.q = (const __nv_bfloat16*)q; p.block_idx = block_idx; p.seq_offsets = seq_offsets; p.seq_lens = seq_lens;

@@ -99,7 +99,12 @@ __device__ __forceinline__ int warp_excl_scan(int v, int lane) {
 }
 
 constexpr int kTopkWarps = 4;
-constexpr int kTopkStage = 160;  // flush threshold (32) + one round of four pushes (4 x 32)
+#ifndef MSA_TOPK_LOADS
+#define MSA_TOPK_LOADS 8
+#endif
+constexpr int kTopkLoads = MSA_TOPK_LOADS;            // coalesced 32-wide loads per round
+constexpr int kTopkRound = 32 * kTopkLoads;           // blocks covered by one round
+constexpr int kTopkStage = 32 + kTopkRound;           // flush threshold (32) + one round of pushes
 constexpr int kTopkLog = 768;    // survivors remembered per row for the index pass
 
 template <int R>
@@ -133,7 +138,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
     const unsigned lt_mask = (1u << lane) - 1u;
 
     // ------------------------------------------------------------------ pass 1: threshold value
-    // A round covers 128 consecutive blocks as four coalesced 32-wide loads, so that compacting
+    // A round covers kTopkRound consecutive blocks as coalesced 32-wide loads, so that compacting
     // the loads one after the other keeps the survivors in block order.
     uint32_t kept[R];
 #pragma unroll
@@ -165,40 +170,46 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
     };
 
     {
+        constexpr int C = kTopkLoads;
         const int n = (int)loc;  // candidates are blocks [0, n); n < 2^31
-        float nxt[4];
+        float nxt[C];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < C; ++c) {
             const int i = c * 32 + lane;
             nxt[c] = i < n ? __ldg(srow + i) : -INFINITY;
         }
-        for (int i0 = 0; i0 < n; i0 += 128) {
-            float x[4];
+        for (int i0 = 0; i0 < n; i0 += kTopkRound) {
+            float x[C];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) x[c] = nxt[c];
+            for (int c = 0; c < C; ++c) x[c] = nxt[c];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {  // next round's loads are in flight while this one is ranked
-                const int i = i0 + 128 + c * 32 + lane;
+            for (int c = 0; c < C; ++c) {  // next round's loads are in flight while this one is ranked
+                const int i = i0 + kTopkRound + c * 32 + lane;
                 nxt[c] = i < n ? __ldg(srow + i) : -INFINITY;
             }
             // While fewer than m keys are kept everything passes; afterwards only strictly better
             // scores can change the m-th best value.  (Out-of-range lanes hold -inf.)
-            unsigned mk[4];
+            unsigned mk[C];
+            unsigned any = 0u;
             if (tau_f == -INFINITY) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) mk[c] = __ballot_sync(0xffffffffu, i0 + c * 32 + lane < n);
+                for (int c = 0; c < C; ++c) mk[c] = __ballot_sync(0xffffffffu, i0 + c * 32 + lane < n);
             } else {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) mk[c] = __ballot_sync(0xffffffffu, x[c] > tau_f);
+                for (int c = 0; c < C; ++c) mk[c] = __ballot_sync(0xffffffffu, x[c] > tau_f);
             }
-            if ((mk[0] | mk[1] | mk[2] | mk[3]) == 0u) continue;
-            // survivors keep block order: component 0's lanes first, then component 1's, ...
-            const int n0 = __popc(mk[0]), n1 = __popc(mk[1]), n2 = __popc(mk[2]), n3 = __popc(mk[3]);
-            const int tot = n0 + n1 + n2 + n3;
-            if (log_ok && n_log + tot > kTopkLog) log_ok = false;
-            const int off[4] = {0, n0, n0 + n1, n0 + n1 + n2};
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < C; ++c) any |= mk[c];
+            if (any == 0u) continue;
+            // survivors keep block order: component 0's lanes first, then component 1's, ...
+            int off[C + 1];
+            off[0] = 0;
+#pragma unroll
+            for (int c = 0; c < C; ++c) off[c + 1] = off[c] + __popc(mk[c]);
+            const int tot = off[C];
+            if (log_ok && n_log + tot > kTopkLog) log_ok = false;
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
                 if (mk[c] & (1u << lane)) {
                     const int rnk = off[c] + __popc(mk[c] & lt_mask);
                     const uint32_t key = topk_key(x[c]);
