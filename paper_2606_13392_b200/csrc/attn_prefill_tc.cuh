@@ -9,7 +9,7 @@
 //   2. attention: a tile's handles are cut into items of 128/G queries; an item stacks those
 //      queries' G heads into one 128-row operand (query concatenation), computes
 //      S = Q K_b^T into TMEM, a row softmax local to the item (one block = one S tile),
-//      P (bf16) to shared memory, O = P V_b into TMEM, and writes the locally normalised
+//      P (bf16) back into TMEM, O = P V_b into TMEM, and writes the locally normalised
 //      partial and its log-sum-exp to the workspace;
 //   3. combine: LSE-weighted merge of each query's partials (Section 4.2, two-phase forward).
 #pragma once
@@ -17,8 +17,6 @@
 #include "tc_common.cuh"
 
 namespace msa {
-
-constexpr int kAttnThreads = 192;  // warp 0: TMA + item walk, warp 1: MMA, warps 2-5: softmax/epilogue
 
 struct RangeParams {
     int64_t q_begin;   // absolute position of the first query of the call
@@ -106,38 +104,70 @@ revidx_scan_kernel(int32_t* __restrict__ cnt, int n_tiles, int qpi, int32_t* __r
 }
 
 // ---------------------------------------------------------------- 2. attention
-template <int BK>
-struct AttnSmem {
-    alignas(1024) uint8_t q[2][128 * 128];   // [d half][row = query*G + head][64 bf16]
-    alignas(1024) uint8_t k[2][BK * 128];    // [d half][key][64 bf16]
-    alignas(1024) uint8_t v[2][BK * 128];
-    alignas(8) uint64_t in_full, s_full, p_full, o_full, drain;
-    uint32_t tmem_base;
-    int abort;
-    // per-item info, double-buffered by item parity
-    int32_t info_block[2], info_r[2], info_nq[2];
-    uint32_t info_handle[2][16];
+constexpr int kAttnInfoRing = 8;  // item descriptors; deeper than the furthest reader lags
+
+struct AttnItemInfo {
+    int32_t block, r, nq;
+    int32_t kb, vb;        // K and V buffers of this item's tile
+    int32_t new_tile;      // first item of its tile in this CTA: wait for the K/V loads
+    int32_t last_of_tile;  // last item of its tile in this CTA: release the K/V buffers
+    int32_t pad;
+    uint32_t handle[16];
 };
 
-// Per-CTA pipeline (two CTAs share an SM):
-//   producer : Q(n+1) boxes as soon as MMA1(n) has read Q(n) (s_full); K/V of a new tile once
-//              MMA2(n) has read V (o_full).
-//   MMA      : in_full(n) -> S = Q K^T -> s_full(n);  p_full(n) -> O = P V -> o_full(n).
-//              MMAs execute in issue order, so S(n+1) may be issued right behind O(n) although
-//              P(n) lives in the columns S(n+1) overwrites.
-//   softmax  : s_full(n) -> read S row, exp2, write P (bf16 pairs) over the S columns ->
-//              p_full(n); o_full(n) -> O row / ell -> partial; then item n+1.
+template <int BK>
+struct AttnSmem {
+    alignas(1024) uint8_t q[2][128 * 256];     // [context][query][head group of 8][d half][8 heads][64 bf16]
+    alignas(1024) uint8_t kv[3][2][BK * 128];  // three tile buffers [d half][key][64 bf16]; roles rotate (see below)
+    alignas(1024) uint8_t ostage[2][128 * 256];  // [context][query][16-byte chunk of d][head]: partials on their way out
+    alignas(8) uint64_t q_full[2], q_empty[2];
+    uint64_t kv_full[3], kv_empty[3];
+    uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort;
+    AttnItemInfo info[kAttnInfoRing];
+};
+
+// K and V tiles rotate through three buffers: the t-th tile a CTA touches keeps K in buffer
+// (2t) mod 3 and V in buffer (2t+1) mod 3.  The next tile's K goes to the third buffer (free since
+// the tile before), its V to this tile's K buffer, which is free as soon as this tile's last
+// S = Q K^T has run, about one softmax before the first O = P V of the next tile needs it: tiles
+// change without a bubble on 1.5x the memory of one tile pair.  Every buffer is used twice per
+// three tiles, so the phase parity of a use depends only on the buffer and the role.
+__device__ __forceinline__ int kv_k_buf(int t) { return (2 * t) % 3; }
+__device__ __forceinline__ int kv_v_buf(int t) { return (2 * t + 1) % 3; }
+__device__ __forceinline__ int kv_k_parity(int kb) { return kb == 1 ? 1 : 0; }   // second use of buffer 1
+__device__ __forceinline__ int kv_v_parity(int vb) { return vb != 1 ? 1 : 0; }   // second use of buffers 0, 2
+
+// One CTA per SM, eleven warps, two items in flight (contexts j = n mod 2, each with its own Q
+// buffer, S/P and O columns in TMEM, softmax group and staging buffer):
+//   warps 0, 10  producers: both walk the CTA's share of the item list head phase after head phase;
+//             per item one TMA box per query into the context's Q buffer (free once S(n-2) has read
+//             it), warp 0 the first half of the queries and warp 10 the second (a warp spends about
+//             a hundred cycles per box it issues); per new tile warp 0 loads K, warp 10 loads V.
+//   warp 1    MMA issuer: S_j = Q(n) K^T as soon as Q(n) has landed, then O_j' = P(n-1) V once
+//             P(n-1) is written.  MMAs execute in issue order, which is what lets S(n+2) reuse
+//             the columns that hold P(n).
+//   warps 2-5 / 6-9  softmax groups: read the S row from TMEM, exp2 with the scale folded in,
+//             write P (bf16 pairs) over the S columns; then O row / ell as bf16 into the
+//             context's staging buffer and one bulk copy per query to the partial buffer.  The
+//             copies drain in the background: an SM moves about 32 bytes of stores per clock, and
+//             as 16-byte stores issued by the softmax warps they stalled those warps for a third
+//             of an item's time.
+constexpr int kAttnThreads = 352;
+
 template <int BK, int G>
-__global__ void __launch_bounds__(kAttnThreads, 2)
+__global__ void __launch_bounds__(kAttnThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, RangeParams p,
                        const int32_t* __restrict__ tile_off, const int32_t* __restrict__ item_off,
                        const uint32_t* __restrict__ handles, float scale_log2e,
                        __nv_bfloat16* __restrict__ o_buf, float* __restrict__ lse_buf, int* status) {
     constexpr int QPI = 128 / G;            // queries per item
-    constexpr int TMEM_COLS = 256;          // S (then P): columns 0..BK-1, O: columns 128..255
-    constexpr uint32_t Q_BOX_BYTES = G * 128;
-    constexpr uint32_t KV_BYTES = 4 * BK * 128;
+    constexpr int TMEM_COLS = 512;          // context j: S/P at j*256, O at j*256 + 128
+    constexpr uint32_t Q_BYTES = G * 256;   // one query's G heads
+    constexpr uint32_t KV_HALF = BK * 128;  // one d half of a K or V tile
     extern __shared__ uint8_t smem_raw[];
     AttnSmem<BK>& sm =
         *reinterpret_cast<AttnSmem<BK>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -146,12 +176,19 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
     const int n_tiles = p.n_blocks * p.H_kv;
     const int phases = n_phases(p);
+    int n_items = 0;  // items of this CTA over all phases (every role walks the same sequence)
+    for (int ph = 0; ph < phases; ++ph) {
+        int lo, hi;
+        phase_items(item_off, p, ph, lo, hi);
+        n_items += max(hi - lo, 0);
+    }
 
     if (threadIdx.x == 0) {
-        mbar_init(&sm.in_full, 1);
-        mbar_init(&sm.s_full, 1);
-        mbar_init(&sm.p_full, 4);
-        mbar_init(&sm.o_full, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sm.q_full[i], 2); mbar_init(&sm.q_empty[i], 1);
+            mbar_init(&sm.s_full[i], 1); mbar_init(&sm.p_full[i], 4); mbar_init(&sm.o_full[i], 1);
+        }
+        for (int i = 0; i < 3; ++i) { mbar_init(&sm.kv_full[i], 1); mbar_init(&sm.kv_empty[i], 1); }
         mbar_init(&sm.drain, 1);
         sm.abort = 0;
         fence_mbar_init();
@@ -164,17 +201,17 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
-    const uint32_t tmem_s = tmem, tmem_o = tmem + 128;
 
-    if (warp == 0) {
-        // ---------------- producer: walks the item list, gathers Q rows, loads K/V tiles
+    if (warp == 0 || warp == 10) {
+        // ---------------- producers
+        const int half = warp == 10 ? 1 : 0;  // warp 10: the second half of the queries, and V
         // Tile metadata lives in registers and is refreshed only when the walk crosses into the
         // next tile; an item's handles follow the previous item's in memory (the handle array is
         // laid out tile after tile), so the next item's handles are fetched one item ahead.
         const int handles_end = tile_off[n_tiles];
-        // Q rows are gathered top_k times each, K/V tiles and partials go by once.
+        // Q rows are gathered top_k times each, K/V tiles go by once.
         const uint64_t pol_q = l2_policy_evict_last(), pol_kv = l2_policy_evict_first();
-        int loaded_tile = -1, n = 0;
+        int loaded_tile = -1, tile_seq = -1, n = 0;
         bool ok = true;
         for (int ph = 0; ph < phases && ok; ++ph) {
             int it_lo, it_hi;
@@ -200,43 +237,62 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 }
                 const int r = ph, b = tile - ph * p.n_blocks;
                 const int nq = min(QPI, p_end - first);
+                const bool new_tile = tile != loaded_tile;
+                const bool last_of_tile = (it + 1 == it_hi) || (i_next <= it + 1);
+                if (new_tile) ++tile_seq;
+                const int kb = kv_k_buf(tile_seq), vb = kv_v_buf(tile_seq);
                 const uint32_t h = lane < nq ? h_next : 0u;
                 {
                     const int nf = first + nq;  // the next item's handles start where this item's end
                     h_next = (it + 1 < it_hi && nf + lane < handles_end) ? handles[nf + lane] : 0u;
                 }
-                // The Q buffer is free once the previous item's first MMA has read it.
-                if (n > 0 && !mbar_wait(&sm.s_full, (n - 1) & 1, abort)) {
+                const int j = n & 1;
+                // The context's Q buffer is free once S(n-2) has read it.
+                if (n >= 2 && !mbar_wait(&sm.q_empty[j], ((n >> 1) - 1) & 1, abort)) {
                     if (lane == 0) report_async(status, kAsyncTimeout, 0x311);
                     ok = false;
                     break;
                 }
-                if (lane < QPI) sm.info_handle[n & 1][lane] = h;
-                if (lane == 0) {
-                    sm.info_block[n & 1] = b; sm.info_r[n & 1] = r; sm.info_nq[n & 1] = nq;
+                // Slot n mod 8 was last read by the epilogue of item n-8, long before S(n-2) ran.
+                AttnItemInfo& inf = sm.info[n % kAttnInfoRing];
+                if (lane < QPI && half == 0) inf.handle[lane] = h;
+                if (lane == 0 && half == 0) {
+                    inf.block = b; inf.r = r; inf.nq = nq; inf.kb = kb; inf.vb = vb;
+                    inf.new_tile = new_tile ? 1 : 0; inf.last_of_tile = last_of_tile ? 1 : 0;
                 }
                 __syncwarp();
-                const bool new_tile = tile != loaded_tile;
-                if (lane == 0)
-                    mbar_arrive_expect_tx(&sm.in_full, nq * 2 * Q_BOX_BYTES + (new_tile ? KV_BYTES : 0u));
+                const int q_lo = half * (QPI / 2), q_hi = min(nq, q_lo + QPI / 2);
+                if (lane == 0) mbar_arrive_expect_tx(&sm.q_full[j], (uint32_t)max(q_hi - q_lo, 0) * Q_BYTES);
                 __syncwarp();
                 // One box per query: its G heads x 128 d, one contiguous read of G*256 bytes, laid
                 // down as [8 heads][d half][8 heads][64 d] so that every 1 KB is one operand atom.
-                if (lane < nq)
-                    tma_load_5d_hint(&sm.q[0][0] + lane * (2 * Q_BOX_BYTES), &tm_q, 0, 0, 0, r * (G / 8),
-                                     (int)(p.q_first + (h >> 8)), &sm.in_full, pol_q);
+                if (lane >= q_lo && lane < q_hi)
+                    tma_load_5d_hint(sm.q[j] + lane * Q_BYTES, &tm_q, 0, 0, 0, r * (G / 8),
+                                     (int)(p.q_first + (h >> 8)), &sm.q_full[j], pol_q);
                 if (new_tile) {
-                    // K/V buffers are free once the previous item's second MMA has read V.
-                    if (n > 0 && !mbar_wait(&sm.o_full, (n - 1) & 1, abort)) {
+                    // K: the buffer was the V buffer of the tile before last (or the K buffer three
+                    // tiles back); V: this buffer held the previous tile's K.
+                    const bool k_wait = tile_seq >= 3 || kv_k_parity(kb) == 1;
+                    const bool v_wait = tile_seq >= 3 || kv_v_parity(vb) == 1;
+                    if (half == 0 && k_wait && !mbar_wait(&sm.kv_empty[kb], kv_k_parity(kb) ^ 1, abort)) {
                         if (lane == 0) report_async(status, kAsyncTimeout, 0x312);
                         ok = false;
                         break;
                     }
-                    if (lane == 0) {
-                        tma_load_3d_hint(sm.k[0], &tm_k, 0, r, b * BK, &sm.in_full, pol_kv);
-                        tma_load_3d_hint(sm.k[1], &tm_k, 64, r, b * BK, &sm.in_full, pol_kv);
-                        tma_load_3d_hint(sm.v[0], &tm_v, 0, r, b * BK, &sm.in_full, pol_kv);
-                        tma_load_3d_hint(sm.v[1], &tm_v, 64, r, b * BK, &sm.in_full, pol_kv);
+                    if (lane == 0 && half == 0) {
+                        mbar_arrive_expect_tx(&sm.kv_full[kb], 2 * KV_HALF);
+                        tma_load_3d_hint(sm.kv[kb][0], &tm_k, 0, r, b * BK, &sm.kv_full[kb], pol_kv);
+                        tma_load_3d_hint(sm.kv[kb][1], &tm_k, 64, r, b * BK, &sm.kv_full[kb], pol_kv);
+                    }
+                    if (half == 1 && v_wait && !mbar_wait(&sm.kv_empty[vb], kv_v_parity(vb) ^ 1, abort)) {
+                        if (lane == 0) report_async(status, kAsyncTimeout, 0x313);
+                        ok = false;
+                        break;
+                    }
+                    if (lane == 0 && half == 1) {
+                        mbar_arrive_expect_tx(&sm.kv_full[vb], 2 * KV_HALF);
+                        tma_load_3d_hint(sm.kv[vb][0], &tm_v, 0, r, b * BK, &sm.kv_full[vb], pol_kv);
+                        tma_load_3d_hint(sm.kv[vb][1], &tm_v, 64, r, b * BK, &sm.kv_full[vb], pol_kv);
                     }
                     loaded_tile = tile;
                 }
@@ -249,33 +305,58 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (lane == 0) {
             constexpr uint32_t idesc_s = make_idesc_bf16(128, BK, false, false);
             constexpr uint32_t idesc_o = make_idesc_bf16(128, 128, false, true);
-            // Q atoms (8 rows x 64 d) of one d half are 2 KB apart; the other half sits 1 KB further.
-            const uint64_t qd0 = make_smem_desc(smem_u32(&sm.q[0][0]), 16, 2048);
-            const uint64_t qd1 = make_smem_desc(smem_u32(&sm.q[0][0]) + 1024, 16, 2048);
-            const uint64_t kd0 = make_smem_desc(smem_u32(sm.k[0]), 16, 1024);
-            const uint64_t kd1 = make_smem_desc(smem_u32(sm.k[1]), 16, 1024);
-            // V as the MN-major B operand: next 64 columns of d are BK*128 bytes away.
-            const uint64_t vd = make_smem_desc(smem_u32(sm.v[0]), BK * 128, 1024);
-            int n_items = 0;
-            for (int ph = 0; ph < phases; ++ph) {
-                int lo, hi;
-                phase_items(item_off, p, ph, lo, hi);
-                n_items += max(hi - lo, 0);
-            }
-            for (int n = 0; n < n_items; ++n) {
-                if (!mbar_wait(&sm.in_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x321); break; }
-                tc_fence_after();
+            int prev_vb = 0, prev_last = 0, prev_new = 0;
+            for (int n = 0; n <= n_items; ++n) {
+                int vb = 0, last = 0, nw = 0;
+                if (n < n_items) {
+                    const int j = n & 1;
+                    if (!mbar_wait(&sm.q_full[j], (n >> 1) & 1, abort)) {
+                        report_async(status, kAsyncTimeout, 0x321);
+                        break;
+                    }
+                    const AttnItemInfo& inf = sm.info[n % kAttnInfoRing];
+                    const int kb = inf.kb;
+                    vb = inf.vb; last = inf.last_of_tile; nw = inf.new_tile;
+                    if (nw && !mbar_wait(&sm.kv_full[kb], kv_k_parity(kb), abort)) {
+                        report_async(status, kAsyncTimeout, 0x322);
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t ts = tmem + j * 256;
+                    // Q atoms (8 rows x 64 d) of one d half are 2 KB apart; the other half sits 1 KB further.
+                    const uint64_t qd0 = make_smem_desc(smem_u32(sm.q[j]), 16, 2048);
+                    const uint64_t qd1 = make_smem_desc(smem_u32(sm.q[j]) + 1024, 16, 2048);
+                    const uint64_t kd0 = make_smem_desc(smem_u32(sm.kv[kb][0]), 16, 1024);
+                    const uint64_t kd1 = make_smem_desc(smem_u32(sm.kv[kb][1]), 16, 1024);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(tmem_s, qd0 + 2 * kk, kd0 + 2 * kk, idesc_s, kk > 0);
+                    for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(ts, qd0 + 2 * kk, kd0 + 2 * kk, idesc_s, kk > 0);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(tmem_s, qd1 + 2 * kk, kd1 + 2 * kk, idesc_s, true);
-                mma_commit(&sm.s_full);
-                if (!mbar_wait(&sm.p_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x323); break; }
-                tc_fence_after();
+                    for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(ts, qd1 + 2 * kk, kd1 + 2 * kk, idesc_s, true);
+                    mma_commit(&sm.q_empty[j]);
+                    mma_commit(&sm.s_full[j]);
+                    if (last) mma_commit(&sm.kv_empty[kb]);
+                }
+                if (n >= 1) {
+                    const int m = n - 1, jm = m & 1;
+                    if (!mbar_wait(&sm.p_full[jm], (m >> 1) & 1, abort)) {
+                        report_async(status, kAsyncTimeout, 0x323);
+                        break;
+                    }
+                    if (prev_new && !mbar_wait(&sm.kv_full[prev_vb], kv_v_parity(prev_vb), abort)) {
+                        report_async(status, kAsyncTimeout, 0x324);
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t ts = tmem + jm * 256, to = ts + 128;
+                    // V as the MN-major B operand: next 64 columns of d are BK*128 bytes away.
+                    const uint64_t vd = make_smem_desc(smem_u32(sm.kv[prev_vb][0]), BK * 128, 1024);
 #pragma unroll
-                for (int kk = 0; kk < BK / 16; ++kk)  // P: 8 packed columns per 16 keys; V: 2048 bytes per 16 keys
-                    mma_bf16_ts(tmem_o, tmem_s + kk * 8, vd + (uint64_t)(kk * 2048 / 16), idesc_o, kk > 0);
-                mma_commit(&sm.o_full);
+                    for (int kk = 0; kk < BK / 16; ++kk)  // P: 8 packed columns per 16 keys; V: 2048 bytes per 16 keys
+                        mma_bf16_ts(to, ts + kk * 8, vd + (uint64_t)(kk * 2048 / 16), idesc_o, kk > 0);
+                    mma_commit(&sm.o_full[jm]);
+                    if (prev_last) mma_commit(&sm.kv_empty[prev_vb]);
+                }
+                prev_vb = vb; prev_last = last; prev_new = nw;
             }
             if (*abort != 0) {
                 mma_commit(&sm.drain);
@@ -284,25 +365,26 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
     } else {
         // ---------------- softmax + epilogue: thread = row of the 128-row operand
+        const int j = (warp - 2) >> 2;  // context: items n = j (mod 2)
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const int qi = row / G, g = row % G;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        int n_items = 0;
-        for (int ph = 0; ph < phases; ++ph) {
-            int lo, hi;
-            phase_items(item_off, p, ph, lo, hi);
-            n_items += max(hi - lo, 0);
-        }
-        const uint64_t pol_o = l2_policy_evict_first();
-        for (int n = 0; n < n_items; ++n) {
-            if (!mbar_wait(&sm.s_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x331); break; }
+        const uint32_t tmem_s = tmem + j * 256, tmem_o = tmem_s + 128;
+        constexpr int QPW = 32 / G;  // queries per warp
+        // staging: this thread's row goes to [query][chunk][head]; lanes < QPW copy one query each
+        uint8_t* stg_row = sm.ostage[j] + (size_t)qi * Q_BYTES + g * 16;
+        const uint8_t* stg_query = sm.ostage[j] + (size_t)(quarter * QPW + lane) * Q_BYTES;
+        for (int n = j; n < n_items; n += 2) {
+            if (!mbar_wait(&sm.s_full[j], (n >> 1) & 1, abort)) { report_async(status, kAsyncTimeout, 0x331); break; }
             tc_fence_after();
-            const int b = sm.info_block[n & 1], r = sm.info_r[n & 1], nq = sm.info_nq[n & 1];
-            const uint32_t h = sm.info_handle[n & 1][qi];
+            const AttnItemInfo& inf = sm.info[n % kAttnInfoRing];
+            const int b = inf.block, r = inf.r, nq = inf.nq;
+            const uint32_t h = inf.handle[qi];
+            // handle of the query whose partial this lane hands to the bulk-copy engine
+            const uint32_t h_copy = inf.handle[(quarter * QPW + lane) & 15];
             const bool valid = qi < nq;
             const int64_t ql = h >> 8;
-            const int slot = h & 0xFF;
             const int64_t pos = p.q_begin + p.q_first + ql;
             // visible columns of this block for this query: 0..lim
             const int64_t lim64 = pos - (int64_t)b * BK;
@@ -343,39 +425,48 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.p_full);
+            if (lane == 0) mbar_arrive(&sm.p_full[j]);
 
-            // ---- epilogue: O row / ell -> bf16 partial, LSE partial
-            if (!mbar_wait(&sm.o_full, n & 1, abort)) { report_async(status, kAsyncTimeout, 0x332); break; }
+            // ---- epilogue: O row / ell -> bf16 partial (via the staging buffer), LSE partial
+            // The copies of the context's previous item have read the staging buffer long ago;
+            // the wait makes that certain.
+            if (lane < QPW) bulk_wait_read_all();
+            if (!mbar_wait(&sm.o_full[j], (n >> 1) & 1, abort)) { report_async(status, kAsyncTimeout, 0x332); break; }
             tc_fence_after();
             const float inv = 1.0f / ell;
-            const int64_t prow = partial_base(ql, r, p) + slot;
-            // Partial layout inside a (query, group, slot) region of G*256 bytes: [16-byte chunk of d][head],
-            // so the G lanes of one query write G*16 contiguous bytes per store instruction.
-            __nv_bfloat16* oreg = o_buf + prow * (G * 128) + g * 8;
-            uint32_t ov[4][32];
+            __syncwarp();
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld_32x32(tmem_o + lane_base + c * 32, ov[c]);
-            tmem_wait_ld();
-            if (valid) {
+            for (int c = 0; c < 4; ++c) {
+                uint32_t ov[32];
+                tmem_ld_32x32(tmem_o + lane_base + c * 32, ov);
+                tmem_wait_ld();
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int j4 = 0; j4 < 4; ++j4) {
+                    uint32_t pk[4];
 #pragma unroll
-                    for (int j4 = 0; j4 < 4; ++j4) {
-                        uint32_t pk[4];
-#pragma unroll
-                        for (int w = 0; w < 4; ++w) {
-                            const __nv_bfloat162 ob = __floats2bfloat162_rn(
-                                __uint_as_float(ov[c][j4 * 8 + 2 * w]) * inv,
-                                __uint_as_float(ov[c][j4 * 8 + 2 * w + 1]) * inv);
-                            pk[w] = *reinterpret_cast<const uint32_t*>(&ob);
-                        }
-                        st_global_v4_hint(oreg + (c * 4 + j4) * (G * 8), pk[0], pk[1], pk[2], pk[3], pol_o);
+                    for (int w = 0; w < 4; ++w) {
+                        const __nv_bfloat162 ob = __floats2bfloat162_rn(__uint_as_float(ov[j4 * 8 + 2 * w]) * inv,
+                                                                        __uint_as_float(ov[j4 * 8 + 2 * w + 1]) * inv);
+                        pk[w] = *reinterpret_cast<const uint32_t*>(&ob);
                     }
+                    *reinterpret_cast<uint4*>(stg_row + (c * 4 + j4) * (G * 16)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
             }
-            if (valid) lse_buf[prow * G + g] = (mc + log2f(ell)) * 0.6931471805599453f;
             tc_fence_before();
+            fence_proxy_async_smem();
+            __syncwarp();
+            // Partial of (query, group, slot): G*256 contiguous bytes, [16-byte chunk of d][head].
+            if (lane < QPW) {
+                if (quarter * QPW + lane < nq) {
+                    const int64_t pr = partial_base((int64_t)(h_copy >> 8), r, p) + (h_copy & 0xFF);
+                    bulk_store(o_buf + pr * (G * 128), stg_query, Q_BYTES);
+                }
+                bulk_commit();
+            }
+            if (valid)
+                lse_buf[(partial_base(ql, r, p) + (h & 0xFF)) * G + g] = (mc + log2f(ell)) * 0.6931471805599453f;
         }
+        if (lane < QPW) bulk_wait_all();  // partials still on their way out
     }
     tc_fence_before();
     __syncthreads();

@@ -394,7 +394,7 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
         attr_set_dev[dev_id] = true;
     }
     const float scale_log2e = r.softmax_scale * 1.4426950408889634f;
-    const int grid_attn = 2 * sm_count();
+    const int grid_attn = sm_count();  // one CTA per SM (all of its shared memory and TMEM)
     for (int64_t q_first = 0; q_first < q_count; q_first += R) {
         RangeParams p;
         p.q_begin = q_begin; p.q_first = q_first;
