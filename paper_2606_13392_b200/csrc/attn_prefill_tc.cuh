@@ -145,7 +145,7 @@ __device__ __forceinline__ int kv_v_parity(int vb) { return vb != 1 ? 1 : 0; }  
 //   warps 0, 10  producers: both walk the CTA's share of the item list head phase after head phase;
 //             per item one TMA box per query into the context's Q buffer (free once S(n-2) has read
 //             it), warp 0 the first half of the queries and warp 10 the second (a warp spends about
-//             a hundred cycles per box it issues); per new tile warp 0 loads K, warp 10 loads V.
+//             a hundred cycles per box it issues); per new tile warp 0 loads K and V.
 //   warp 1    MMA issuer: S_j = Q(n) K^T as soon as Q(n) has landed, then O_j' = P(n-1) V once
 //             P(n-1) is written.  MMAs execute in issue order, which is what lets S(n+2) reuse
 //             the columns that hold P(n).
@@ -204,7 +204,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
     if (warp == 0 || warp == 10) {
         // ---------------- producers
-        const int half = warp == 10 ? 1 : 0;  // warp 10: the second half of the queries, and V
+        const int half = warp == 10 ? 1 : 0;  // warp 10: the second half of the queries
         // Tile metadata lives in registers and is refreshed only when the walk crosses into the
         // next tile; an item's handles follow the previous item's in memory (the handle array is
         // laid out tile after tile), so the next item's handles are fetched one item ahead.
@@ -271,7 +271,10 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                                      (int)(p.q_first + (h >> 8)), &sm.q_full[j], pol_q);
                 if (new_tile) {
                     // K: the buffer was the V buffer of the tile before last (or the K buffer three
-                    // tiles back); V: this buffer held the previous tile's K.
+                    // tiles back); V: this buffer held the previous tile's K.  One warp does all the
+                    // waiting on a buffer's barrier: a parity wait is only right for a waiter that
+                    // has seen every earlier phase complete, and a second warp waiting for every
+                    // other phase could be two phases behind and be let through a phase early.
                     const bool k_wait = tile_seq >= 3 || kv_k_parity(kb) == 1;
                     const bool v_wait = tile_seq >= 3 || kv_v_parity(vb) == 1;
                     if (half == 0 && k_wait && !mbar_wait(&sm.kv_empty[kb], kv_k_parity(kb) ^ 1, abort)) {
@@ -284,12 +287,12 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         tma_load_3d_hint(sm.kv[kb][0], &tm_k, 0, r, b * BK, &sm.kv_full[kb], pol_kv);
                         tma_load_3d_hint(sm.kv[kb][1], &tm_k, 64, r, b * BK, &sm.kv_full[kb], pol_kv);
                     }
-                    if (half == 1 && v_wait && !mbar_wait(&sm.kv_empty[vb], kv_v_parity(vb) ^ 1, abort)) {
+                    if (half == 0 && v_wait && !mbar_wait(&sm.kv_empty[vb], kv_v_parity(vb) ^ 1, abort)) {
                         if (lane == 0) report_async(status, kAsyncTimeout, 0x313);
                         ok = false;
                         break;
                     }
-                    if (lane == 0 && half == 1) {
+                    if (lane == 0 && half == 0) {
                         mbar_arrive_expect_tx(&sm.kv_full[vb], 2 * KV_HALF);
                         tma_load_3d_hint(sm.kv[vb][0], &tm_v, 0, r, b * BK, &sm.kv_full[vb], pol_kv);
                         tma_load_3d_hint(sm.kv[vb][1], &tm_v, 64, r, b * BK, &sm.kv_full[vb], pol_kv);

@@ -100,6 +100,14 @@ def test_c3_shape_small_workspace_many_passes():
     assert torch.equal(o1, o2) and torch.equal(l1, l2)
 
 
+def test_single_item_tiles_many_ranges():
+    # Few selections per query and the smallest workspace: nearly every (block, head) tile of a
+    # query range holds a single item, so the K/V tile buffers change owner with every item.
+    cfg = CONFIGS["c3"].scaled(name="c3-lone", T=4096 + 19, top_k=4)
+    mn, _ = B.msa_prefill_forward_workspace_bytes(B.shape_of(cfg), cfg.T)
+    run_prefill_case(cfg, sharp=False, n_sample=96, ws_bytes=mn)
+
+
 @pytest.mark.parametrize("T,Hq,Hkv,Bk,k,d,di", [
     (1, 8, 1, 64, 8, 128, 64),        # a single token
     (63, 8, 1, 64, 8, 128, 64),       # less than one block
