@@ -174,10 +174,10 @@ def oracle_sample_size(cfg: MSAConfig) -> int:
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     # c4: captured at full size with a one-pass metric set (profiles/launch_list_and_dram_c4.md)
     ("c4", "index_scores"): 38.85e9, ("c4", "topk_select"): 17.62e9,
-    # (attention: 16.7 GB read + 33.7 GB written; half of the Q gathers now hit L2)
-    ("c4", "attn_prefill"): 50.7e9, ("c4", "combine"): 34.30e9,
-    # c3: c3-16k captures scaled by (query, group, block) pairs per launch (profiles/*_c3-16k.md)
-    ("c3", "attn_prefill"): 48.3e9, ("c3", "combine"): 26.8e9,
+    # (attention: 18.5 GB read + 33.7 GB written; half of the Q gathers hit L2)
+    ("c4", "attn_prefill"): 52.2e9, ("c4", "combine"): 34.30e9,
+    # c3: captured at full size with the same one-pass metric set (profiles/launch_list_and_dram_c4.md)
+    ("c3", "attn_prefill"): 39.96e9, ("c3", "combine"): 27.55e9,
     # c5: c5-small captures scaled by the selected K/V (resp. cached index keys) streamed
     ("c5", "attn_decode"): 1.106e9, ("c5", "index_scores_decode"): 2.47e9,
 }

@@ -437,6 +437,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             if (!mbar_wait(&sm.o_full[j], (n >> 1) & 1, abort)) { report_async(status, kAsyncTimeout, 0x332); break; }
             tc_fence_after();
             const float inv = 1.0f / ell;
+            const float2 inv2 = make_float2(inv, inv);
             __syncwarp();
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -447,9 +448,10 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 for (int j4 = 0; j4 < 4; ++j4) {
                     uint32_t pk[4];
 #pragma unroll
-                    for (int w = 0; w < 4; ++w) {
-                        const __nv_bfloat162 ob = __floats2bfloat162_rn(__uint_as_float(ov[j4 * 8 + 2 * w]) * inv,
-                                                                        __uint_as_float(ov[j4 * 8 + 2 * w + 1]) * inv);
+                    for (int w = 0; w < 4; ++w) {  // packed two-float multiply: half the instructions
+                        const float2 o2 = __fmul2_rn(make_float2(__uint_as_float(ov[j4 * 8 + 2 * w]),
+                                                                 __uint_as_float(ov[j4 * 8 + 2 * w + 1])), inv2);
+                        const __nv_bfloat162 ob = __floats2bfloat162_rn(o2.x, o2.y);
                         pk[w] = *reinterpret_cast<const uint32_t*>(&ob);
                     }
                     *reinterpret_cast<uint4*>(stg_row + (c * 4 + j4) * (G * 16)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
