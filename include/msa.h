@@ -201,6 +201,29 @@ msa_status_t msa_prefill_forward_workspace_bytes(const msa_shape_t* shape, int64
                                                  size_t* min_bytes, size_t* preferred_bytes);
 
 /*
+ * Whole path, prefill, for a batch of sequences of different lengths packed token-major
+ * (Section 4.2 names variable-length sequences as a source of uneven tile work; blocks are
+ * counted from each sequence's own first token, every sequence is causal on its own and no
+ * quantity of Eq. 6-8 crosses a sequence boundary).  Sequence s owns rows
+ * cu_seqlens[s] .. cu_seqlens[s+1]-1 of q, k, v, q_idx, k_idx, out, lse and block_idx;
+ * cu_seqlens is a HOST array of n_seqs+1 non-decreasing row offsets (int64), cu_seqlens[0] >= 0.
+ * block_idx holds block numbers relative to the row's own sequence.  Sequences of length 0 are
+ * skipped.  The sequences are run one after the other through the single-sequence path on
+ * `stream`; workspace >= msa_prefill_forward_varlen_workspace_bytes (the largest single
+ * sequence's need).  Errors: MSA_ERR_INVALID_ARG for a NULL or decreasing cu_seqlens or
+ * n_seqs < 0, otherwise as msa_prefill_forward.
+ */
+msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q, const void* k,
+                                        const void* v, const void* q_idx, const void* k_idx,
+                                        const int64_t* cu_seqlens, int32_t n_seqs, void* out,
+                                        float* lse, int32_t* block_idx, void* workspace,
+                                        size_t workspace_bytes, msa_stream_t stream);
+
+msa_status_t msa_prefill_forward_varlen_workspace_bytes(const msa_shape_t* shape,
+                                                        const int64_t* cu_seqlens, int32_t n_seqs,
+                                                        size_t* min_bytes, size_t* preferred_bytes);
+
+/*
  * Same, from HOST buffers: copies q, k, v, q_idx, k_idx host->device into the staging
  * area at the front of `workspace`, runs the three stages, copies `out` (and lse,
  * block_idx when non-NULL) back, and synchronises before returning.  The copies run on a

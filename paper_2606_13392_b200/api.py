@@ -28,6 +28,24 @@ def prefill_forward(cfg: MSAConfig, x: Dict[str, torch.Tensor], workspace: Optio
     return out, lse, block_idx
 
 
+def prefill_forward_varlen(cfg: MSAConfig, x: Dict[str, torch.Tensor], cu_seqlens,
+                           workspace: Optional[torch.Tensor] = None, want_lse: bool = True):
+    """The same for sequences packed token-major; cu_seqlens: n_seqs+1 row offsets (host ints).
+    block_idx holds block numbers relative to each row's own sequence."""
+    shape = B.shape_of(cfg)
+    T = x["q"].shape[0]
+    dev = x["q"].device
+    out = torch.empty_like(x["q"])
+    lse = torch.empty((T, cfg.n_q_heads), dtype=torch.float32, device=dev) if want_lse else None
+    block_idx = torch.empty((T, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32, device=dev)
+    if workspace is None:
+        _, pf = B.msa_prefill_forward_varlen_workspace_bytes(shape, cu_seqlens)
+        workspace = B.alloc_workspace(pf, dev)
+    B.msa_prefill_forward_varlen(shape, x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"], cu_seqlens, out, lse,
+                                 block_idx, workspace)
+    return out, lse, block_idx
+
+
 def index_scores(cfg: MSAConfig, q_idx: torch.Tensor, k_idx: torch.Tensor, q_begin: int, q_count: int,
                  kv_len: Optional[int] = None) -> torch.Tensor:
     """Eq. 6 for rows [q_begin, q_begin+q_count); q_idx holds the whole sequence's rows."""

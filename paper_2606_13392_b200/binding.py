@@ -28,7 +28,8 @@ EXPORTS = [
     "msa_sparse_attn_prefill_workspace_bytes", "msa_sparse_attn_prefill_static",
     "msa_sparse_attn_decode",
     "msa_sparse_attn_decode_workspace_bytes", "msa_prefill_forward",
-    "msa_prefill_forward_workspace_bytes", "msa_prefill_forward_host",
+    "msa_prefill_forward_workspace_bytes", "msa_prefill_forward_varlen",
+    "msa_prefill_forward_varlen_workspace_bytes", "msa_prefill_forward_host",
     "msa_prefill_forward_host_workspace_bytes", "msa_decode_forward", "msa_decode_forward_host",
     "msa_launch_count", "msa_profile_begin", "msa_profile_end",
 ]
@@ -228,6 +229,30 @@ def msa_prefill_forward(shape, q, k, v, q_idx, k_idx, T, out, lse, block_idx, wo
                                      _dev(workspace),
                                      c_sz(workspace.numel() * workspace.element_size()),
                                      _stream(stream)), "msa_prefill_forward")
+
+
+def _cu_array(cu_seqlens):
+    cu = [int(c) for c in cu_seqlens]
+    return (c_i64 * len(cu))(*cu), len(cu) - 1
+
+
+def msa_prefill_forward_varlen_workspace_bytes(shape, cu_seqlens) -> Tuple[int, int]:
+    arr, n = _cu_array(cu_seqlens)
+    mn, pf = c_sz(0), c_sz(0)
+    _check(lib().msa_prefill_forward_varlen_workspace_bytes(ctypes.byref(shape), arr, c_i32(n),
+                                                            ctypes.byref(mn), ctypes.byref(pf)),
+           "msa_prefill_forward_varlen_workspace_bytes")
+    return int(mn.value), int(pf.value)
+
+
+def msa_prefill_forward_varlen(shape, q, k, v, q_idx, k_idx, cu_seqlens, out, lse, block_idx, workspace,
+                               stream=None):
+    arr, n = _cu_array(cu_seqlens)
+    _check(lib().msa_prefill_forward_varlen(ctypes.byref(shape), _dev(q), _dev(k), _dev(v), _dev(q_idx),
+                                            _dev(k_idx), arr, c_i32(n), _dev(out), _dev(lse),
+                                            _dev(block_idx), _dev(workspace),
+                                            c_sz(workspace.numel() * workspace.element_size()),
+                                            _stream(stream)), "msa_prefill_forward_varlen")
 
 
 def msa_prefill_forward_host_workspace_bytes(shape, T) -> Tuple[int, int]:

@@ -856,6 +856,64 @@ static msa_status_t prefill_stages_1_2(const msa_shape_t* shape, const Resolved&
     return MSA_OK;
 }
 
+static msa_status_t check_cu_seqlens(const int64_t* cu, int32_t n_seqs) {
+    if (n_seqs < 0 || cu == nullptr || cu[0] < 0) return MSA_ERR_INVALID_ARG;
+    for (int32_t i = 0; i < n_seqs; ++i)
+        if (cu[i + 1] < cu[i]) return MSA_ERR_INVALID_ARG;
+    return MSA_OK;
+}
+
+msa_status_t msa_prefill_forward_varlen_workspace_bytes(const msa_shape_t* shape,
+                                                        const int64_t* cu_seqlens, int32_t n_seqs,
+                                                        size_t* min_bytes, size_t* preferred_bytes) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if ((s = check_cu_seqlens(cu_seqlens, n_seqs)) != MSA_OK) return s;
+    size_t mn = kAlign, pf = kAlign;
+    for (int32_t i = 0; i < n_seqs; ++i) {
+        size_t a = 0, b = 0;
+        if ((s = msa_prefill_forward_workspace_bytes(shape, cu_seqlens[i + 1] - cu_seqlens[i], &a, &b)) != MSA_OK)
+            return s;
+        if (a > mn) mn = a;
+        if (b > pf) pf = b;
+    }
+    if (min_bytes) *min_bytes = mn;
+    if (preferred_bytes) *preferred_bytes = pf;
+    return MSA_OK;
+}
+
+msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q, const void* k,
+                                        const void* v, const void* q_idx, const void* k_idx,
+                                        const int64_t* cu_seqlens, int32_t n_seqs, void* out,
+                                        float* lse, int32_t* block_idx, void* workspace,
+                                        size_t workspace_bytes, msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if ((s = check_cu_seqlens(cu_seqlens, n_seqs)) != MSA_OK) return s;
+    if (n_seqs == 0 || cu_seqlens[n_seqs] == cu_seqlens[0]) return MSA_OK;
+    if (!q || !k || !v || !q_idx || !k_idx || !out || !block_idx) return MSA_ERR_INVALID_ARG;
+    size_t need = 0;
+    if ((s = msa_prefill_forward_varlen_workspace_bytes(shape, cu_seqlens, n_seqs, &need, nullptr)) != MSA_OK)
+        return s;
+    if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
+    // Every sequence is an independent problem: the single-sequence path on row-offset pointers.
+    const size_t q_row = (size_t)r.H_q * r.d * 2, kv_row = (size_t)r.H_kv * r.d * 2;
+    const size_t qi_row = (size_t)r.H_kv * r.d_idx * 2, ki_row = (size_t)r.d_idx * 2;
+    for (int32_t i = 0; i < n_seqs; ++i) {
+        const int64_t o = cu_seqlens[i], T = cu_seqlens[i + 1] - o;
+        if (T == 0) continue;
+        s = msa_prefill_forward(shape, (const char*)q + o * q_row, (const char*)k + o * kv_row,
+                                (const char*)v + o * kv_row, (const char*)q_idx + o * qi_row,
+                                (const char*)k_idx + o * ki_row, T, (char*)out + o * q_row,
+                                lse ? lse + o * r.H_q : nullptr, block_idx + o * (int64_t)r.H_kv * r.k, workspace,
+                                workspace_bytes, stream);
+        if (s != MSA_OK) return s;
+    }
+    return MSA_OK;
+}
+
 static size_t host_staging_bytes(const Resolved& r, int64_t T, size_t off[8]) {
     size_t o = 0;
     off[0] = o; o += align_up((size_t)T * r.H_q * r.d * 2);      // q

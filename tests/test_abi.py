@@ -89,6 +89,23 @@ def test_workspace_queries(lib):
     assert code == 3
 
 
+def test_varlen_validation_and_workspace(lib):
+    shape = B.shape_of(CONFIGS["c3"])
+    one = ctypes.c_void_p(256)  # non-null, never dereferenced on these paths
+    i64x3 = (ctypes.c_int64 * 3)
+    args = lambda cu, n: (ctypes.byref(shape), one, one, one, one, one, cu, ctypes.c_int32(n), one, None, one,
+                          one, ctypes.c_size_t(16), None)
+    assert lib.msa_prefill_forward_varlen(*args(None, 2)) == 1                  # no offsets
+    assert lib.msa_prefill_forward_varlen(*args(i64x3(0, 500, 400), 2)) == 1    # decreasing
+    assert lib.msa_prefill_forward_varlen(*args(i64x3(0, 0, 0), 2)) == 0        # nothing to do
+    assert lib.msa_prefill_forward_varlen(*args(i64x3(0, 500, 900), -1)) == 1
+    assert lib.msa_prefill_forward_varlen(*args(i64x3(0, 500, 900), 2)) == 3    # workspace too small
+    # the batch needs what its longest sequence needs
+    mn, pf = B.msa_prefill_forward_varlen_workspace_bytes(shape, [0, 300, 5000, 5100])
+    m1, p1 = B.msa_prefill_forward_workspace_bytes(shape, 4700)
+    assert (mn, pf) == (m1, p1)
+
+
 def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "missing.so"))

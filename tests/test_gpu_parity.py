@@ -100,6 +100,43 @@ def test_c3_shape_small_workspace_many_passes():
     assert torch.equal(o1, o2) and torch.equal(l1, l2)
 
 
+def test_varlen_batch_equals_sequence_by_sequence():
+    # Packed sequences of different lengths (one shorter than a block, one empty): every sequence
+    # must come out exactly as from its own single-sequence call, and one of them is checked
+    # against the oracle through the packed call's outputs.
+    cfg = CONFIGS["c3"].scaled(name="c3-varlen", T=0, top_k=8)
+    lens = [1000, 37, 0, 4096 + 5, 129, 2500]
+    cu = np.concatenate([[0], np.cumsum(lens)]).tolist()
+    total = cu[-1]
+    x = make_prefill_inputs(cfg.scaled(T=total), DEV, sharp=False)
+    out, lse, I = api.prefill_forward_varlen(cfg.scaled(T=total), x, cu)
+    torch.cuda.synchronize()
+    _assert_clean()
+    for s, L in enumerate(lens):
+        if L == 0:
+            continue
+        a, b = cu[s], cu[s + 1]
+        xs = {n: t[a:b].contiguous() for n, t in x.items()}
+        o1, l1, i1 = api.prefill_forward(cfg.scaled(T=L), xs)
+        torch.cuda.synchronize()
+        assert torch.equal(I[a:b], i1), "sequence %d index lists" % s
+        assert torch.equal(out[a:b], o1) and torch.equal(lse[a:b], l1), "sequence %d outputs" % s
+    # oracle on the fourth sequence, positions relative to that sequence
+    s = 3
+    a, b, L = cu[s], cu[s + 1], lens[s]
+    pos = sample_positions(L, cfg.block_size, cfg.top_k, 64, 11)
+    pos_t = torch.from_numpy(pos).to(DEV)
+    kb, vb, kib = to_bits(x["k"][a:b]), to_bits(x["v"][a:b]), to_bits(x["k_idx"][a:b])
+    qb, qib = to_bits(x["q"][a:b][pos_t]), to_bits(x["q_idx"][a:b][pos_t])
+    M_ref = oracle.index_scores(qib, kib, pos, cfg.block_size)
+    I_ref = oracle.topk_select(M_ref, pos, L, cfg.block_size, cfg.top_k)
+    I_gpu = I[a:b][pos_t].cpu().numpy()
+    exact, n_rows = check_selection(I_gpu, I_ref, M_ref, pos, cfg.block_size, cfg.top_k)
+    assert exact >= 0.999
+    O_ref, LSE_ref = oracle.sparse_attn(qb, kb, vb, I_gpu, pos, cfg.block_size)
+    check_attn(out[a:b][pos_t].float().cpu().numpy(), lse[a:b][pos_t].cpu().numpy(), O_ref, LSE_ref, "varlen")
+
+
 def test_single_item_tiles_many_ranges():
     # Few selections per query and the smallest workspace: nearly every (block, head) tile of a
     # query range holds a single item, so the K/V tile buffers change owner with every item.
