@@ -93,6 +93,23 @@ def topk_select(M, pos, L: int, block_size: int, top_k: int) -> np.ndarray:
     return I
 
 
+def index_lse(q_idx, k_idx, I, pos, block_size: int, scale: Optional[float] = None) -> np.ndarray:
+    """Section 4.3 (LSE fusion): log-sum-exp of the index scores over the visible tokens of the
+    selected blocks.  q_idx [n,H_kv,d_idx] u16, k_idx [L,d_idx] u16, I [n,H_kv,k] int32 -> [n,H_kv] f64."""
+    q_idx, k_idx, pos = _u16(q_idx), _u16(k_idx), _pos(pos)
+    I = np.ascontiguousarray(I, dtype=np.int32)
+    n, H_kv, d_idx = q_idx.shape
+    L = k_idx.shape[0]
+    assert k_idx.shape[1] == d_idx and len(pos) == n and I.shape[:2] == (n, H_kv)
+    if scale is None:
+        scale = 1.0 / np.sqrt(d_idx)
+    out = np.empty((n, H_kv), dtype=np.float64)
+    _load().msa_oracle_index_lse(_p(q_idx), _p(k_idx), _p(I), _p(pos), ctypes.c_int64(n),
+                                 ctypes.c_int64(L), H_kv, d_idx, block_size, I.shape[2],
+                                 ctypes.c_double(scale), _p(out))
+    return out
+
+
 def sparse_attn(q, K, V, I, pos, block_size: int, scale: Optional[float] = None):
     """Eq. 8.  q [n,H_q,d] u16, K,V [L,H_kv,d] u16, I [n,H_kv,k] -> (O [n,H_q,d], LSE [n,H_q]) f64."""
     q, K, V, pos = _u16(q), _u16(K), _u16(V), _pos(pos)

@@ -74,6 +74,45 @@ void msa_oracle_index_scores(const uint16_t* q_idx, const uint16_t* k_idx,
     }
 }
 
+/*
+ * Section 4.3, "LSE fusion": the log-sum-exp of the index branch over the selected blocks,
+ *   LSE_idx[i,r] = log sum over b in I[i,r], j in block b, j <= i of exp(S[i,r,j])
+ * with S as in Eq. 6 (natural logarithm).  The paper obtains it by reducing per-block
+ * log-sum-exps over the Top-k blocks; here it is the definition written out as one sum,
+ * stabilised by the largest selected score.  Entries of I below 0 are padding.
+ * q_idx: [n, H_kv, d_idx]; k_idx: [L, d_idx]; I: [n, H_kv, k]; out: [n, H_kv].
+ */
+void msa_oracle_index_lse(const uint16_t* q_idx, const uint16_t* k_idx, const int32_t* I,
+                          const int64_t* pos, int64_t n, int64_t L, int H_kv, int d_idx,
+                          int B_k, int k, double scale, double* out) {
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t a = 0; a < n * H_kv; ++a) {
+        const int64_t qi = a / H_kv;
+        const int64_t i = pos[qi];
+        const uint16_t* qrow = q_idx + a * (int64_t)d_idx;
+        const int32_t* sel = I + a * (int64_t)k;
+        double best = -INFINITY, sum = 0.0;
+        for (int pass = 0; pass < 2; ++pass) {  /* pass 0: the largest score; pass 1: the sum */
+            for (int t = 0; t < k; ++t) {
+                if (sel[t] < 0) continue;
+                const int64_t j0 = (int64_t)sel[t] * B_k;
+                int64_t j1 = j0 + B_k;
+                if (j1 > L) j1 = L;
+                for (int64_t j = j0; j < j1 && j <= i; ++j) {
+                    const uint16_t* krow = k_idx + j * (int64_t)d_idx;
+                    double s = 0.0;
+                    for (int c = 0; c < d_idx; ++c)
+                        s += bf16_to_double(qrow[c]) * bf16_to_double(krow[c]);
+                    s *= scale;
+                    if (pass == 0) { if (s > best) best = s; }
+                    else sum += exp(s - best);
+                }
+            }
+        }
+        out[a] = (best == -INFINITY) ? -INFINITY : best + log(sum);
+    }
+}
+
 typedef struct {
     double score;
     int32_t block;

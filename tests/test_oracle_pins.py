@@ -348,6 +348,50 @@ def test_group_sharing_uses_adjacent_heads():
 
 
 # ---------------------------------------------------------------- P5: printed FLOPs ratio
+def test_index_lse_brute_force_dense_limit_and_bounds():
+    # Section 4.3 (LSE fusion).  (a) token-by-token enumeration; (b) with every visible block
+    # selected it is the log-sum-exp of the whole causal score row, which scipy computes from an
+    # einsum; (c) it is the log-sum-exp of per-block log-sum-exps (the reduction the paper
+    # describes), for any split of the list; (d) it lies between the largest selected block score
+    # and that plus the log of the number of tokens summed.
+    from scipy.special import logsumexp
+    cfg, x = tiny(T=61, Hq=4, Hkv=2, Bk=4, k=4, di=8, seed=21)
+    pos = np.arange(cfg.T)
+    M = oracle.index_scores(x["q_idx"], x["k_idx"], pos, cfg.block_size)
+    I = oracle.topk_select(M, pos, cfg.T, cfg.block_size, cfg.top_k)
+    got = oracle.index_lse(x["q_idx"], x["k_idx"], I, pos, cfg.block_size)
+    qi, ki = f64(x["q_idx"]), f64(x["k_idx"])
+    for i in range(cfg.T):
+        for r in range(cfg.n_kv_heads):
+            blocks = [b for b in I[i, r] if b >= 0]
+            z = np.array([np.dot(qi[i, r], ki[j]) / np.sqrt(cfg.idx_dim)
+                          for j in range(i + 1) if j // cfg.block_size in blocks])
+            want = np.log(np.exp(z - z.max()).sum()) + z.max()
+            assert abs(got[i, r] - want) < 1e-12
+            # (d)
+            top = max(M[i, r, b] for b in blocks)
+            assert top - 1e-12 <= got[i, r] <= top + np.log(len(z)) + 1e-12
+            # (c): two sub-lists, each padded with -1
+            if len(blocks) >= 2:
+                a, b2 = blocks[:1], blocks[1:]
+                Ia = np.full((1, 1, cfg.top_k), -1, np.int32); Ia[0, 0, :len(a)] = a
+                Ib = np.full((1, 1, cfg.top_k), -1, np.int32); Ib[0, 0, :len(b2)] = b2
+                la = oracle.index_lse(x["q_idx"][i:i + 1, r:r + 1], x["k_idx"], Ia, [i], cfg.block_size)[0, 0]
+                lb = oracle.index_lse(x["q_idx"][i:i + 1, r:r + 1], x["k_idx"], Ib, [i], cfg.block_size)[0, 0]
+                assert abs(np.logaddexp(la, lb) - got[i, r]) < 1e-12
+    # (b)
+    k_all = cfg.n_blocks
+    I_all = oracle.topk_select(M, pos, cfg.T, cfg.block_size, k_all)
+    dense = oracle.index_lse(x["q_idx"], x["k_idx"], I_all, pos, cfg.block_size)
+    S = np.einsum("irc,jc->irj", qi, ki) / np.sqrt(cfg.idx_dim)
+    causal = np.arange(cfg.T)[None, :] <= np.arange(cfg.T)[:, None]
+    S = np.where(causal[:, None, :], S, -np.inf)
+    np.testing.assert_allclose(dense, logsumexp(S, axis=-1), rtol=0, atol=1e-12)
+    # an all-padding list has nothing to sum
+    I_none = np.full((1, 1, 3), -1, np.int32)
+    assert np.isneginf(oracle.index_lse(x["q_idx"][:1, :1], x["k_idx"], I_none, [0], cfg.block_size)[0, 0])
+
+
 def test_flops_model_printed_ratio():
     path = os.path.join(os.path.dirname(__file__), "golden", "flops_reduction_1m.txt")
     vals = {}
