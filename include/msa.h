@@ -188,6 +188,28 @@ msa_status_t msa_sparse_attn_decode_workspace_bytes(const msa_shape_t* shape, in
                                                     size_t* min_bytes);
 
 /* ------------------------------------------------------------------------------------
+ * Index-branch log-sum-exp over the selected blocks (Section 4.3, "LSE fusion": the forward
+ * emits LSE_idx so that the sparse-KL backward need not recompute it):
+ *   lse_idx[i,r] = log sum over b in block_idx[i,r,:], j in block b, j <= q_begin+i of
+ *                  exp(<q_idx[i,r,:], k_idx[j,:]> * index_scale)            (natural log)
+ * q_idx [q_count,H_kv,d_idx] bf16 (rows of the range), k_idx [kv_len,d_idx] bf16, block_idx
+ * [q_count,H_kv,k] int32 as written by msa_topk_select (entries < 0 are padding), lse_idx
+ * [q_count,H_kv] float32 (out; -inf for a row with no valid entry).  Runs after Top-k, KV-outer
+ * over the (block, head) tiles like the attention, on warp-level tensor-core MMAs for
+ * d_idx in {64,128} and B_k in {64,128}; any other shape takes a plain kernel that needs no
+ * workspace.  workspace >= msa_index_lse_prefill_workspace_bytes (device, 16-byte aligned).
+ * Errors as msa_sparse_attn_prefill; a block index outside [-1, loc] sets the async status.
+ */
+msa_status_t msa_index_lse_prefill(const msa_shape_t* shape, const void* q_idx, const void* k_idx,
+                                   const int32_t* block_idx, int64_t q_begin, int64_t q_count,
+                                   int64_t kv_len, float* lse_idx, void* workspace,
+                                   size_t workspace_bytes, msa_stream_t stream);
+
+msa_status_t msa_index_lse_prefill_workspace_bytes(const msa_shape_t* shape, int64_t q_count,
+                                                   int64_t kv_len, size_t* min_bytes,
+                                                   size_t* preferred_bytes);
+
+/* ------------------------------------------------------------------------------------
  * Whole path, prefill (Algorithm 1, lines 3-5) for one sequence of T tokens: runs stage 1
  * and 2 over query chunks sized to the workspace, then stage 3.  block_idx [T,H_kv,k] is
  * an output (required); lse may be NULL.  workspace >= msa_prefill_forward_workspace_bytes.
@@ -281,8 +303,9 @@ int64_t msa_launch_count(void);
  * msa_profile_begin() and msa_profile_end() every kernel launch of the library is
  * bracketed by CUDA events on its stream; msa_profile_end() synchronises the device and
  * returns, per stage, the summed device time in milliseconds and the number of launches
- * (arrays of 8: 0 index scoring, 1 top-k, 2 reverse index/schedule, 3 prefill attention,
- * 4 combine, 5 decode index scoring, 6 decode attention, 7 decode combine).  The first
+ * (arrays of 9: 0 index scoring, 1 top-k, 2 reverse index/schedule, 3 prefill attention,
+ * 4 combine, 5 decode index scoring, 6 decode attention, 7 decode combine, 8 index-branch
+ * log-sum-exp).  The first
  * msa_profile_begin() creates the event pool (8192 launches); MSA_ERR_UNSUPPORTED from
  * msa_profile_end() means the pool ran out and the sums are partial.  Not thread-safe.
  */

@@ -46,6 +46,22 @@ def prefill_forward_varlen(cfg: MSAConfig, x: Dict[str, torch.Tensor], cu_seqlen
     return out, lse, block_idx
 
 
+def index_lse(cfg: MSAConfig, q_idx: torch.Tensor, k_idx: torch.Tensor, block_idx: torch.Tensor,
+              q_begin: int = 0, q_count: Optional[int] = None, kv_len: Optional[int] = None,
+              workspace_bytes: Optional[int] = None) -> torch.Tensor:
+    """Section 4.3: log-sum-exp of the index scores over the selected blocks, rows
+    [q_begin, q_begin+q_count); q_idx and block_idx hold the whole sequence's rows."""
+    shape = B.shape_of(cfg)
+    kv_len = k_idx.shape[0] if kv_len is None else kv_len
+    q_count = q_idx.shape[0] - q_begin if q_count is None else q_count
+    out = torch.empty((q_count, cfg.n_kv_heads), dtype=torch.float32, device=q_idx.device)
+    mn, pf = B.msa_index_lse_prefill_workspace_bytes(shape, q_count, kv_len)
+    ws = B.alloc_workspace(pf if workspace_bytes is None else max(mn, workspace_bytes), q_idx.device)
+    B.msa_index_lse_prefill(shape, q_idx[q_begin:q_begin + q_count], k_idx, block_idx[q_begin:q_begin + q_count],
+                            q_begin, q_count, kv_len, out, ws)
+    return out
+
+
 def index_scores(cfg: MSAConfig, q_idx: torch.Tensor, k_idx: torch.Tensor, q_begin: int, q_count: int,
                  kv_len: Optional[int] = None) -> torch.Tensor:
     """Eq. 6 for rows [q_begin, q_begin+q_count); q_idx holds the whole sequence's rows."""

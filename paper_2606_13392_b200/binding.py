@@ -27,7 +27,8 @@ EXPORTS = [
     "msa_topk_select", "msa_topk_select_decode", "msa_sparse_attn_prefill",
     "msa_sparse_attn_prefill_workspace_bytes", "msa_sparse_attn_prefill_static",
     "msa_sparse_attn_decode",
-    "msa_sparse_attn_decode_workspace_bytes", "msa_prefill_forward",
+    "msa_sparse_attn_decode_workspace_bytes", "msa_index_lse_prefill",
+    "msa_index_lse_prefill_workspace_bytes", "msa_prefill_forward",
     "msa_prefill_forward_workspace_bytes", "msa_prefill_forward_varlen",
     "msa_prefill_forward_varlen_workspace_bytes", "msa_prefill_forward_host",
     "msa_prefill_forward_host_workspace_bytes", "msa_decode_forward", "msa_decode_forward_host",
@@ -108,7 +109,7 @@ def launch_count() -> int:
 
 
 STAGES = ["index_scores", "topk_select", "schedule", "attn_prefill", "combine",
-          "index_scores_decode", "attn_decode", "combine_decode"]
+          "index_scores_decode", "attn_decode", "combine_decode", "index_lse"]
 
 
 def profile_begin() -> None:
@@ -117,10 +118,10 @@ def profile_begin() -> None:
 
 def profile_end():
     """-> {stage: (ms, launches)} summed since profile_begin(); synchronises the device."""
-    ms = (ctypes.c_float * 8)()
-    n = (c_i64 * 8)()
+    ms = (ctypes.c_float * len(STAGES))()
+    n = (c_i64 * len(STAGES))()
     _check(lib().msa_profile_end(ms, n), "msa_profile_end")
-    return {STAGES[i]: (float(ms[i]), int(n[i])) for i in range(8)}
+    return {STAGES[i]: (float(ms[i]), int(n[i])) for i in range(len(STAGES))}
 
 
 def check_async_status() -> Tuple[int, int]:
@@ -229,6 +230,22 @@ def msa_prefill_forward(shape, q, k, v, q_idx, k_idx, T, out, lse, block_idx, wo
                                      _dev(workspace),
                                      c_sz(workspace.numel() * workspace.element_size()),
                                      _stream(stream)), "msa_prefill_forward")
+
+
+def msa_index_lse_prefill_workspace_bytes(shape, q_count, kv_len) -> Tuple[int, int]:
+    mn, pf = c_sz(0), c_sz(0)
+    _check(lib().msa_index_lse_prefill_workspace_bytes(ctypes.byref(shape), c_i64(q_count), c_i64(kv_len),
+                                                       ctypes.byref(mn), ctypes.byref(pf)),
+           "msa_index_lse_prefill_workspace_bytes")
+    return int(mn.value), int(pf.value)
+
+
+def msa_index_lse_prefill(shape, q_idx, k_idx, block_idx, q_begin, q_count, kv_len, lse_idx, workspace,
+                          stream=None):
+    _check(lib().msa_index_lse_prefill(ctypes.byref(shape), _dev(q_idx), _dev(k_idx), _dev(block_idx),
+                                       c_i64(q_begin), c_i64(q_count), c_i64(kv_len), _dev(lse_idx),
+                                       _dev(workspace), c_sz(workspace.numel() * workspace.element_size()),
+                                       _stream(stream)), "msa_index_lse_prefill")
 
 
 def _cu_array(cu_seqlens):

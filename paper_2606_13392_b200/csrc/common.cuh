@@ -55,7 +55,8 @@ enum Stage : int {
     kStageIndexDecode = 5,
     kStageAttnDecode = 6,
     kStageCombineDecode = 7,
-    kNumStages = 8
+    kStageIndexLse = 8,   // Section 4.3: index-branch log-sum-exp over the selected blocks
+    kNumStages = 9
 };
 
 // Wraps one kernel launch: counts it and, while profiling is on, brackets it with CUDA

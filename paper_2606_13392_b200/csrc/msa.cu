@@ -10,6 +10,7 @@
 #include "topk.cuh"
 #include "index_scores_tc.cuh"
 #include "attn_prefill_tc.cuh"
+#include "index_lse.cuh"
 #include "decode.cuh"
 
 namespace msa {
@@ -508,6 +509,98 @@ static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const v
     return launch_status();
 }
 
+// ---------------------------------------------------------------------- index-branch LSE (Section 4.3)
+static bool index_lse_fast(const Resolved& r) {
+    return (r.d_idx == 64 || r.d_idx == 128) && (r.B_k == 64 || r.B_k == 128);
+}
+
+// Workspace for ranges of R queries: [cnt | tile_off | item_off] per tile, handles, rank, partials.
+struct LsePlan {
+    size_t off_cnt, off_tile_off, off_item_off, off_handles, off_rank, off_part, total;
+};
+
+static LsePlan lse_plan(const Resolved& r, int64_t kv_len, int64_t R) {
+    LsePlan p;
+    const size_t n_tiles = (size_t)ceil_div64(kv_len, r.B_k) * r.H_kv + 1;
+    const size_t pairs = (size_t)R * r.H_kv * r.k;
+    size_t o = 0;
+    p.off_cnt = o; o += align_up(n_tiles * 4);
+    p.off_tile_off = o; o += align_up(n_tiles * 4);
+    p.off_item_off = o; o += align_up(n_tiles * 4);
+    p.off_handles = o; o += align_up(pairs * 4);
+    p.off_rank = o; o += align_up(pairs * 4);
+    p.off_part = o; o += align_up(pairs * 4);
+    p.total = o;
+    return p;
+}
+
+template <int BK, int DIDX>
+static msa_status_t run_index_lse(const Resolved& r, const void* q_idx, const void* k_idx,
+                                  const int32_t* block_idx, int64_t q_begin, int64_t q_count, int64_t kv_len,
+                                  float* lse_idx, void* ws, size_t ws_bytes, cudaStream_t st) {
+    const size_t fixed = lse_plan(r, kv_len, 0).total + 4 * kAlign;
+    if (ws_bytes <= fixed) return MSA_ERR_WORKSPACE;
+    int64_t R = (int64_t)((ws_bytes - fixed) / ((size_t)r.H_kv * r.k * 12));
+    if (R > q_count) R = q_count;
+    if (R > (1 << 23)) R = 1 << 23;  // handles keep the query in 24 bits
+    if (R <= 0) return MSA_ERR_WORKSPACE;
+    const LsePlan pl = lse_plan(r, kv_len, R);
+    char* w = static_cast<char*>(ws);
+    int32_t* cnt = (int32_t*)(w + pl.off_cnt);
+    int32_t* tile_off = (int32_t*)(w + pl.off_tile_off);
+    int32_t* item_off = (int32_t*)(w + pl.off_item_off);
+    uint32_t* handles = (uint32_t*)(w + pl.off_handles);
+    uint32_t* rank = (uint32_t*)(w + pl.off_rank);
+    float* part = (float*)(w + pl.off_part);
+    int* status = async_status_ptr();
+    if (status == nullptr) return MSA_ERR_CUDA;
+    const size_t smem = (size_t)(BK + kLseItemQueries) * (DIDX + 8) * 2 + kLseItemQueries * 4;
+    static bool attr_set_dev[64] = {false};  // the attribute is per device
+    const int dev_id = current_device();
+    if (!attr_set_dev[dev_id]) {
+        if (cudaFuncSetAttribute(index_lse_kernel<BK, DIDX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+            cudaSuccess)
+            return MSA_ERR_CUDA;
+        attr_set_dev[dev_id] = true;
+    }
+    const float scale_log2e = r.index_scale * 1.4426950408889634f;
+    const int grid = sm_count() * (smem > 48 * 1024 ? 3 : 4);
+    for (int64_t q_first = 0; q_first < q_count; q_first += R) {
+        RangeParams p;
+        p.q_begin = q_begin; p.q_first = q_first;
+        p.q_count = (int32_t)((q_count - q_first) < R ? (q_count - q_first) : R);
+        p.n_blocks = (int32_t)ceil_div64(q_begin + q_first + p.q_count, BK);
+        p.H_kv = r.H_kv; p.top_k = r.k;
+        const int n_tiles = p.n_blocks * r.H_kv;
+        const unsigned eg = (unsigned)ceil_div64((int64_t)p.q_count * r.H_kv, 8);  // 8 warps (rows) per CTA
+        if (cudaMemsetAsync(cnt, 0, (size_t)(n_tiles + 1) * 4, st) != cudaSuccess) return MSA_ERR_CUDA;
+        {
+            StageScope sc(kStageSchedule, st);
+            revidx_kernel<BK><<<eg, 256, 0, st>>>(block_idx, p, 0, cnt, tile_off, rank, handles, status);
+        }
+        {
+            StageScope sc(kStageSchedule, st);
+            revidx_scan_kernel<<<1, 1024, 0, st>>>(cnt, n_tiles, kLseItemQueries, tile_off, item_off);
+        }
+        {
+            StageScope sc(kStageSchedule, st);
+            revidx_kernel<BK><<<eg, 256, 0, st>>>(block_idx, p, 1, cnt, tile_off, rank, handles, status);
+        }
+        {
+            StageScope sc(kStageIndexLse, st);
+            index_lse_kernel<BK, DIDX><<<grid, kLseThreads, smem, st>>>(
+                (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx, p, kv_len, tile_off, item_off, handles,
+                scale_log2e, part);
+        }
+        {
+            StageScope sc(kStageIndexLse, st);
+            index_lse_reduce_kernel<BK><<<eg, 256, 0, st>>>(block_idx, p, part, lse_idx);
+        }
+        if (cudaPeekAtLastError() != cudaSuccess) return MSA_ERR_CUDA;
+    }
+    return MSA_OK;
+}
+
 }  // namespace msa
 
 using namespace msa;
@@ -687,6 +780,62 @@ msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, co
     }
     return run_attn_generic(r, q, k, v, block_idx, prefill_rows(q_begin, kv_len, r.B_k), q_count, out,
                             lse, st);
+}
+
+// ---------------------------------------------------------------------- index-branch LSE (Section 4.3)
+msa_status_t msa_index_lse_prefill_workspace_bytes(const msa_shape_t* shape, int64_t q_count,
+                                                   int64_t kv_len, size_t* min_bytes,
+                                                   size_t* preferred_bytes) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if (q_count < 0 || kv_len < 0) return MSA_ERR_INVALID_ARG;
+    size_t mn = kAlign, pf = kAlign;
+    if (index_lse_fast(r) && q_count > 0) {
+        const int64_t r_min = q_count < 256 ? q_count : 256;
+        const int64_t r_pref = q_count < 131072 ? q_count : 131072;
+        mn = lse_plan(r, kv_len, r_min).total + 8 * kAlign;
+        pf = lse_plan(r, kv_len, r_pref).total + 8 * kAlign;
+    }
+    if (min_bytes) *min_bytes = mn;
+    if (preferred_bytes) *preferred_bytes = pf;
+    return MSA_OK;
+}
+
+msa_status_t msa_index_lse_prefill(const msa_shape_t* shape, const void* q_idx, const void* k_idx,
+                                   const int32_t* block_idx, int64_t q_begin, int64_t q_count,
+                                   int64_t kv_len, float* lse_idx, void* workspace,
+                                   size_t workspace_bytes, msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if ((s = check_range(q_begin, q_count, kv_len)) != MSA_OK) return s;
+    if (q_count == 0) return MSA_OK;
+    if (!q_idx || !k_idx || !block_idx || !lse_idx || !aligned16(q_idx) || !aligned16(k_idx))
+        return MSA_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (index_lse_fast(r) && kv_len < 2147483647LL) {
+        size_t need = 0;
+        msa_index_lse_prefill_workspace_bytes(shape, q_count, kv_len, &need, nullptr);
+        if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
+        if (r.B_k == 64 && r.d_idx == 64)
+            return run_index_lse<64, 64>(r, q_idx, k_idx, block_idx, q_begin, q_count, kv_len, lse_idx, workspace, workspace_bytes, st);
+        if (r.B_k == 64)
+            return run_index_lse<64, 128>(r, q_idx, k_idx, block_idx, q_begin, q_count, kv_len, lse_idx, workspace, workspace_bytes, st);
+        if (r.d_idx == 64)
+            return run_index_lse<128, 64>(r, q_idx, k_idx, block_idx, q_begin, q_count, kv_len, lse_idx, workspace, workspace_bytes, st);
+        return run_index_lse<128, 128>(r, q_idx, k_idx, block_idx, q_begin, q_count, kv_len, lse_idx, workspace, workspace_bytes, st);
+    }
+    const int64_t rows = q_count * r.H_kv;
+    const int64_t grid = ceil_div64(rows, 8);
+    if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
+    {
+        StageScope sc(kStageIndexLse, st);
+        index_lse_generic_kernel<<<(unsigned)grid, 256, 0, st>>>(
+            (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx, block_idx, q_begin, q_count, kv_len, r.H_kv,
+            r.d_idx, r.B_k, r.k, r.index_scale, lse_idx);
+    }
+    return launch_status();
 }
 
 // Scratch of msa_sparse_attn_prefill_static: part of the library's device image, so no call

@@ -137,6 +137,37 @@ def test_varlen_batch_equals_sequence_by_sequence():
     check_attn(out[a:b][pos_t].float().cpu().numpy(), lse[a:b][pos_t].cpu().numpy(), O_ref, LSE_ref, "varlen")
 
 
+@pytest.mark.parametrize("name,T,Hq,Hkv,Bk,k,di,sharp", [
+    ("c3 shape", 6144 + 77, 64, 8, 128, 64, 64, False),
+    ("c3 shape, sharp", 5000, 64, 8, 128, 16, 64, True),
+    ("paper regime", 4096 + 3, 64, 4, 128, 16, 128, True),
+    ("B_k 64", 3000, 16, 2, 64, 8, 64, True),
+    ("generic shape", 700, 6, 3, 16, 5, 32, True),
+])
+def test_index_lse_matches_oracle(name, T, Hq, Hkv, Bk, k, di, sharp):
+    # Section 4.3: log-sum-exp of the index scores over the visible tokens of the selected blocks,
+    # on the GPU's own selection; full sequence on the GPU, sampled rows in the oracle; the
+    # smallest workspace as well (many query ranges).
+    cfg = MSAConfig("lse", "prefill", T, Hq, Hkv, Bk, k, head_dim=128, idx_dim=di, seed=T)
+    x = make_prefill_inputs(cfg, DEV, sharp=sharp)
+    _, _, I = api.prefill_forward(cfg, x)
+    got = api.index_lse(cfg, x["q_idx"], x["k_idx"], I)
+    got_small = api.index_lse(cfg, x["q_idx"], x["k_idx"], I, workspace_bytes=0)
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert torch.equal(got, got_small)
+    pos = sample_positions(T, Bk, k, 160, 5)
+    pos_t = torch.from_numpy(pos).to(DEV)
+    want = oracle.index_lse(to_bits(x["q_idx"][pos_t]), to_bits(x["k_idx"]), I[pos_t].cpu().numpy(), pos, Bk)
+    err = np.abs(got[pos_t].cpu().numpy().astype(np.float64) - want)
+    assert np.isfinite(want).all() and err.max() <= 2e-3, (name, float(err.max()))
+    # a sub-range call gives the same rows
+    q0, qc = T // 3, min(500, T - T // 3)
+    sub = api.index_lse(cfg, x["q_idx"], x["k_idx"], I, q_begin=q0, q_count=qc)
+    torch.cuda.synchronize()
+    assert torch.equal(sub, got[q0:q0 + qc])
+
+
 def test_single_item_tiles_many_ranges():
     # Few selections per query and the smallest workspace: nearly every (block, head) tile of a
     # query range holds a single item, so the K/V tile buffers change owner with every item.
