@@ -168,9 +168,9 @@ def oracle_sample_size(cfg: MSAConfig) -> int:
 
 # ----------------------------------------------------------------------------- main
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the stage kernels,
-# from the ncu captures summarised under profiles/ (captured on the reduced workloads named
-# there and scaled to a full launch by the units processed, as the design doc explains).  None =
-# not captured.
+# from the ncu captures summarised under profiles/ (c3, c4: one-pass captures at full size; c5:
+# captured on the reduced workload named there and scaled to a full launch by the bytes streamed,
+# which the traffic is proportional to).  None = not captured.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     # c4: captured at full size with a one-pass metric set (profiles/launch_list_and_dram_c4.md)
     ("c4", "index_scores"): 38.85e9, ("c4", "topk_select"): 17.62e9,
