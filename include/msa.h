@@ -188,6 +188,19 @@ msa_status_t msa_sparse_attn_decode_workspace_bytes(const msa_shape_t* shape, in
                                                     size_t* min_bytes);
 
 /* ------------------------------------------------------------------------------------
+ * Eq. 6 and Eq. 7 in one kernel (the indexer only needs block-wise maxima, so the score
+ * matrix M need not exist): block_idx [q_count,H_kv,k] int32 exactly as msa_index_scores
+ * followed by msa_topk_select would write it (same scaled fp32 maxima, same tie rule, same
+ * list format).  Every epilogue thread of the scoring kernel keeps the best 15 earlier blocks
+ * of its row in registers, so this form exists for top_k <= 16, d_idx in {64,128}, B_k in
+ * {64,128} and q_count >= 32; anything else returns MSA_ERR_UNSUPPORTED and the two separate
+ * calls are the way.  msa_prefill_forward uses it whenever the shape allows.  No workspace.
+ */
+msa_status_t msa_index_topk_fused(const msa_shape_t* shape, const void* q_idx, const void* k_idx,
+                                  int64_t q_begin, int64_t q_count, int64_t kv_len, int32_t* block_idx,
+                                  msa_stream_t stream);
+
+/* ------------------------------------------------------------------------------------
  * Index-branch log-sum-exp over the selected blocks (Section 4.3, "LSE fusion": the forward
  * emits LSE_idx so that the sparse-KL backward need not recompute it):
  *   lse_idx[i,r] = log sum over b in block_idx[i,r,:], j in block b, j <= q_begin+i of

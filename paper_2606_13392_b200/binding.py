@@ -27,7 +27,7 @@ EXPORTS = [
     "msa_topk_select", "msa_topk_select_decode", "msa_sparse_attn_prefill",
     "msa_sparse_attn_prefill_workspace_bytes", "msa_sparse_attn_prefill_static",
     "msa_sparse_attn_decode",
-    "msa_sparse_attn_decode_workspace_bytes", "msa_index_lse_prefill",
+    "msa_sparse_attn_decode_workspace_bytes", "msa_index_topk_fused", "msa_index_lse_prefill",
     "msa_index_lse_prefill_workspace_bytes", "msa_prefill_forward",
     "msa_prefill_forward_workspace_bytes", "msa_prefill_forward_varlen",
     "msa_prefill_forward_varlen_workspace_bytes", "msa_prefill_forward_host",
@@ -230,6 +230,12 @@ def msa_prefill_forward(shape, q, k, v, q_idx, k_idx, T, out, lse, block_idx, wo
                                      _dev(workspace),
                                      c_sz(workspace.numel() * workspace.element_size()),
                                      _stream(stream)), "msa_prefill_forward")
+
+
+def msa_index_topk_fused(shape, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, stream=None):
+    _check(lib().msa_index_topk_fused(ctypes.byref(shape), _dev(q_idx), _dev(k_idx), c_i64(q_begin),
+                                      c_i64(q_count), c_i64(kv_len), _dev(block_idx), _stream(stream)),
+           "msa_index_topk_fused")
 
 
 def msa_index_lse_prefill_workspace_bytes(shape, q_count, kv_len) -> Tuple[int, int]:

@@ -35,11 +35,22 @@ struct IdxSmem {
     int abort;
 };
 
-template <int BK, int NH, int DI, int ST>
+// FK = 0: the block maxima are written to `scores` (Eq. 6).  FK > 0 (fused Eq. 6 + Eq. 7 for
+// top_k <= FK + 1, NH <= 2): nothing is written to `scores`; every epilogue thread keeps the FK best
+// earlier blocks of its (row, head) among the blocks it sees (its half of every key tile) in
+// registers, sorted by (score descending, block ascending); at the end the two halves of a row
+// are merged through the shared memory the key tiles no longer need and the index list goes to
+// block_idx, ascending, the local block last, padded with -1: the same list msa_topk_select
+// writes, since both rank the same scaled fp32 maxima with the same tie rule.
+constexpr int kIdxFuseKeep = 15;
+
+template <int BK, int NH, int DI, int ST, int FK = 0>
 __global__ void __launch_bounds__(kIdxThreads, 1)
 index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        int64_t q_begin, int64_t q_count, int H_kv, float scale,
-                       float* __restrict__ scores, int64_t ld_scores, int64_t n_cols, int* status) {
+                       float* __restrict__ scores, int64_t ld_scores, int64_t n_cols, int* status,
+                       int32_t* __restrict__ block_idx = nullptr, int top_k = 0) {
+    static_assert(FK == 0 || NH <= 2, "the fused form keeps its candidates in registers");
     extern __shared__ uint8_t smem_raw[];
     IdxSmem<NH, DI, ST>& sm =
         *reinterpret_cast<IdxSmem<NH, DI, ST>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -133,11 +144,22 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const bool valid_row = q < q_count;
         const int64_t loc = pos / BK;
         bool live = true;
+        constexpr int FKN = FK > 0 ? FK : 1;
+        float ts[NH][FKN];   // fused form: best earlier blocks seen by this thread, per head
+        int32_t tb[NH][FKN];
+        if constexpr (FK > 0) {
+#pragma unroll
+            for (int h = 0; h < NH; ++h)
+#pragma unroll
+                for (int i = 0; i < FK; ++i) { ts[h][i] = -INFINITY; tb[h][i] = -1; }
+        }
         for (int t = 0; live && t < n_tiles; ++t) {
             const int64_t key0 = (int64_t)t * kIdxTileK + half * 128;
             const bool need_mask = key0 + 127 > pos;
             const int lim = (int)(pos - key0);  // columns 0..lim are visible (may be negative)
+#pragma unroll(FK > 0 ? NH : 1)
             for (int h = 0; h < NH; ++h) {
+                if (FK > 0 && !live) break;
                 const int u = t * NH + h, buf = u & 1;
                 if (!mbar_wait(&sm.acc_full[buf], (u >> 1) & 1, abort)) {
                     report_async(status, kAsyncTimeout, 0x105);
@@ -146,28 +168,65 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 }
                 tc_fence_after();
                 const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + buf * kIdxTileK + half * 128;
-                uint32_t v[4][32];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld_32x32(taddr + c * 32, v[c]);
-                tmem_wait_ld();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
-
                 constexpr int NB = 128 / BK;  // blocks in this thread's 128 columns
                 float best[NB];
 #pragma unroll
                 for (int i = 0; i < NB; ++i) best[i] = -INFINITY;
-                if (need_mask) {
+                if constexpr (FK > 0) {
+                    // 32 columns at a time: the candidate lists need the registers
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t v[32];
+                        tmem_ld_32x32(taddr + c * 32, v);
+                        tmem_wait_ld();
+                        if (c == 3) {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
+                        }
+                        if (need_mask) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (c * 32 + e > lim) v[c][e] = 0xFF800000u;  // -inf
+                            for (int e = 0; e < 32; ++e)
+                                if (c * 32 + e > lim) v[e] = 0xFF800000u;  // -inf
+                        }
+                        best[(c * 32) / BK] = fmaxf(best[(c * 32) / BK], tree_max32(v));
+                    }
+                } else {
+                    uint32_t v[4][32];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) tmem_ld_32x32(taddr + c * 32, v[c]);
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
+                    if (need_mask) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                if (c * 32 + e > lim) v[c][e] = 0xFF800000u;  // -inf
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) best[(c * 32) / BK] = fmaxf(best[(c * 32) / BK], tree_max32(v[c]));
                 }
+                if constexpr (FK > 0) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) best[(c * 32) / BK] = fmaxf(best[(c * 32) / BK], tree_max32(v[c]));
-                if (valid_row) {
+                    for (int i = 0; i < NB; ++i) {
+                        const int64_t b = key0 / BK + i;
+                        const float x = best[i] * scale;
+                        // ranked: earlier blocks only; a later equal score never passes an earlier one
+                        if (valid_row && b < loc && x > ts[h][FK - 1]) {
+                            ts[h][FK - 1] = x; tb[h][FK - 1] = (int32_t)b;
+#pragma unroll
+                            for (int e = FK - 1; e > 0; --e) {
+                                if (ts[h][e] > ts[h][e - 1]) {
+                                    const float fs = ts[h][e]; ts[h][e] = ts[h][e - 1]; ts[h][e - 1] = fs;
+                                    const int32_t fb = tb[h][e]; tb[h][e] = tb[h][e - 1]; tb[h][e - 1] = fb;
+                                }
+                            }
+                        }
+                    }
+                } else if (valid_row) {
                     float* out_row = scores + (q * H_kv + r0 + h) * ld_scores;
 #pragma unroll
                     for (int i = 0; i < NB; ++i) {
@@ -177,8 +236,50 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 }
             }
         }
+        if constexpr (FK > 0) {
+            // Merge the two halves of every row.  All MMAs have completed (the last accumulator was
+            // read), so the key-tile stages are free: [half][row][head][FK] scores, then blocks.
+            float* xs = reinterpret_cast<float*>(&sm.b[0][0][0]);
+            int32_t* xb = reinterpret_cast<int32_t*>(xs + 2 * kIdxTileQ * NH * FK);
+            static_assert(sizeof(sm.b) >= 2 * kIdxTileQ * NH * FK * 8 + kIdxTileQ * NH * 16 * 4, "exchange area");
+            int32_t* xo = xb + 2 * kIdxTileQ * NH * FK;  // [row][head][16] merged picks
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+#pragma unroll
+            for (int h = 0; h < NH; ++h)
+#pragma unroll
+                for (int i = 0; i < FK; ++i) {
+                    xs[((half * kIdxTileQ + row) * NH + h) * FK + i] = ts[h][i];
+                    xb[((half * kIdxTileQ + row) * NH + h) * FK + i] = tb[h][i];
+                }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            // thread (row, half) finishes head `half` (and, with one head per CTA, half 0 does it)
+            const int m = top_k - 1;
+            for (int h = half; h < NH; h += 2) {
+                if (!valid_row || !live) break;
+                const float* sa = xs + ((0 * kIdxTileQ + row) * NH + h) * FK;
+                const float* sb = xs + ((1 * kIdxTileQ + row) * NH + h) * FK;
+                const int32_t* ba = xb + ((0 * kIdxTileQ + row) * NH + h) * FK;
+                const int32_t* bb = xb + ((1 * kIdxTileQ + row) * NH + h) * FK;
+                int32_t* pick = xo + (row * NH + h) * 16;
+                int ia = 0, ib = 0, c = 0;
+                while (c < m) {  // best first; equal scores: the lower block
+                    const bool ha = ia < FK && ba[ia] >= 0, hb = ib < FK && bb[ib] >= 0;
+                    if (!ha && !hb) break;
+                    const bool take_a = ha && (!hb || sa[ia] > sb[ib] || (sa[ia] == sb[ib] && ba[ia] < bb[ib]));
+                    pick[c++] = take_a ? ba[ia++] : bb[ib++];
+                }
+                for (int i = 1; i < c; ++i) {  // ascending block order
+                    const int32_t v = pick[i];
+                    int j2 = i - 1;
+                    while (j2 >= 0 && pick[j2] > v) { pick[j2 + 1] = pick[j2]; --j2; }
+                    pick[j2 + 1] = v;
+                }
+                int32_t* orow = block_idx + (q * H_kv + r0 + h) * (int64_t)top_k;
+                for (int i = 0; i < top_k; ++i) orow[i] = i < c ? pick[i] : (i == c ? (int32_t)loc : -1);
+            }
+        }
         // Blocks with no visible token: -inf (Eq. 6).  Warp ew fills rows ew, ew+8, ...
-        for (int rr = ew; rr < kIdxTileQ; rr += 8) {
+        for (int rr = ew; FK == 0 && rr < kIdxTileQ; rr += 8) {
             const int64_t qq = q0 + rr;
             if (qq >= q_count) break;
             for (int h = 0; h < NH; ++h) {

@@ -116,10 +116,10 @@ bool encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64
 }
 
 // ---------------------------------------------------------------------- stage 1
-template <int BK, int NH, int DI>
+template <int BK, int NH, int DI, int FK = 0>
 static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                     int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
-                                    int64_t n_cols, cudaStream_t st) {
+                                    int64_t n_cols, cudaStream_t st, int32_t* block_idx = nullptr) {
     // key-tile stages: what fits beside the NH*DI query atoms in 227 KB of shared memory (at most 3)
     constexpr int ST = (NH * DI * 16 + 3 * DI * 32 <= 224) ? 3 : 2;
     static_assert(NH * DI * 16 + ST * DI * 32 <= 224, "shared memory budget");
@@ -139,7 +139,7 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
     static bool attr_set_dev[64] = {false};  // the attribute is per device
     const int dev_id = current_device();
     if (!attr_set_dev[dev_id]) {
-        if (cudaFuncSetAttribute(index_scores_tc_kernel<BK, NH, DI, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(index_scores_tc_kernel<BK, NH, DI, ST, FK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem) != cudaSuccess)
             return MSA_ERR_CUDA;
         attr_set_dev[dev_id] = true;
@@ -148,8 +148,8 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
     if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
     {
         StageScope sc(kStageIndex, st);
-        index_scores_tc_kernel<BK, NH, DI, ST><<<(unsigned)grid, kIdxThreads, smem, st>>>(
-            tm_q, tm_k, q_begin, q_count, r.H_kv, r.index_scale, scores, ld_scores, n_cols, status);
+        index_scores_tc_kernel<BK, NH, DI, ST, FK><<<(unsigned)grid, kIdxThreads, smem, st>>>(
+            tm_q, tm_k, q_begin, q_count, r.H_kv, r.index_scale, scores, ld_scores, n_cols, status, block_idx, r.k);
     }
     return launch_status();
 }
@@ -171,6 +171,32 @@ static msa_status_t launch_index_tc_bk(const Resolved& r, const void* q_idx, con
     }
     if (nh == 2) return launch_index_tc<BK, 2, DI>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
     return launch_index_tc<BK, 1, DI>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+}
+
+// Eq. 6 and Eq. 7 in one kernel, no score matrix (top_k <= 16 on the tensor-core path).
+static bool index_topk_fused_ok(const Resolved& r, int64_t q_count, int64_t kv_len) {
+    return r.k <= kIdxFuseKeep + 1 && (r.d_idx == 64 || r.d_idx == 128) && (r.B_k == 64 || r.B_k == 128) &&
+           kv_len < 2147483647LL && q_count >= 32;
+}
+
+template <int BK, int DI>
+static msa_status_t launch_index_fused_bk(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
+                                          int64_t q_count, int64_t kv_len, int32_t* block_idx, cudaStream_t st) {
+    if (r.H_kv % 2 == 0)
+        return launch_index_tc<BK, 2, DI, kIdxFuseKeep>(r, q_idx, k_idx, q_begin, q_count, kv_len, nullptr, 0, 0, st,
+                                                        block_idx);
+    return launch_index_tc<BK, 1, DI, kIdxFuseKeep>(r, q_idx, k_idx, q_begin, q_count, kv_len, nullptr, 0, 0, st,
+                                                    block_idx);
+}
+
+static msa_status_t run_index_topk_fused(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
+                                         int64_t q_count, int64_t kv_len, int32_t* block_idx, cudaStream_t st) {
+    if (r.d_idx == 64) {
+        if (r.B_k == 64) return launch_index_fused_bk<64, 1>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
+        return launch_index_fused_bk<128, 1>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
+    }
+    if (r.B_k == 64) return launch_index_fused_bk<64, 2>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
+    return launch_index_fused_bk<128, 2>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
 }
 
 static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const void* k_idx,
@@ -682,6 +708,19 @@ msa_status_t msa_index_scores(const msa_shape_t* shape, const void* q_idx, const
                             ld_scores, (cudaStream_t)stream);
 }
 
+msa_status_t msa_index_topk_fused(const msa_shape_t* shape, const void* q_idx, const void* k_idx,
+                                  int64_t q_begin, int64_t q_count, int64_t kv_len, int32_t* block_idx,
+                                  msa_stream_t stream) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if ((s = check_range(q_begin, q_count, kv_len)) != MSA_OK) return s;
+    if (q_count == 0) return MSA_OK;
+    if (!q_idx || !k_idx || !block_idx || !aligned16(q_idx) || !aligned16(k_idx)) return MSA_ERR_INVALID_ARG;
+    if (!index_topk_fused_ok(r, q_count, kv_len)) return MSA_ERR_UNSUPPORTED;
+    return run_index_topk_fused(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, (cudaStream_t)stream);
+}
+
 msa_status_t msa_index_scores_decode(const msa_shape_t* shape, const void* q_idx,
                                      const void* k_idx_cache, const int64_t* seq_offsets,
                                      const int32_t* seq_lens, int32_t batch, int64_t max_seq_len,
@@ -988,6 +1027,8 @@ static msa_status_t prefill_stages_1_2(const msa_shape_t* shape, const Resolved&
                                        const void* k_idx, int64_t T, int32_t* block_idx, void* workspace,
                                        size_t workspace_bytes, msa_stream_t stream) {
     msa_status_t s = MSA_OK;
+    if (index_topk_fused_ok(r, T, T))  // no score matrix, no chunks
+        return run_index_topk_fused(r, q_idx, k_idx, 0, T, T, block_idx, (cudaStream_t)stream);
     const int64_t ld = score_ld(T, r.B_k);
     const int64_t chunk = pick_score_chunk(r, T, workspace_bytes);
     if (chunk <= 0) return MSA_ERR_WORKSPACE;

@@ -168,6 +168,36 @@ def test_index_lse_matches_oracle(name, T, Hq, Hkv, Bk, k, di, sharp):
     assert torch.equal(sub, got[q0:q0 + qc])
 
 
+@pytest.mark.parametrize("T,Hq,Hkv,Bk,k,di,ties", [
+    (4096 + 77, 64, 4, 128, 16, 128, False),   # the paper's regime
+    (3000, 16, 2, 64, 8, 64, False),           # B_k 64: two blocks per thread and key tile
+    (2500, 24, 3, 128, 16, 64, False),         # an odd number of index heads: one head per CTA
+    (2048 + 5, 8, 1, 128, 1, 64, False),       # k = 1: the local block only
+    (5000, 32, 4, 128, 12, 128, True),         # many exactly equal scores
+])
+def test_fused_index_topk_equals_separate_calls(T, Hq, Hkv, Bk, k, di, ties):
+    # Eq. 6 + Eq. 7 in one kernel must write the very list the two calls write (ties included).
+    cfg = MSAConfig("fused", "prefill", T, Hq, Hkv, Bk, k, head_dim=128, idx_dim=di, seed=T)
+    x = make_prefill_inputs(cfg, DEV, sharp=True)
+    if ties:  # keys repeat with period 7 blocks: block maxima of different blocks coincide exactly
+        period = 7 * Bk
+        x["k_idx"] = x["k_idx"][:period].repeat((T + period - 1) // period, 1)[:T].contiguous()
+    shape = B.shape_of(cfg)
+    I_f = torch.full((T, Hkv, k), -7, dtype=torch.int32, device=DEV)
+    B.msa_index_topk_fused(shape, x["q_idx"], x["k_idx"], 0, T, T, I_f)
+    M = api.index_scores(cfg, x["q_idx"], x["k_idx"], 0, T)
+    I_s = api.topk_select(cfg, M, 0, T)
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert torch.equal(I_f, I_s), int((I_f != I_s).any(dim=2).sum())
+    # a range that starts inside the sequence
+    q0, qc = T // 2 + 3, T - (T // 2 + 3)
+    I_r = torch.full((qc, Hkv, k), -7, dtype=torch.int32, device=DEV)
+    B.msa_index_topk_fused(shape, x["q_idx"][q0:], x["k_idx"], q0, qc, T, I_r)
+    torch.cuda.synchronize()
+    assert torch.equal(I_r, I_s[q0:])
+
+
 def test_single_item_tiles_many_ranges():
     # Few selections per query and the smallest workspace: nearly every (block, head) tile of a
     # query range holds a single item, so the K/V tile buffers change owner with every item.
