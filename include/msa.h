@@ -27,6 +27,15 @@
  *   - Fast kernels are specialised for d_h = 128, d_idx in {64,128}, B_k in {64,128},
  *     G in {8,16} (decode index scoring: H_kv <= 8); other shapes (d_h, d_idx multiples
  *     of 8, d_h <= 256, d_idx <= 128) run on generic kernels.  k is limited to 1..128.
+ *   - Host threads: the library keeps a little state per process (the pool of CUDA events
+ *     and the copy stream of the *_host calls, the profiling hooks, cached kernel
+ *     attributes per device).  Calls from several host threads must be serialised by the
+ *     caller; calls on different streams from one thread are fine, but two calls that are
+ *     in flight at the same time must not share a workspace.
+ *   - Beyond the four stage calls there are: whole-path calls (msa_prefill_forward,
+ *     msa_prefill_forward_varlen, msa_decode_forward and their *_host forms), the fused
+ *     Eq. 6 + Eq. 7 call msa_index_topk_fused (top_k <= 16), and the index branch's
+ *     log-sum-exp msa_index_lse_prefill (Section 4.3).
  */
 #ifndef MSA_H_
 #define MSA_H_
