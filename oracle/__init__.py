@@ -64,9 +64,18 @@ def n_threads() -> int:
     return len(os.sched_getaffinity(0))
 
 
+def _idx(a) -> np.ndarray:
+    """Index-branch operand: bf16 bit patterns (uint16) or fp8 E4M3 bit patterns (uint8)."""
+    a = np.asarray(a)
+    assert a.dtype in (np.uint16, np.uint8), "index operands are uint16 (bf16) or uint8 (E4M3) bit patterns"
+    return np.ascontiguousarray(a)
+
+
 def index_scores(q_idx, k_idx, pos, block_size: int, scale: Optional[float] = None) -> np.ndarray:
-    """Eq. 6.  q_idx [n,H_kv,d_idx] u16, k_idx [L,d_idx] u16, pos [n] -> M [n,H_kv,B] f64."""
-    q_idx, k_idx, pos = _u16(q_idx), _u16(k_idx), _pos(pos)
+    """Eq. 6.  q_idx [n,H_kv,d_idx], k_idx [L,d_idx] (both u16 = bf16 or both u8 = E4M3), pos [n]
+    -> M [n,H_kv,B] f64."""
+    q_idx, k_idx, pos = _idx(q_idx), _idx(k_idx), _pos(pos)
+    assert q_idx.dtype == k_idx.dtype
     n, H_kv, d_idx = q_idx.shape
     L = k_idx.shape[0]
     assert k_idx.shape[1] == d_idx and len(pos) == n
@@ -77,7 +86,7 @@ def index_scores(q_idx, k_idx, pos, block_size: int, scale: Optional[float] = No
     M = np.empty((n, H_kv, B), dtype=np.float64)
     _load().msa_oracle_index_scores(_p(q_idx), _p(k_idx), _p(pos), ctypes.c_int64(n),
                                     ctypes.c_int64(L), H_kv, d_idx, block_size,
-                                    ctypes.c_double(scale), _p(M))
+                                    ctypes.c_double(scale), _p(M), int(q_idx.dtype == np.uint8))
     return M
 
 
@@ -96,7 +105,8 @@ def topk_select(M, pos, L: int, block_size: int, top_k: int) -> np.ndarray:
 def index_lse(q_idx, k_idx, I, pos, block_size: int, scale: Optional[float] = None) -> np.ndarray:
     """Section 4.3 (LSE fusion): log-sum-exp of the index scores over the visible tokens of the
     selected blocks.  q_idx [n,H_kv,d_idx] u16, k_idx [L,d_idx] u16, I [n,H_kv,k] int32 -> [n,H_kv] f64."""
-    q_idx, k_idx, pos = _u16(q_idx), _u16(k_idx), _pos(pos)
+    q_idx, k_idx, pos = _idx(q_idx), _idx(k_idx), _pos(pos)
+    assert q_idx.dtype == k_idx.dtype
     I = np.ascontiguousarray(I, dtype=np.int32)
     n, H_kv, d_idx = q_idx.shape
     L = k_idx.shape[0]
@@ -106,7 +116,7 @@ def index_lse(q_idx, k_idx, I, pos, block_size: int, scale: Optional[float] = No
     out = np.empty((n, H_kv), dtype=np.float64)
     _load().msa_oracle_index_lse(_p(q_idx), _p(k_idx), _p(I), _p(pos), ctypes.c_int64(n),
                                  ctypes.c_int64(L), H_kv, d_idx, block_size, I.shape[2],
-                                 ctypes.c_double(scale), _p(out))
+                                 ctypes.c_double(scale), _p(out), int(q_idx.dtype == np.uint8))
     return out
 
 

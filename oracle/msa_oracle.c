@@ -38,6 +38,26 @@ static inline double bf16_to_double(uint16_t b) {
 }
 
 /*
+ * fp8 E4M3 ("fn" flavour: no infinities, S.1111.111 is NaN) widened exactly: 1 sign bit, 4
+ * exponent bits with bias 7, 3 mantissa bits; exponent 0 is subnormal, m/8 * 2^-6.
+ * (The paper states that its kernels also support fp8, Section 4.2; this build accepts the
+ * index branch's operands in that format.)
+ */
+static inline double e4m3_to_double(uint8_t b) {
+    const int sign = b >> 7, e = (b >> 3) & 15, m = b & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m / 8.0, -6);
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+/* element c of an index-branch row stored as bf16 (idx_fp8 = 0) or E4M3 (idx_fp8 = 1) */
+static inline double idx_elem(const void* row, int c, int idx_fp8) {
+    return idx_fp8 ? e4m3_to_double(((const uint8_t*)row)[c]) : bf16_to_double(((const uint16_t*)row)[c]);
+}
+
+/*
  * Eq. 6: token-level index scores and their block-wise causal maximum.
  *   S[i,r,j] = <Q_idx[i,r,:], K_idx[j,:]> * scale           for j <= i
  *   M[i,r,b] = max over j in block b with j <= i of S[i,r,j]
@@ -45,16 +65,17 @@ static inline double bf16_to_double(uint16_t b) {
  * q_idx: [n, H_kv, d_idx] rows for the listed positions; k_idx: [L, d_idx] (one shared
  * index key head, Eq. 5); M: [n, H_kv, B] with B = ceil(L / B_k).
  */
-void msa_oracle_index_scores(const uint16_t* q_idx, const uint16_t* k_idx,
+void msa_oracle_index_scores(const void* q_idx, const void* k_idx,
                              const int64_t* pos, int64_t n, int64_t L, int H_kv,
-                             int d_idx, int B_k, double scale, double* M) {
+                             int d_idx, int B_k, double scale, double* M, int idx_fp8) {
     const int64_t B = (L + B_k - 1) / B_k;
+    const int64_t eb = idx_fp8 ? 1 : 2;  /* bytes per index element */
 #pragma omp parallel for schedule(dynamic, 1)
     for (int64_t a = 0; a < n * H_kv; ++a) {
         const int64_t qi = a / H_kv;
         const int r = (int)(a % H_kv);
         const int64_t i = pos[qi];
-        const uint16_t* qrow = q_idx + (qi * H_kv + r) * (int64_t)d_idx;
+        const char* qrow = (const char*)q_idx + (qi * H_kv + r) * (int64_t)d_idx * eb;
         double* Mrow = M + (qi * H_kv + r) * B;
         for (int64_t b = 0; b < B; ++b) {
             double best = -INFINITY;
@@ -62,10 +83,10 @@ void msa_oracle_index_scores(const uint16_t* q_idx, const uint16_t* k_idx,
             int64_t j1 = j0 + B_k;
             if (j1 > L) j1 = L;
             for (int64_t j = j0; j < j1 && j <= i; ++j) {
-                const uint16_t* krow = k_idx + j * (int64_t)d_idx;
+                const char* krow = (const char*)k_idx + j * (int64_t)d_idx * eb;
                 double s = 0.0;
                 for (int c = 0; c < d_idx; ++c)
-                    s += bf16_to_double(qrow[c]) * bf16_to_double(krow[c]);
+                    s += idx_elem(qrow, c, idx_fp8) * idx_elem(krow, c, idx_fp8);
                 s *= scale;
                 if (s > best) best = s;
             }
@@ -82,14 +103,15 @@ void msa_oracle_index_scores(const uint16_t* q_idx, const uint16_t* k_idx,
  * stabilised by the largest selected score.  Entries of I below 0 are padding.
  * q_idx: [n, H_kv, d_idx]; k_idx: [L, d_idx]; I: [n, H_kv, k]; out: [n, H_kv].
  */
-void msa_oracle_index_lse(const uint16_t* q_idx, const uint16_t* k_idx, const int32_t* I,
+void msa_oracle_index_lse(const void* q_idx, const void* k_idx, const int32_t* I,
                           const int64_t* pos, int64_t n, int64_t L, int H_kv, int d_idx,
-                          int B_k, int k, double scale, double* out) {
+                          int B_k, int k, double scale, double* out, int idx_fp8) {
+    const int64_t eb = idx_fp8 ? 1 : 2;
 #pragma omp parallel for schedule(dynamic, 1)
     for (int64_t a = 0; a < n * H_kv; ++a) {
         const int64_t qi = a / H_kv;
         const int64_t i = pos[qi];
-        const uint16_t* qrow = q_idx + a * (int64_t)d_idx;
+        const char* qrow = (const char*)q_idx + a * (int64_t)d_idx * eb;
         const int32_t* sel = I + a * (int64_t)k;
         double best = -INFINITY, sum = 0.0;
         for (int pass = 0; pass < 2; ++pass) {  /* pass 0: the largest score; pass 1: the sum */
@@ -99,10 +121,10 @@ void msa_oracle_index_lse(const uint16_t* q_idx, const uint16_t* k_idx, const in
                 int64_t j1 = j0 + B_k;
                 if (j1 > L) j1 = L;
                 for (int64_t j = j0; j < j1 && j <= i; ++j) {
-                    const uint16_t* krow = k_idx + j * (int64_t)d_idx;
+                    const char* krow = (const char*)k_idx + j * (int64_t)d_idx * eb;
                     double s = 0.0;
                     for (int c = 0; c < d_idx; ++c)
-                        s += bf16_to_double(qrow[c]) * bf16_to_double(krow[c]);
+                        s += idx_elem(qrow, c, idx_fp8) * idx_elem(krow, c, idx_fp8);
                     s *= scale;
                     if (pass == 0) { if (s > best) best = s; }
                     else sum += exp(s - best);

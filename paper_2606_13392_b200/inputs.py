@@ -44,6 +44,7 @@ class MSAConfig:
     planted_frac: float = 0.0
     planted_shift: float = 0.0
     seq_lens: Tuple[int, ...] = ()
+    idx_fp8: bool = False  # index-branch operands (Q_idx, K_idx) rounded to fp8 E4M3 instead of bf16
 
     @property
     def group(self) -> int:
@@ -146,6 +147,8 @@ def make_prefill_inputs(cfg: MSAConfig, device="cpu", sharp: bool = False):
     v = _draw(gen, T, (cfg.n_kv_heads, d), s_main, device)
     q_idx = _draw(gen, T, (cfg.n_kv_heads, di), s_idx, device)
     k_idx = _draw(gen, T, (di,), s_idx, device, tok_mask, sh_idx)
+    if cfg.idx_fp8:  # the same draws, stored in the narrower format
+        q_idx, k_idx = q_idx.to(torch.float8_e4m3fn), k_idx.to(torch.float8_e4m3fn)
     return {"q": q, "k": k, "v": v, "q_idx": q_idx, "k_idx": k_idx}
 
 
@@ -169,6 +172,8 @@ def make_decode_inputs(cfg: MSAConfig, device="cpu", sharp: bool = False):
     v_cache = _draw(gen, total, (cfg.n_kv_heads, d), s_main, device)
     q_idx = _draw(gen, batch, (cfg.n_kv_heads, di), s_idx, device)
     k_idx_cache = _draw(gen, total, (di,), s_idx, device)
+    if cfg.idx_fp8:
+        q_idx, k_idx_cache = q_idx.to(torch.float8_e4m3fn), k_idx_cache.to(torch.float8_e4m3fn)
     offs = np.concatenate([[0], np.cumsum(lens)[:-1]]).astype(np.int64)
     return {
         "q": q, "q_idx": q_idx, "k_cache": k_cache, "v_cache": v_cache,
@@ -204,7 +209,9 @@ def sample_positions(T: int, block_size: int, top_k: int, n: int, seed: int) -> 
 
 
 def to_bits(t: torch.Tensor) -> np.ndarray:
-    """bf16 tensor (any device) -> contiguous numpy uint16 array of its bit patterns."""
+    """bf16 (or fp8 E4M3) tensor, any device -> contiguous numpy uint16 (uint8) array of its bit patterns."""
+    if t.dtype == torch.float8_e4m3fn:
+        return t.detach().contiguous().cpu().view(torch.uint8).numpy()
     assert t.dtype == torch.bfloat16
     return t.detach().contiguous().cpu().view(torch.uint16).numpy()
 

@@ -392,6 +392,40 @@ def test_index_lse_brute_force_dense_limit_and_bounds():
     assert np.isneginf(oracle.index_lse(x["q_idx"][:1, :1], x["k_idx"], I_none, [0], cfg.block_size)[0, 0])
 
 
+def test_fp8_index_operands_decode_and_scores():
+    # The oracle's E4M3 decoding against torch's own conversion for all 256 codes (through a
+    # one-element score: q = code, k = 1.0), and Eq. 6 on fp8 operands against an einsum on the
+    # torch-decoded values.
+    codes = np.arange(256, dtype=np.uint8)
+    want = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    one = torch.tensor([1.0]).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    q = codes.reshape(256, 1, 1)                    # [n, H_kv=1, d_idx=1]
+    k = np.repeat(one.reshape(1, 1), 256, axis=0)   # [L, 1]: every key is 1.0
+    M = oracle.index_scores(q, k, np.arange(256), block_size=1, scale=1.0)
+    got = np.array([M[i, 0, i] for i in range(256)])
+    finite = np.isfinite(want)
+    assert np.array_equal(got[finite], want[finite])
+    assert list(np.nonzero(~finite)[0]) == [0x7F, 0xFF]  # the two NaN codes; a NaN is never a maximum
+    cfg = MSAConfig("tiny8", "prefill", 50, 4, 2, 4, 3, head_dim=8, idx_dim=16, seed=5, idx_fp8=True)
+    t = make_prefill_inputs(cfg, "cpu", sharp=True)
+    assert t["q_idx"].dtype == torch.float8_e4m3fn
+    qi, ki = t["q_idx"].to(torch.float64).numpy(), t["k_idx"].to(torch.float64).numpy()
+    pos = np.arange(cfg.T)
+    M = oracle.index_scores(to_bits(t["q_idx"]), to_bits(t["k_idx"]), pos, cfg.block_size)
+    S = np.einsum("irc,jc->irj", qi, ki) / np.sqrt(cfg.idx_dim)
+    causal = np.arange(cfg.T)[None, :] <= np.arange(cfg.T)[:, None]
+    S = np.where(causal[:, None, :], S, -np.inf)
+    pad = cfg.n_blocks * cfg.block_size - cfg.T
+    S = np.pad(S, ((0, 0), (0, 0), (0, pad)), constant_values=-np.inf)
+    np.testing.assert_allclose(M, S.reshape(cfg.T, cfg.n_kv_heads, cfg.n_blocks, cfg.block_size).max(-1),
+                               rtol=1e-12, atol=1e-14)
+    # and the log-sum-exp of the same operands, dense limit
+    from scipy.special import logsumexp
+    I_all = oracle.topk_select(M, pos, cfg.T, cfg.block_size, cfg.n_blocks)
+    dense = oracle.index_lse(to_bits(t["q_idx"]), to_bits(t["k_idx"]), I_all, pos, cfg.block_size)
+    np.testing.assert_allclose(dense, logsumexp(S, axis=-1), rtol=0, atol=1e-12)
+
+
 def test_flops_model_printed_ratio():
     path = os.path.join(os.path.dirname(__file__), "golden", "flops_reduction_1m.txt")
     vals = {}
