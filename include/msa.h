@@ -67,6 +67,11 @@ typedef struct {
     int32_t top_k;       /* k, blocks per (query, group) including the local one  */
     float softmax_scale; /* 0 => 1/sqrt(d_h)   (Eq. 1, Eq. 8)                     */
     float index_scale;   /* 0 => 1/sqrt(d_idx) (Eq. 6)                            */
+    int32_t idx_fp8;     /* 0: q_idx / k_idx are bf16.  1: they are fp8 E4M3      */
+                         /* (Section 4.2), one byte per element, d_idx % 16 == 0; */
+                         /* every "bf16" below then reads "fp8" for those two     */
+                         /* operands.  Codes 0x7F / 0xFF (NaN) must not occur.    */
+                         /* Any other value: MSA_ERR_INVALID_ARG.                 */
 } msa_shape_t;
 
 typedef void* msa_stream_t; /* a cudaStream_t */

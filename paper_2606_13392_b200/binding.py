@@ -39,7 +39,8 @@ EXPORTS = [
 class MsaShape(ctypes.Structure):
     _fields_ = [("n_q_heads", c_i32), ("n_kv_heads", c_i32), ("head_dim", c_i32),
                 ("idx_dim", c_i32), ("block_size", c_i32), ("top_k", c_i32),
-                ("softmax_scale", ctypes.c_float), ("index_scale", ctypes.c_float)]
+                ("softmax_scale", ctypes.c_float), ("index_scale", ctypes.c_float),
+                ("idx_fp8", c_i32)]
 
 
 class MsaError(RuntimeError):
@@ -72,7 +73,7 @@ def status_string(code: int) -> str:
 
 def shape_of(cfg: MSAConfig, softmax_scale: float = 0.0, index_scale: float = 0.0) -> MsaShape:
     return MsaShape(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.idx_dim, cfg.block_size,
-                    cfg.top_k, softmax_scale, index_scale)
+                    cfg.top_k, softmax_scale, index_scale, 1 if cfg.idx_fp8 else 0)
 
 
 def _ptr(t) -> c_vp:
@@ -86,6 +87,15 @@ def _dev(t: Optional[torch.Tensor]):
     if t is not None:
         assert t.is_cuda, "device pointer expected"
     return _ptr(t)
+
+
+def _idx(shape, t: Optional[torch.Tensor], host: bool = False):
+    """An index-branch operand: its element size must match the shape's idx_fp8 flag."""
+    if t is not None:
+        want = 1 if shape.idx_fp8 else 2
+        assert t.element_size() == want, "index operand element size %d, shape expects %d" % (
+            t.element_size(), want)
+    return _host(t) if host else _dev(t)
 
 
 def _host(t: Optional[torch.Tensor]):
@@ -133,14 +143,14 @@ def check_async_status() -> Tuple[int, int]:
 
 # ------------------------------------------------------------------ the four stages
 def msa_index_scores(shape, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, stream=None):
-    _check(lib().msa_index_scores(ctypes.byref(shape), _dev(q_idx), _dev(k_idx), c_i64(q_begin),
+    _check(lib().msa_index_scores(ctypes.byref(shape), _idx(shape, q_idx), _idx(shape, k_idx), c_i64(q_begin),
                                   c_i64(q_count), c_i64(kv_len), _dev(scores), c_i64(ld_scores),
                                   _stream(stream)), "msa_index_scores")
 
 
 def msa_index_scores_decode(shape, q_idx, k_idx_cache, seq_offsets, seq_lens, batch, max_seq_len,
                             scores, ld_scores, stream=None):
-    _check(lib().msa_index_scores_decode(ctypes.byref(shape), _dev(q_idx), _dev(k_idx_cache),
+    _check(lib().msa_index_scores_decode(ctypes.byref(shape), _idx(shape, q_idx), _idx(shape, k_idx_cache),
                                          _dev(seq_offsets), _dev(seq_lens), c_i32(batch),
                                          c_i64(max_seq_len), _dev(scores), c_i64(ld_scores),
                                          _stream(stream)), "msa_index_scores_decode")
@@ -225,15 +235,15 @@ def msa_prefill_forward_workspace_bytes(shape, T) -> Tuple[int, int]:
 
 
 def msa_prefill_forward(shape, q, k, v, q_idx, k_idx, T, out, lse, block_idx, workspace, stream=None):
-    _check(lib().msa_prefill_forward(ctypes.byref(shape), _dev(q), _dev(k), _dev(v), _dev(q_idx),
-                                     _dev(k_idx), c_i64(T), _dev(out), _dev(lse), _dev(block_idx),
+    _check(lib().msa_prefill_forward(ctypes.byref(shape), _dev(q), _dev(k), _dev(v), _idx(shape, q_idx),
+                                     _idx(shape, k_idx), c_i64(T), _dev(out), _dev(lse), _dev(block_idx),
                                      _dev(workspace),
                                      c_sz(workspace.numel() * workspace.element_size()),
                                      _stream(stream)), "msa_prefill_forward")
 
 
 def msa_index_topk_fused(shape, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, stream=None):
-    _check(lib().msa_index_topk_fused(ctypes.byref(shape), _dev(q_idx), _dev(k_idx), c_i64(q_begin),
+    _check(lib().msa_index_topk_fused(ctypes.byref(shape), _idx(shape, q_idx), _idx(shape, k_idx), c_i64(q_begin),
                                       c_i64(q_count), c_i64(kv_len), _dev(block_idx), _stream(stream)),
            "msa_index_topk_fused")
 
@@ -248,7 +258,7 @@ def msa_index_lse_prefill_workspace_bytes(shape, q_count, kv_len) -> Tuple[int, 
 
 def msa_index_lse_prefill(shape, q_idx, k_idx, block_idx, q_begin, q_count, kv_len, lse_idx, workspace,
                           stream=None):
-    _check(lib().msa_index_lse_prefill(ctypes.byref(shape), _dev(q_idx), _dev(k_idx), _dev(block_idx),
+    _check(lib().msa_index_lse_prefill(ctypes.byref(shape), _idx(shape, q_idx), _idx(shape, k_idx), _dev(block_idx),
                                        c_i64(q_begin), c_i64(q_count), c_i64(kv_len), _dev(lse_idx),
                                        _dev(workspace), c_sz(workspace.numel() * workspace.element_size()),
                                        _stream(stream)), "msa_index_lse_prefill")
@@ -271,8 +281,8 @@ def msa_prefill_forward_varlen_workspace_bytes(shape, cu_seqlens) -> Tuple[int, 
 def msa_prefill_forward_varlen(shape, q, k, v, q_idx, k_idx, cu_seqlens, out, lse, block_idx, workspace,
                                stream=None):
     arr, n = _cu_array(cu_seqlens)
-    _check(lib().msa_prefill_forward_varlen(ctypes.byref(shape), _dev(q), _dev(k), _dev(v), _dev(q_idx),
-                                            _dev(k_idx), arr, c_i32(n), _dev(out), _dev(lse),
+    _check(lib().msa_prefill_forward_varlen(ctypes.byref(shape), _dev(q), _dev(k), _dev(v), _idx(shape, q_idx),
+                                            _idx(shape, k_idx), arr, c_i32(n), _dev(out), _dev(lse),
                                             _dev(block_idx), _dev(workspace),
                                             c_sz(workspace.numel() * workspace.element_size()),
                                             _stream(stream)), "msa_prefill_forward_varlen")
@@ -290,7 +300,7 @@ def msa_prefill_forward_host(shape, q, k, v, q_idx, k_idx, T, out, lse, block_id
                              stream=None):
     """q..k_idx, out, lse, block_idx are HOST tensors (pinned for full copy rate)."""
     _check(lib().msa_prefill_forward_host(ctypes.byref(shape), _host(q), _host(k), _host(v),
-                                          _host(q_idx), _host(k_idx), c_i64(T), _host(out),
+                                          _idx(shape, q_idx, True), _idx(shape, k_idx, True), c_i64(T), _host(out),
                                           _host(lse), _host(block_idx), _dev(workspace),
                                           c_sz(workspace.numel() * workspace.element_size()),
                                           _stream(stream)), "msa_prefill_forward_host")
@@ -299,8 +309,8 @@ def msa_prefill_forward_host(shape, q, k, v, q_idx, k_idx, T, out, lse, block_id
 def msa_decode_forward(shape, q, q_idx, k_cache, v_cache, k_idx_cache, cache_tokens, seq_offsets,
                        seq_lens, batch, max_seq_len, scores, ld_scores, block_idx, out, lse,
                        workspace, stream=None):
-    _check(lib().msa_decode_forward(ctypes.byref(shape), _dev(q), _dev(q_idx), _dev(k_cache),
-                                    _dev(v_cache), _dev(k_idx_cache), c_i64(cache_tokens),
+    _check(lib().msa_decode_forward(ctypes.byref(shape), _dev(q), _idx(shape, q_idx), _dev(k_cache),
+                                    _dev(v_cache), _idx(shape, k_idx_cache), c_i64(cache_tokens),
                                     _dev(seq_offsets), _dev(seq_lens), c_i32(batch),
                                     c_i64(max_seq_len), _dev(scores), c_i64(ld_scores),
                                     _dev(block_idx), _dev(out), _dev(lse), _dev(workspace),
@@ -311,9 +321,9 @@ def msa_decode_forward(shape, q, q_idx, k_cache, v_cache, k_idx_cache, cache_tok
 def msa_decode_forward_host(shape, q_host, q_idx_host, q_dev, q_idx_dev, k_cache, v_cache,
                             k_idx_cache, cache_tokens, seq_offsets, seq_lens, batch, max_seq_len,
                             scores, ld_scores, block_idx, out_dev, out_host, workspace, stream=None):
-    _check(lib().msa_decode_forward_host(ctypes.byref(shape), _host(q_host), _host(q_idx_host),
-                                         _dev(q_dev), _dev(q_idx_dev), _dev(k_cache), _dev(v_cache),
-                                         _dev(k_idx_cache), c_i64(cache_tokens), _dev(seq_offsets),
+    _check(lib().msa_decode_forward_host(ctypes.byref(shape), _host(q_host), _idx(shape, q_idx_host, True),
+                                         _dev(q_dev), _idx(shape, q_idx_dev), _dev(k_cache), _dev(v_cache),
+                                         _idx(shape, k_idx_cache), c_i64(cache_tokens), _dev(seq_offsets),
                                          _dev(seq_lens), c_i32(batch), c_i64(max_seq_len),
                                          _dev(scores), c_i64(ld_scores), _dev(block_idx),
                                          _dev(out_dev), _host(out_host), _dev(workspace),

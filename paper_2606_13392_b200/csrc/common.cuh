@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -27,6 +28,19 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) {
 // Two packed bf16 (low half first) -> two floats.
 __device__ __forceinline__ float2 bf16x2_to_float2(uint32_t u) {
     return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+}
+
+// fp8 E4M3 ("fn": bias 7, no infinities, 0x7F / 0xFF are NaN) to fp32; exact.
+__device__ __forceinline__ float e4m3_to_float(uint8_t b) {
+    const __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)b, __NV_E4M3);
+    return __half2float(__half(h));
+}
+
+// Element c of an index-branch row stored as fp8 E4M3 (F8) or bf16.
+template <bool F8>
+__device__ __forceinline__ float idx_elem(const void* row, int c) {
+    if constexpr (F8) return e4m3_to_float(static_cast<const uint8_t*>(row)[c]);
+    else return __bfloat162float(static_cast<const __nv_bfloat16*>(row)[c]);
 }
 
 __device__ __forceinline__ float warp_max(float v) {

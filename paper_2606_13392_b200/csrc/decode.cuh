@@ -22,6 +22,16 @@ __device__ __forceinline__ void mma_m16n8k16_bf16(float (&c)[4], uint32_t a0, ui
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// fp8 E4M3 operands, 32 contraction elements: the same register roles as m16n8k16 with four
+// fp8 per register instead of two bf16.
+__device__ __forceinline__ void mma_m16n8k32_e4m3(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                  uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t smem_addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -47,9 +57,12 @@ __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
 // The contraction index is permuted identically in A and B so that a lane's B fragment for
 // two consecutive k-steps is one 16-byte load: within a 32-wide segment of d, lane quad
 // position t owns d[8t..8t+7]; k-step 0 uses d[8t..8t+3], k-step 1 uses d[8t+4..8t+7].
+// F8: rows of 64*NSEG fp8 E4M3 occupy the same bytes as 32*NSEG bf16, and the fp8 MMA takes 32
+// contraction elements from the registers that hold 16 bf16, so the same loads feed it: within a
+// 64-wide segment of d, lane quad position t owns d[16t..16t+15].
 constexpr int kIdxDecWarps = 8;
 
-template <int UNROLL, int NSEG>
+template <int UNROLL, int NSEG, bool F8 = false>
 __global__ void __launch_bounds__(kIdxDecWarps * 32)
 index_scores_decode_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_bfloat16* __restrict__ k_idx,
                            const int64_t* __restrict__ seq_offsets, const int32_t* __restrict__ seq_lens,
@@ -116,8 +129,13 @@ index_scores_decode_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_b
                     float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                     for (int seg = 0; seg < NSEG; ++seg) {
-                        mma_m16n8k16_bf16(c, qa[seg * 4], 0u, qa[seg * 4 + 1], 0u, kv[u][seg].x, kv[u][seg].y);
-                        mma_m16n8k16_bf16(c, qa[seg * 4 + 2], 0u, qa[seg * 4 + 3], 0u, kv[u][seg].z, kv[u][seg].w);
+                        if constexpr (F8) {
+                            mma_m16n8k32_e4m3(c, qa[seg * 4], 0u, qa[seg * 4 + 1], 0u, kv[u][seg].x, kv[u][seg].y);
+                            mma_m16n8k32_e4m3(c, qa[seg * 4 + 2], 0u, qa[seg * 4 + 3], 0u, kv[u][seg].z, kv[u][seg].w);
+                        } else {
+                            mma_m16n8k16_bf16(c, qa[seg * 4], 0u, qa[seg * 4 + 1], 0u, kv[u][seg].x, kv[u][seg].y);
+                            mma_m16n8k16_bf16(c, qa[seg * 4 + 2], 0u, qa[seg * 4 + 3], 0u, kv[u][seg].z, kv[u][seg].w);
+                        }
                     }
                     // c[0], c[1]: group g, keys nt*8 + 2t, +1
                     const int key = nt * 8 + 2 * t;

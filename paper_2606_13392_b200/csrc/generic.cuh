@@ -31,10 +31,10 @@ struct RowMap {
 
 // Eq. 6.  One warp per (query row, key block): lanes stride over the block's visible
 // tokens, each lane scoring one K_idx row against all H_kv index query heads.
-template <int WARPS>
+// F8: the operands are fp8 E4M3 instead of bf16 (Section 4.2).
+template <int WARPS, bool F8>
 __global__ void __launch_bounds__(WARPS * 32)
-index_scores_generic_kernel(const __nv_bfloat16* __restrict__ q_idx,
-                            const __nv_bfloat16* __restrict__ k_idx, RowMap rows,
+index_scores_generic_kernel(const void* __restrict__ q_idx, const void* __restrict__ k_idx, RowMap rows,
                             int64_t n_chunks, int H_kv, int d_idx, int B_k, float scale,
                             float* __restrict__ scores, int64_t ld_scores) {
     extern __shared__ float q_s[];  // [H_kv][d_idx]
@@ -44,9 +44,9 @@ index_scores_generic_kernel(const __nv_bfloat16* __restrict__ q_idx,
     int64_t pos, len, base;
     rows.get(row, pos, len, base);
 
-    const __nv_bfloat16* qrow = q_idx + row * (int64_t)H_kv * d_idx;
-    for (int t = threadIdx.x; t < H_kv * d_idx; t += WARPS * 32)
-        q_s[t] = __bfloat162float(qrow[t]);
+    constexpr int ELT = F8 ? 1 : 2;
+    const char* qrow = static_cast<const char*>(q_idx) + row * (int64_t)H_kv * d_idx * ELT;
+    for (int t = threadIdx.x; t < H_kv * d_idx; t += WARPS * 32) q_s[t] = idx_elem<F8>(qrow, t);
     __syncthreads();
 
     const int64_t b = chunk * WARPS + warp;
@@ -65,14 +65,23 @@ index_scores_generic_kernel(const __nv_bfloat16* __restrict__ q_idx,
     for (int r = 0; r < kMaxKvHeadsGeneric; ++r) best[r] = -INFINITY;
 
     for (int64_t j = j0 + lane; j < j_end; j += 32) {
-        const uint4* krow = reinterpret_cast<const uint4*>(k_idx + (base + j) * (int64_t)d_idx);
+        const char* krow = static_cast<const char*>(k_idx) + (base + j) * (int64_t)d_idx * ELT;
         float acc[kMaxKvHeadsGeneric];
 #pragma unroll
         for (int r = 0; r < kMaxKvHeadsGeneric; ++r) acc[r] = 0.f;
         for (int c = 0; c < d_idx / 8; ++c) {
-            const uint4 kv = __ldg(krow + c);
-            const float2 k0 = bf16x2_to_float2(kv.x), k1 = bf16x2_to_float2(kv.y);
-            const float2 k2 = bf16x2_to_float2(kv.z), k3 = bf16x2_to_float2(kv.w);
+            float2 k0, k1, k2, k3;  // eight consecutive elements of the key row
+            if constexpr (F8) {
+                const uint2 kv = __ldg(reinterpret_cast<const uint2*>(krow) + c);
+                k0 = make_float2(e4m3_to_float(kv.x & 0xFF), e4m3_to_float((kv.x >> 8) & 0xFF));
+                k1 = make_float2(e4m3_to_float((kv.x >> 16) & 0xFF), e4m3_to_float(kv.x >> 24));
+                k2 = make_float2(e4m3_to_float(kv.y & 0xFF), e4m3_to_float((kv.y >> 8) & 0xFF));
+                k3 = make_float2(e4m3_to_float((kv.y >> 16) & 0xFF), e4m3_to_float(kv.y >> 24));
+            } else {
+                const uint4 kv = __ldg(reinterpret_cast<const uint4*>(krow) + c);
+                k0 = bf16x2_to_float2(kv.x); k1 = bf16x2_to_float2(kv.y);
+                k2 = bf16x2_to_float2(kv.z); k3 = bf16x2_to_float2(kv.w);
+            }
 #pragma unroll
             for (int r = 0; r < kMaxKvHeadsGeneric; ++r) {
                 if (r < H_kv) {

@@ -187,8 +187,9 @@ index_lse_reduce_kernel(const int32_t* __restrict__ block_idx, RangeParams p, co
 
 // Any shape (no tensor cores, no reuse of key blocks between queries): one warp per (query,
 // head) row walks its selected blocks; lanes take keys, the row's sum is kept online.
+template <bool F8>
 __global__ void __launch_bounds__(256)
-index_lse_generic_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_bfloat16* __restrict__ k_idx,
+index_lse_generic_kernel(const void* __restrict__ q_idx, const void* __restrict__ k_idx,
                          const int32_t* __restrict__ block_idx, int64_t q_begin, int64_t q_count, int64_t kv_len,
                          int H_kv, int d_idx, int B_k, int top_k, float scale, float* __restrict__ lse_idx) {
     const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -196,7 +197,8 @@ index_lse_generic_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_bfl
     if (row >= q_count * H_kv) return;
     const int64_t q = row / H_kv;
     const int64_t pos = q_begin + q, loc = pos / B_k;
-    const __nv_bfloat16* qrow = q_idx + row * d_idx;
+    constexpr int ELT = F8 ? 1 : 2;
+    const char* qrow = static_cast<const char*>(q_idx) + row * d_idx * ELT;
     const int32_t* sel = block_idx + row * top_k;
     float mx = -INFINITY, sum = 0.f;
     for (int s = 0; s < top_k; ++s) {
@@ -205,9 +207,9 @@ index_lse_generic_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_bfl
         for (int t = lane; t < B_k; t += 32) {
             const int64_t j = (int64_t)b * B_k + t;
             if (j > pos || j >= kv_len) continue;
-            const __nv_bfloat16* krow = k_idx + j * d_idx;
+            const char* krow = static_cast<const char*>(k_idx) + j * d_idx * ELT;
             float dot = 0.f;
-            for (int c = 0; c < d_idx; ++c) dot = fmaf(__bfloat162float(qrow[c]), __bfloat162float(krow[c]), dot);
+            for (int c = 0; c < d_idx; ++c) dot = fmaf(idx_elem<F8>(qrow, c), idx_elem<F8>(krow, c), dot);
             const float x = dot * scale;
             if (x > mx) { sum = sum * expf(mx - x) + 1.f; mx = x; }
             else sum += expf(x - mx);

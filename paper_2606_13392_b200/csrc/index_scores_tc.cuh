@@ -44,13 +44,19 @@ struct IdxSmem {
 // writes, since both rank the same scaled fp32 maxima with the same tie rule.
 constexpr int kIdxFuseKeep = 15;
 
-template <int BK, int NH, int DI, int ST, int FK = 0>
+//
+// F8: the operands are fp8 E4M3 (Section 4.2), d_idx = 128 bytes = one swizzle atom (DI = 1).
+// The tiles are the same bytes in the same places as 64 bf16 per row, so the tensor maps, the
+// shared-memory layout and the descriptor walk are unchanged; only the MMA kind differs (32
+// contraction elements per 32-byte step instead of 16).
+template <int BK, int NH, int DI, int ST, int FK = 0, bool F8 = false>
 __global__ void __launch_bounds__(kIdxThreads, 1)
 index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        int64_t q_begin, int64_t q_count, int H_kv, float scale,
                        float* __restrict__ scores, int64_t ld_scores, int64_t n_cols, int* status,
                        int32_t* __restrict__ block_idx = nullptr, int top_k = 0) {
     static_assert(FK == 0 || NH <= 2, "the fused form keeps its candidates in registers");
+    static_assert(!F8 || DI == 1, "fp8 index vectors are one 128-byte atom");
     extern __shared__ uint8_t smem_raw[];
     IdxSmem<NH, DI, ST>& sm =
         *reinterpret_cast<IdxSmem<NH, DI, ST>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -100,7 +106,8 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(kIdxTileQ, kIdxTileK, false, false);
+            constexpr uint32_t idesc =
+                F8 ? make_idesc_e4m3(kIdxTileQ, kIdxTileK) : make_idesc_bf16(kIdxTileQ, kIdxTileK, false, false);
             bool ok = mbar_wait(&sm.a_full, 0, abort);
             if (!ok) report_async(status, kAsyncTimeout, 0x102);
             for (int t = 0; ok && t < n_tiles; ++t) {
@@ -122,8 +129,12 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         const uint64_t a_desc = make_smem_desc(smem_u32(sm.a[h][a]), 16, 1024);
                         const uint64_t b_desc = make_smem_desc(smem_u32(sm.b[s][a]), 16, 1024);
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)  // 16 bf16 = 32 bytes = 2 descriptor units per K step
-                            mma_bf16_ss(tmem + buf * kIdxTileK, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (a | kk) > 0);
+                        for (int kk = 0; kk < 4; ++kk) {  // 32 bytes (16 bf16 or 32 fp8) = 2 descriptor units per K step
+                            if constexpr (F8)
+                                mma_e4m3_ss(tmem + buf * kIdxTileK, a_desc + 2 * kk, b_desc + 2 * kk, idesc, kk > 0);
+                            else
+                                mma_bf16_ss(tmem + buf * kIdxTileK, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (a | kk) > 0);
+                        }
                     }
                     mma_commit(&sm.acc_full[buf]);
                 }

@@ -49,6 +49,8 @@ int* async_status_ptr() {
 struct Resolved {
     int H_q, H_kv, G, d, d_idx, B_k, k;
     float softmax_scale, index_scale;
+    bool idx_fp8;                                        // index-branch operands are fp8 E4M3 (else bf16)
+    size_t idx_elt() const { return idx_fp8 ? 1 : 2; }  // bytes per index-branch element
 };
 
 static msa_status_t resolve(const msa_shape_t* s, Resolved& r) {
@@ -65,6 +67,9 @@ static msa_status_t resolve(const msa_shape_t* s, Resolved& r) {
     if (!(s->softmax_scale >= 0.f) || !(s->index_scale >= 0.f)) return MSA_ERR_INVALID_ARG;
     r.softmax_scale = s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf((float)r.d);
     r.index_scale = s->index_scale > 0.f ? s->index_scale : 1.0f / sqrtf((float)r.d_idx);
+    if (s->idx_fp8 != 0 && s->idx_fp8 != 1) return MSA_ERR_INVALID_ARG;
+    r.idx_fp8 = s->idx_fp8 == 1;
+    if (r.idx_fp8 && r.d_idx % 16 != 0) return MSA_ERR_UNSUPPORTED;  // 16-byte rows
     return MSA_OK;
 }
 
@@ -116,7 +121,9 @@ bool encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64
 }
 
 // ---------------------------------------------------------------------- stage 1
-template <int BK, int NH, int DI, int FK = 0>
+// F8: fp8 E4M3 operands with d_idx = 128; the bytes of a row are laid out like 64 bf16, so the
+// tensor maps below (bf16 element type, used only to move bytes) serve both.
+template <int BK, int NH, int DI, int FK = 0, bool F8 = false>
 static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                     int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
                                     int64_t n_cols, cudaStream_t st, int32_t* block_idx = nullptr) {
@@ -139,7 +146,7 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
     static bool attr_set_dev[64] = {false};  // the attribute is per device
     const int dev_id = current_device();
     if (!attr_set_dev[dev_id]) {
-        if (cudaFuncSetAttribute(index_scores_tc_kernel<BK, NH, DI, ST, FK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(index_scores_tc_kernel<BK, NH, DI, ST, FK, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem) != cudaSuccess)
             return MSA_ERR_CUDA;
         attr_set_dev[dev_id] = true;
@@ -148,7 +155,7 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
     if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
     {
         StageScope sc(kStageIndex, st);
-        index_scores_tc_kernel<BK, NH, DI, ST, FK><<<(unsigned)grid, kIdxThreads, smem, st>>>(
+        index_scores_tc_kernel<BK, NH, DI, ST, FK, F8><<<(unsigned)grid, kIdxThreads, smem, st>>>(
             tm_q, tm_k, q_begin, q_count, r.H_kv, r.index_scale, scores, ld_scores, n_cols, status, block_idx, r.k);
     }
     return launch_status();
@@ -157,7 +164,7 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
 // Heads sharing one key tile per CTA: the most (8, 4, 2, 1; at most 2 when d_idx = 128, for
 // shared memory) that divide H_kv and still leave at least two CTAs per SM, so that short
 // chunks keep the machine full.
-template <int BK, int DI>
+template <int BK, int DI, bool F8 = false>
 static msa_status_t launch_index_tc_bk(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                        int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
                                        int64_t n_cols, cudaStream_t st) {
@@ -166,31 +173,39 @@ static msa_status_t launch_index_tc_bk(const Resolved& r, const void* q_idx, con
     for (int cand = (DI == 1 ? 8 : 2); cand > 1; cand >>= 1)
         if (r.H_kv % cand == 0 && n_qtiles * (r.H_kv / cand) >= 2 * sm_count()) { nh = cand; break; }
     if constexpr (DI == 1) {
-        if (nh == 8) return launch_index_tc<BK, 8, DI>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
-        if (nh == 4) return launch_index_tc<BK, 4, DI>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+        if (nh == 8) return launch_index_tc<BK, 8, DI, 0, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+        if (nh == 4) return launch_index_tc<BK, 4, DI, 0, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
     }
-    if (nh == 2) return launch_index_tc<BK, 2, DI>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
-    return launch_index_tc<BK, 1, DI>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    if (nh == 2) return launch_index_tc<BK, 2, DI, 0, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    return launch_index_tc<BK, 1, DI, 0, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+}
+
+// Shapes of the tensor-core index kernel: one or two 128-byte atoms per index vector.
+static bool index_tc_ok(const Resolved& r) {
+    return (r.idx_fp8 ? r.d_idx == 128 : (r.d_idx == 64 || r.d_idx == 128)) && (r.B_k == 64 || r.B_k == 128);
 }
 
 // Eq. 6 and Eq. 7 in one kernel, no score matrix (top_k <= 16 on the tensor-core path).
 static bool index_topk_fused_ok(const Resolved& r, int64_t q_count, int64_t kv_len) {
-    return r.k <= kIdxFuseKeep + 1 && (r.d_idx == 64 || r.d_idx == 128) && (r.B_k == 64 || r.B_k == 128) &&
-           kv_len < 2147483647LL && q_count >= 32;
+    return r.k <= kIdxFuseKeep + 1 && index_tc_ok(r) && kv_len < 2147483647LL && q_count >= 32;
 }
 
-template <int BK, int DI>
+template <int BK, int DI, bool F8 = false>
 static msa_status_t launch_index_fused_bk(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                           int64_t q_count, int64_t kv_len, int32_t* block_idx, cudaStream_t st) {
     if (r.H_kv % 2 == 0)
-        return launch_index_tc<BK, 2, DI, kIdxFuseKeep>(r, q_idx, k_idx, q_begin, q_count, kv_len, nullptr, 0, 0, st,
+        return launch_index_tc<BK, 2, DI, kIdxFuseKeep, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, nullptr, 0, 0, st,
                                                         block_idx);
-    return launch_index_tc<BK, 1, DI, kIdxFuseKeep>(r, q_idx, k_idx, q_begin, q_count, kv_len, nullptr, 0, 0, st,
+    return launch_index_tc<BK, 1, DI, kIdxFuseKeep, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, nullptr, 0, 0, st,
                                                     block_idx);
 }
 
 static msa_status_t run_index_topk_fused(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                          int64_t q_count, int64_t kv_len, int32_t* block_idx, cudaStream_t st) {
+    if (r.idx_fp8) {
+        if (r.B_k == 64) return launch_index_fused_bk<64, 1, true>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
+        return launch_index_fused_bk<128, 1, true>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
+    }
     if (r.d_idx == 64) {
         if (r.B_k == 64) return launch_index_fused_bk<64, 1>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
         return launch_index_fused_bk<128, 1>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
@@ -203,9 +218,12 @@ static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const
                                      const RowMap& rows, int64_t n_rows, float* scores,
                                      int64_t ld_scores, cudaStream_t st) {
     if (n_rows == 0 || rows.n_cols == 0) return MSA_OK;
-    if (rows.seq_lens == nullptr && (r.d_idx == 64 || r.d_idx == 128) && (r.B_k == 64 || r.B_k == 128) &&
-        rows.kv_len < 2147483647LL && n_rows >= 32) {
+    if (rows.seq_lens == nullptr && index_tc_ok(r) && rows.kv_len < 2147483647LL && n_rows >= 32) {
         const int64_t qb = rows.q_begin, kl = rows.kv_len, nc = rows.n_cols;
+        if (r.idx_fp8) {
+            if (r.B_k == 64) return launch_index_tc_bk<64, 1, true>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
+            return launch_index_tc_bk<128, 1, true>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
+        }
         if (r.d_idx == 64) {
             if (r.B_k == 64) return launch_index_tc_bk<64, 1>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
             return launch_index_tc_bk<128, 1>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
@@ -220,9 +238,12 @@ static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const
     const size_t smem = sizeof(float) * (size_t)r.H_kv * r.d_idx;
     {
         StageScope sc(rows.seq_lens ? kStageIndexDecode : kStageIndex, st);
-        index_scores_generic_kernel<WARPS><<<(unsigned)grid, WARPS * 32, smem, st>>>(
-            (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx, rows, n_chunks, r.H_kv, r.d_idx,
-            r.B_k, r.index_scale, scores, ld_scores);
+        if (r.idx_fp8)
+            index_scores_generic_kernel<WARPS, true><<<(unsigned)grid, WARPS * 32, smem, st>>>(
+                q_idx, k_idx, rows, n_chunks, r.H_kv, r.d_idx, r.B_k, r.index_scale, scores, ld_scores);
+        else
+            index_scores_generic_kernel<WARPS, false><<<(unsigned)grid, WARPS * 32, smem, st>>>(
+                q_idx, k_idx, rows, n_chunks, r.H_kv, r.d_idx, r.B_k, r.index_scale, scores, ld_scores);
     }
     return launch_status();
 }
@@ -463,14 +484,20 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
 }
 
 // ---------------------------------------------------------------------- decode path
-static bool index_decode_fast(const Resolved& r) { return (r.d_idx == 64 || r.d_idx == 128) && r.H_kv <= 8; }
+static bool index_decode_fast(const Resolved& r) {
+    return (r.idx_fp8 ? r.d_idx == 128 : (r.d_idx == 64 || r.d_idx == 128)) && r.H_kv <= 8;
+}
 
 static msa_status_t run_index_decode(const Resolved& r, const void* q_idx, const void* k_idx_cache,
                                      const int64_t* seq_offsets, const int32_t* seq_lens, int batch,
                                      int64_t n_cols, float* scores, int64_t ld_scores, cudaStream_t st) {
     const int grid = sm_count() * 4;
     StageScope sc(kStageIndexDecode, st);
-    if (r.d_idx == 64)
+    if (r.idx_fp8)  // 128 fp8 per row: the bytes of 64 bf16
+        index_scores_decode_kernel<8, 2, true><<<grid, kIdxDecWarps * 32, 0, st>>>(
+            (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx_cache, seq_offsets, seq_lens, batch, r.H_kv,
+            r.B_k, r.index_scale, scores, ld_scores, n_cols);
+    else if (r.d_idx == 64)
         index_scores_decode_kernel<8, 2><<<grid, kIdxDecWarps * 32, 0, st>>>(
             (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx_cache, seq_offsets, seq_lens, batch, r.H_kv,
             r.B_k, r.index_scale, scores, ld_scores, n_cols);
@@ -536,8 +563,8 @@ static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const v
 }
 
 // ---------------------------------------------------------------------- index-branch LSE (Section 4.3)
-static bool index_lse_fast(const Resolved& r) {
-    return (r.d_idx == 64 || r.d_idx == 128) && (r.B_k == 64 || r.B_k == 128);
+static bool index_lse_fast(const Resolved& r) {  // bf16 operands; fp8 takes the generic kernel
+    return !r.idx_fp8 && (r.d_idx == 64 || r.d_idx == 128) && (r.B_k == 64 || r.B_k == 128);
 }
 
 // Workspace for ranges of R queries: [cnt | tile_off | item_off] per tile, handles, rank, partials.
@@ -870,9 +897,12 @@ msa_status_t msa_index_lse_prefill(const msa_shape_t* shape, const void* q_idx, 
     if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
     {
         StageScope sc(kStageIndexLse, st);
-        index_lse_generic_kernel<<<(unsigned)grid, 256, 0, st>>>(
-            (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx, block_idx, q_begin, q_count, kv_len, r.H_kv,
-            r.d_idx, r.B_k, r.k, r.index_scale, lse_idx);
+        if (r.idx_fp8)
+            index_lse_generic_kernel<true><<<(unsigned)grid, 256, 0, st>>>(
+                q_idx, k_idx, block_idx, q_begin, q_count, kv_len, r.H_kv, r.d_idx, r.B_k, r.k, r.index_scale, lse_idx);
+        else
+            index_lse_generic_kernel<false><<<(unsigned)grid, 256, 0, st>>>(
+                q_idx, k_idx, block_idx, q_begin, q_count, kv_len, r.H_kv, r.d_idx, r.B_k, r.k, r.index_scale, lse_idx);
     }
     return launch_status();
 }
@@ -1035,7 +1065,7 @@ static msa_status_t prefill_stages_1_2(const msa_shape_t* shape, const Resolved&
     float* scores = static_cast<float*>(workspace);
     for (int64_t q0 = 0; q0 < T; q0 += chunk) {
         const int64_t qc = (T - q0) < chunk ? (T - q0) : chunk;
-        const char* qi = static_cast<const char*>(q_idx) + (size_t)q0 * r.H_kv * r.d_idx * 2;
+        const char* qi = static_cast<const char*>(q_idx) + (size_t)q0 * r.H_kv * r.d_idx * r.idx_elt();
         // Only keys up to the chunk's last query are visible, so score that prefix.
         const int64_t kv_vis = q0 + qc;
         s = msa_index_scores(shape, qi, k_idx, q0, qc, kv_vis, scores, ld, stream);
@@ -1090,7 +1120,7 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
     if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
     // Every sequence is an independent problem: the single-sequence path on row-offset pointers.
     const size_t q_row = (size_t)r.H_q * r.d * 2, kv_row = (size_t)r.H_kv * r.d * 2;
-    const size_t qi_row = (size_t)r.H_kv * r.d_idx * 2, ki_row = (size_t)r.d_idx * 2;
+    const size_t qi_row = (size_t)r.H_kv * r.d_idx * r.idx_elt(), ki_row = (size_t)r.d_idx * r.idx_elt();
     for (int32_t i = 0; i < n_seqs; ++i) {
         const int64_t o = cu_seqlens[i], T = cu_seqlens[i + 1] - o;
         if (T == 0) continue;
@@ -1109,8 +1139,8 @@ static size_t host_staging_bytes(const Resolved& r, int64_t T, size_t off[8]) {
     off[0] = o; o += align_up((size_t)T * r.H_q * r.d * 2);      // q
     off[1] = o; o += align_up((size_t)T * r.H_kv * r.d * 2);     // k
     off[2] = o; o += align_up((size_t)T * r.H_kv * r.d * 2);     // v
-    off[3] = o; o += align_up((size_t)T * r.H_kv * r.d_idx * 2); // q_idx
-    off[4] = o; o += align_up((size_t)T * r.d_idx * 2);          // k_idx
+    off[3] = o; o += align_up((size_t)T * r.H_kv * r.d_idx * r.idx_elt()); // q_idx
+    off[4] = o; o += align_up((size_t)T * r.d_idx * r.idx_elt());          // k_idx
     off[5] = o; o += align_up((size_t)T * r.H_q * r.d * 2);      // out
     off[6] = o; o += align_up((size_t)T * r.H_q * 4);            // lse
     off[7] = o; o += align_up((size_t)T * r.H_kv * r.k * 4);     // block_idx
@@ -1158,8 +1188,8 @@ msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_ho
     if (cudaEventRecord(e_in, st) != cudaSuccess || cudaStreamWaitEvent(copy, e_in, 0) != cudaSuccess) return MSA_ERR_CUDA;
     const void* src[5] = {q_host, k_host, v_host, q_idx_host, k_idx_host};
     const size_t nbytes[5] = {(size_t)T * r.H_q * r.d * 2, (size_t)T * r.H_kv * r.d * 2,
-                              (size_t)T * r.H_kv * r.d * 2, (size_t)T * r.H_kv * r.d_idx * 2,
-                              (size_t)T * r.d_idx * 2};
+                              (size_t)T * r.H_kv * r.d * 2, (size_t)T * r.H_kv * r.d_idx * r.idx_elt(),
+                              (size_t)T * r.d_idx * r.idx_elt()};
     const int order[5] = {4, 3, 1, 2, 0};  // k_idx, q_idx, k, v, q
     for (int j = 0; j < 5; ++j) {
         const int i = order[j];
@@ -1224,7 +1254,7 @@ msa_status_t msa_decode_forward_host(const msa_shape_t* shape, const void* q_hos
     if (batch == 0) return MSA_OK;
     if (!q_host || !q_idx_host || !q_dev || !q_idx_dev || !out_dev || !out_host) return MSA_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    const size_t qb = (size_t)batch * r.H_q * r.d * 2, qib = (size_t)batch * r.H_kv * r.d_idx * 2;
+    const size_t qb = (size_t)batch * r.H_q * r.d * 2, qib = (size_t)batch * r.H_kv * r.d_idx * r.idx_elt();
     if (cudaMemcpyAsync(q_dev, q_host, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return MSA_ERR_CUDA;
     if (cudaMemcpyAsync(q_idx_dev, q_idx_host, qib, cudaMemcpyHostToDevice, st) != cudaSuccess) return MSA_ERR_CUDA;
     s = msa_decode_forward(shape, q_dev, q_idx_dev, k_cache, v_cache, k_idx_cache, cache_tokens,

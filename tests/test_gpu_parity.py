@@ -33,7 +33,7 @@ def run_prefill_case(cfg: MSAConfig, sharp: bool, n_sample: int, ws_bytes=None):
     pos_t = torch.from_numpy(pos).to(DEV)
     # the oracle needs every key/value row but only the sampled query rows
     kb, vb, kib = to_bits(x["k"]), to_bits(x["v"]), to_bits(x["k_idx"])
-    qb, qib = to_bits(x["q"][pos_t]), to_bits(x["q_idx"][pos_t])
+    qb, qib = to_bits(x["q"][pos_t]), to_bits(x["q_idx"])[pos]
 
     # --- whole path on the GPU
     out, lse, I = api.prefill_forward(cfg, x, workspace_bytes=ws_bytes)
@@ -420,3 +420,94 @@ def test_decode_g16_b64():
     cfg = MSAConfig("dec-g16", "decode", 0, 32, 2, 64, 12, head_dim=128, idx_dim=64, seed=8,
                     seq_lens=(70, 640, 641, 7000))
     run_decode_case(cfg, True)
+
+
+# ----------------------------------------------------------------- fp8 E4M3 index operands (Section 4.2)
+@pytest.mark.parametrize("name,T,Hq,Hkv,Bk,k,di,sharp", [
+    ("paper regime, fused selection", 6144 + 77, 64, 4, 128, 16, 128, True),
+    ("paper regime, diffuse", 5000, 64, 4, 128, 16, 128, False),
+    ("8 index heads, k 64", 7000, 64, 8, 128, 64, 128, True),
+    ("B_k 64", 4096 + 9, 16, 2, 64, 24, 128, True),
+    ("short range, generic kernel", 20, 16, 2, 64, 4, 128, True),
+    ("generic shape", 700, 6, 3, 16, 5, 32, True),
+])
+def test_fp8_index_prefill(name, T, Hq, Hkv, Bk, k, di, sharp):
+    cfg = MSAConfig("f8", "prefill", T, Hq, Hkv, Bk, k, head_dim=128 if Hq > 6 else 64, idx_dim=di, seed=T,
+                    idx_fp8=True)
+    stats = run_prefill_case(cfg, sharp, n_sample=200)
+    assert stats["exact_sets"] >= 0.999, (name, stats)
+    print("fp8", name, stats)
+
+
+def test_fp8_fused_equals_separate_calls_and_small_workspace():
+    cfg = MSAConfig("f8-fused", "prefill", 9000, 64, 4, 128, 16, head_dim=128, idx_dim=128, seed=12, idx_fp8=True)
+    x = make_prefill_inputs(cfg, DEV, sharp=True)
+    shape = B.shape_of(cfg)
+    T = cfg.T
+    I_f = torch.full((T, 4, 16), -7, dtype=torch.int32, device=DEV)
+    B.msa_index_topk_fused(shape, x["q_idx"], x["k_idx"], 0, T, T, I_f)
+    M = api.index_scores(cfg, x["q_idx"], x["k_idx"], 0, T)
+    I_s = api.topk_select(cfg, M, 0, T)
+    mn, pf = B.msa_prefill_forward_workspace_bytes(shape, T)
+    o1, l1, i1 = api.prefill_forward(cfg, x, workspace_bytes=pf)
+    o2, l2, i2 = api.prefill_forward(cfg, x, workspace_bytes=mn)  # several ranges: q_idx offsets in bytes
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert torch.equal(I_f, I_s) and torch.equal(i1, I_s) and torch.equal(i2, I_s)
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
+
+
+def test_fp8_varlen_equals_sequence_by_sequence():
+    cfg = MSAConfig("f8-varlen", "prefill", 0, 64, 4, 128, 16, head_dim=128, idx_dim=128, seed=4, idx_fp8=True)
+    lens = [1000, 37, 0, 4096 + 5, 2500]
+    cu = np.concatenate([[0], np.cumsum(lens)]).tolist()
+    x = make_prefill_inputs(cfg.scaled(T=cu[-1]), DEV, sharp=True)
+    out, lse, I = api.prefill_forward_varlen(cfg.scaled(T=cu[-1]), x, cu)
+    torch.cuda.synchronize()
+    _assert_clean()
+    for s, L in enumerate(lens):
+        if L == 0:
+            continue
+        a, b = cu[s], cu[s + 1]
+        xs = {n: t[a:b].contiguous() for n, t in x.items()}
+        o1, l1, i1 = api.prefill_forward(cfg.scaled(T=L), xs)
+        torch.cuda.synchronize()
+        assert torch.equal(I[a:b], i1) and torch.equal(out[a:b], o1) and torch.equal(lse[a:b], l1), s
+
+
+@pytest.mark.parametrize("Hkv,di,lens", [
+    (4, 128, (1, 130, 4096, 5000, 30000, 16384 + 64)),   # streaming tensor-core kernel
+    (3, 32, (5, 16, 17, 400, 1000)),                     # generic kernel
+])
+def test_fp8_index_decode(Hkv, di, lens):
+    big = di == 128
+    cfg = MSAConfig("f8-dec", "decode", 0, 64 if big else 6, Hkv, 128 if big else 16, 16 if big else 5,
+                    head_dim=128 if big else 64, idx_dim=di, seed=21, seq_lens=lens, idx_fp8=True)
+    res = run_decode_case(cfg, True)
+    assert np.mean([r["exact"] for r in res]) >= 0.95
+
+
+def test_fp8_index_lse_matches_oracle():
+    cfg = MSAConfig("f8-lse", "prefill", 3000, 64, 4, 128, 16, head_dim=128, idx_dim=128, seed=6, idx_fp8=True)
+    x = make_prefill_inputs(cfg, DEV, sharp=True)
+    _, _, I = api.prefill_forward(cfg, x)
+    got = api.index_lse(cfg, x["q_idx"], x["k_idx"], I)
+    torch.cuda.synchronize()
+    _assert_clean()
+    pos = sample_positions(cfg.T, 128, 16, 160, 5)
+    pos_t = torch.from_numpy(pos).to(DEV)
+    want = oracle.index_lse(to_bits(x["q_idx"])[pos], to_bits(x["k_idx"]), I[pos_t].cpu().numpy(), pos, 128)
+    err = np.abs(got[pos_t].cpu().numpy().astype(np.float64) - want)
+    assert np.isfinite(want).all() and err.max() <= 2e-3, float(err.max())
+
+
+def test_fp8_flag_and_operand_size_must_agree():
+    cfg = MSAConfig("f8-bad", "prefill", 256, 16, 2, 64, 4, head_dim=128, idx_dim=128, seed=1)
+    x = make_prefill_inputs(cfg, DEV)  # bf16 index operands
+    shape = B.shape_of(cfg.scaled(idx_fp8=True))
+    with pytest.raises(AssertionError):
+        B.msa_index_scores(shape, x["q_idx"], x["k_idx"], 0, 256, 256,
+                           torch.empty((256, 2, 4), device=DEV), 4)
+    shape.idx_fp8 = 2
+    with pytest.raises(B.MsaError):
+        B.msa_prefill_forward_workspace_bytes(shape, 256)
