@@ -73,7 +73,7 @@ def decode_work(cfg: MSAConfig):
     n_sel = np.minimum(k, loc + 1)
     tokens = (n_sel - 1) * Bk + ((lens - 1) % Bk) + 1
     return {
-        "index_bytes": 2.0 * cfg.idx_dim * float(lens.sum()),
+        "index_bytes": (1.0 if cfg.idx_fp8 else 2.0) * cfg.idx_dim * float(lens.sum()),
         "index_flops": 2.0 * cfg.n_kv_heads * cfg.idx_dim * float(lens.sum()),
         "attn_bytes": 2.0 * 2 * cfg.n_kv_heads * cfg.head_dim * float(tokens.sum()),
         "attn_flops": 4.0 * cfg.n_q_heads * cfg.head_dim * float(tokens.sum()),
@@ -194,6 +194,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-others", action="store_true")
+    ap.add_argument("--index-lse", action="store_true",
+                    help="prefill: also time the index-branch log-sum-exp (Section 4.3) on the step's selection; "
+                         "reported beside the step, not part of it")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -256,12 +259,13 @@ def base_line(cfg: MSAConfig, args, n_gpus: int):
 
 
 def describe(cfg: MSAConfig) -> str:
+    f8 = ", index operands fp8 E4M3" if cfg.idx_fp8 else ""
     if cfg.mode == "prefill":
-        return ("prefill fwd, batch 1, T=%d causal, %d q heads / %d kv heads, d_h=%d, d_idx=%d, B_k=%d, k=%d"
-                % (cfg.T, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.idx_dim, cfg.block_size, cfg.top_k))
-    return ("decode, batch %d (lens %s), %d q heads / %d kv heads, d_h=%d, d_idx=%d, B_k=%d, k=%d"
+        return ("prefill fwd, batch 1, T=%d causal, %d q heads / %d kv heads, d_h=%d, d_idx=%d, B_k=%d, k=%d%s"
+                % (cfg.T, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.idx_dim, cfg.block_size, cfg.top_k, f8))
+    return ("decode, batch %d (lens %s), %d q heads / %d kv heads, d_h=%d, d_idx=%d, B_k=%d, k=%d%s"
             % (len(cfg.seq_lens), sorted(set(cfg.seq_lens)), cfg.n_q_heads, cfg.n_kv_heads,
-               cfg.head_dim, cfg.idx_dim, cfg.block_size, cfg.top_k))
+               cfg.head_dim, cfg.idx_dim, cfg.block_size, cfg.top_k, f8))
 
 
 def run_reference(cfg: MSAConfig, args):
@@ -388,8 +392,12 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
             bound, work = spec[name]
             if bound == "tensor":
                 ach = work / (per_step_ms * 1e-3) / 1e12
-                ent.update(bound="tensor", achieved=ach, unit="TFLOP/s", peak=tf_s, frac=ach / tf_s,
-                           frac_of_burst_peak=ach / tf_b)
+                # an fp8 contraction: the measured bf16 peaks times the nominal fp8 / bf16 ratio of 2
+                mul = 2.0 if (cfg.idx_fp8 and name == "index_scores") else 1.0
+                ent.update(bound="tensor", achieved=ach, unit="TFLOP/s", peak=tf_s * mul, frac=ach / (tf_s * mul),
+                           frac_of_burst_peak=ach / (tf_b * mul))
+                if mul != 1.0:
+                    ent["peak_dtype"] = "fp8 = measured bf16 x 2 (nominal ratio)"
             else:
                 ach = work / (per_step_ms * 1e-3) / 1e9
                 ent.update(bound="hbm", achieved=ach, unit="GB/s", peak=hbm, frac=ach / hbm)
@@ -420,6 +428,31 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
         torch.cuda.empty_cache()
         line["e2e"] = run_e2e(cfg, shape, x, B, dev, min(steps, 3), world)
 
+    # ---- training-side forward output, timed on its own (Section 4.3)
+    if getattr(args, "index_lse", False) and cfg.mode == "prefill":
+        mn_l, pf_l = B.msa_index_lse_prefill_workspace_bytes(shape, T, T)
+        ws_l = B.alloc_workspace(pf_l, dev)
+        lse_idx = torch.empty((T, cfg.n_kv_heads), dtype=torch.float32, device=dev)
+
+        def lse_step():
+            B.msa_index_lse_prefill(shape, x["q_idx"], x["k_idx"], block_idx, 0, T, T, lse_idx, ws_l)
+        for _ in range(2):
+            lse_step()
+        torch.cuda.synchronize()
+        n_rep = min(steps, 3)
+        e0.record(stream)
+        for _ in range(n_rep):
+            lse_step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / n_rep
+        w = prefill_work(cfg)
+        # one dot product of d_idx per (query, index head, visible token of a selected block)
+        flops = w["attn_flops"] / (4.0 * cfg.n_q_heads * cfg.head_dim) * 2.0 * cfg.n_kv_heads * cfg.idx_dim
+        line["index_lse"] = {"ms": ms, "bound": "tensor", "achieved": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                             "peak": peaks["bf16_tflops"], "frac": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+        del ws_l, lse_idx
+
     # ---- the oracle on this machine's host cores (bounded sample)
     if cpu:
         import oracle
@@ -429,7 +462,8 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
             rng = np.random.default_rng(123)
             pos = np.sort(rng.choice(cfg.T, size=min(n, cfg.T), replace=False)).astype(np.int64)
             pt = torch.from_numpy(pos).to(dev)
-            qb, qib = to_bits(x["q"][pt]), to_bits(x["q_idx"][pt])
+            qb = to_bits(x["q"][pt])
+            qib = (x["q_idx"].view(torch.uint8)[pt].cpu().numpy() if cfg.idx_fp8 else to_bits(x["q_idx"][pt]))
             t0 = time.perf_counter()
             oracle.msa_forward(qb, xb["k"], xb["v"], qib, xb["k_idx"], pos, cfg.block_size, cfg.top_k)
             dt = time.perf_counter() - t0

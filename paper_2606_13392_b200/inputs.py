@@ -72,6 +72,11 @@ CONFIGS: Dict[str, MSAConfig] = {
     "p1m": MSAConfig("p1m", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=7),
     "pdec": MSAConfig("pdec", "decode", 1048576, 64, 4, 128, 16, idx_dim=128, seed=8,
                       seq_lens=(131072,) * 16 + (1048576,) * 16),
+    # The same regime with the index-branch operands stored in fp8 E4M3 (Section 4.2).
+    "p128k-f8": MSAConfig("p128k-f8", "prefill", 131072, 64, 4, 128, 16, idx_dim=128, seed=6, idx_fp8=True),
+    "p1m-f8": MSAConfig("p1m-f8", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=7, idx_fp8=True),
+    "pdec-f8": MSAConfig("pdec-f8", "decode", 1048576, 64, 4, 128, 16, idx_dim=128, seed=8,
+                         seq_lens=(131072,) * 16 + (1048576,) * 16, idx_fp8=True),
     # Reduced cases of the same shapes, small enough for multi-pass profiler captures
     # (inputs still larger than L2).
     "c3-16k": MSAConfig("c3-16k", "prefill", 16384, 64, 8, 128, 64, seed=2,
