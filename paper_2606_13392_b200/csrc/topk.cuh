@@ -13,6 +13,9 @@
 //           block; only rows with more survivors than the log holds are walked a second time.
 //           Index order makes the output list ascending with no final sort; the local block
 //           is appended by construction (never ranked).
+// Both passes are written over a "stream" (elements in ascending block order); long rows run them
+// twice, on the maxima of runs of 8 blocks and then on the blocks of the runs that matter (see
+// "two-level selection" below).
 #pragma once
 
 #include "common.cuh"
@@ -105,47 +108,41 @@ constexpr int kTopkWarps = 4;
 constexpr int kTopkLoads = MSA_TOPK_LOADS;            // coalesced 32-wide loads per round
 constexpr int kTopkRound = 32 * kTopkLoads;           // blocks covered by one round
 constexpr int kTopkStage = 32 + kTopkRound;           // flush threshold (32) + one round of pushes
-constexpr int kTopkLog = 768;    // survivors remembered per row for the index pass
+constexpr int kTopkLog = 512;    // survivors remembered per row for the index pass
 
-template <int R>
-__global__ void __launch_bounds__(kTopkWarps * 32)
-topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap rows,
-                   int64_t n_rows, int H_kv, int B_k, int top_k, int32_t* __restrict__ block_idx) {
-    __shared__ uint32_t stg_all[kTopkWarps][kTopkStage];
-    __shared__ uint2 log_all[kTopkWarps][kTopkLog];   // (key, block) of every survivor, in index order
-    __shared__ int32_t out_all[kTopkWarps][32 * R];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * kTopkWarps + warp;
-    if (row >= n_rows) return;
-    int64_t pos, len, base;
-    rows.get(row / H_kv, pos, len, base);
-    const int64_t loc = pos / B_k;
-    int32_t* orow = block_idx + row * (int64_t)top_k;
+// A row as the selection sees it: element i of n has a score and a block index; the elements come
+// in ascending block order.
+struct TopkPlainStream {            // blocks [0, n) of a score row
+    const float* srow;
+    int n;
+    __device__ __forceinline__ float score(int i) const { return i < n ? __ldg(srow + i) : -INFINITY; }
+    __device__ __forceinline__ bool in(int i) const { return i < n; }
+    __device__ __forceinline__ uint32_t block(int i) const { return (uint32_t)i; }
+};
 
-    if (loc <= top_k - 1) {  // every visible block is selected
-        for (int e = lane; e < top_k; e += 32) orow[e] = (e <= loc) ? e : -1;
-        return;
-    }
-    const int m = top_k - 1;  // ranked entries; candidates are blocks [0, loc)
-    if (m == 0) {
-        for (int e = lane; e < top_k; e += 32) orow[e] = (e == 0) ? (int32_t)loc : -1;
-        return;
-    }
-    const float* srow = scores + row * ld_scores;
-    uint32_t* stg = stg_all[warp];
-    uint2* logb = log_all[warp];
-    int32_t* outb = out_all[warp];
+// Per-warp scratch of the selection.
+struct TopkScratch {
+    uint32_t* stg;   // [kTopkStage] survivors waiting to be merged
+    uint2* logb;     // [log_cap] (key, block) of every survivor, in block order
+    int log_cap;
+};
+
+// Pass 1: the sorted keys of the m best scores of the stream (kept), a log of every element that
+// passed the filter when it was seen (all selected blocks are among them), its length, and
+// whether the log holds them all.  floor_f: a score strictly below every score that may be
+// selected (-inf if none is known); only elements above it are looked at.
+template <int R, class Stream>
+__device__ __forceinline__ void topk_pass1(const Stream& st, int m, float floor_f, const TopkScratch& sc,
+                                           uint32_t (&kept)[R], int& n_log, bool& log_ok, int lane) {
     const unsigned lt_mask = (1u << lane) - 1u;
-
-    // ------------------------------------------------------------------ pass 1: threshold value
-    // A round covers kTopkRound consecutive blocks as coalesced 32-wide loads, so that compacting
-    // the loads one after the other keeps the survivors in block order.
-    uint32_t kept[R];
+    uint32_t* stg = sc.stg;
+    uint2* logb = sc.logb;
 #pragma unroll
     for (int s = 0; s < R; ++s) kept[s] = 0;  // 0 is below every real key
-    float tau_f = -INFINITY;                   // score of the current m-th best (strict filter)
-    int cnt = 0, n_log = 0;
-    bool log_ok = true;
+    float tau_f = floor_f;                     // strict filter: the current m-th best, or the floor
+    int cnt = 0;
+    n_log = 0;
+    log_ok = true;
 
     auto flush = [&](bool all) {
         __syncwarp();
@@ -165,75 +162,77 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         if (lane < rem) stg[lane] = carry;
         cnt = rem;
         const uint32_t tau = element_at<R>(kept, m - 1);
-        tau_f = tau != 0u ? topk_key_score(tau) : -INFINITY;
+        const float t_kept = tau != 0u ? topk_key_score(tau) : -INFINITY;
+        tau_f = fmaxf(t_kept, floor_f);
         __syncwarp();
     };
 
-    {
-        constexpr int C = kTopkLoads;
-        const int n = (int)loc;  // candidates are blocks [0, n); n < 2^31
-        float nxt[C];
+    constexpr int C = kTopkLoads;
+    const int n = st.n;
+    float nxt[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) nxt[c] = st.score(c * 32 + lane);
+    // A round covers kTopkRound consecutive elements as coalesced 32-wide loads, so that compacting
+    // the loads one after the other keeps the survivors in block order.
+    for (int i0 = 0; i0 < n; i0 += kTopkRound) {
+        float x[C];
+#pragma unroll
+        for (int c = 0; c < C; ++c) x[c] = nxt[c];
+#pragma unroll
+        for (int c = 0; c < C; ++c)  // next round's loads are in flight while this one is ranked
+            nxt[c] = st.score(i0 + kTopkRound + c * 32 + lane);
+        // While fewer than m keys are kept (and no floor is known) everything passes; afterwards
+        // only strictly better scores can change the m-th best value.
+        unsigned mk[C];
+        unsigned any = 0u;
+        if (tau_f == -INFINITY) {
+#pragma unroll
+            for (int c = 0; c < C; ++c) mk[c] = __ballot_sync(0xffffffffu, st.in(i0 + c * 32 + lane));
+        } else {
+#pragma unroll
+            for (int c = 0; c < C; ++c) mk[c] = __ballot_sync(0xffffffffu, x[c] > tau_f);
+        }
+#pragma unroll
+        for (int c = 0; c < C; ++c) any |= mk[c];
+        if (any == 0u) continue;
+        // survivors keep block order: component 0's lanes first, then component 1's, ...
+        int off[C + 1];
+        off[0] = 0;
+#pragma unroll
+        for (int c = 0; c < C; ++c) off[c + 1] = off[c] + __popc(mk[c]);
+        const int tot = off[C];
+        if (log_ok && n_log + tot > sc.log_cap) log_ok = false;
 #pragma unroll
         for (int c = 0; c < C; ++c) {
-            const int i = c * 32 + lane;
-            nxt[c] = i < n ? __ldg(srow + i) : -INFINITY;
+            if (mk[c] & (1u << lane)) {
+                const int rnk = off[c] + __popc(mk[c] & lt_mask);
+                const uint32_t key = topk_key(x[c]);
+                stg[cnt + rnk] = key;
+                if (log_ok) logb[n_log + rnk] = make_uint2(key, st.block(i0 + c * 32 + lane));
+            }
         }
-        for (int i0 = 0; i0 < n; i0 += kTopkRound) {
-            float x[C];
-#pragma unroll
-            for (int c = 0; c < C; ++c) x[c] = nxt[c];
-#pragma unroll
-            for (int c = 0; c < C; ++c) {  // next round's loads are in flight while this one is ranked
-                const int i = i0 + kTopkRound + c * 32 + lane;
-                nxt[c] = i < n ? __ldg(srow + i) : -INFINITY;
-            }
-            // While fewer than m keys are kept everything passes; afterwards only strictly better
-            // scores can change the m-th best value.  (Out-of-range lanes hold -inf.)
-            unsigned mk[C];
-            unsigned any = 0u;
-            if (tau_f == -INFINITY) {
-#pragma unroll
-                for (int c = 0; c < C; ++c) mk[c] = __ballot_sync(0xffffffffu, i0 + c * 32 + lane < n);
-            } else {
-#pragma unroll
-                for (int c = 0; c < C; ++c) mk[c] = __ballot_sync(0xffffffffu, x[c] > tau_f);
-            }
-#pragma unroll
-            for (int c = 0; c < C; ++c) any |= mk[c];
-            if (any == 0u) continue;
-            // survivors keep block order: component 0's lanes first, then component 1's, ...
-            int off[C + 1];
-            off[0] = 0;
-#pragma unroll
-            for (int c = 0; c < C; ++c) off[c + 1] = off[c] + __popc(mk[c]);
-            const int tot = off[C];
-            if (log_ok && n_log + tot > kTopkLog) log_ok = false;
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                if (mk[c] & (1u << lane)) {
-                    const int rnk = off[c] + __popc(mk[c] & lt_mask);
-                    const uint32_t key = topk_key(x[c]);
-                    stg[cnt + rnk] = key;
-                    if (log_ok) logb[n_log + rnk] = make_uint2(key, (uint32_t)(i0 + c * 32 + lane));
-                }
-            }
-            cnt += tot;
-            n_log += tot;
-            if (cnt >= 32) flush(false);
-        }
-        flush(true);
+        cnt += tot;
+        n_log += tot;
+        if (cnt >= 32) flush(false);
     }
-    const uint32_t tau = element_at<R>(kept, m - 1);  // key of the m-th best score (loc > m, so it exists)
+    flush(true);
+}
+
+// Pass 2: every block whose key beats the threshold plus, among the blocks that tie with it, the
+// first ones in block order until m are taken; written ascending to outb[0..m).  Every selected
+// block survived the filter when it was seen (its score beat the threshold of that moment), so
+// the log holds them all, in block order; only a row with more survivors than the log holds is
+// walked a second time.
+template <int R, class Stream>
+__device__ __forceinline__ void topk_pass2(const Stream& st, int m, const TopkScratch& sc,
+                                           const uint32_t (&kept)[R], int n_log, bool log_ok, int32_t* outb,
+                                           int lane) {
+    const unsigned lt_mask = (1u << lane) - 1u;
+    const uint32_t tau = element_at<R>(kept, m - 1);  // key of the m-th best score (the stream has more than m elements)
     int n_gt = 0;                                      // kept keys strictly above the threshold
 #pragma unroll
     for (int s = 0; s < R; ++s) n_gt += __popc(__ballot_sync(0xffffffffu, (s * 32 + lane) < m && kept[s] > tau));
     const int need_ties = m - n_gt;                    // blocks equal to the threshold still to take
-
-    // ------------------------------------------------------------------ pass 2: indices, ascending
-    // Every selected block survived the filter when it was seen (its score beat the threshold
-    // of that moment), so the log holds them all, in block order; ties with the final threshold
-    // are taken first come, first served.  Only a row with more survivors than the log holds
-    // is walked a second time.
     int out_cnt = 0, ties_seen = 0;
     auto take_in_order = [&](uint32_t key, uint32_t blk, bool in) {
         const bool gt = in && key > tau, eq = in && key == tau;
@@ -254,17 +253,161 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         for (int e0 = 0; e0 < n_log && out_cnt < m; e0 += 32) {
             const int e = e0 + lane;
             uint2 kv = make_uint2(0u, 0u);
-            if (e < n_log) kv = logb[e];
+            if (e < n_log) kv = sc.logb[e];
             take_in_order(kv.x, kv.y, e < n_log);
         }
     } else {
-        for (int64_t i0 = 0; i0 < loc && out_cnt < m; i0 += 32) {
-            const int64_t i = i0 + lane;
-            const float x = i < loc ? __ldg(srow + i) : 0.f;
-            take_in_order(topk_key(x), (uint32_t)i, i < loc);
+        for (int i0 = 0; i0 < st.n && out_cnt < m; i0 += 32) {
+            const int i = i0 + lane;
+            const bool in = st.in(i);
+            const float x = in ? st.score(i) : 0.f;
+            take_in_order(topk_key(x), st.block(i), in);
         }
     }
     __syncwarp();
+}
+
+// Rows with at most top_k visible blocks, or top_k = 1: no ranking.  Returns true if the row is done.
+__device__ __forceinline__ bool topk_trivial_row(int64_t loc, int top_k, int32_t* orow, int lane) {
+    if (loc <= top_k - 1) {  // every visible block is selected
+        for (int e = lane; e < top_k; e += 32) orow[e] = (e <= loc) ? e : -1;
+        return true;
+    }
+    if (top_k == 1) {
+        for (int e = lane; e < top_k; e += 32) orow[e] = (e == 0) ? (int32_t)loc : -1;
+        return true;
+    }
+    return false;
+}
+
+// ------------------------------------------------------------------ two-level selection (long rows)
+// A long row is selected in three steps, the last two of which touch a fraction of it:
+//   1. tau0 = a value that the maxima of at least m runs of kTopkRunBlocks consecutive blocks reach
+//      (runs that lie wholly before the local block): m different blocks score at least tau0, so
+//      the m-th best block score is at least tau0 (one streaming pass, 8 scores per lane and load
+//      pair, no merge networks);
+//   2. the candidate runs - those whose maximum reaches tau0, plus the run that holds the local
+//      block - are listed in ascending order (every selected block is in one of them);
+//   3. the blocks of the candidate runs form a stream in block order, and the two passes above
+//      select from it exactly what they would select from the whole row, ties included.
+// The merge networks, which dominate a one-level selection, then run on about a third of the
+// survivors (run maxima first, then the few blocks above tau0).
+constexpr int kTopkRunBlocks = 8;
+constexpr int kTopkMaxRuns = 1024;     // candidate list capacity (rows of up to 8192 blocks)
+
+struct TopkRunMaxStream {  // element i: maximum of blocks [8i, 8i+8); rows are 16-byte aligned
+    const float* srow;
+    int n;
+    __device__ __forceinline__ float score(int i) const {
+        if (i >= n) return -INFINITY;
+        const float4* p = reinterpret_cast<const float4*>(srow) + 2 * i;
+        const float4 a = __ldg(p), b = __ldg(p + 1);
+        return fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w)));
+    }
+    __device__ __forceinline__ bool in(int i) const { return i < n; }
+    __device__ __forceinline__ uint32_t block(int i) const { return (uint32_t)i; }
+};
+
+struct TopkGatherStream {  // element i: block i % 8 of candidate run i / 8; blocks from loc on do not rank
+    const float* srow;
+    const uint16_t* run;   // candidate runs, ascending
+    int n;                 // 8 * number of candidate runs
+    int loc;
+    __device__ __forceinline__ uint32_t block(int i) const {
+        return (uint32_t)run[i >> 3] * kTopkRunBlocks + (uint32_t)(i & 7);
+    }
+    __device__ __forceinline__ bool in(int i) const { return i < n && (int)block(i) < loc; }
+    __device__ __forceinline__ float score(int i) const { return in(i) ? __ldg(srow + block(i)) : -INFINITY; }
+};
+
+template <int R>
+__global__ void __launch_bounds__(kTopkWarps * 32)
+topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap rows,
+                   int64_t n_rows, int H_kv, int B_k, int top_k, int32_t* __restrict__ block_idx) {
+    __shared__ uint32_t stg_all[kTopkWarps][kTopkStage];
+    __shared__ uint2 log_all[kTopkWarps][kTopkLog];   // (key, block) of every survivor, in index order
+    __shared__ uint16_t run_all[kTopkWarps][kTopkMaxRuns + 2];
+    __shared__ int32_t out_all[kTopkWarps][32 * R];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * kTopkWarps + warp;
+    if (row >= n_rows) return;
+    int64_t pos, len, base;
+    rows.get(row / H_kv, pos, len, base);
+    const int64_t loc = pos / B_k;
+    int32_t* orow = block_idx + row * (int64_t)top_k;
+    if (topk_trivial_row(loc, top_k, orow, lane)) return;
+    const int m = top_k - 1;  // ranked entries; candidates are blocks [0, loc), loc < 2^31
+    const float* srow = scores + row * ld_scores;
+    const TopkScratch sc{stg_all[warp], log_all[warp], kTopkLog};
+    int32_t* outb = out_all[warp];
+    uint32_t kept[R];
+    int n_log;
+    bool log_ok;
+    const int64_t n_full = loc / kTopkRunBlocks;  // runs wholly before the local block
+    if (n_full < 4 * m || n_full > kTopkMaxRuns) {  // short row (or one beyond the list): one level
+        const TopkPlainStream st{srow, (int)loc};
+        topk_pass1<R>(st, m, -INFINITY, sc, kept, n_log, log_ok, lane);
+        topk_pass2<R>(st, m, sc, kept, n_log, log_ok, outb, lane);
+    } else {
+        // 1. A threshold from the run maxima.  Any value that m run maxima reach will do, so no exact
+        // selection: every lane keeps the S = 2R largest of the maxima it sees (sorted registers, no
+        // branches), the 32 S kept values - maxima of different runs - are sorted once, and tau0 is
+        // the m-th largest of them (the exact m-th largest run maximum unless one lane saw more than S
+        // of the m largest, and then a little lower).
+        const TopkRunMaxStream rs{srow, (int)n_full};
+        constexpr int S = 2 * R;
+        float top[S];
+#pragma unroll
+        for (int i = 0; i < S; ++i) top[i] = -INFINITY;
+        for (int g0 = 0; g0 < (int)n_full; g0 += 32 * 4) {
+            float x[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) x[u] = rs.score(g0 + u * 32 + lane);  // -inf beyond n_full
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                float v = x[u];
+#pragma unroll
+                for (int i = 0; i < S; ++i) {
+                    const float hi = fmaxf(top[i], v);
+                    v = fminf(top[i], v);
+                    top[i] = hi;
+                }
+            }
+        }
+        uint32_t tk[S];
+#pragma unroll
+        for (int i = 0; i < S; ++i) tk[i] = topk_key(top[i]);
+#pragma unroll
+        for (int size = 2; size <= 32 * S; size <<= 1) {
+#pragma unroll
+            for (int stride = size >> 1; stride > 0; stride >>= 1) bitonic_stage<S>(tk, lane, size, stride);
+        }
+        const float tau0 = topk_key_score(element_at<S>(tk, m - 1));  // 32 S >= 2 m values
+        // 2. candidate runs, ascending (the row was just read: these loads hit L1 or L2)
+        uint16_t* run = run_all[warp];
+        const unsigned lt_mask = (1u << lane) - 1u;
+        int n_run = 0;
+        for (int g0 = 0; g0 < (int)n_full; g0 += 32) {
+            const int g = g0 + lane;
+            const bool c = rs.score(g) >= tau0;  // -inf beyond n_full; tau0 is a real score
+            const unsigned cm = __ballot_sync(0xffffffffu, c);
+            if (c) run[n_run + __popc(cm & lt_mask)] = (uint16_t)g;
+            n_run += __popc(cm);
+        }
+        if (n_full * kTopkRunBlocks < loc) {  // the run that holds the local block
+            if (lane == 0) run[n_run] = (uint16_t)n_full;
+            ++n_run;
+        }
+        __syncwarp();
+        // 3. select among the candidates' blocks; scores below tau0 cannot be selected.  The floor
+        // only has to lie below tau0: a hair below it, whatever its sign or size.
+        const float floor_f = tau0 - fmaxf(fabsf(tau0) * 1e-6f, 1e-30f);
+        const TopkGatherStream gs{srow, run, n_run * kTopkRunBlocks, (int)loc};
+        topk_pass1<R>(gs, m, floor_f, sc, kept, n_log, log_ok, lane);
+        topk_pass2<R>(gs, m, sc, kept, n_log, log_ok, outb, lane);
+    }
+    // Block order makes the list ascending with no final sort; the local block is appended by
+    // construction (never ranked).
     for (int e = lane; e < top_k; e += 32) orow[e] = e < m ? outb[e] : (e == m ? (int32_t)loc : -1);
 }
 

@@ -511,3 +511,58 @@ def test_fp8_flag_and_operand_size_must_agree():
     shape.idx_fp8 = 2
     with pytest.raises(B.MsaError):
         B.msa_prefill_forward_workspace_bytes(shape, 256)
+
+
+# ----------------------------------------------------------------- two-level Top-k on long rows
+@pytest.mark.parametrize("T,Hq,Hkv,k,di,ties,sharp", [
+    (100000 + 77, 16, 2, 20, 64, False, True),
+    (100000 + 77, 16, 2, 20, 64, True, True),     # many exactly equal scores (and equal run maxima)
+    (140000, 32, 4, 24, 128, True, False),
+    (300000 + 5, 64, 8, 64, 64, False, False),    # the headline shape's head layout and k
+])
+def test_two_level_topk_long_rows_bit_exact(T, Hq, Hkv, k, di, ties, sharp):
+    # Rows of 4 (k-1) runs of 8 blocks and more are selected in two levels (run maxima first, then
+    # only the runs that can hold a selected block).  The lists must be the oracle's on the very
+    # scores the GPU computed (fp32, exact in fp64), ties included, and the whole-path call must
+    # give the same lists as the separate calls.
+    cfg = MSAConfig("top2", "prefill", T, Hq, Hkv, 128, k, head_dim=128, idx_dim=di, seed=T + k)
+    x = make_prefill_inputs(cfg, DEV, sharp=sharp)
+    if ties:  # keys repeat with period 7 blocks: block maxima of different blocks coincide exactly
+        period = 7 * 128
+        x["k_idx"] = x["k_idx"][:period].repeat((T + period - 1) // period, 1)[:T].contiguous()
+    _, _, I = api.prefill_forward(cfg, x)
+    torch.cuda.synchronize()
+    _assert_clean()
+    first_long = 4 * (k - 1) * 8 * 128  # rows from here on take the two-level path
+    assert T > first_long + 4096
+    nb = cfg.n_blocks
+    for q0, qc in [(first_long - 150, 300), ((first_long + T) // 2 + 11, 400), (T - 384, 384)]:
+        M = api.index_scores(cfg, x["q_idx"], x["k_idx"], q0, qc)
+        I_s = api.topk_select(cfg, M, q0, T)
+        torch.cuda.synchronize()
+        assert torch.equal(I[q0:q0 + qc], I_s), (q0, int((I[q0:q0 + qc] != I_s).any(dim=2).sum()))
+        I_ref = oracle.topk_select(M[:, :, :nb].double().cpu().numpy(), np.arange(q0, q0 + qc), T, 128, k)
+        assert np.array_equal(I_s.cpu().numpy(), I_ref), q0
+
+
+@pytest.mark.parametrize("n_blocks,k,levels", [(3000, 20, 0), (8192, 64, 0), (8192, 64, 5), (5000, 33, 3),
+                                               (9000, 17, 0)])
+def test_two_level_topk_on_arbitrary_long_score_rows(n_blocks, k, levels):
+    # Top-k alone on synthetic score rows: continuous values, and values from a handful of levels
+    # (whole runs tie, the threshold is shared by hundreds of blocks); rows at many positions,
+    # including ones beyond the candidate list's capacity (n_blocks 9000), which take one level.
+    Bk = 16
+    T = n_blocks * Bk
+    cfg = MSAConfig("top2-raw", "prefill", T, 4, 2, Bk, k, head_dim=64, idx_dim=32, seed=n_blocks)
+    g = torch.Generator().manual_seed(n_blocks + k)
+    ld = B.score_ld(T, Bk)
+    pos = np.unique(np.concatenate([np.arange(T - 40, T), np.linspace(4 * (k - 1) * 8 * Bk - 20, T - 1, 150).astype(np.int64)]))
+    runs = np.split(pos, np.where(np.diff(pos) != 1)[0] + 1)
+    for run in runs:
+        q0, qc = int(run[0]), len(run)
+        M = torch.randn((qc, 2, ld), generator=g)
+        if levels:
+            M = torch.randint(0, levels, (qc, 2, ld), generator=g).float() * 0.5 - 1.0
+        I = api.topk_select(cfg, M.to(DEV), q0, T).cpu().numpy()
+        I_ref = oracle.topk_select(M[:, :, :n_blocks].double().numpy(), np.arange(q0, q0 + qc), T, Bk, k)
+        assert np.array_equal(I, I_ref), (q0, qc)
