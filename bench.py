@@ -194,6 +194,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-others", action="store_true")
+    ap.add_argument("--topk-table", action="store_true",
+                    help="time Top-k alone on the four (rows, scores per row, k) shapes of the paper's Top-k "
+                         "latency table (Section 4.1, Table 1) and print one JSON line; not the headline metric")
     ap.add_argument("--index-lse", action="store_true",
                     help="prefill: also time the index-branch log-sum-exp (Section 4.3) on the step's selection; "
                          "reported beside the step, not part of it")
@@ -214,6 +217,10 @@ def main():
     from paper_2606_13392_b200 import binding as B
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
+    if args.topk_table:
+        if rank == 0:
+            topk_table(B, dev, load_peaks())
+        return
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     peaks = load_peaks()
@@ -233,6 +240,51 @@ def main():
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def topk_table(B, dev, peaks):
+    """Top-k alone on N independent rows of n_scores fp32 block scores, k selected (Table 1's shapes).
+
+    A row is a decode row whose local block is block n_scores: the n_scores blocks before it are
+    ranked and k of them selected (top_k = k + 1 with the forced local block).  The paper's figures
+    (another GPU) are printed beside ours as context.
+    """
+    shapes = [(131072, 1024, 16, 779.0), (131072, 2048, 32, 1991.0), (524288, 4096, 16, 7880.0),
+              (524288, 8192, 32, 21326.0)]
+    H_kv, Bk = 8, 128
+    out = []
+    for n_rows, n_scores, k, paper_us in shapes:
+        cfg = MSAConfig("topk-table", "decode", 0, 64, H_kv, Bk, k + 1)
+        shape = B.shape_of(cfg)
+        batch = n_rows // H_kv
+        ld = B.score_ld((n_scores + 1) * Bk, Bk)
+        g = torch.Generator(device=dev).manual_seed(n_scores)
+        scores = torch.empty((batch, H_kv, ld), dtype=torch.float32, device=dev)
+        for b0 in range(0, batch, 4096):  # drawn in pieces: the largest matrix is 17 GB
+            scores[b0:b0 + 4096].normal_(generator=g)
+        seq_lens = torch.full((batch,), n_scores * Bk + 1, dtype=torch.int32, device=dev)
+        idx = torch.empty((batch, H_kv, k + 1), dtype=torch.int32, device=dev)
+        stream = torch.cuda.current_stream()
+        for _ in range(3):
+            B.msa_topk_select_decode(shape, scores, ld, seq_lens, batch, idx)
+        torch.cuda.synchronize()
+        reps = 10
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            B.msa_topk_select_decode(shape, scores, ld, seq_lens, batch, idx)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        gbs = n_rows * n_scores * 4.0 / (us * 1e-6) / 1e9
+        assert bool((idx[:, :, k] == n_scores).all()) and bool((idx[:, :, :k] >= 0).all())
+        out.append({"rows": n_rows, "scores_per_row": n_scores, "k": k, "us": us, "GB/s": gbs,
+                    "frac_of_hbm": gbs / peaks["hbm_gbs"], "paper_us_other_gpu": paper_us})
+        del scores, idx
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "topk_latency_us", "unit": "us", "higher_is_better": False, "dtype": "f32",
+                      "data": "synthetic", "l2": "inputs larger than L2 (126 MB)", "shapes": out,
+                      "peak_source": "of " + peaks["_source"]}))
 
 
 def rank_seed(seed: int, rank: int) -> int:

@@ -344,7 +344,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
     int n_log;
     bool log_ok;
     const int64_t n_full = loc / kTopkRunBlocks;  // runs wholly before the local block
-    if (n_full < 4 * m || n_full > kTopkMaxRuns) {  // short row (or one beyond the list): one level
+    if (n_full < 2 * m || n_full > kTopkMaxRuns) {  // short row (or one beyond the list): one level
         const TopkPlainStream st{srow, (int)loc};
         topk_pass1<R>(st, m, -INFINITY, sc, kept, n_log, log_ok, lane);
         topk_pass2<R>(st, m, sc, kept, n_log, log_ok, outb, lane);
@@ -359,13 +359,21 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         float top[S];
 #pragma unroll
         for (int i = 0; i < S; ++i) top[i] = -INFINITY;
+        float* runmax = reinterpret_cast<float*>(log_all[warp]);  // the log is not in use before step 3
+        static_assert(kTopkLog * sizeof(uint2) >= kTopkMaxRuns * sizeof(float), "run maxima share the log");
+        float nx[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) nx[u] = rs.score(u * 32 + lane);  // -inf beyond n_full
         for (int g0 = 0; g0 < (int)n_full; g0 += 32 * 4) {
             float x[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) x[u] = rs.score(g0 + u * 32 + lane);  // -inf beyond n_full
+            for (int u = 0; u < 4; ++u) x[u] = nx[u];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) nx[u] = rs.score(g0 + 128 + u * 32 + lane);  // in flight during the inserts
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 float v = x[u];
+                if (g0 + u * 32 + lane < (int)n_full) runmax[g0 + u * 32 + lane] = v;
 #pragma unroll
                 for (int i = 0; i < S; ++i) {
                     const float hi = fmaxf(top[i], v);
@@ -383,13 +391,14 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
             for (int stride = size >> 1; stride > 0; stride >>= 1) bitonic_stage<S>(tk, lane, size, stride);
         }
         const float tau0 = topk_key_score(element_at<S>(tk, m - 1));  // 32 S >= 2 m values
-        // 2. candidate runs, ascending (the row was just read: these loads hit L1 or L2)
+        // 2. candidate runs, ascending (their maxima wait in shared memory)
         uint16_t* run = run_all[warp];
         const unsigned lt_mask = (1u << lane) - 1u;
         int n_run = 0;
+        __syncwarp();
         for (int g0 = 0; g0 < (int)n_full; g0 += 32) {
             const int g = g0 + lane;
-            const bool c = rs.score(g) >= tau0;  // -inf beyond n_full; tau0 is a real score
+            const bool c = g < (int)n_full && runmax[g] >= tau0;  // tau0 is a real score
             const unsigned cm = __ballot_sync(0xffffffffu, c);
             if (c) run[n_run + __popc(cm & lt_mask)] = (uint16_t)g;
             n_run += __popc(cm);

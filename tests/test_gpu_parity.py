@@ -521,7 +521,7 @@ def test_fp8_flag_and_operand_size_must_agree():
     (300000 + 5, 64, 8, 64, 64, False, False),    # the headline shape's head layout and k
 ])
 def test_two_level_topk_long_rows_bit_exact(T, Hq, Hkv, k, di, ties, sharp):
-    # Rows of 4 (k-1) runs of 8 blocks and more are selected in two levels (run maxima first, then
+    # Rows of 2 (k-1) runs of 8 blocks and more are selected in two levels (run maxima first, then
     # only the runs that can hold a selected block).  The lists must be the oracle's on the very
     # scores the GPU computed (fp32, exact in fp64), ties included, and the whole-path call must
     # give the same lists as the separate calls.
@@ -533,7 +533,7 @@ def test_two_level_topk_long_rows_bit_exact(T, Hq, Hkv, k, di, ties, sharp):
     _, _, I = api.prefill_forward(cfg, x)
     torch.cuda.synchronize()
     _assert_clean()
-    first_long = 4 * (k - 1) * 8 * 128  # rows from here on take the two-level path
+    first_long = 2 * (k - 1) * 8 * 128  # rows from here on take the two-level path
     assert T > first_long + 4096
     nb = cfg.n_blocks
     for q0, qc in [(first_long - 150, 300), ((first_long + T) // 2 + 11, 400), (T - 384, 384)]:
@@ -556,7 +556,7 @@ def test_two_level_topk_on_arbitrary_long_score_rows(n_blocks, k, levels):
     cfg = MSAConfig("top2-raw", "prefill", T, 4, 2, Bk, k, head_dim=64, idx_dim=32, seed=n_blocks)
     g = torch.Generator().manual_seed(n_blocks + k)
     ld = B.score_ld(T, Bk)
-    pos = np.unique(np.concatenate([np.arange(T - 40, T), np.linspace(4 * (k - 1) * 8 * Bk - 20, T - 1, 150).astype(np.int64)]))
+    pos = np.unique(np.concatenate([np.arange(T - 40, T), np.linspace(2 * (k - 1) * 8 * Bk - 20, T - 1, 150).astype(np.int64)]))
     runs = np.split(pos, np.where(np.diff(pos) != 1)[0] + 1)
     for run in runs:
         q0, qc = int(run[0]), len(run)
