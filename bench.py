@@ -480,6 +480,27 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
         torch.cuda.empty_cache()
         line["e2e"] = run_e2e(cfg, shape, x, B, dev, min(steps, 3), world)
 
+    # ---- the same decode step replayed from a CUDA graph (serving loops capture it once)
+    if cfg.mode == "decode":
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(stream)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                step()
+            for _ in range(3):
+                g.replay()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(side)
+            for _ in range(steps):
+                g.replay()
+            g1.record(side)
+        torch.cuda.synchronize()
+        g_ms = g0.elapsed_time(g1) / steps
+        line["cuda_graph"] = {"ms_per_step": g_ms, "value": world * units / (g_ms * 1e-3), "unit": line["unit"],
+                              "note": "this rank's step captured once and replayed; not max over ranks"}
+        del g
+
     # ---- training-side forward output, timed on its own (Section 4.3)
     if getattr(args, "index_lse", False) and cfg.mode == "prefill":
         mn_l, pf_l = B.msa_index_lse_prefill_workspace_bytes(shape, T, T)

@@ -81,6 +81,8 @@ CONFIGS: Dict[str, MSAConfig] = {
     # (inputs still larger than L2).
     "c3-16k": MSAConfig("c3-16k", "prefill", 16384, 64, 8, 128, 64, seed=2,
                         planted_frac=0.05, planted_shift=2.0),
+    # A light decode step (8 sequences of 32K): launch gaps weigh as much as the kernels.
+    "c5-light": MSAConfig("c5-light", "decode", 32768, 64, 8, 128, 64, seed=4, seq_lens=(32768,) * 8),
     "c5-small": MSAConfig("c5-small", "decode", 131072, 64, 8, 128, 64, seed=4,
                           seq_lens=(32768,) * 8 + (131072,) * 8),
 }

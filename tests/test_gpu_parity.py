@@ -566,3 +566,68 @@ def test_two_level_topk_on_arbitrary_long_score_rows(n_blocks, k, levels):
         I = api.topk_select(cfg, M.to(DEV), q0, T).cpu().numpy()
         I_ref = oracle.topk_select(M[:, :, :n_blocks].double().numpy(), np.arange(q0, q0 + qc), T, Bk, k)
         assert np.array_equal(I, I_ref), (q0, qc)
+
+
+# ----------------------------------------------------------------- CUDA graphs
+def test_decode_and_prefill_calls_replay_from_a_cuda_graph():
+    # A decode step is a handful of short kernels: serving loops capture it once and replay it.
+    # The calls must be capturable (no allocation, no synchronisation, no host read inside) and a
+    # replay on new inputs in the same buffers must give what a plain call gives.
+    cfg = CONFIGS["c5"].scaled(name="c5-graph", seq_lens=(129, 4096, 20000, 16384 + 64))
+    x = make_decode_inputs(cfg, DEV, sharp=True)
+    shape = B.shape_of(cfg)
+    batch, max_len = len(cfg.seq_lens), int(max(cfg.seq_lens))
+    ld = B.score_ld(max_len, cfg.block_size)
+    scores = torch.empty((batch, cfg.n_kv_heads, ld), dtype=torch.float32, device=DEV)
+    I = torch.empty((batch, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32, device=DEV)
+    out = torch.empty_like(x["q"])
+    lse = torch.empty((batch, cfg.n_q_heads), dtype=torch.float32, device=DEV)
+    ws = B.alloc_workspace(B.msa_sparse_attn_decode_workspace_bytes(shape, batch), DEV)
+
+    def step():
+        B.msa_decode_forward(shape, x["q"], x["q_idx"], x["k_cache"], x["v_cache"], x["k_idx_cache"],
+                             x["k_cache"].shape[0], x["seq_offsets"], x["seq_lens"], batch, max_len,
+                             scores, ld, I, out, lse, ws)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):  # warm-up outside the capture (attributes are set on first use)
+        step()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    # new queries in the captured buffers
+    x2 = make_decode_inputs(cfg.scaled(seed=cfg.seed + 1), DEV, sharp=True)
+    x["q"].copy_(x2["q"])
+    x["q_idx"].copy_(x2["q_idx"])
+    g.replay()
+    torch.cuda.synchronize()
+    _assert_clean()
+    got = (out.clone(), lse.clone(), I.clone())
+    out.zero_(); lse.zero_(); I.zero_()
+    step()
+    torch.cuda.synchronize()
+    assert torch.equal(got[2], I) and torch.equal(got[0], out) and torch.equal(got[1], lse)
+
+    # the prefill call, same way
+    pcfg = CONFIGS["c3"].scaled(name="c3-graph", T=3000)
+    px = make_prefill_inputs(pcfg, DEV, sharp=True)
+    pshape = B.shape_of(pcfg)
+    po = torch.empty_like(px["q"])
+    pl = torch.empty((pcfg.T, pcfg.n_q_heads), dtype=torch.float32, device=DEV)
+    pi = torch.empty((pcfg.T, pcfg.n_kv_heads, pcfg.top_k), dtype=torch.int32, device=DEV)
+    pws = B.alloc_workspace(B.msa_prefill_forward_workspace_bytes(pshape, pcfg.T)[1], DEV)
+
+    def pstep():
+        B.msa_prefill_forward(pshape, px["q"], px["k"], px["v"], px["q_idx"], px["k_idx"], pcfg.T, po, pl, pi, pws)
+    with torch.cuda.stream(side):
+        pstep()
+    torch.cuda.synchronize()
+    want = (po.clone(), pl.clone(), pi.clone())
+    pg = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(pg):
+        pstep()
+    po.zero_(); pl.zero_(); pi.zero_()
+    pg.replay()
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert torch.equal(want[2], pi) and torch.equal(want[0], po) and torch.equal(want[1], pl)
