@@ -47,14 +47,15 @@ def load_peaks():
 def prefill_work(cfg: MSAConfig):
     """Algorithmic FLOPs/bytes of one prefill pass (formulas: Section 3.3 and Section 4.2)."""
     T, Bk, k = cfg.T, cfg.block_size, cfg.top_k
-    i = np.arange(T, dtype=np.int64)
+    lens = cfg.seq_lens if cfg.seq_lens else (T,)  # packed sequences: positions restart in each
+    i = np.concatenate([np.arange(n, dtype=np.int64) for n in lens])
     loc = i // Bk
     n_sel = np.minimum(k, loc + 1)
     tokens = (n_sel - 1) * Bk + (i % Bk) + 1          # visible tokens of the selected blocks
     pairs = int(n_sel.sum()) * cfg.n_kv_heads          # (query, group, block) pairs
     gd2 = 2 * cfg.group * cfg.head_dim                 # bytes of one (query, group) bf16 row set
     return {
-        "index_flops": float(cfg.n_kv_heads) * cfg.idx_dim * T * (T + 1),
+        "index_flops": float(cfg.n_kv_heads) * cfg.idx_dim * float(sum(float(n) * (n + 1) for n in lens)),
         "attn_flops": 4.0 * cfg.n_q_heads * cfg.head_dim * float(tokens.sum()),
         "topk_bytes": 4.0 * cfg.n_kv_heads * float((loc + 1).sum()) + 4.0 * T * cfg.n_kv_heads * k,
         # KV-outer with bf16 partials: K+V once, per pair Q gather + partial write, final O
@@ -224,8 +225,9 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     peaks = load_peaks()
-    line = measure(cfg, args, rank, world, dev, B, peaks, dist, e2e=not args.no_e2e,
-                   cpu=(world == 1 and not args.no_cpu_baseline))
+    packed = cfg.mode == "prefill" and bool(cfg.seq_lens)  # no host-buffer call and no oracle leg for packed batches
+    line = measure(cfg, args, rank, world, dev, B, peaks, dist, e2e=not args.no_e2e and not packed,
+                   cpu=(world == 1 and not args.no_cpu_baseline and not packed))
     others = {}
     for name in extras:
         torch.cuda.empty_cache()
@@ -312,6 +314,11 @@ def base_line(cfg: MSAConfig, args, n_gpus: int):
 
 def describe(cfg: MSAConfig) -> str:
     f8 = ", index operands fp8 E4M3" if cfg.idx_fp8 else ""
+    if cfg.mode == "prefill" and cfg.seq_lens:
+        return ("prefill fwd, %d packed sequences of %s tokens (%d in all), causal, %d q heads / %d kv heads, d_h=%d, "
+                "d_idx=%d, B_k=%d, k=%d%s"
+                % (len(cfg.seq_lens), "/".join(str(n) for n in cfg.seq_lens), cfg.T, cfg.n_q_heads, cfg.n_kv_heads,
+                   cfg.head_dim, cfg.idx_dim, cfg.block_size, cfg.top_k, f8))
     if cfg.mode == "prefill":
         return ("prefill fwd, batch 1, T=%d causal, %d q heads / %d kv heads, d_h=%d, d_idx=%d, B_k=%d, k=%d%s"
                 % (cfg.T, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.idx_dim, cfg.block_size, cfg.top_k, f8))
@@ -368,9 +375,19 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
         ws = B.alloc_workspace(pf, dev)
         units = T
 
-        def step():
-            B.msa_prefill_forward(shape, x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"], T, out, lse,
-                                  block_idx, ws)
+        if cfg.seq_lens:  # packed sequences of these lengths (they sum to T)
+            assert sum(cfg.seq_lens) == T
+            cu = np.concatenate([[0], np.cumsum(cfg.seq_lens)]).tolist()
+            mn, pf = B.msa_prefill_forward_varlen_workspace_bytes(shape, cu)
+            ws = B.alloc_workspace(pf, dev)
+
+            def step():
+                B.msa_prefill_forward_varlen(shape, x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"], cu, out, lse,
+                                             block_idx, ws)
+        else:
+            def step():
+                B.msa_prefill_forward(shape, x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"], T, out, lse,
+                                      block_idx, ws)
     else:
         x = make_decode_inputs(mycfg, dev)
         batch = len(cfg.seq_lens)

@@ -81,6 +81,10 @@ CONFIGS: Dict[str, MSAConfig] = {
     # (inputs still larger than L2).
     "c3-16k": MSAConfig("c3-16k", "prefill", 16384, 64, 8, 128, 64, seed=2,
                         planted_frac=0.05, planted_shift=2.0),
+    # Variable-length batched prefill (Section 4.2 mentions variable-length sequences): sequences of
+    # mixed lengths packed token-major, 1M tokens in all, the paper's regime.  seq_lens = the lengths.
+    "pvar": MSAConfig("pvar", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=9,
+                      seq_lens=(524288, 262144, 131072, 65536, 32768, 16384, 8192, 4096, 2048, 1024, 512, 512)),
     # A light decode step (8 sequences of 32K): launch gaps weigh as much as the kernels.
     "c5-light": MSAConfig("c5-light", "decode", 32768, 64, 8, 128, 64, seed=4, seq_lens=(32768,) * 8),
     "c5-small": MSAConfig("c5-small", "decode", 131072, 64, 8, 128, 64, seed=4,
