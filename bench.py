@@ -174,7 +174,7 @@ def oracle_sample_size(cfg: MSAConfig) -> int:
 # which the traffic is proportional to).  None = not captured.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
     # c4: captured at full size with a one-pass metric set (profiles/launch_list_and_dram_c4.md)
-    ("c4", "index_scores"): 38.85e9, ("c4", "topk_select"): 17.62e9,
+    ("c4", "index_scores"): 38.85e9, ("c4", "topk_select"): 17.89e9,
     # (attention: 18.5 GB read + 33.7 GB written; half of the Q gathers hit L2)
     ("c4", "attn_prefill"): 52.2e9, ("c4", "combine"): 34.30e9,
     # c3: captured at full size with the same one-pass metric set (profiles/launch_list_and_dram_c4.md)
