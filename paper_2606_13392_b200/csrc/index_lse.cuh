@@ -42,11 +42,12 @@ index_lse_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_bfloat16* _
                  const int32_t* __restrict__ item_off, const uint32_t* __restrict__ handles,
                  float scale_log2e, float* __restrict__ part) {
     constexpr int LD = DIDX + 8;  // padded row (bf16): conflict-free ldmatrix
+    constexpr int CH = DIDX / 8;  // 16-byte chunks per row
+    constexpr int NCH = kLseItemQueries * CH / kLseThreads;  // chunks of a query tile gathered by one thread
     extern __shared__ __align__(16) uint8_t lse_smem[];
-    __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(lse_smem);       // [BK][LD]
-    __nv_bfloat16* Qs = Ks + BK * LD;                                     // [128][LD]
-    uint32_t* hs = reinterpret_cast<uint32_t*>(Qs + kLseItemQueries * LD);  // [128] handles
-    __shared__ int s_tile, s_first, s_nq;
+    __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(lse_smem);        // [BK][LD]
+    __nv_bfloat16* Qs0 = Ks + BK * LD;                                     // [2][128][LD]: this item's and the next one's queries
+    uint32_t* hs0 = reinterpret_cast<uint32_t*>(Qs0 + 2 * kLseItemQueries * LD);  // [2][128] handles
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = p.n_blocks * p.H_kv;
     const int total_items = item_off[n_tiles];
@@ -54,10 +55,11 @@ index_lse_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_bfloat16* _
     // a contiguous share of the item list per CTA: consecutive items mostly share their key block
     const int per_cta = (total_items + (int)gridDim.x - 1) / (int)gridDim.x;
     const int it_lo = min(total_items, (int)blockIdx.x * per_cta), it_hi = min(total_items, it_lo + per_cta);
-    int loaded_tile = -1;
-    // thread 0 walks the tile list: a search for the first item, then steps
-    int w_tile = 0, w_next = 0;
-    if (threadIdx.x == 0 && it_lo < it_hi) {  // last tile whose first item is <= it_lo (skips empty tiles)
+    if (it_lo >= it_hi) return;
+    // Every thread walks the tile list for the item being fetched (uniform loads): a search for the
+    // first item, then steps.
+    int w_tile, w_next;
+    {   // last tile whose first item is <= it_lo (skips empty tiles)
         int lo = 0, hi = n_tiles;
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -66,23 +68,48 @@ index_lse_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_bfloat16* _
         w_tile = lo;
         w_next = item_off[lo + 1];
     }
-    for (int it = it_lo; it < it_hi; ++it) {
-        if (threadIdx.x == 0) {
-            while (w_next <= it) {  // crossed into the next non-empty tile
-                ++w_tile;
-                w_next = item_off[w_tile + 1];
-            }
-            s_tile = w_tile;
-            const int first = tile_off[w_tile] + (it - item_off[w_tile]) * kLseItemQueries;
-            s_first = first;
-            s_nq = min(kLseItemQueries, tile_off[w_tile + 1] - first);
+    // The gather of item `it` into buffer `buf`: per row its handle, then DIDX*2 bytes of its index
+    // vector as asynchronous 16-byte copies; the next item's gather is in flight while this item's
+    // scores are computed.
+    auto fetch = [&](int it, int buf, int& tile, int& nq) {
+        while (w_next <= it) {  // crossed into the next non-empty tile
+            ++w_tile;
+            w_next = item_off[w_tile + 1];
         }
-        __syncthreads();
-        const int tile = s_tile, first = s_first, nq = s_nq;
+        tile = w_tile;
+        const int first = tile_off[w_tile] + (it - item_off[w_tile]) * kLseItemQueries;
+        nq = min(kLseItemQueries, tile_off[w_tile + 1] - first);
+        const int r = tile / p.n_blocks;
+        __nv_bfloat16* Qs = Qs0 + buf * (kLseItemQueries * LD);
+        uint32_t* hs = hs0 + buf * kLseItemQueries;
+        uint32_t hh[NCH];
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            const int row = ((int)threadIdx.x + j * kLseThreads) / CH;
+            hh[j] = row < nq ? __ldg(handles + first + row) : 0u;
+        }
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            const int e = (int)threadIdx.x + j * kLseThreads, row = e / CH, ch = e % CH;
+            if (ch == 0) hs[row] = hh[j];
+            if (row < nq) {  // rows past nq keep stale (finite or not, never written back) data
+                const int64_t ql = hh[j] >> 8;
+                const __nv_bfloat16* src = q_idx + ((p.q_first + ql) * p.H_kv + r) * DIDX + ch * 8;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(Qs + row * LD + ch * 8)), "l"(src)
+                             : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    int loaded_tile = -1;
+    int tile, nq;
+    fetch(it_lo, 0, tile, nq);
+    for (int it = it_lo; it < it_hi; ++it) {
+        const int buf = (it - it_lo) & 1;
+        int tile_n = 0, nq_n = 0;
+        if (it + 1 < it_hi) fetch(it + 1, buf ^ 1, tile_n, nq_n);
         const int r = tile / p.n_blocks, b = tile - r * p.n_blocks;  // tiles are numbered head after head
-        if (threadIdx.x < kLseItemQueries) hs[threadIdx.x] = threadIdx.x < nq ? handles[first + threadIdx.x] : 0u;
         // K_idx block: BK rows of DIDX bf16, 16-byte chunks; rows past the sequence are zero (masked below)
-        constexpr int CH = DIDX / 8;
         for (int e = threadIdx.x; tile != loaded_tile && e < BK * CH; e += kLseThreads) {
             const int row = e / CH, ch = e % CH;
             const int64_t j = (int64_t)b * BK + row;
@@ -90,17 +117,11 @@ index_lse_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_bfloat16* _
             if (j < kv_len) v = __ldg(reinterpret_cast<const uint4*>(k_idx + j * DIDX) + ch);
             *reinterpret_cast<uint4*>(Ks + row * LD + ch * 8) = v;
         }
-        __syncthreads();  // handles visible
-        for (int e = threadIdx.x; e < kLseItemQueries * CH; e += kLseThreads) {
-            const int row = e / CH, ch = e % CH;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (row < nq) {
-                const int64_t ql = hs[row] >> 8;
-                v = __ldg(reinterpret_cast<const uint4*>(q_idx + ((p.q_first + ql) * p.H_kv + r) * DIDX) + ch);
-            }
-            *reinterpret_cast<uint4*>(Qs + row * LD + ch * 8) = v;
-        }
-        __syncthreads();
+        if (it + 1 < it_hi) asm volatile("cp.async.wait_group 1;" ::: "memory");
+        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();  // this item's queries and handles, and the key block, are in shared memory
+        const __nv_bfloat16* Qs = Qs0 + buf * (kLseItemQueries * LD);
+        const uint32_t* hs = hs0 + buf * kLseItemQueries;
 
         // scores of 16 queries (this warp) x BK keys
         float acc[BK / 8][4];
@@ -147,7 +168,9 @@ index_lse_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_bfloat16* _
                 part[((int64_t)(h >> 8) * p.H_kv + r) * p.top_k + (h & 0xFF)] = (mx + log2f(sum)) * 0.6931471805599453f;
         }
         loaded_tile = tile;
-        __syncthreads();  // shared tiles are reused by the next item
+        __syncthreads();  // this buffer and the key block are free for the gathers and loads of later items
+        tile = tile_n;
+        nq = nq_n;
     }
 }
 

@@ -607,7 +607,7 @@ static msa_status_t run_index_lse(const Resolved& r, const void* q_idx, const vo
     float* part = (float*)(w + pl.off_part);
     int* status = async_status_ptr();
     if (status == nullptr) return MSA_ERR_CUDA;
-    const size_t smem = (size_t)(BK + kLseItemQueries) * (DIDX + 8) * 2 + kLseItemQueries * 4;
+    const size_t smem = (size_t)(BK + 2 * kLseItemQueries) * (DIDX + 8) * 2 + 2 * kLseItemQueries * 4;
     static bool attr_set_dev[64] = {false};  // the attribute is per device
     const int dev_id = current_device();
     if (!attr_set_dev[dev_id]) {
@@ -617,7 +617,9 @@ static msa_status_t run_index_lse(const Resolved& r, const void* q_idx, const vo
         attr_set_dev[dev_id] = true;
     }
     const float scale_log2e = r.index_scale * 1.4426950408889634f;
-    const int grid = sm_count() * (smem > 48 * 1024 ? 3 : 4);
+    int per_sm = (int)((227 * 1024) / (smem + 1024));  // resident CTAs by shared memory, at most 4
+    if (per_sm > 4) per_sm = 4;
+    const int grid = sm_count() * per_sm;
     for (int64_t q_first = 0; q_first < q_count; q_first += R) {
         RangeParams p;
         p.q_begin = q_begin; p.q_first = q_first;
