@@ -539,8 +539,15 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
         w = prefill_work(cfg)
         # one dot product of d_idx per (query, index head, visible token of a selected block)
         flops = w["attn_flops"] / (4.0 * cfg.n_q_heads * cfg.head_dim) * 2.0 * cfg.n_kv_heads * cfg.idx_dim
-        line["index_lse"] = {"ms": ms, "bound": "tensor", "achieved": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
-                             "peak": peaks["bf16_tflops"], "frac": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+        # Bound by the exponential unit, one exp2 per score: 16 per clock and SM (4 sub-partitions x 4 lanes)
+        # x 148 SMs x 1.965 GHz = 4.65e12 per second; the 2*d_idx FLOPs per score need 5-10 % of the tensor peak.
+        n_exp = flops / (2.0 * cfg.idx_dim)
+        xu_peak = 16 * 148 * 1.965e9
+        line["index_lse"] = {"ms": ms, "bound": "alu", "achieved": n_exp / (ms * 1e-3) / 1e9, "unit": "Gexp/s",
+                             "peak": xu_peak / 1e9, "frac": n_exp / (ms * 1e-3) / xu_peak,
+                             "peak_source": "derived: 16 exp2 per clock and SM x 148 SMs x 1.965 GHz",
+                             "tensor_tflops": flops / (ms * 1e-3) / 1e12,
+                             "includes": "reverse index, the per-item kernel and the slot reduction"}
         del ws_l, lse_idx
 
     # ---- the oracle on this machine's host cores (bounded sample)

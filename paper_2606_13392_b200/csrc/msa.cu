@@ -607,7 +607,7 @@ static msa_status_t run_index_lse(const Resolved& r, const void* q_idx, const vo
     float* part = (float*)(w + pl.off_part);
     int* status = async_status_ptr();
     if (status == nullptr) return MSA_ERR_CUDA;
-    const size_t smem = (size_t)(BK + 2 * kLseItemQueries) * (DIDX + 8) * 2 + 2 * kLseItemQueries * 4;
+    const size_t smem = (size_t)(BK + 2 * kLseItemQueries) * DIDX * 2 + 2 * kLseItemQueries * 4 + 1024;
     static bool attr_set_dev[64] = {false};  // the attribute is per device
     const int dev_id = current_device();
     if (!attr_set_dev[dev_id]) {
@@ -645,7 +645,7 @@ static msa_status_t run_index_lse(const Resolved& r, const void* q_idx, const vo
             StageScope sc(kStageIndexLse, st);
             index_lse_kernel<BK, DIDX><<<grid, kLseThreads, smem, st>>>(
                 (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx, p, kv_len, tile_off, item_off, handles,
-                scale_log2e, part);
+                scale_log2e, part, status);
         }
         {
             StageScope sc(kStageIndexLse, st);
