@@ -52,3 +52,20 @@ def test_c5_decode_full_batch():
     assert np.mean([r["exact"] for r in res]) >= 0.99
     print("c5", res[0], res[-1])
     _free()
+
+
+# The paper's own regime at full length (bench workloads p1m, p1m-f8, pdec-f8): fused index + Top-k,
+# G = 16 attention, fp8 index operands.
+@pytest.mark.parametrize("name", ["p1m", "p1m-f8"])
+def test_paper_regime_1m_sampled(name):
+    stats = run_prefill_case(CONFIGS[name], True, n_sample=96)
+    assert stats["exact_sets"] >= 0.995
+    print(name, stats)
+    _free()
+
+
+def test_paper_regime_decode_fp8_full_batch():
+    res = run_decode_case(CONFIGS["pdec-f8"], True)
+    assert len(res) == 32
+    assert np.mean([r["exact"] for r in res]) >= 0.99
+    _free()
