@@ -371,6 +371,17 @@ struct HostOutHook {
 };
 static HostOutHook g_out_hook;
 
+// Copy-in hook of the same call: Q is uploaded in pieces on the copy stream, an event after each;
+// a query range's attention waits only for the piece that holds its last row (its reverse index
+// and the ranges before it run while later pieces are still on their way).
+struct HostInHook {
+    bool on = false;
+    int64_t piece_rows = 0;
+    int n_pieces = 0;
+    cudaEvent_t ev[256];
+};
+static HostInHook g_in_hook;
+
 static cudaEvent_t next_sync_event() {
     constexpr int kPool = 2048;
     static cudaEvent_t pool[kPool];
@@ -463,6 +474,11 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
         {
             StageScope sc(kStageSchedule, st);
             revidx_kernel<BK><<<eg, 256, 0, st>>>(block_idx, p, 1, cnt, tile_off, rank, handles, status);
+        }
+        if (g_in_hook.on && q_begin == 0) {  // the range's Q rows must have arrived
+            int piece = (int)((q_first + p.q_count - 1) / g_in_hook.piece_rows);
+            if (piece >= g_in_hook.n_pieces) piece = g_in_hook.n_pieces - 1;
+            if (cudaStreamWaitEvent(st, g_in_hook.ev[piece], 0) != cudaSuccess) return MSA_ERR_CUDA;
         }
         {
             StageScope sc(kStageAttn, st);
@@ -1185,32 +1201,54 @@ msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_ho
     // while the next one is computed.
     static cudaStream_t copy = nullptr;
     if (copy == nullptr && cudaStreamCreateWithFlags(&copy, cudaStreamNonBlocking) != cudaSuccess) return MSA_ERR_CUDA;
-    cudaEvent_t e_in = next_sync_event(), e_idx = next_sync_event(), e_all = next_sync_event();
-    if (!e_in || !e_idx || !e_all) return MSA_ERR_CUDA;
+    cudaEvent_t e_in = next_sync_event(), e_idx = next_sync_event(), e_kv = next_sync_event();
+    if (!e_in || !e_idx || !e_kv) return MSA_ERR_CUDA;
     if (cudaEventRecord(e_in, st) != cudaSuccess || cudaStreamWaitEvent(copy, e_in, 0) != cudaSuccess) return MSA_ERR_CUDA;
     const void* src[5] = {q_host, k_host, v_host, q_idx_host, k_idx_host};
     const size_t nbytes[5] = {(size_t)T * r.H_q * r.d * 2, (size_t)T * r.H_kv * r.d * 2,
                               (size_t)T * r.H_kv * r.d * 2, (size_t)T * r.H_kv * r.d_idx * r.idx_elt(),
                               (size_t)T * r.d_idx * r.idx_elt()};
-    const int order[5] = {4, 3, 1, 2, 0};  // k_idx, q_idx, k, v, q
-    for (int j = 0; j < 5; ++j) {
+    const int order[4] = {4, 3, 1, 2};  // k_idx, q_idx, k, v; then Q in pieces
+    for (int j = 0; j < 4; ++j) {
         const int i = order[j];
         if (cudaMemcpyAsync(w + off[i], src[i], nbytes[i], cudaMemcpyHostToDevice, copy) != cudaSuccess)
             return MSA_ERR_CUDA;
         if (j == 1 && cudaEventRecord(e_idx, copy) != cudaSuccess) return MSA_ERR_CUDA;
     }
-    if (cudaEventRecord(e_all, copy) != cudaSuccess) return MSA_ERR_CUDA;
+    if (cudaEventRecord(e_kv, copy) != cudaSuccess) return MSA_ERR_CUDA;
+    {
+        HostInHook& ih = g_in_hook;
+        int64_t piece = 16384;  // rows per piece: a few milliseconds of transfer, at most 256 pieces
+        while (ceil_div64(T, piece) > 256) piece *= 2;
+        ih.piece_rows = piece;
+        ih.n_pieces = (int)ceil_div64(T, piece);
+        const size_t rb = (size_t)r.H_q * r.d * 2;
+        for (int i = 0; i < ih.n_pieces; ++i) {
+            const int64_t r0 = (int64_t)i * piece, rows = (T - r0) < piece ? (T - r0) : piece;
+            ih.ev[i] = next_sync_event();
+            if (!ih.ev[i] ||
+                cudaMemcpyAsync(w + off[0] + (size_t)r0 * rb, (const char*)q_host + (size_t)r0 * rb, (size_t)rows * rb,
+                                cudaMemcpyHostToDevice, copy) != cudaSuccess ||
+                cudaEventRecord(ih.ev[i], copy) != cudaSuccess)
+                return MSA_ERR_CUDA;
+        }
+    }
     float* lse_dev = lse_host ? (float*)(w + off[6]) : nullptr;
     int32_t* bi_dev = (int32_t*)(w + off[7]);
     if (cudaStreamWaitEvent(st, e_idx, 0) != cudaSuccess) return MSA_ERR_CUDA;
     s = prefill_stages_1_2(shape, r, w + off[3], w + off[4], T, bi_dev, w + stage, workspace_bytes - stage, stream);
     if (s != MSA_OK) return s;
-    if (cudaStreamWaitEvent(st, e_all, 0) != cudaSuccess) return MSA_ERR_CUDA;
+    if (cudaStreamWaitEvent(st, e_kv, 0) != cudaSuccess) return MSA_ERR_CUDA;
+    // The tensor-core path waits for Q range by range; any other path waits for all of it here.
+    g_in_hook.on = attn_tc_supported(r) && T < 2147483647LL;
+    if (!g_in_hook.on && cudaStreamWaitEvent(st, g_in_hook.ev[g_in_hook.n_pieces - 1], 0) != cudaSuccess)
+        return MSA_ERR_CUDA;
     g_out_hook.on = true; g_out_hook.copy = copy; g_out_hook.out_host = (char*)out_host;
     g_out_hook.lse_host = lse_host; g_out_hook.rows_copied = 0;
     s = msa_sparse_attn_prefill(shape, w + off[0], w + off[1], w + off[2], bi_dev, 0, T, T, w + off[5], lse_dev,
                                 w + stage, workspace_bytes - stage, stream);
     g_out_hook.on = false;
+    g_in_hook.on = false;
     if (s != MSA_OK) return s;
     if (g_out_hook.rows_copied < T) {  // rows the per-range hook did not cover (generic kernel path)
         const msa_status_t hs = hook_copy_rows(r, w + off[5], lse_dev, g_out_hook.rows_copied,
