@@ -380,7 +380,33 @@ struct HostInHook {
     int n_pieces = 0;
     cudaEvent_t ev[256];
 };
-static HostInHook g_in_hook;
+static cudaEvent_t next_sync_event();
+static HostInHook g_in_hook;      // Q rows, waited for by the attention of each query range
+static HostInHook g_in_idx_hook;  // Q_idx rows, waited for by the scoring of each query chunk
+
+static msa_status_t wait_rows(const HostInHook& h, int64_t last_row, cudaStream_t st) {
+    if (!h.on) return MSA_OK;
+    int piece = (int)(last_row / h.piece_rows);
+    if (piece >= h.n_pieces) piece = h.n_pieces - 1;
+    return cudaStreamWaitEvent(st, h.ev[piece], 0) == cudaSuccess ? MSA_OK : MSA_ERR_CUDA;
+}
+// Uploads `rows` rows of `row_bytes` each in pieces on the copy stream, an event after each piece.
+static msa_status_t upload_in_pieces(HostInHook& h, char* dst, const void* src, int64_t rows, size_t row_bytes,
+                                     int64_t piece, cudaStream_t copy) {
+    while (ceil_div64(rows, piece) > 256) piece *= 2;
+    h.piece_rows = piece;
+    h.n_pieces = (int)ceil_div64(rows, piece);
+    for (int i = 0; i < h.n_pieces; ++i) {
+        const int64_t r0 = (int64_t)i * piece, n = (rows - r0) < piece ? (rows - r0) : piece;
+        h.ev[i] = next_sync_event();
+        if (!h.ev[i] ||
+            cudaMemcpyAsync(dst + (size_t)r0 * row_bytes, (const char*)src + (size_t)r0 * row_bytes, (size_t)n * row_bytes,
+                            cudaMemcpyHostToDevice, copy) != cudaSuccess ||
+            cudaEventRecord(h.ev[i], copy) != cudaSuccess)
+            return MSA_ERR_CUDA;
+    }
+    return MSA_OK;
+}
 
 static cudaEvent_t next_sync_event() {
     constexpr int kPool = 2048;
@@ -475,11 +501,8 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
             StageScope sc(kStageSchedule, st);
             revidx_kernel<BK><<<eg, 256, 0, st>>>(block_idx, p, 1, cnt, tile_off, rank, handles, status);
         }
-        if (g_in_hook.on && q_begin == 0) {  // the range's Q rows must have arrived
-            int piece = (int)((q_first + p.q_count - 1) / g_in_hook.piece_rows);
-            if (piece >= g_in_hook.n_pieces) piece = g_in_hook.n_pieces - 1;
-            if (cudaStreamWaitEvent(st, g_in_hook.ev[piece], 0) != cudaSuccess) return MSA_ERR_CUDA;
-        }
+        if (q_begin == 0 && wait_rows(g_in_hook, q_first + p.q_count - 1, st) != MSA_OK)  // the range's Q rows
+            return MSA_ERR_CUDA;
         {
             StageScope sc(kStageAttn, st);
             attn_prefill_tc_kernel<BK, G><<<grid_attn, kAttnThreads, smem, st>>>(
@@ -1075,8 +1098,10 @@ static msa_status_t prefill_stages_1_2(const msa_shape_t* shape, const Resolved&
                                        const void* k_idx, int64_t T, int32_t* block_idx, void* workspace,
                                        size_t workspace_bytes, msa_stream_t stream) {
     msa_status_t s = MSA_OK;
-    if (index_topk_fused_ok(r, T, T))  // no score matrix, no chunks
+    if (index_topk_fused_ok(r, T, T)) {  // no score matrix, no chunks
+        if (wait_rows(g_in_idx_hook, T - 1, (cudaStream_t)stream) != MSA_OK) return MSA_ERR_CUDA;
         return run_index_topk_fused(r, q_idx, k_idx, 0, T, T, block_idx, (cudaStream_t)stream);
+    }
     const int64_t ld = score_ld(T, r.B_k);
     const int64_t chunk = pick_score_chunk(r, T, workspace_bytes);
     if (chunk <= 0) return MSA_ERR_WORKSPACE;
@@ -1086,6 +1111,7 @@ static msa_status_t prefill_stages_1_2(const msa_shape_t* shape, const Resolved&
         const char* qi = static_cast<const char*>(q_idx) + (size_t)q0 * r.H_kv * r.d_idx * r.idx_elt();
         // Only keys up to the chunk's last query are visible, so score that prefix.
         const int64_t kv_vis = q0 + qc;
+        if (wait_rows(g_in_idx_hook, q0 + qc - 1, (cudaStream_t)stream) != MSA_OK) return MSA_ERR_CUDA;
         s = msa_index_scores(shape, qi, k_idx, q0, qc, kv_vis, scores, ld, stream);
         if (s != MSA_OK) return s;
         s = msa_topk_select(shape, scores, ld, q0, qc, kv_vis, block_idx + (size_t)q0 * r.H_kv * r.k, stream);
@@ -1208,35 +1234,22 @@ msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_ho
     const size_t nbytes[5] = {(size_t)T * r.H_q * r.d * 2, (size_t)T * r.H_kv * r.d * 2,
                               (size_t)T * r.H_kv * r.d * 2, (size_t)T * r.H_kv * r.d_idx * r.idx_elt(),
                               (size_t)T * r.d_idx * r.idx_elt()};
-    const int order[4] = {4, 3, 1, 2};  // k_idx, q_idx, k, v; then Q in pieces
-    for (int j = 0; j < 4; ++j) {
-        const int i = order[j];
-        if (cudaMemcpyAsync(w + off[i], src[i], nbytes[i], cudaMemcpyHostToDevice, copy) != cudaSuccess)
-            return MSA_ERR_CUDA;
-        if (j == 1 && cudaEventRecord(e_idx, copy) != cudaSuccess) return MSA_ERR_CUDA;
-    }
+    // Order on the copy stream: K_idx, Q_idx, K, V, Q; Q_idx and Q go in pieces with an event after each,
+    // so that every scoring chunk and every attention range waits only for its own rows.
+    if (cudaMemcpyAsync(w + off[4], src[4], nbytes[4], cudaMemcpyHostToDevice, copy) != cudaSuccess) return MSA_ERR_CUDA;
+    if (cudaEventRecord(e_idx, copy) != cudaSuccess) return MSA_ERR_CUDA;
+    const size_t qi_rb = (size_t)r.H_kv * r.d_idx * r.idx_elt(), q_rb = (size_t)r.H_q * r.d * 2;
+    if (upload_in_pieces(g_in_idx_hook, w + off[3], src[3], T, qi_rb, 65536, copy) != MSA_OK) return MSA_ERR_CUDA;
+    for (int i = 1; i <= 2; ++i)
+        if (cudaMemcpyAsync(w + off[i], src[i], nbytes[i], cudaMemcpyHostToDevice, copy) != cudaSuccess) return MSA_ERR_CUDA;
     if (cudaEventRecord(e_kv, copy) != cudaSuccess) return MSA_ERR_CUDA;
-    {
-        HostInHook& ih = g_in_hook;
-        int64_t piece = 16384;  // rows per piece: a few milliseconds of transfer, at most 256 pieces
-        while (ceil_div64(T, piece) > 256) piece *= 2;
-        ih.piece_rows = piece;
-        ih.n_pieces = (int)ceil_div64(T, piece);
-        const size_t rb = (size_t)r.H_q * r.d * 2;
-        for (int i = 0; i < ih.n_pieces; ++i) {
-            const int64_t r0 = (int64_t)i * piece, rows = (T - r0) < piece ? (T - r0) : piece;
-            ih.ev[i] = next_sync_event();
-            if (!ih.ev[i] ||
-                cudaMemcpyAsync(w + off[0] + (size_t)r0 * rb, (const char*)q_host + (size_t)r0 * rb, (size_t)rows * rb,
-                                cudaMemcpyHostToDevice, copy) != cudaSuccess ||
-                cudaEventRecord(ih.ev[i], copy) != cudaSuccess)
-                return MSA_ERR_CUDA;
-        }
-    }
+    if (upload_in_pieces(g_in_hook, w + off[0], src[0], T, q_rb, 16384, copy) != MSA_OK) return MSA_ERR_CUDA;
     float* lse_dev = lse_host ? (float*)(w + off[6]) : nullptr;
     int32_t* bi_dev = (int32_t*)(w + off[7]);
     if (cudaStreamWaitEvent(st, e_idx, 0) != cudaSuccess) return MSA_ERR_CUDA;
+    g_in_idx_hook.on = true;
     s = prefill_stages_1_2(shape, r, w + off[3], w + off[4], T, bi_dev, w + stage, workspace_bytes - stage, stream);
+    g_in_idx_hook.on = false;
     if (s != MSA_OK) return s;
     if (cudaStreamWaitEvent(st, e_kv, 0) != cudaSuccess) return MSA_ERR_CUDA;
     // The tensor-core path waits for Q range by range; any other path waits for all of it here.
