@@ -234,7 +234,7 @@ def main():
         res = measure(CONFIGS[name], args, rank, world, dev, B, peaks, dist, e2e=not args.no_e2e, cpu=False)
         if rank == 0:
             others[name] = {k: res[k] for k in ("metric", "value", "unit", "ms_per_step", "gpu_launches",
-                                                 "roofline", "kernels", "e2e", "config") if k in res}
+                                                 "roofline", "kernels", "e2e", "cuda_graph", "config") if k in res}
     if rank == 0:
         if others:
             line["others"] = others
@@ -491,12 +491,6 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
     if cfg.mode == "prefill":
         line["tflops_total"] = (w["index_flops"] + w["attn_flops"]) / (ms_step * 1e-3) / 1e12
 
-    # ---- end to end from host buffers (copies inside the timed region)
-    if e2e:
-        del out, lse, ws
-        torch.cuda.empty_cache()
-        line["e2e"] = run_e2e(cfg, shape, x, B, dev, min(steps, 3), world)
-
     # ---- the same decode step replayed from a CUDA graph (serving loops capture it once)
     if cfg.mode == "decode":
         side = torch.cuda.Stream(device=dev)
@@ -549,6 +543,12 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
                              "tensor_tflops": flops / (ms * 1e-3) / 1e12,
                              "includes": "reverse index, the per-item kernel and the slot reduction"}
         del ws_l, lse_idx
+
+    # ---- end to end from host buffers (copies inside the timed region)
+    if e2e:
+        del out, lse, ws
+        torch.cuda.empty_cache()
+        line["e2e"] = run_e2e(cfg, shape, x, B, dev, min(steps, 3), world)
 
     # ---- the oracle on this machine's host cores (bounded sample)
     if cpu:
