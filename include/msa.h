@@ -278,8 +278,9 @@ msa_status_t msa_prefill_forward_varlen_workspace_bytes(const msa_shape_t* shape
  * block_idx when non-NULL) back, and synchronises before returning.  The copies run on a
  * second stream owned by the library (created on first use) and overlap the kernels: the
  * index inputs are uploaded first so that stages 1-2 start while Q, K and V are still in
- * flight, and each finished query range of the output is copied back while the next one is
- * computed.  Host buffers should be page-locked for the copies to run at full rate and to
+ * flight; q_idx and q go up in pieces of rows, and a scoring chunk or the attention of a query
+ * range waits only for the piece that holds its last row; each finished query range of the
+ * output is copied back while the next one is computed.  Host buffers should be page-locked for the copies to run at full rate and to
  * overlap at all.
  * workspace >= msa_prefill_forward_host_workspace_bytes.
  */
