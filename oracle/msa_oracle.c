@@ -53,6 +53,11 @@ static inline double e4m3_to_double(uint8_t b) {
 }
 
 /* element c of an index-branch row stored as bf16 (idx_fp8 = 0) or E4M3 (idx_fp8 = 1) */
+/* Element e of a K or V tensor stored as fp8 E4M3 (Section 4.2: the kernels also support fp8) or bf16. */
+static inline double kv_elem(const void* base, int64_t e, int kv_fp8) {
+    return kv_fp8 ? e4m3_to_double(((const uint8_t*)base)[e]) : bf16_to_double(((const uint16_t*)base)[e]);
+}
+
 static inline double idx_elem(const void* row, int c, int idx_fp8) {
     return idx_fp8 ? e4m3_to_double(((const uint8_t*)row)[c]) : bf16_to_double(((const uint16_t*)row)[c]);
 }
@@ -197,10 +202,10 @@ void msa_oracle_topk_select(const double* M, const int64_t* pos, int64_t n, int6
  * q: [n,H_q,d]; K,V: [L,H_kv,d]; I: [n,H_kv,k] (entries < 0 are padding);
  * O: [n,H_q,d]; LSE: [n,H_q].
  */
-void msa_oracle_sparse_attn(const uint16_t* q, const uint16_t* K, const uint16_t* V,
+void msa_oracle_sparse_attn(const uint16_t* q, const void* K, const void* V,
                             const int32_t* I, const int64_t* pos, int64_t n, int64_t L,
                             int H_q, int H_kv, int d, int B_k, int k, double scale,
-                            double* O, double* LSE) {
+                            double* O, double* LSE, int kv_fp8) {
     const int G = H_q / H_kv;
 #pragma omp parallel for schedule(dynamic, 1)
     for (int64_t a = 0; a < n * H_q; ++a) {
@@ -217,10 +222,10 @@ void msa_oracle_sparse_attn(const uint16_t* q, const uint16_t* K, const uint16_t
             if (sel[s] < 0) continue;
             const int64_t j0 = (int64_t)sel[s] * B_k;
             for (int64_t j = j0; j < j0 + B_k && j < L && j <= i; ++j) {
-                const uint16_t* krow = K + (j * H_kv + r) * (int64_t)d;
+                const int64_t krow = (j * H_kv + r) * (int64_t)d;  /* element offset; K, V hold bf16 or fp8 E4M3 */
                 double acc = 0.0;
                 for (int c = 0; c < d; ++c)
-                    acc += bf16_to_double(qrow[c]) * bf16_to_double(krow[c]);
+                    acc += bf16_to_double(qrow[c]) * kv_elem(K, krow + c, kv_fp8);
                 z[nt] = acc * scale;
                 tok[nt] = j;
                 ++nt;
@@ -235,8 +240,8 @@ void msa_oracle_sparse_attn(const uint16_t* q, const uint16_t* K, const uint16_t
         for (int c = 0; c < d; ++c) orow[c] = 0.0;
         for (int64_t t = 0; t < nt; ++t) {
             const double w = exp(z[t] - mx) / ell;
-            const uint16_t* vrow = V + (tok[t] * H_kv + r) * (int64_t)d;
-            for (int c = 0; c < d; ++c) orow[c] += w * bf16_to_double(vrow[c]);
+            const int64_t vrow = (tok[t] * H_kv + r) * (int64_t)d;
+            for (int c = 0; c < d; ++c) orow[c] += w * kv_elem(V, vrow + c, kv_fp8);
         }
         LSE[a] = mx + log(ell);
         free(z);

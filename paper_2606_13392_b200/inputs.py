@@ -45,6 +45,7 @@ class MSAConfig:
     planted_shift: float = 0.0
     seq_lens: Tuple[int, ...] = ()
     idx_fp8: bool = False  # index-branch operands (Q_idx, K_idx) rounded to fp8 E4M3 instead of bf16
+    kv_fp8: bool = False   # decode: the K and V caches are stored in fp8 E4M3 (Q stays bf16)
 
     @property
     def group(self) -> int:
@@ -185,6 +186,8 @@ def make_decode_inputs(cfg: MSAConfig, device="cpu", sharp: bool = False):
     k_idx_cache = _draw(gen, total, (di,), s_idx, device)
     if cfg.idx_fp8:
         q_idx, k_idx_cache = q_idx.to(torch.float8_e4m3fn), k_idx_cache.to(torch.float8_e4m3fn)
+    if cfg.kv_fp8:  # the same draws, stored in the narrower format
+        k_cache, v_cache = k_cache.to(torch.float8_e4m3fn), v_cache.to(torch.float8_e4m3fn)
     offs = np.concatenate([[0], np.cumsum(lens)[:-1]]).astype(np.int64)
     return {
         "q": q, "q_idx": q_idx, "k_cache": k_cache, "v_cache": v_cache,

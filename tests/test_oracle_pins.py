@@ -13,7 +13,7 @@ import pytest
 import torch
 
 import oracle
-from paper_2606_13392_b200.inputs import (MSAConfig, bits_to_f32, make_prefill_inputs,
+from paper_2606_13392_b200.inputs import (MSAConfig, bits_to_f32, make_decode_inputs, make_prefill_inputs,
                                           to_bits)
 
 
@@ -442,3 +442,24 @@ def test_flops_model_printed_ratio():
     # closed forms of the two terms
     assert oracle.flops_gqa(10, 3, 5) == 2 * 3 * 5 * 100
     assert oracle.flops_msa(10, 4, 2, 5, 7, 3, 2) == 2 * 7 * 100 + 4 * 4 * 5 * 10 * 3 * 2
+
+
+def test_fp8_kv_sparse_attention_equals_bf16_of_the_same_values():
+    # Section 4.2 (the kernels also support fp8): K and V stored as fp8 E4M3.  Every E4M3 value is
+    # exactly a bf16 value, so the oracle on fp8 K/V must give, bit for bit, what it gives on the bf16
+    # tensors torch converts those fp8 tensors to (an independent decoding), and a visibly different
+    # result from the unrounded bf16 caches.
+    cfg = MSAConfig("kv8", "decode", 0, 8, 2, 16, 3, head_dim=32, idx_dim=16, seed=5, seq_lens=(70, 33), kv_fp8=True)
+    x = make_decode_inputs(cfg, "cpu", sharp=True)
+    assert x["k_cache"].dtype == torch.float8_e4m3fn and x["q"].dtype == torch.bfloat16
+    L = cfg.seq_lens[0]
+    K8, V8 = x["k_cache"][:L], x["v_cache"][:L]
+    pos = np.array([L - 1])
+    I = np.array([[[0, 2, 4], [1, 3, 4]]], dtype=np.int32)
+    q = to_bits(x["q"][:1])
+    O8, L8 = oracle.sparse_attn(q, to_bits(K8), to_bits(V8), I, pos, cfg.block_size)
+    Ob, Lb = oracle.sparse_attn(q, to_bits(K8.to(torch.bfloat16)), to_bits(V8.to(torch.bfloat16)), I, pos, cfg.block_size)
+    assert np.array_equal(O8, Ob) and np.array_equal(L8, Lb)
+    xb = make_decode_inputs(cfg.scaled(kv_fp8=False), "cpu", sharp=True)
+    Of, _ = oracle.sparse_attn(q, to_bits(xb["k_cache"][:L]), to_bits(xb["v_cache"][:L]), I, pos, cfg.block_size)
+    assert 1e-4 < np.abs(Of - O8).max() < 0.2  # the rounding of K and V is there, and is small
