@@ -76,7 +76,7 @@ def decode_work(cfg: MSAConfig):
     return {
         "index_bytes": (1.0 if cfg.idx_fp8 else 2.0) * cfg.idx_dim * float(lens.sum()),
         "index_flops": 2.0 * cfg.n_kv_heads * cfg.idx_dim * float(lens.sum()),
-        "attn_bytes": 2.0 * 2 * cfg.n_kv_heads * cfg.head_dim * float(tokens.sum()),
+        "attn_bytes": (1.0 if cfg.kv_fp8 else 2.0) * 2 * cfg.n_kv_heads * cfg.head_dim * float(tokens.sum()),
         "attn_flops": 4.0 * cfg.n_q_heads * cfg.head_dim * float(tokens.sum()),
     }
 
@@ -313,7 +313,7 @@ def base_line(cfg: MSAConfig, args, n_gpus: int):
 
 
 def describe(cfg: MSAConfig) -> str:
-    f8 = ", index operands fp8 E4M3" if cfg.idx_fp8 else ""
+    f8 = (", index operands fp8 E4M3" if cfg.idx_fp8 else "") + (", K/V caches fp8 E4M3" if cfg.kv_fp8 else "")
     if cfg.mode == "prefill" and cfg.seq_lens:
         return ("prefill fwd, %d packed sequences of %s tokens (%d in all), causal, %d q heads / %d kv heads, d_h=%d, "
                 "d_idx=%d, B_k=%d, k=%d%s"

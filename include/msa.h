@@ -72,6 +72,12 @@ typedef struct {
                          /* every "bf16" below then reads "fp8" for those two     */
                          /* operands.  Codes 0x7F / 0xFF (NaN) must not occur.    */
                          /* Any other value: MSA_ERR_INVALID_ARG.                 */
+    int32_t kv_fp8;      /* 0: K and V are bf16.  1: the decode calls read k_cache */
+                         /* and v_cache as fp8 E4M3 (Section 4.2), one byte per   */
+                         /* element; Q stays bf16 and must lie in the normal range */
+                         /* of fp16 (it is multiplied as fp16).  Needs d_h = 128,  */
+                         /* G in {8,16}, B_k in {64,128}; the prefill calls return */
+                         /* MSA_ERR_UNSUPPORTED.  Other values: INVALID_ARG.       */
 } msa_shape_t;
 
 typedef void* msa_stream_t; /* a cudaStream_t */

@@ -40,7 +40,7 @@ class MsaShape(ctypes.Structure):
     _fields_ = [("n_q_heads", c_i32), ("n_kv_heads", c_i32), ("head_dim", c_i32),
                 ("idx_dim", c_i32), ("block_size", c_i32), ("top_k", c_i32),
                 ("softmax_scale", ctypes.c_float), ("index_scale", ctypes.c_float),
-                ("idx_fp8", c_i32)]
+                ("idx_fp8", c_i32), ("kv_fp8", c_i32)]
 
 
 class MsaError(RuntimeError):
@@ -73,7 +73,7 @@ def status_string(code: int) -> str:
 
 def shape_of(cfg: MSAConfig, softmax_scale: float = 0.0, index_scale: float = 0.0) -> MsaShape:
     return MsaShape(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.idx_dim, cfg.block_size,
-                    cfg.top_k, softmax_scale, index_scale, 1 if cfg.idx_fp8 else 0)
+                    cfg.top_k, softmax_scale, index_scale, 1 if cfg.idx_fp8 else 0, 1 if cfg.kv_fp8 else 0)
 
 
 def _ptr(t) -> c_vp:
@@ -96,6 +96,14 @@ def _idx(shape, t: Optional[torch.Tensor], host: bool = False):
         assert t.element_size() == want, "index operand element size %d, shape expects %d" % (
             t.element_size(), want)
     return _host(t) if host else _dev(t)
+
+
+def _kv(shape, t: Optional[torch.Tensor]):
+    """A K or V cache of a decode call: its element size must match the shape's kv_fp8 flag."""
+    if t is not None:
+        want = 1 if shape.kv_fp8 else 2
+        assert t.element_size() == want, "K/V cache element size %d, shape expects %d" % (t.element_size(), want)
+    return _dev(t)
 
 
 def _host(t: Optional[torch.Tensor]):
@@ -217,7 +225,7 @@ def msa_sparse_attn_decode_workspace_bytes(shape, batch) -> int:
 
 def msa_sparse_attn_decode(shape, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch,
                            block_idx, out, lse, workspace, stream=None):
-    _check(lib().msa_sparse_attn_decode(ctypes.byref(shape), _dev(q), _dev(k_cache), _dev(v_cache),
+    _check(lib().msa_sparse_attn_decode(ctypes.byref(shape), _dev(q), _kv(shape, k_cache), _kv(shape, v_cache),
                                         c_i64(cache_tokens), _dev(seq_offsets), _dev(seq_lens),
                                         c_i32(batch), _dev(block_idx), _dev(out), _dev(lse),
                                         _dev(workspace),
@@ -309,8 +317,8 @@ def msa_prefill_forward_host(shape, q, k, v, q_idx, k_idx, T, out, lse, block_id
 def msa_decode_forward(shape, q, q_idx, k_cache, v_cache, k_idx_cache, cache_tokens, seq_offsets,
                        seq_lens, batch, max_seq_len, scores, ld_scores, block_idx, out, lse,
                        workspace, stream=None):
-    _check(lib().msa_decode_forward(ctypes.byref(shape), _dev(q), _idx(shape, q_idx), _dev(k_cache),
-                                    _dev(v_cache), _idx(shape, k_idx_cache), c_i64(cache_tokens),
+    _check(lib().msa_decode_forward(ctypes.byref(shape), _dev(q), _idx(shape, q_idx), _kv(shape, k_cache),
+                                    _kv(shape, v_cache), _idx(shape, k_idx_cache), c_i64(cache_tokens),
                                     _dev(seq_offsets), _dev(seq_lens), c_i32(batch),
                                     c_i64(max_seq_len), _dev(scores), c_i64(ld_scores),
                                     _dev(block_idx), _dev(out), _dev(lse), _dev(workspace),
@@ -322,7 +330,7 @@ def msa_decode_forward_host(shape, q_host, q_idx_host, q_dev, q_idx_dev, k_cache
                             k_idx_cache, cache_tokens, seq_offsets, seq_lens, batch, max_seq_len,
                             scores, ld_scores, block_idx, out_dev, out_host, workspace, stream=None):
     _check(lib().msa_decode_forward_host(ctypes.byref(shape), _host(q_host), _idx(shape, q_idx_host, True),
-                                         _dev(q_dev), _idx(shape, q_idx_dev), _dev(k_cache), _dev(v_cache),
+                                         _dev(q_dev), _idx(shape, q_idx_dev), _kv(shape, k_cache), _kv(shape, v_cache),
                                          _idx(shape, k_idx_cache), c_i64(cache_tokens), _dev(seq_offsets),
                                          _dev(seq_lens), c_i32(batch), c_i64(max_seq_len),
                                          _dev(scores), c_i64(ld_scores), _dev(block_idx),

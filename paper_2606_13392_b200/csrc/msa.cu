@@ -12,6 +12,7 @@
 #include "attn_prefill_tc.cuh"
 #include "index_lse.cuh"
 #include "decode.cuh"
+#include "decode_kv8.cuh"
 
 namespace msa {
 
@@ -49,6 +50,7 @@ int* async_status_ptr() {
 struct Resolved {
     int H_q, H_kv, G, d, d_idx, B_k, k;
     float softmax_scale, index_scale;
+    bool kv_fp8;                                         // decode: the K and V caches are fp8 E4M3 (else bf16)
     bool idx_fp8;                                        // index-branch operands are fp8 E4M3 (else bf16)
     size_t idx_elt() const { return idx_fp8 ? 1 : 2; }  // bytes per index-branch element
 };
@@ -70,6 +72,8 @@ static msa_status_t resolve(const msa_shape_t* s, Resolved& r) {
     if (s->idx_fp8 != 0 && s->idx_fp8 != 1) return MSA_ERR_INVALID_ARG;
     r.idx_fp8 = s->idx_fp8 == 1;
     if (r.idx_fp8 && r.d_idx % 16 != 0) return MSA_ERR_UNSUPPORTED;  // 16-byte rows
+    if (s->kv_fp8 != 0 && s->kv_fp8 != 1) return MSA_ERR_INVALID_ARG;
+    r.kv_fp8 = s->kv_fp8 == 1;
     return MSA_OK;
 }
 
@@ -558,26 +562,29 @@ static size_t decode_ws_bytes(const Resolved& r, int batch) {
     return align_up(parts * r.G * 128 * 4) + align_up(parts * 2 * r.G * 4) + kAlign;
 }
 
-template <int BK, int G>
+// KV8: the caches hold fp8 E4M3; a key row of 128 bytes is moved as 64 two-byte elements (one box per tile).
+template <int BK, int G, bool KV8 = false>
 static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const void* k_cache, const void* v_cache,
                                        int64_t cache_tokens, const int64_t* seq_offsets, const int32_t* seq_lens,
                                        int batch, const int32_t* block_idx, void* out, float* lse, void* ws,
                                        cudaStream_t st) {
     CUtensorMap tm_k, tm_v;
-    const uint64_t kd[3] = {128, (uint64_t)r.H_kv, (uint64_t)cache_tokens};
-    const uint64_t ks[2] = {256, (uint64_t)r.H_kv * 256};
+    const uint64_t row_b = KV8 ? 128 : 256;  // bytes of one head's key or value vector
+    const uint64_t kd[3] = {row_b / 2, (uint64_t)r.H_kv, (uint64_t)cache_tokens};
+    const uint64_t ks[2] = {row_b, (uint64_t)r.H_kv * row_b};
     const uint32_t kb[3] = {64, 1, (uint32_t)BK};
     if (!encode_tmap_bf16(&tm_k, k_cache, 3, kd, ks, kb) || !encode_tmap_bf16(&tm_v, v_cache, 3, kd, ks, kb))
         return MSA_ERR_CUDA;
     int* status = async_status_ptr();
     if (status == nullptr) return MSA_ERR_CUDA;
-    const size_t smem = sizeof(DecSmem<BK>) + 1024;
+    const size_t smem = (KV8 ? sizeof(DecKv8Smem<BK>) : sizeof(DecSmem<BK>)) + 1024;
     static bool attr_set_dev[64] = {false};  // the attribute is per device
     const int dev_id = current_device();
     if (!attr_set_dev[dev_id]) {
-        if (cudaFuncSetAttribute(attn_decode_kernel<BK, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-            cudaSuccess)
-            return MSA_ERR_CUDA;
+        const cudaError_t e =
+            KV8 ? cudaFuncSetAttribute(attn_decode_kv8_kernel<BK, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                : cudaFuncSetAttribute(attn_decode_kernel<BK, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return MSA_ERR_CUDA;
         attr_set_dev[dev_id] = true;
     }
     DecParams p;
@@ -591,7 +598,10 @@ static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const v
     const int grid = n_items < sm_count() ? n_items : sm_count();
     {
         StageScope sc(kStageAttnDecode, st);
-        attn_decode_kernel<BK, G><<<grid, kDecThreads, smem, st>>>(tm_k, tm_v, p, status);
+        if constexpr (KV8)
+            attn_decode_kv8_kernel<BK, G><<<grid, kDecThreads, smem, st>>>(tm_k, tm_v, p, status);
+        else
+            attn_decode_kernel<BK, G><<<grid, kDecThreads, smem, st>>>(tm_k, tm_v, p, status);
     }
     {
         StageScope sc(kStageCombineDecode, st);
@@ -867,6 +877,7 @@ msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, co
     Resolved r;
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
+    if (r.kv_fp8) return MSA_ERR_UNSUPPORTED;  // fp8 K/V caches: decode calls only
     if ((s = check_range(q_begin, q_count, kv_len)) != MSA_OK) return s;
     if (q_count == 0) return MSA_OK;
     if (!q || !k || !v || !block_idx || !out || !aligned16(q) || !aligned16(k) || !aligned16(v) ||
@@ -976,6 +987,7 @@ msa_status_t msa_sparse_attn_prefill_static(const msa_shape_t* shape, const void
     Resolved r;
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
+    if (r.kv_fp8) return MSA_ERR_UNSUPPORTED;  // fp8 K/V caches: decode calls only
     if ((s = check_range(q_begin, q_count, kv_len)) != MSA_OK) return s;
     if (q_count == 0) return MSA_OK;
     if (!q || !k || !v || !block_idx || !out || !aligned16(q) || !aligned16(k) || !aligned16(v) ||
@@ -1026,6 +1038,17 @@ msa_status_t msa_sparse_attn_decode(const msa_shape_t* shape, const void* q, con
     size_t need = 0;
     msa_sparse_attn_decode_workspace_bytes(shape, batch, &need);
     if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
+    if (r.kv_fp8) {  // fp8 caches: the streaming tensor-core kernel only
+        if (!attn_decode_fast(r) || cache_tokens >= 2147483647LL) return MSA_ERR_UNSUPPORTED;
+        cudaStream_t st = (cudaStream_t)stream;
+        if (r.B_k == 64 && r.G == 8)
+            return run_attn_decode_tc<64, 8, true>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch, block_idx, out, lse, workspace, st);
+        if (r.B_k == 64)
+            return run_attn_decode_tc<64, 16, true>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch, block_idx, out, lse, workspace, st);
+        if (r.G == 8)
+            return run_attn_decode_tc<128, 8, true>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch, block_idx, out, lse, workspace, st);
+        return run_attn_decode_tc<128, 16, true>(r, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens, batch, block_idx, out, lse, workspace, st);
+    }
     if (attn_decode_fast(r) && cache_tokens < 2147483647LL) {
         cudaStream_t st = (cudaStream_t)stream;
         if (r.B_k == 64 && r.G == 8)
@@ -1081,6 +1104,7 @@ msa_status_t msa_prefill_forward(const msa_shape_t* shape, const void* q, const 
     Resolved r;
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
+    if (r.kv_fp8) return MSA_ERR_UNSUPPORTED;  // fp8 K/V caches: decode calls only
     if (T < 0) return MSA_ERR_INVALID_ARG;
     if (T == 0) return MSA_OK;
     if (!q || !k || !v || !q_idx || !k_idx || !out || !block_idx) return MSA_ERR_INVALID_ARG;
@@ -1212,6 +1236,7 @@ msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_ho
     Resolved r;
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
+    if (r.kv_fp8) return MSA_ERR_UNSUPPORTED;  // fp8 K/V caches: decode calls only
     if (T < 0) return MSA_ERR_INVALID_ARG;
     if (T == 0) return MSA_OK;
     if (!q_host || !k_host || !v_host || !q_idx_host || !k_idx_host || !out_host)

@@ -631,3 +631,41 @@ def test_decode_and_prefill_calls_replay_from_a_cuda_graph():
     torch.cuda.synchronize()
     _assert_clean()
     assert torch.equal(want[2], pi) and torch.equal(want[0], po) and torch.equal(want[1], pl)
+
+
+# ----------------------------------------------------------------- fp8 E4M3 K/V caches (decode, Section 4.2)
+@pytest.mark.parametrize("Hq,Hkv,Bk,k,lens", [
+    (64, 8, 128, 64, (1, 127, 128, 129, 8192, 8200, 20000, 16384 + 64)),   # G = 8
+    (64, 4, 128, 16, (1, 130, 4096, 5000, 30000)),                          # G = 16, the paper's regime
+    (32, 2, 64, 12, (70, 640, 641, 7000)),                                  # G = 16, B_k = 64
+    (16, 2, 64, 40, (3000, 64, 65)),                                        # G = 8, B_k = 64, several splits
+])
+@pytest.mark.parametrize("sharp", [False, True])
+def test_fp8_kv_cache_decode(Hq, Hkv, Bk, k, lens, sharp):
+    # K and V are dequantised exactly in registers, so against the oracle on the same fp8 values the
+    # result must hold the bf16 path's tolerances.
+    cfg = MSAConfig("kv8", "decode", 0, Hq, Hkv, Bk, k, head_dim=128, idx_dim=64, seed=len(lens) + k, seq_lens=lens,
+                    kv_fp8=True)
+    res = run_decode_case(cfg, sharp)
+    assert np.mean([r["exact"] for r in res]) >= 0.95
+
+
+def test_fp8_kv_and_index_decode_together():
+    cfg = MSAConfig("kv8-idx8", "decode", 0, 64, 4, 128, 16, head_dim=128, idx_dim=128, seed=3,
+                    seq_lens=(129, 4096, 40000), kv_fp8=True, idx_fp8=True)
+    run_decode_case(cfg, True)
+
+
+def test_fp8_kv_cache_is_rejected_where_it_is_not_supported():
+    cfg = MSAConfig("kv8-bad", "prefill", 512, 64, 8, 128, 4, head_dim=128, idx_dim=64, seed=1, kv_fp8=True)
+    x = make_prefill_inputs(cfg.scaled(kv_fp8=False), DEV)
+    with pytest.raises(B.MsaError) as e:
+        api.prefill_forward(cfg, x)
+    assert e.value.code == 2  # MSA_ERR_UNSUPPORTED
+    dcfg = MSAConfig("kv8-odd", "decode", 0, 6, 3, 16, 5, head_dim=64, idx_dim=32, seed=3, seq_lens=(5, 400), kv_fp8=True)
+    xd = make_decode_inputs(dcfg, DEV)
+    with pytest.raises(B.MsaError) as e:
+        api.decode_forward(dcfg, xd)
+    assert e.value.code == 2
+    with pytest.raises(AssertionError):  # bf16 caches with the flag set
+        api.decode_forward(dcfg, make_decode_inputs(dcfg.scaled(kv_fp8=False), DEV))
