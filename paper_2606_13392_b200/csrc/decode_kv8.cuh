@@ -3,7 +3,8 @@
 // The structure of attn_decode_kernel - persistent CTAs, a producer warp streaming the selected
 // blocks through a TMA ring, four consumer warps with 32 keys of every block each, online softmax
 // in registers, per-warp partials - with tiles of half the bytes (a key row is one 128-byte swizzle
-// atom) and a deeper ring.  K and V are dequantised in registers: E4M3 -> f16 is exact and one
+// atom), two CTAs per SM (six tiles of 16 KB each) and tensor maps with a 128-byte L2 promotion (a
+// head's 128-byte row has other heads' rows as neighbours; a 256-byte promotion fetched them too).  K and V are dequantised in registers: E4M3 -> f16 is exact and one
 // instruction per pair, so both products run as f16 MMAs with Q converted to f16 (exact for bf16
 // values in f16's normal range) and P rounded to f16: the result differs from the bf16-cache
 // kernel's only by the rounding of K and V to fp8.  The contraction index of Q K^T and the row
@@ -17,7 +18,7 @@
 
 namespace msa {
 
-constexpr int kDecKv8Stages = 10;
+constexpr int kDecKv8Stages = 6;  // 96 KB at B_k = 128: two CTAs per SM, eight consumer warps to hide the dequantisation
 
 template <int BK>
 struct DecKv8Smem {
@@ -40,12 +41,16 @@ __device__ __forceinline__ void mma_m16n8k16_f16(float (&c)[4], uint32_t a0, uin
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Two fp8 E4M3 (low 16 bits, lower byte first) -> two f16 (exact).  (Integer bit moves instead of the
-// conversion instruction - sign and the seven other bits shifted to their f16 places, a factor 2^8
-// folded into the scales - were measured at the same speed.)
-__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two) {
-    const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(two & 0xFFFFu), __NV_E4M3);
-    return (uint32_t)h.x | ((uint32_t)h.y << 16);
+// Four fp8 E4M3 (bytes x0 .. x3 of a register) -> two registers of two f16 each, (x0, x1) and (x2, x3);
+// exact.  (Integer bit moves instead of the conversion instruction - sign and the seven other bits
+// shifted to their f16 places, a factor 2^8 folded into the scales - were measured at the same speed.)
+__device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t four, uint32_t& lo, uint32_t& hi) {
+    asm("{\n\t.reg .b16 a, b;\n\t"
+        "mov.b32 {a, b}, %2;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %0, a;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %1, b;\n\t}"
+        : "=r"(lo), "=r"(hi)
+        : "r"(four));
 }
 
 // Two bf16 (lower half first) -> two f16, round to nearest.
@@ -56,7 +61,7 @@ __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t two) {
 }
 
 template <int BK, int G>
-__global__ void __launch_bounds__(kDecThreads, 1)
+__global__ void __launch_bounds__(kDecThreads, 2)
 attn_decode_kv8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    DecParams p, int* status) {
     constexpr int KPW = BK / 4;    // keys per consumer warp
@@ -175,8 +180,9 @@ attn_decode_kv8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {  // chunk 4 q4 + j: this lane holds its bytes 4t .. 4t+3 of key g
                             const int ks = q4 * 4 + j;
-                            mma_m16n8k16_f16(c[nt], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], e4m3x2_to_f16x2(r4[j] & 0xFFFFu),
-                                             e4m3x2_to_f16x2(r4[j] >> 16));
+                            uint32_t b0, b1;
+                            e4m3x4_to_f16x2x2(r4[j], b0, b1);
+                            mma_m16n8k16_f16(c[nt], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
                         }
                     }
                 }
@@ -242,10 +248,10 @@ attn_decode_kv8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
                             const uint32_t lo = r4[half * 2], hi = r4[half * 2 + 1];  // keys 2t, 2t+1 and 8 + 2t, 8 + 2t + 1
-                            const uint32_t a0 = e4m3x2_to_f16x2(__byte_perm(lo, 0u, 0x4420));  // d even: (key 2t, key 2t+1)
-                            const uint32_t a1 = e4m3x2_to_f16x2(__byte_perm(lo, 0u, 0x4431));  // d odd
-                            const uint32_t a2 = e4m3x2_to_f16x2(__byte_perm(hi, 0u, 0x4420));
-                            const uint32_t a3 = e4m3x2_to_f16x2(__byte_perm(hi, 0u, 0x4431));
+                            // bytes (key 2t: d even, d odd; key 2t+1: d even, d odd) -> (d even: both keys; d odd: both keys)
+                            uint32_t a0, a1, a2, a3;
+                            e4m3x4_to_f16x2x2(__byte_perm(lo, 0u, 0x3120), a0, a1);
+                            e4m3x4_to_f16x2x2(__byte_perm(hi, 0u, 0x3120), a2, a3);
 #pragma unroll
                             for (int hg = 0; hg < HG; ++hg)
                                 mma_m16n8k16_f16(acc[hg][mp * 2 + half], a0, a1, a2, a3, pb[hg][ks][0], pb[hg][ks][1]);

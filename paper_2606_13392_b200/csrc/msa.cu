@@ -111,8 +111,10 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// promote_128: rows of 128 bytes whose neighbours in memory belong to other CTAs (fp8 K/V rows of one
+// head): a 256-byte L2 promotion would fetch the neighbour's row from DRAM as well.
 bool encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
-                      const uint64_t* strides_bytes, const uint32_t* box) {
+                      const uint64_t* strides_bytes, const uint32_t* box, bool promote_128) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
     cuuint64_t gdim[5], gstr[5];
@@ -120,7 +122,8 @@ bool encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64
     for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
     for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i];
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstr, bx, es,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              promote_128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -573,7 +576,7 @@ static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const v
     const uint64_t kd[3] = {row_b / 2, (uint64_t)r.H_kv, (uint64_t)cache_tokens};
     const uint64_t ks[2] = {row_b, (uint64_t)r.H_kv * row_b};
     const uint32_t kb[3] = {64, 1, (uint32_t)BK};
-    if (!encode_tmap_bf16(&tm_k, k_cache, 3, kd, ks, kb) || !encode_tmap_bf16(&tm_v, v_cache, 3, kd, ks, kb))
+    if (!encode_tmap_bf16(&tm_k, k_cache, 3, kd, ks, kb, KV8) || !encode_tmap_bf16(&tm_v, v_cache, 3, kd, ks, kb, KV8))
         return MSA_ERR_CUDA;
     int* status = async_status_ptr();
     if (status == nullptr) return MSA_ERR_CUDA;
@@ -595,7 +598,8 @@ static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const v
     p.part_o = (float*)ws;
     p.part_ml = (float*)((char*)ws + align_up(parts * G * 128 * 4));
     const int n_items = batch * r.H_kv * p.n_split;
-    const int grid = n_items < sm_count() ? n_items : sm_count();
+    const int ctas = sm_count() * (KV8 ? 2 : 1);  // the fp8 kernel's tiles are half as large: two CTAs per SM
+    const int grid = n_items < ctas ? n_items : ctas;
     {
         StageScope sc(kStageAttnDecode, st);
         if constexpr (KV8)

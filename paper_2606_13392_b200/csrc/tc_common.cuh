@@ -328,6 +328,6 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t 
 // the byte stride of dim i+1.  Returns false if the driver entry point is unavailable or
 // the encode fails.
 bool encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
-                      const uint64_t* strides_bytes, const uint32_t* box);
+                      const uint64_t* strides_bytes, const uint32_t* box, bool promote_128 = false);
 
 }  // namespace msa
