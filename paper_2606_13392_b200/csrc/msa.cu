@@ -531,7 +531,7 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
 
 // ---------------------------------------------------------------------- decode path
 static bool index_decode_fast(const Resolved& r) {
-    return (r.idx_fp8 ? r.d_idx == 128 : (r.d_idx == 64 || r.d_idx == 128)) && r.H_kv <= 8;
+    return (r.d_idx == 64 || r.d_idx == 128) && r.H_kv <= 8;
 }
 
 static msa_status_t run_index_decode(const Resolved& r, const void* q_idx, const void* k_idx_cache,
@@ -539,7 +539,11 @@ static msa_status_t run_index_decode(const Resolved& r, const void* q_idx, const
                                      int64_t n_cols, float* scores, int64_t ld_scores, cudaStream_t st) {
     const int grid = sm_count() * 4;
     StageScope sc(kStageIndexDecode, st);
-    if (r.idx_fp8)  // 128 fp8 per row: the bytes of 64 bf16
+    if (r.idx_fp8 && r.d_idx == 64)  // 64 fp8 per row: one 64-byte segment
+        index_scores_decode_kernel<16, 1, true><<<grid, kIdxDecWarps * 32, 0, st>>>(
+            (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx_cache, seq_offsets, seq_lens, batch, r.H_kv,
+            r.B_k, r.index_scale, scores, ld_scores, n_cols);
+    else if (r.idx_fp8)  // 128 fp8 per row: the bytes of 64 bf16
         index_scores_decode_kernel<8, 2, true><<<grid, kIdxDecWarps * 32, 0, st>>>(
             (const __nv_bfloat16*)q_idx, (const __nv_bfloat16*)k_idx_cache, seq_offsets, seq_lens, batch, r.H_kv,
             r.B_k, r.index_scale, scores, ld_scores, n_cols);

@@ -82,10 +82,12 @@ CONFIGS: Dict[str, MSAConfig] = {
     # (inputs still larger than L2).
     "c3-16k": MSAConfig("c3-16k", "prefill", 16384, 64, 8, 128, 64, seed=2,
                         planted_frac=0.05, planted_shift=2.0),
-    # Decode with the K/V caches stored in fp8 E4M3 (C5's shapes), and the paper's regime with both the
-    # cached index keys and the K/V caches in fp8.
+    # Decode with the K/V caches stored in fp8 E4M3 (C5's shapes), with the cached index keys in fp8 as
+    # well (c5-f8), and the paper's regime with both in fp8.
     "c5-kv8": MSAConfig("c5-kv8", "decode", 1048576, 64, 8, 128, 64, seed=4,
                         seq_lens=(131072,) * 16 + (1048576,) * 16, kv_fp8=True),
+    "c5-f8": MSAConfig("c5-f8", "decode", 1048576, 64, 8, 128, 64, seed=4,
+                       seq_lens=(131072,) * 16 + (1048576,) * 16, idx_fp8=True, kv_fp8=True),
     "pdec-f8kv": MSAConfig("pdec-f8kv", "decode", 1048576, 64, 4, 128, 16, idx_dim=128, seed=8,
                            seq_lens=(131072,) * 16 + (1048576,) * 16, idx_fp8=True, kv_fp8=True),
     "c5-small-kv8": MSAConfig("c5-small-kv8", "decode", 131072, 64, 8, 128, 64, seed=4,

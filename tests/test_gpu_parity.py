@@ -669,3 +669,11 @@ def test_fp8_kv_cache_is_rejected_where_it_is_not_supported():
     assert e.value.code == 2
     with pytest.raises(AssertionError):  # bf16 caches with the flag set
         api.decode_forward(dcfg, make_decode_inputs(dcfg.scaled(kv_fp8=False), DEV))
+
+
+def test_fp8_index_decode_d_idx_64():
+    # fp8 index keys of 64 elements (C5's shapes): a 64-byte row is one segment of the streaming kernel.
+    cfg = MSAConfig("f8-dec64", "decode", 0, 64, 8, 128, 64, head_dim=128, idx_dim=64, seed=21,
+                    seq_lens=(1, 130, 4096, 5000, 30000, 16384 + 64), idx_fp8=True, kv_fp8=True)
+    res = run_decode_case(cfg, True)
+    assert np.mean([r["exact"] for r in res]) >= 0.95
