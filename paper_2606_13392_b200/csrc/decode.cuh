@@ -152,7 +152,7 @@ index_scores_decode_kernel(const __nv_bfloat16* __restrict__ q_idx, const __nv_b
 }
 
 // ------------------------------------------------------------------ stage 3, decode
-constexpr int kDecStages = 6;
+constexpr int kDecStages = 3;         // 96 KB of tiles at B_k = 128: two CTAs per SM (measured a little ahead of one CTA with six)
 constexpr int kDecThreads = 160;      // warp 0: TMA producer, warps 1-4: consumers
 constexpr int kDecBlocksPerItem = 8;  // selected blocks streamed by one work item
 constexpr int kDecPartsPerItem = 4;   // one partial per consumer warp
@@ -183,7 +183,7 @@ __device__ __forceinline__ uint32_t dec_tile_addr(uint32_t tile_base, int key, i
 }
 
 template <int BK, int G>
-__global__ void __launch_bounds__(kDecThreads, 1)
+__global__ void __launch_bounds__(kDecThreads, 2)
 attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                    DecParams p, int* status) {
     constexpr int KPW = BK / 4;    // keys per consumer warp

@@ -602,7 +602,7 @@ static msa_status_t run_attn_decode_tc(const Resolved& r, const void* q, const v
     p.part_o = (float*)ws;
     p.part_ml = (float*)((char*)ws + align_up(parts * G * 128 * 4));
     const int n_items = batch * r.H_kv * p.n_split;
-    const int ctas = sm_count() * (KV8 ? 2 : 1);  // the fp8 kernel's tiles are half as large: two CTAs per SM
+    const int ctas = sm_count() * 2;
     const int grid = n_items < ctas ? n_items : ctas;
     {
         StageScope sc(kStageAttnDecode, st);
