@@ -402,19 +402,48 @@ attn_decode_combine_kernel(const float* __restrict__ part_o, const float* __rest
     const int r = h / G, g = h - r * G;
     const int n_parts = n_split * kDecPartsPerItem;
     const int64_t p0 = ((int64_t)seq * H_kv + r) * n_parts;
-    float M = -INFINITY;
-    for (int i = lane; i < n_parts; i += 32) M = fmaxf(M, part_ml[(p0 + i) * (2 * G) + g]);
+    // Lane i holds the weight of parts i, i + 32, ... (the maxima and sums are read once, in parallel);
+    // the partial rows are then accumulated four at a time, their loads independent of one another.
+    constexpr int kMaxSlots = 4;  // n_parts <= 128: top_k <= 128 -> n_split <= 16, four parts each = 64
+    float wv[kMaxSlots], M = -INFINITY;
+#pragma unroll
+    for (int u = 0; u < kMaxSlots; ++u) {
+        const int i = lane + 32 * u;
+        wv[u] = i < n_parts ? part_ml[(p0 + i) * (2 * G) + g] : -INFINITY;
+        M = fmaxf(M, wv[u]);
+    }
     M = warp_max(M);
     float L = 0.f;
+#pragma unroll
+    for (int u = 0; u < kMaxSlots; ++u) {
+        const int i = lane + 32 * u;
+        wv[u] = wv[u] > -INFINITY ? exp2f(wv[u] - M) : 0.f;  // a part with no visible key weighs nothing
+        if (i < n_parts && wv[u] > 0.f) L += wv[u] * part_ml[(p0 + i) * (2 * G) + G + g];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int i = 0; i < n_parts; ++i) {
-        const float mi = part_ml[(p0 + i) * (2 * G) + g];
-        if (mi == -INFINITY) continue;
-        const float wgt = exp2f(mi - M);
-        L += wgt * part_ml[(p0 + i) * (2 * G) + G + g];
-        const float4 o = *reinterpret_cast<const float4*>(part_o + ((p0 + i) * G + g) * 128 + lane * 4);
-        acc[0] = fmaf(wgt, o.x, acc[0]); acc[1] = fmaf(wgt, o.y, acc[1]);
-        acc[2] = fmaf(wgt, o.z, acc[2]); acc[3] = fmaf(wgt, o.w, acc[3]);
+    const float* orow = part_o + (p0 * G + g) * 128 + lane * 4;
+    for (int i0 = 0; i0 < n_parts; i0 += 4) {
+        float4 o[4];
+        float w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = i0 + j;
+            float wi = 0.f;
+#pragma unroll
+            for (int u = 0; u < kMaxSlots; ++u)
+                if (u == (i >> 5)) wi = wv[u];
+            w[j] = __shfl_sync(0xffffffffu, wi, i & 31);
+            o[j] = i < n_parts ? *reinterpret_cast<const float4*>(orow + (int64_t)i * G * 128) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (w[j] > 0.f) {  // (an unweighted part may hold anything)
+                acc[0] = fmaf(w[j], o[j].x, acc[0]); acc[1] = fmaf(w[j], o[j].y, acc[1]);
+                acc[2] = fmaf(w[j], o[j].z, acc[2]); acc[3] = fmaf(w[j], o[j].w, acc[3]);
+            }
+        }
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
     const __nv_bfloat162 o01 = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv);
