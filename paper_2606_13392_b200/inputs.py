@@ -96,6 +96,11 @@ CONFIGS: Dict[str, MSAConfig] = {
     # mixed lengths packed token-major, 1M tokens in all, the paper's regime.  seq_lens = the lengths.
     "pvar": MSAConfig("pvar", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=9,
                       seq_lens=(524288, 262144, 131072, 65536, 32768, 16384, 8192, 4096, 2048, 1024, 512, 512)),
+    # The same token count as many short sequences (a training batch): 128 of 8K, 512 of 2K.
+    "pvar-8k": MSAConfig("pvar-8k", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=10,
+                         seq_lens=(8192,) * 128),
+    "pvar-2k": MSAConfig("pvar-2k", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=11,
+                         seq_lens=(2048,) * 512),
     # A light decode step (8 sequences of 32K): launch gaps weigh as much as the kernels.
     "c5-light": MSAConfig("c5-light", "decode", 32768, 64, 8, 128, 64, seed=4, seq_lens=(32768,) * 8),
     "c5-small": MSAConfig("c5-small", "decode", 131072, 64, 8, 128, 64, seed=4,
