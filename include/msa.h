@@ -263,9 +263,14 @@ msa_status_t msa_prefill_forward_workspace_bytes(const msa_shape_t* shape, int64
  * cu_seqlens[s] .. cu_seqlens[s+1]-1 of q, k, v, q_idx, k_idx, out, lse and block_idx;
  * cu_seqlens is a HOST array of n_seqs+1 non-decreasing row offsets (int64), cu_seqlens[0] >= 0.
  * block_idx holds block numbers relative to the row's own sequence.  Sequences of length 0 are
- * skipped.  The sequences are run one after the other through the single-sequence path on
- * `stream`; workspace >= msa_prefill_forward_varlen_workspace_bytes (the largest single
- * sequence's need).  Errors: MSA_ERR_INVALID_ARG for a NULL or decreasing cu_seqlens or
+ * skipped.  Every sequence runs through the single-sequence path: long ones one after the other
+ * on `stream` with the whole workspace; sequences of at most 8192 tokens, when a quarter of the
+ * workspace holds one's preferred size, in turn on four streams owned by the library (created on
+ * first use), each with its own quarter, which start behind the work `stream` holds at the call
+ * and which `stream` waits for before the call returns (events only: the call may be captured
+ * into a CUDA graph).  Results do not depend on which way a sequence ran.
+ * workspace >= msa_prefill_forward_varlen_workspace_bytes' minimum (the largest single
+ * sequence's need; its preferred size has room for the four quarters).  Errors: MSA_ERR_INVALID_ARG for a NULL or decreasing cu_seqlens or
  * n_seqs < 0, otherwise as msa_prefill_forward.
  */
 msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q, const void* k,

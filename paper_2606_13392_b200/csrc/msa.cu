@@ -1159,6 +1159,12 @@ static msa_status_t check_cu_seqlens(const int64_t* cu, int32_t n_seqs) {
     return MSA_OK;
 }
 
+// Sequences of at most kVarlenSmallTokens leave much of the GPU idle at the ends of their kernels:
+// such sequences, independent problems, run on up to kVarlenLanes streams of the library's own, each
+// on its own slice of the workspace, forked from and joined to the caller's stream with events.
+constexpr int kVarlenLanes = 4;
+constexpr int64_t kVarlenSmallTokens = 8192;
+
 msa_status_t msa_prefill_forward_varlen_workspace_bytes(const msa_shape_t* shape,
                                                         const int64_t* cu_seqlens, int32_t n_seqs,
                                                         size_t* min_bytes, size_t* preferred_bytes) {
@@ -1166,14 +1172,16 @@ msa_status_t msa_prefill_forward_varlen_workspace_bytes(const msa_shape_t* shape
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
     if ((s = check_cu_seqlens(cu_seqlens, n_seqs)) != MSA_OK) return s;
-    size_t mn = kAlign, pf = kAlign;
+    size_t mn = kAlign, pf = kAlign, pf_small = 0;
     for (int32_t i = 0; i < n_seqs; ++i) {
         size_t a = 0, b = 0;
-        if ((s = msa_prefill_forward_workspace_bytes(shape, cu_seqlens[i + 1] - cu_seqlens[i], &a, &b)) != MSA_OK)
-            return s;
+        const int64_t T = cu_seqlens[i + 1] - cu_seqlens[i];
+        if ((s = msa_prefill_forward_workspace_bytes(shape, T, &a, &b)) != MSA_OK) return s;
         if (a > mn) mn = a;
         if (b > pf) pf = b;
+        if (T <= kVarlenSmallTokens && b > pf_small) pf_small = b;
     }
+    if (n_seqs > 1 && kVarlenLanes * align_up(pf_small) > pf) pf = kVarlenLanes * align_up(pf_small);
     if (min_bytes) *min_bytes = mn;
     if (preferred_bytes) *preferred_bytes = pf;
     return MSA_OK;
@@ -1197,17 +1205,63 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
     // Every sequence is an independent problem: the single-sequence path on row-offset pointers.
     const size_t q_row = (size_t)r.H_q * r.d * 2, kv_row = (size_t)r.H_kv * r.d * 2;
     const size_t qi_row = (size_t)r.H_kv * r.d_idx * r.idx_elt(), ki_row = (size_t)r.d_idx * r.idx_elt();
-    for (int32_t i = 0; i < n_seqs; ++i) {
+    cudaStream_t st = (cudaStream_t)stream;
+    static cudaStream_t lanes[kVarlenLanes] = {};
+    const size_t slice = (workspace_bytes / kVarlenLanes) & ~(size_t)(kAlign - 1);
+    bool forked[kVarlenLanes] = {};   // lanes that hold work since the last join
+    cudaEvent_t fork_ev = nullptr;    // marks the caller's stream after the last join
+    int next_lane = 0;
+    auto join = [&]() -> bool {
+        for (int l = 0; l < kVarlenLanes; ++l) {
+            if (!forked[l]) continue;
+            cudaEvent_t e = next_sync_event();
+            if (!e || cudaEventRecord(e, lanes[l]) != cudaSuccess || cudaStreamWaitEvent(st, e, 0) != cudaSuccess)
+                return false;
+            forked[l] = false;
+        }
+        fork_ev = nullptr;
+        return true;
+    };
+    msa_status_t result = MSA_OK;
+    for (int32_t i = 0; i < n_seqs && result == MSA_OK; ++i) {
         const int64_t o = cu_seqlens[i], T = cu_seqlens[i + 1] - o;
         if (T == 0) continue;
-        s = msa_prefill_forward(shape, (const char*)q + o * q_row, (const char*)k + o * kv_row,
-                                (const char*)v + o * kv_row, (const char*)q_idx + o * qi_row,
-                                (const char*)k_idx + o * ki_row, T, (char*)out + o * q_row,
-                                lse ? lse + o * r.H_q : nullptr, block_idx + o * (int64_t)r.H_kv * r.k, workspace,
-                                workspace_bytes, stream);
-        if (s != MSA_OK) return s;
+        size_t mn = 0, pf = 0;
+        if ((result = msa_prefill_forward_workspace_bytes(shape, T, &mn, &pf)) != MSA_OK) break;
+        const bool on_lane = n_seqs > 1 && T <= kVarlenSmallTokens && pf <= slice;
+        cudaStream_t run = st;
+        char* ws = (char*)workspace;
+        size_t ws_bytes = workspace_bytes;
+        if (on_lane) {
+            const int l = next_lane;
+            next_lane = (next_lane + 1) % kVarlenLanes;
+            if (lanes[l] == nullptr && cudaStreamCreateWithFlags(&lanes[l], cudaStreamNonBlocking) != cudaSuccess) {
+                result = MSA_ERR_CUDA;
+                break;
+            }
+            if (!forked[l]) {  // the lane starts behind what the caller's stream holds now
+                if (fork_ev == nullptr) {
+                    fork_ev = next_sync_event();
+                    if (!fork_ev || cudaEventRecord(fork_ev, st) != cudaSuccess) { result = MSA_ERR_CUDA; break; }
+                }
+                if (cudaStreamWaitEvent(lanes[l], fork_ev, 0) != cudaSuccess) { result = MSA_ERR_CUDA; break; }
+                forked[l] = true;
+            }
+            run = lanes[l];
+            ws += (size_t)l * slice;
+            ws_bytes = slice;
+        } else if (!join()) {  // the whole workspace: behind every lane
+            result = MSA_ERR_CUDA;
+            break;
+        }
+        result = msa_prefill_forward(shape, (const char*)q + o * q_row, (const char*)k + o * kv_row,
+                                     (const char*)v + o * kv_row, (const char*)q_idx + o * qi_row,
+                                     (const char*)k_idx + o * ki_row, T, (char*)out + o * q_row,
+                                     lse ? lse + o * r.H_q : nullptr, block_idx + o * (int64_t)r.H_kv * r.k, ws,
+                                     ws_bytes, (msa_stream_t)run);
     }
-    return MSA_OK;
+    if (!join() && result == MSA_OK) result = MSA_ERR_CUDA;  // (also on an error: no lane is left unjoined)
+    return result;
 }
 
 static size_t host_staging_bytes(const Resolved& r, int64_t T, size_t off[8]) {

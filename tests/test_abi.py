@@ -100,9 +100,15 @@ def test_varlen_validation_and_workspace(lib):
     assert lib.msa_prefill_forward_varlen(*args(i64x3(0, 0, 0), 2)) == 0        # nothing to do
     assert lib.msa_prefill_forward_varlen(*args(i64x3(0, 500, 900), -1)) == 1
     assert lib.msa_prefill_forward_varlen(*args(i64x3(0, 500, 900), 2)) == 3    # workspace too small
-    # the batch needs what its longest sequence needs
+    # the batch needs what its longest sequence needs; the preferred size has room for four short
+    # sequences (at most 8192 tokens) side by side
     mn, pf = B.msa_prefill_forward_varlen_workspace_bytes(shape, [0, 300, 5000, 5100])
     m1, p1 = B.msa_prefill_forward_workspace_bytes(shape, 4700)
+    assert mn == m1 and 4 * p1 <= pf <= 4 * p1 + 4 * 1024
+    mn, pf = B.msa_prefill_forward_varlen_workspace_bytes(shape, [0, 300, 300, 200300])
+    m2, p2 = B.msa_prefill_forward_workspace_bytes(shape, 200000)
+    assert (mn, pf) == (m2, p2)
+    mn, pf = B.msa_prefill_forward_varlen_workspace_bytes(shape, [0, 4700])
     assert (mn, pf) == (m1, p1)
 
 

@@ -137,6 +137,35 @@ def test_varlen_batch_equals_sequence_by_sequence():
     check_attn(out[a:b][pos_t].float().cpu().numpy(), lse[a:b][pos_t].cpu().numpy(), O_ref, LSE_ref, "varlen")
 
 
+@pytest.mark.parametrize("ws", ["preferred", "minimum"])
+def test_varlen_short_sequences_side_by_side_and_long_ones_between(ws):
+    # Short sequences run on the library's own streams, each on a quarter of the workspace; a long
+    # one (more than 8192 tokens) waits for them, takes the whole workspace, and the next short ones
+    # start behind it.  With the minimum workspace everything runs on the caller's stream.  Either
+    # way every sequence must come out exactly as from its own call.
+    cfg = CONFIGS["c3"].scaled(name="c3-varlen-mix", T=0, top_k=8)
+    lens = [3000, 700, 9000, 0, 500, 64, 100, 2000, 1500, 12000, 300, 8192]
+    cu = np.concatenate([[0], np.cumsum(lens)]).tolist()
+    total = cu[-1]
+    x = make_prefill_inputs(cfg.scaled(T=total), DEV, sharp=False)
+    shape = B.shape_of(cfg.scaled(T=total))
+    mn, pf = B.msa_prefill_forward_varlen_workspace_bytes(shape, cu)
+    workspace = B.alloc_workspace(pf if ws == "preferred" else mn, DEV)
+    for rep in range(2):  # (the second call starts behind the first one's joins)
+        out, lse, I = api.prefill_forward_varlen(cfg.scaled(T=total), x, cu, workspace=workspace)
+    torch.cuda.synchronize()
+    _assert_clean()
+    for s, L in enumerate(lens):
+        if L == 0:
+            continue
+        a, b = cu[s], cu[s + 1]
+        xs = {n: t[a:b].contiguous() for n, t in x.items()}
+        o1, l1, i1 = api.prefill_forward(cfg.scaled(T=L), xs)
+        torch.cuda.synchronize()
+        assert torch.equal(I[a:b], i1), "sequence %d index lists" % s
+        assert torch.equal(out[a:b], o1) and torch.equal(lse[a:b], l1), "sequence %d outputs" % s
+
+
 @pytest.mark.parametrize("name,T,Hq,Hkv,Bk,k,di,sharp", [
     ("c3 shape", 6144 + 77, 64, 8, 128, 64, 64, False),
     ("c3 shape, sharp", 5000, 64, 8, 128, 16, 64, True),
@@ -631,6 +660,32 @@ def test_decode_and_prefill_calls_replay_from_a_cuda_graph():
     torch.cuda.synchronize()
     _assert_clean()
     assert torch.equal(want[2], pi) and torch.equal(want[0], po) and torch.equal(want[1], pl)
+
+    # the packed call: its short sequences fork onto the library's streams inside the capture
+    lens = [700, 3000, 9000, 64, 1500]
+    cu = np.concatenate([[0], np.cumsum(lens)]).tolist()
+    vcfg = CONFIGS["c3"].scaled(name="c3-graph-varlen", T=cu[-1], top_k=8)
+    vx = make_prefill_inputs(vcfg, DEV, sharp=True)
+    vshape = B.shape_of(vcfg)
+    vo = torch.empty_like(vx["q"])
+    vl = torch.empty((vcfg.T, vcfg.n_q_heads), dtype=torch.float32, device=DEV)
+    vi = torch.empty((vcfg.T, vcfg.n_kv_heads, vcfg.top_k), dtype=torch.int32, device=DEV)
+    vws = B.alloc_workspace(B.msa_prefill_forward_varlen_workspace_bytes(vshape, cu)[1], DEV)
+
+    def vstep():
+        B.msa_prefill_forward_varlen(vshape, vx["q"], vx["k"], vx["v"], vx["q_idx"], vx["k_idx"], cu, vo, vl, vi, vws)
+    with torch.cuda.stream(side):
+        vstep()
+    torch.cuda.synchronize()
+    want = (vo.clone(), vl.clone(), vi.clone())
+    vg = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(vg):
+        vstep()
+    vo.zero_(); vl.zero_(); vi.zero_()
+    vg.replay()
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert torch.equal(want[2], vi) and torch.equal(want[0], vo) and torch.equal(want[1], vl)
 
 
 # ----------------------------------------------------------------- fp8 E4M3 K/V caches (decode, Section 4.2)
