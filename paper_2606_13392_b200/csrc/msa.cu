@@ -19,7 +19,7 @@ namespace msa {
 static std::atomic<int64_t> g_launches{0};
 
 // Optional per-stage timing: a fixed pool of event pairs, created by msa_profile_begin().
-constexpr int kProfSlots = 8192;
+constexpr int kProfSlots = 16384;
 static bool g_prof_on = false;
 static int g_prof_used = 0;
 static cudaEvent_t g_prof_ev[kProfSlots][2];
