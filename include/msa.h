@@ -72,12 +72,20 @@ typedef struct {
                          /* every "bf16" below then reads "fp8" for those two     */
                          /* operands.  Codes 0x7F / 0xFF (NaN) must not occur.    */
                          /* Any other value: MSA_ERR_INVALID_ARG.                 */
-    int32_t kv_fp8;      /* 0: K and V are bf16.  1: the decode calls read k_cache */
-                         /* and v_cache as fp8 E4M3 (Section 4.2), one byte per   */
-                         /* element; Q stays bf16 and must lie in the normal range */
-                         /* of fp16 (it is multiplied as fp16).  Needs d_h = 128,  */
-                         /* G in {8,16}, B_k in {64,128}; the prefill calls return */
-                         /* MSA_ERR_UNSUPPORTED.  Other values: INVALID_ARG.       */
+    int32_t kv_fp8;      /* 0: K and V are bf16.  1: k / v (prefill) and k_cache / */
+                         /* v_cache (decode) are fp8 E4M3 (Section 4.2), one byte  */
+                         /* per element, dequantised exactly; Q stays bf16.        */
+                         /* Decode: needs d_h = 128, G in {8,16}, B_k in {64,128}, */
+                         /* and Q in the normal range of fp16 (it is multiplied as */
+                         /* fp16).  Prefill (msa_sparse_attn_prefill,              */
+                         /* msa_prefill_forward, msa_prefill_forward_varlen):      */
+                         /* d_h % 16 == 0; the call widens the kv_len visible rows */
+                         /* to bf16 in its workspace first (the *_workspace_bytes  */
+                         /* results include 4 * kv_len * H_kv * d_h bytes for it)  */
+                         /* and then computes as with bf16 K and V holding the     */
+                         /* same values.  The host-buffer and allocation-free      */
+                         /* prefill calls return MSA_ERR_UNSUPPORTED with the      */
+                         /* flag.  Other values: INVALID_ARG.                      */
 } msa_shape_t;
 
 typedef void* msa_stream_t; /* a cudaStream_t */

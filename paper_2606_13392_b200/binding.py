@@ -99,7 +99,7 @@ def _idx(shape, t: Optional[torch.Tensor], host: bool = False):
 
 
 def _kv(shape, t: Optional[torch.Tensor]):
-    """A K or V cache of a decode call: its element size must match the shape's kv_fp8 flag."""
+    """A K or V tensor (device): its element size must match the shape's kv_fp8 flag."""
     if t is not None:
         want = 1 if shape.kv_fp8 else 2
         assert t.element_size() == want, "K/V cache element size %d, shape expects %d" % (t.element_size(), want)
@@ -187,7 +187,7 @@ def msa_sparse_attn_prefill_workspace_bytes(shape, q_count, kv_len) -> Tuple[int
 
 def msa_sparse_attn_prefill(shape, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse,
                             workspace, stream=None):
-    _check(lib().msa_sparse_attn_prefill(ctypes.byref(shape), _dev(q), _dev(k), _dev(v),
+    _check(lib().msa_sparse_attn_prefill(ctypes.byref(shape), _dev(q), _kv(shape, k), _kv(shape, v),
                                          _dev(block_idx), c_i64(q_begin), c_i64(q_count),
                                          c_i64(kv_len), _dev(out), _dev(lse), _dev(workspace),
                                          c_sz(workspace.numel() * workspace.element_size()),
@@ -243,7 +243,7 @@ def msa_prefill_forward_workspace_bytes(shape, T) -> Tuple[int, int]:
 
 
 def msa_prefill_forward(shape, q, k, v, q_idx, k_idx, T, out, lse, block_idx, workspace, stream=None):
-    _check(lib().msa_prefill_forward(ctypes.byref(shape), _dev(q), _dev(k), _dev(v), _idx(shape, q_idx),
+    _check(lib().msa_prefill_forward(ctypes.byref(shape), _dev(q), _kv(shape, k), _kv(shape, v), _idx(shape, q_idx),
                                      _idx(shape, k_idx), c_i64(T), _dev(out), _dev(lse), _dev(block_idx),
                                      _dev(workspace),
                                      c_sz(workspace.numel() * workspace.element_size()),
@@ -289,7 +289,7 @@ def msa_prefill_forward_varlen_workspace_bytes(shape, cu_seqlens) -> Tuple[int, 
 def msa_prefill_forward_varlen(shape, q, k, v, q_idx, k_idx, cu_seqlens, out, lse, block_idx, workspace,
                                stream=None):
     arr, n = _cu_array(cu_seqlens)
-    _check(lib().msa_prefill_forward_varlen(ctypes.byref(shape), _dev(q), _dev(k), _dev(v), _idx(shape, q_idx),
+    _check(lib().msa_prefill_forward_varlen(ctypes.byref(shape), _dev(q), _kv(shape, k), _kv(shape, v), _idx(shape, q_idx),
                                             _idx(shape, k_idx), arr, c_i32(n), _dev(out), _dev(lse),
                                             _dev(block_idx), _dev(workspace),
                                             c_sz(workspace.numel() * workspace.element_size()),

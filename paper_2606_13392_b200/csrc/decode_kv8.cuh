@@ -60,6 +60,29 @@ __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t two) {
     return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+// fp8 E4M3 -> bf16, exact (every E4M3 value is a bf16 value): the prefill calls run on bf16 copies of
+// fp8 K/V caches.  One thread per 16 elements; n16 = elements / 16.
+__global__ void __launch_bounds__(256)
+e4m3_to_bf16_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int64_t n16) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (int64_t)gridDim.x * blockDim.x) {
+        const uint4 in = __ldg(src + i);
+        const uint32_t w[4] = {in.x, in.y, in.z, in.w};
+        uint32_t o[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t lo, hi;
+            e4m3x4_to_f16x2x2(w[j], lo, hi);
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&lo));
+            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&hi));
+            const __nv_bfloat162 ab = __floats2bfloat162_rn(a.x, a.y), bb = __floats2bfloat162_rn(b.x, b.y);
+            o[2 * j] = *reinterpret_cast<const uint32_t*>(&ab);
+            o[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&bb);
+        }
+        dst[2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
 template <int BK, int G>
 __global__ void __launch_bounds__(kDecThreads, 2)
 attn_decode_kv8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,

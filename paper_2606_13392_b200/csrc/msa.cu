@@ -50,7 +50,8 @@ int* async_status_ptr() {
 struct Resolved {
     int H_q, H_kv, G, d, d_idx, B_k, k;
     float softmax_scale, index_scale;
-    bool kv_fp8;                                         // decode: the K and V caches are fp8 E4M3 (else bf16)
+    bool kv_fp8;                                         // the K and V caches are fp8 E4M3 (else bf16)
+    size_t kv_elt() const { return kv_fp8 ? 1 : 2; }    // bytes per K/V element
     bool idx_fp8;                                        // index-branch operands are fp8 E4M3 (else bf16)
     size_t idx_elt() const { return idx_fp8 ? 1 : 2; }  // bytes per index-branch element
 };
@@ -855,6 +856,13 @@ msa_status_t msa_topk_select_decode(const msa_shape_t* shape, const float* score
     return run_topk(r, scores, ld_scores, rows, batch, block_idx, (cudaStream_t)stream);
 }
 
+// A prefill call on fp8 K/V caches runs on bf16 copies of the rows it can see (E4M3 -> bf16 is
+// exact): the caches are read once more per call, 3 bytes of traffic per element, against the
+// partial buffers' hundreds of bytes per (query, head).
+static size_t kv_copy_bytes(const Resolved& r, int64_t kv_len) {
+    return align_up((size_t)kv_len * r.H_kv * r.d * 2);
+}
+
 msa_status_t msa_sparse_attn_prefill_workspace_bytes(const msa_shape_t* shape, int64_t q_count,
                                                      int64_t kv_len, size_t* min_bytes,
                                                      size_t* preferred_bytes) {
@@ -873,6 +881,10 @@ msa_status_t msa_sparse_attn_prefill_workspace_bytes(const msa_shape_t* shape, i
         mn = attn_plan(r, kv_len, r_min).total + 8 * kAlign;
         pf = attn_plan(r, kv_len, r_pref).total + 8 * kAlign;
     }
+    if (r.kv_fp8) {  // bf16 copies of the visible K and V rows in front
+        mn += 2 * kv_copy_bytes(r, kv_len);
+        pf += 2 * kv_copy_bytes(r, kv_len);
+    }
     if (min_bytes) *min_bytes = mn;
     if (preferred_bytes) *preferred_bytes = pf;
     return MSA_OK;
@@ -885,7 +897,6 @@ msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, co
     Resolved r;
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
-    if (r.kv_fp8) return MSA_ERR_UNSUPPORTED;  // fp8 K/V caches: decode calls only
     if ((s = check_range(q_begin, q_count, kv_len)) != MSA_OK) return s;
     if (q_count == 0) return MSA_OK;
     if (!q || !k || !v || !block_idx || !out || !aligned16(q) || !aligned16(k) || !aligned16(v) ||
@@ -895,6 +906,27 @@ msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, co
     msa_sparse_attn_prefill_workspace_bytes(shape, q_count, kv_len, &need, nullptr);
     if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    if (r.kv_fp8) {  // bf16 copies of the visible rows, then the bf16 path on the rest of the workspace
+        if (r.d % 16 != 0) return MSA_ERR_UNSUPPORTED;  // the conversion moves 16 elements per thread
+        const size_t cb = kv_copy_bytes(r, kv_len);
+        const int64_t n16 = kv_len * r.H_kv * r.d / 16;
+        char* kb = (char*)workspace;
+        char* vb = kb + cb;
+        const unsigned grid = (unsigned)(n16 < 148 * 8 * 256 ? ceil_div64(n16 > 0 ? n16 : 1, 256) : 148 * 8);
+        {
+            StageScope sc(kStageAttn, st);
+            e4m3_to_bf16_kernel<<<grid, 256, 0, st>>>((const uint4*)k, (uint4*)kb, n16);
+        }
+        {
+            StageScope sc(kStageAttn, st);
+            e4m3_to_bf16_kernel<<<grid, 256, 0, st>>>((const uint4*)v, (uint4*)vb, n16);
+        }
+        if (cudaPeekAtLastError() != cudaSuccess) return MSA_ERR_CUDA;
+        msa_shape_t wide = *shape;
+        wide.kv_fp8 = 0;
+        return msa_sparse_attn_prefill(&wide, q, kb, vb, block_idx, q_begin, q_count, kv_len, out, lse,
+                                       (char*)workspace + 2 * cb, workspace_bytes - 2 * cb, stream);
+    }
     if (attn_tc_supported(r) && kv_len < 2147483647LL) {
         if (r.B_k == 64 && r.G == 8)
             return run_attn_prefill_tc<64, 8>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
@@ -1112,7 +1144,6 @@ msa_status_t msa_prefill_forward(const msa_shape_t* shape, const void* q, const 
     Resolved r;
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
-    if (r.kv_fp8) return MSA_ERR_UNSUPPORTED;  // fp8 K/V caches: decode calls only
     if (T < 0) return MSA_ERR_INVALID_ARG;
     if (T == 0) return MSA_OK;
     if (!q || !k || !v || !q_idx || !k_idx || !out || !block_idx) return MSA_ERR_INVALID_ARG;
@@ -1203,7 +1234,7 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
         return s;
     if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
     // Every sequence is an independent problem: the single-sequence path on row-offset pointers.
-    const size_t q_row = (size_t)r.H_q * r.d * 2, kv_row = (size_t)r.H_kv * r.d * 2;
+    const size_t q_row = (size_t)r.H_q * r.d * 2, kv_row = (size_t)r.H_kv * r.d * r.kv_elt();
     const size_t qi_row = (size_t)r.H_kv * r.d_idx * r.idx_elt(), ki_row = (size_t)r.d_idx * r.idx_elt();
     cudaStream_t st = (cudaStream_t)stream;
     static cudaStream_t lanes[kVarlenLanes] = {};

@@ -45,7 +45,7 @@ class MSAConfig:
     planted_shift: float = 0.0
     seq_lens: Tuple[int, ...] = ()
     idx_fp8: bool = False  # index-branch operands (Q_idx, K_idx) rounded to fp8 E4M3 instead of bf16
-    kv_fp8: bool = False   # decode: the K and V caches are stored in fp8 E4M3 (Q stays bf16)
+    kv_fp8: bool = False   # the K and V caches are stored in fp8 E4M3 (Q stays bf16)
 
     @property
     def group(self) -> int:
@@ -78,6 +78,11 @@ CONFIGS: Dict[str, MSAConfig] = {
     "p1m-f8": MSAConfig("p1m-f8", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=7, idx_fp8=True),
     "pdec-f8": MSAConfig("pdec-f8", "decode", 1048576, 64, 4, 128, 16, idx_dim=128, seed=8,
                          seq_lens=(131072,) * 16 + (1048576,) * 16, idx_fp8=True),
+    # Prefill onto fp8 K/V caches (widened to bf16 inside the call), index operands in fp8 as well.
+    "p128k-f8kv": MSAConfig("p128k-f8kv", "prefill", 131072, 64, 4, 128, 16, idx_dim=128, seed=6,
+                            idx_fp8=True, kv_fp8=True),
+    "p1m-f8kv": MSAConfig("p1m-f8kv", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=7,
+                          idx_fp8=True, kv_fp8=True),
     # Reduced cases of the same shapes, small enough for multi-pass profiler captures
     # (inputs still larger than L2).
     "c3-16k": MSAConfig("c3-16k", "prefill", 16384, 64, 8, 128, 64, seed=2,
@@ -176,6 +181,8 @@ def make_prefill_inputs(cfg: MSAConfig, device="cpu", sharp: bool = False):
     k_idx = _draw(gen, T, (di,), s_idx, device, tok_mask, sh_idx)
     if cfg.idx_fp8:  # the same draws, stored in the narrower format
         q_idx, k_idx = q_idx.to(torch.float8_e4m3fn), k_idx.to(torch.float8_e4m3fn)
+    if cfg.kv_fp8:  # prefill onto fp8 caches: K and V rounded to E4M3, Q stays bf16
+        k, v = k.to(torch.float8_e4m3fn), v.to(torch.float8_e4m3fn)
     return {"q": q, "k": k, "v": v, "q_idx": q_idx, "k_idx": k_idx}
 
 

@@ -711,11 +711,72 @@ def test_fp8_kv_and_index_decode_together():
     run_decode_case(cfg, True)
 
 
+@pytest.mark.parametrize("Hq,Hkv,Bk,k,T,d", [
+    (64, 8, 128, 16, 6144 + 77, 128),   # tensor-core attention path, ragged last block
+    (64, 4, 128, 16, 4096 + 1, 128),    # the paper's regime (G = 16)
+    (16, 2, 64, 6, 1500, 128),          # B_k = 64
+    (6, 3, 16, 5, 333, 64),             # generic kernels
+])
+@pytest.mark.parametrize("sharp", [False, True])
+def test_fp8_kv_cache_prefill(Hq, Hkv, Bk, k, T, d, sharp):
+    # Prefill onto fp8 K/V caches: the kernels run on exact bf16 copies of the fp8 values, so the
+    # result must (a) hold the bf16 path's tolerances against the oracle on the fp8 values and
+    # (b) equal, bit for bit, the bf16 call on the same values widened by torch.
+    cfg = MSAConfig("kv8-prefill", "prefill", T, Hq, Hkv, Bk, k, head_dim=d, idx_dim=64, seed=T % 97, kv_fp8=True)
+    stats = run_prefill_case(cfg, sharp, n_sample=256)
+    assert stats["exact_sets"] >= 0.999
+    x = make_prefill_inputs(cfg, DEV, sharp=sharp)
+    o8, l8, i8 = api.prefill_forward(cfg, x)
+    wide = dict(x, k=x["k"].to(torch.bfloat16), v=x["v"].to(torch.bfloat16))
+    o16, l16, i16 = api.prefill_forward(cfg.scaled(kv_fp8=False), wide)
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert torch.equal(i8, i16) and torch.equal(o8, o16) and torch.equal(l8, l16)
+
+
+def test_fp8_kv_cache_prefill_query_range_and_small_workspace():
+    # A chunk of new queries [q_begin, q_begin + q_count) against a longer fp8 cache, with the
+    # smallest workspace the library accepts: same numbers as the preferred size, and as the oracle.
+    cfg = MSAConfig("kv8-chunk", "prefill", 5000, 64, 8, 128, 8, head_dim=128, idx_dim=64, seed=11, kv_fp8=True)
+    x = make_prefill_inputs(cfg, DEV, sharp=True)
+    _, _, I = api.prefill_forward(cfg, x)
+    q0, qc, L = 3000, 1203, 4500  # the cache holds more rows than the call may see
+    o1, l1 = api.sparse_attn_prefill(cfg, x["q"][q0:q0 + qc], x["k"][:L], x["v"][:L], I[q0:q0 + qc].contiguous(), q0)
+    o2, l2 = api.sparse_attn_prefill(cfg, x["q"][q0:q0 + qc], x["k"][:L], x["v"][:L], I[q0:q0 + qc].contiguous(), q0,
+                                     workspace_bytes=1)
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
+    pos = np.arange(q0, q0 + qc)[::7]
+    O_ref, LSE_ref = oracle.sparse_attn(to_bits(x["q"][q0:q0 + qc][::7]), to_bits(x["k"][:L]), to_bits(x["v"][:L]),
+                                        I[q0:q0 + qc][::7].cpu().numpy(), pos, cfg.block_size)
+    check_attn(o1[::7].float().cpu().numpy(), l1[::7].cpu().numpy(), O_ref, LSE_ref, "kv8-chunk")
+
+
+def test_fp8_kv_cache_prefill_varlen_equals_sequence_by_sequence():
+    cfg = MSAConfig("kv8-varlen", "prefill", 0, 64, 8, 128, 8, head_dim=128, idx_dim=64, seed=5, kv_fp8=True)
+    lens = [700, 0, 2048 + 3, 129]
+    cu = np.concatenate([[0], np.cumsum(lens)]).tolist()
+    x = make_prefill_inputs(cfg.scaled(T=cu[-1]), DEV, sharp=True)
+    out, lse, I = api.prefill_forward_varlen(cfg, x, cu)
+    for a, b in zip(cu[:-1], cu[1:]):
+        if b == a:
+            continue
+        o1, l1, i1 = api.prefill_forward(cfg.scaled(T=b - a), {n: t[a:b] for n, t in x.items()})
+        assert torch.equal(out[a:b], o1) and torch.equal(lse[a:b], l1) and torch.equal(I[a:b], i1)
+    torch.cuda.synchronize()
+    _assert_clean()
+
+
 def test_fp8_kv_cache_is_rejected_where_it_is_not_supported():
     cfg = MSAConfig("kv8-bad", "prefill", 512, 64, 8, 128, 4, head_dim=128, idx_dim=64, seed=1, kv_fp8=True)
-    x = make_prefill_inputs(cfg.scaled(kv_fp8=False), DEV)
-    with pytest.raises(B.MsaError) as e:
-        api.prefill_forward(cfg, x)
+    x = make_prefill_inputs(cfg, DEV)
+    with pytest.raises(AssertionError):  # bf16 K/V with the flag set
+        api.prefill_forward(cfg, make_prefill_inputs(cfg.scaled(kv_fp8=False), DEV))
+    I = torch.zeros((cfg.T, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32, device=DEV)
+    out, lse = torch.empty_like(x["q"]), torch.empty((cfg.T, cfg.n_q_heads), dtype=torch.float32, device=DEV)
+    with pytest.raises(B.MsaError) as e:  # the allocation-free variant takes bf16 K/V only
+        B.msa_sparse_attn_prefill_static(B.shape_of(cfg), x["q"], x["k"], x["v"], I, 0, cfg.T, cfg.T, out, lse)
     assert e.value.code == 2  # MSA_ERR_UNSUPPORTED
     dcfg = MSAConfig("kv8-odd", "decode", 0, 6, 3, 16, 5, head_dim=64, idx_dim=32, seed=3, seq_lens=(5, 400), kv_fp8=True)
     xd = make_decode_inputs(dcfg, DEV)
