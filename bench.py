@@ -226,8 +226,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     peaks = load_peaks()
     packed = cfg.mode == "prefill" and bool(cfg.seq_lens)  # no host-buffer call and no oracle leg for packed batches
-    no_host = packed or (cfg.mode == "prefill" and cfg.kv_fp8)  # fp8 K/V caches live on the device: no host-buffer prefill call
-    line = measure(cfg, args, rank, world, dev, B, peaks, dist, e2e=not args.no_e2e and not no_host,
+    line = measure(cfg, args, rank, world, dev, B, peaks, dist, e2e=not args.no_e2e and not packed,
                    cpu=(world == 1 and not args.no_cpu_baseline and not packed))
     others = {}
     for name in extras:

@@ -83,9 +83,10 @@ typedef struct {
                          /* to bf16 in its workspace first (the *_workspace_bytes  */
                          /* results include 4 * kv_len * H_kv * d_h bytes for it)  */
                          /* and then computes as with bf16 K and V holding the     */
-                         /* same values.  The host-buffer and allocation-free      */
-                         /* prefill calls return MSA_ERR_UNSUPPORTED with the      */
-                         /* flag.  Other values: INVALID_ARG.                      */
+                         /* same values (msa_prefill_forward_host uploads the fp8  */
+                         /* bytes and does the same).  The allocation-free prefill */
+                         /* call returns MSA_ERR_UNSUPPORTED with the flag.  Other */
+                         /* values: INVALID_ARG.                                   */
 } msa_shape_t;
 
 typedef void* msa_stream_t; /* a cudaStream_t */

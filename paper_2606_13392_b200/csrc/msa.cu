@@ -1298,8 +1298,8 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
 static size_t host_staging_bytes(const Resolved& r, int64_t T, size_t off[8]) {
     size_t o = 0;
     off[0] = o; o += align_up((size_t)T * r.H_q * r.d * 2);      // q
-    off[1] = o; o += align_up((size_t)T * r.H_kv * r.d * 2);     // k
-    off[2] = o; o += align_up((size_t)T * r.H_kv * r.d * 2);     // v
+    off[1] = o; o += align_up((size_t)T * r.H_kv * r.d * r.kv_elt());  // k
+    off[2] = o; o += align_up((size_t)T * r.H_kv * r.d * r.kv_elt());  // v
     off[3] = o; o += align_up((size_t)T * r.H_kv * r.d_idx * r.idx_elt()); // q_idx
     off[4] = o; o += align_up((size_t)T * r.d_idx * r.idx_elt());          // k_idx
     off[5] = o; o += align_up((size_t)T * r.H_q * r.d * 2);      // out
@@ -1329,7 +1329,6 @@ msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_ho
     Resolved r;
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
-    if (r.kv_fp8) return MSA_ERR_UNSUPPORTED;  // fp8 K/V caches: decode calls only
     if (T < 0) return MSA_ERR_INVALID_ARG;
     if (T == 0) return MSA_OK;
     if (!q_host || !k_host || !v_host || !q_idx_host || !k_idx_host || !out_host)
@@ -1349,8 +1348,8 @@ msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_ho
     if (!e_in || !e_idx || !e_kv) return MSA_ERR_CUDA;
     if (cudaEventRecord(e_in, st) != cudaSuccess || cudaStreamWaitEvent(copy, e_in, 0) != cudaSuccess) return MSA_ERR_CUDA;
     const void* src[5] = {q_host, k_host, v_host, q_idx_host, k_idx_host};
-    const size_t nbytes[5] = {(size_t)T * r.H_q * r.d * 2, (size_t)T * r.H_kv * r.d * 2,
-                              (size_t)T * r.H_kv * r.d * 2, (size_t)T * r.H_kv * r.d_idx * r.idx_elt(),
+    const size_t nbytes[5] = {(size_t)T * r.H_q * r.d * 2, (size_t)T * r.H_kv * r.d * r.kv_elt(),
+                              (size_t)T * r.H_kv * r.d * r.kv_elt(), (size_t)T * r.H_kv * r.d_idx * r.idx_elt(),
                               (size_t)T * r.d_idx * r.idx_elt()};
     // Order on the copy stream: K_idx, Q_idx, K, V, Q; Q_idx and Q go in pieces with an event after each,
     // so that every scoring chunk and every attention range waits only for its own rows.

@@ -361,14 +361,15 @@ def test_bad_block_index_is_reported_not_dereferenced():
     assert B.check_async_status()[0] == 0  # cleared
 
 
-@pytest.mark.parametrize("name,T,ws_scale", [("c1", 2048, 1.0), ("c3", 5000, 0.0), ("c3", 9001, 1.0), ("odd", 300, 1.0)])
+@pytest.mark.parametrize("name,T,ws_scale", [("c1", 2048, 1.0), ("c3", 5000, 0.0), ("c3", 9001, 1.0), ("odd", 300, 1.0),
+                                             ("c3-kv8", 5000, 0.0), ("c3-kv8", 9001, 1.0)])
 def test_host_forward_matches_device_forward(name, T, ws_scale):
     # The host-buffer form (copies overlapped with compute on a second stream, output copied
     # back range by range) must give exactly what the device form gives.
     if name == "odd":
         cfg = MSAConfig("odd", "prefill", T, 4, 2, 8, 3, head_dim=32, idx_dim=16, seed=1)  # generic kernels
     else:
-        cfg = CONFIGS[name].scaled(name=name + "-host", T=T)
+        cfg = CONFIGS[name[:2]].scaled(name=name + "-host", T=T, kv_fp8=name.endswith("kv8"))  # kv8: K, V uploaded as fp8
     shape = B.shape_of(cfg)
     x = make_prefill_inputs(cfg, DEV, sharp=True)
     out, lse, I = api.prefill_forward(cfg, x)
