@@ -55,8 +55,8 @@ def test_c5_decode_full_batch():
 
 
 # The paper's own regime at full length (bench workloads p1m, p1m-f8, pdec-f8): fused index + Top-k,
-# G = 16 attention, fp8 index operands.
-@pytest.mark.parametrize("name", ["p1m", "p1m-f8"])
+# G = 16 attention, fp8 index operands, and prefill onto fp8 K/V caches (p1m-f8kv).
+@pytest.mark.parametrize("name", ["p1m", "p1m-f8", "p1m-f8kv"])
 def test_paper_regime_1m_sampled(name):
     stats = run_prefill_case(CONFIGS[name], True, n_sample=96)
     assert stats["exact_sets"] >= 0.995
