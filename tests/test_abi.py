@@ -81,6 +81,21 @@ def test_workspace_queries(lib):
         amn, apf = B.msa_sparse_attn_prefill_workspace_bytes(shape, cfg.T, cfg.T)
         assert 0 < amn <= apf <= pf
     assert B.msa_sparse_attn_decode_workspace_bytes(B.shape_of(CONFIGS["c5"]), 32) > 0
+    # fp8 K/V caches: room for the bf16 copies of the visible K and V rows in front of the rest,
+    # and half the K/V staging in the host-buffer call
+    for name, q_count, kv_len in (("c3", 1000, 131072), ("p1m", 1048576, 1048576), ("c1", 7, 100)):
+        cfg = CONFIGS[name]
+        s16, s8 = B.shape_of(cfg), B.shape_of(cfg.scaled(kv_fp8=True))
+        copies = 2 * ((kv_len * cfg.n_kv_heads * cfg.head_dim * 2 + 255) // 256 * 256)
+        a16 = B.msa_sparse_attn_prefill_workspace_bytes(s16, q_count, kv_len)
+        a8 = B.msa_sparse_attn_prefill_workspace_bytes(s8, q_count, kv_len)
+        assert a8 == (a16[0] + copies, a16[1] + copies)
+    s16, s8 = B.shape_of(CONFIGS["c3"]), B.shape_of(CONFIGS["c3"].scaled(kv_fp8=True))
+    T = CONFIGS["c3"].T
+    kv_bytes = T * 8 * 128
+    h16, h8 = B.msa_prefill_forward_host_workspace_bytes(s16, T), B.msa_prefill_forward_host_workspace_bytes(s8, T)
+    f16, f8 = B.msa_prefill_forward_workspace_bytes(s16, T), B.msa_prefill_forward_workspace_bytes(s8, T)
+    assert h8[0] - f8[0] == h16[0] - f16[0] - 2 * kv_bytes
     # a workspace below the minimum is refused before any launch
     shape = B.shape_of(CONFIGS["c2"])
     one = ctypes.c_void_p(256)  # non-null, never dereferenced on this path
