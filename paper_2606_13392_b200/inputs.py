@@ -87,6 +87,10 @@ CONFIGS: Dict[str, MSAConfig] = {
     # (inputs still larger than L2).
     "c3-16k": MSAConfig("c3-16k", "prefill", 16384, 64, 8, 128, 64, seed=2,
                         planted_frac=0.05, planted_shift=2.0),
+    # 320 query tiles: the smallest length at which index scoring runs in its full-size form (all
+    # eight index heads of a query tile in one CTA).
+    "c3-40k": MSAConfig("c3-40k", "prefill", 40960, 64, 8, 128, 64, seed=2,
+                        planted_frac=0.05, planted_shift=2.0),
     # Decode with the K/V caches stored in fp8 E4M3 (C5's shapes), with the cached index keys in fp8 as
     # well (c5-f8), and the paper's regime with both in fp8.
     "c5-kv8": MSAConfig("c5-kv8", "decode", 1048576, 64, 8, 128, 64, seed=4,
