@@ -168,19 +168,29 @@ def oracle_sample_size(cfg: MSAConfig) -> int:
 
 
 # ----------------------------------------------------------------------------- main
-# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the stage kernels,
-# from the ncu captures summarised under profiles/ (c3, c4: one-pass captures at full size; c5:
-# captured on the reduced workload named there and scaled to a full launch by the bytes streamed,
-# which the traffic is proportional to).  None = not captured.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    # c4: captured at full size with a one-pass metric set (profiles/launch_list_and_dram_c4.md)
-    ("c4", "index_scores"): 38.85e9, ("c4", "topk_select"): 17.89e9,
-    # (attention: 18.5 GB read + 33.7 GB written; half of the Q gathers hit L2)
-    ("c4", "attn_prefill"): 52.2e9, ("c4", "combine"): 34.30e9,
-    # c3: captured at full size with the same one-pass metric set (profiles/launch_list_and_dram_c4.md)
-    ("c3", "attn_prefill"): 39.96e9, ("c3", "combine"): 27.55e9,
-    # c5: c5-small captures scaled by the selected K/V (resp. cached index keys) streamed
-    ("c5", "attn_decode"): 1.106e9, ("c5", "index_scores_decode"): 2.47e9,
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the stage kernels, from
+# ncu captures.  Every entry says what was captured (workload, kernel form) and how it was brought
+# to a full launch of the benchmarked workload: "scale" multiplies the captured bytes by the ratio
+# of the units the two launches process (traffic grows in proportion to them).  An entry goes
+# stale when its kernel changes; `kernel` names the form that was captured so that this shows.
+NCU_TRAFFIC = {
+    ("c4", "index_scores"): {"bytes": 38.85e9, "captured": "c4, one 32768-query chunk",
+                             "kernel": "index_scores_tc_kernel<128,8,1,3>", "scale": 1.0},
+    ("c4", "topk_select"): {"bytes": 17.89e9, "captured": "c4, one 32768-query chunk",
+                            "kernel": "topk_select_kernel<2>", "scale": 1.0},
+    # attention: 18.5 GB read + 33.7 GB written per query range; half of the Q gathers hit L2
+    ("c4", "attn_prefill"): {"bytes": 52.2e9, "captured": "c4, one query range",
+                             "kernel": "attn_prefill_tc_kernel<128,8>, one CTA per SM", "scale": 1.0},
+    ("c4", "combine"): {"bytes": 34.30e9, "captured": "c4, one query range", "kernel": "combine_kernel<128,8>",
+                        "scale": 1.0},
+    ("c3", "attn_prefill"): {"bytes": 39.96e9, "captured": "c3, one query range",
+                             "kernel": "attn_prefill_tc_kernel<128,8>, one CTA per SM", "scale": 1.0},
+    ("c3", "combine"): {"bytes": 27.55e9, "captured": "c3, one query range", "kernel": "combine_kernel<128,8>",
+                        "scale": 1.0},
+    ("c5", "attn_decode"): {"bytes": 1.106e9, "captured": "c5-small (8 x 32K + 8 x 128K tokens)",
+                            "kernel": "attn_decode_kernel<128,8>", "scale": "selected K/V bytes streamed, c5 / c5-small"},
+    ("c5", "index_scores_decode"): {"bytes": 2.47e9, "captured": "c5-small", "kernel": "index_scores_decode_kernel<8,2>",
+                                    "scale": "cached index keys streamed, c5 / c5-small"},
 }
 
 
@@ -267,14 +277,15 @@ def topk_table(B, dev, peaks):
         seq_lens = torch.full((batch,), n_scores * Bk + 1, dtype=torch.int32, device=dev)
         idx = torch.empty((batch, H_kv, k + 1), dtype=torch.int32, device=dev)
         stream = torch.cuda.current_stream()
+        max_len = n_scores * Bk + 1
         for _ in range(3):
-            B.msa_topk_select_decode(shape, scores, ld, seq_lens, batch, idx)
+            B.msa_topk_select_decode(shape, scores, ld, seq_lens, batch, max_len, idx)
         torch.cuda.synchronize()
         reps = 10
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(reps):
-            B.msa_topk_select_decode(shape, scores, ld, seq_lens, batch, idx)
+            B.msa_topk_select_decode(shape, scores, ld, seq_lens, batch, max_len, idx)
         e1.record(stream)
         torch.cuda.synchronize()
         us = e0.elapsed_time(e1) / reps * 1e3
@@ -470,12 +481,29 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
             else:
                 ach = work / (per_step_ms * 1e-3) / 1e9
                 ent.update(bound="hbm", achieved=ach, unit="GB/s", peak=hbm, frac=ach / hbm)
-            tr = NCU_TRAFFIC_BYTES_PER_LAUNCH.get((cfg.name, name))
-            ent["traffic"] = tr
+            tr = NCU_TRAFFIC.get((cfg.name, name))
+            ent["traffic"] = tr["bytes"] if tr else None
+            if tr:
+                ent["traffic_source"] = {k: v for k, v in tr.items() if k != "bytes"}
+                # measured DRAM bytes over the measured time: the fraction of the copy bandwidth the
+                # kernel really draws (the algorithmic figure above counts bytes that L2 may serve)
+                per_launch_ms = per_step_ms / max(n / steps, 1e-9)
+                ent["dram_gbs"] = tr["bytes"] / (per_launch_ms * 1e-3) / 1e9
+                ent["dram_frac"] = ent["dram_gbs"] / hbm
+            if ent["frac"] > 1.0:
+                ent["note"] = ("above 1.0: the numerator is algorithmic work; part of it is served from L2, and the "
+                               "denominator is a measured copy / cuBLAS rate, not a hardware limit")
         kern[name] = ent
     if cfg.mode == "prefill" and "attn_prefill" in kern:
         kern["attn_prefill"]["tensor_tflops"] = w["attn_flops"] / (kern["attn_prefill"]["ms_per_step"] * 1e-3) / 1e12
         kern["attn_prefill"]["tensor_frac_of_sustained_peak"] = kern["attn_prefill"]["tensor_tflops"] / tf_s
+        kern["attn_prefill"]["tensor_frac_of_burst_peak"] = kern["attn_prefill"]["tensor_tflops"] / tf_b
+        if "combine" in kern:  # Eq. 8 end to end: the partials' pass and their merge as one stage
+            both = kern["attn_prefill"]["ms_per_step"] + kern["combine"]["ms_per_step"]
+            tfl = w["attn_flops"] / (both * 1e-3) / 1e12
+            kern["attn_plus_combine"] = {"ms_per_step": both, "tensor_tflops": tfl,
+                                         "tensor_frac_of_sustained_peak": tfl / tf_s,
+                                         "tensor_frac_of_burst_peak": tfl / tf_b}
     dom = max((n for n in kern if "bound" in kern[n]), key=lambda n: kern[n]["ms_per_step"], default=None)
     if dom is not None:
         d = kern[dom]
@@ -548,7 +576,7 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
     if e2e:
         del out, lse, ws
         torch.cuda.empty_cache()
-        line["e2e"] = run_e2e(cfg, shape, x, B, dev, min(steps, 3), world)
+        line["e2e"] = run_e2e(cfg, shape, x, B, dev, max(5, min(steps, 10)), world)
 
     # ---- the oracle on this machine's host cores (bounded sample)
     if cpu:

@@ -27,11 +27,14 @@
  *   - Fast kernels are specialised for d_h = 128, d_idx in {64,128}, B_k in {64,128},
  *     G in {8,16} (decode index scoring: H_kv <= 8); other shapes (d_h, d_idx multiples
  *     of 8, d_h <= 256, d_idx <= 128) run on generic kernels.  k is limited to 1..128.
- *   - Host threads: the library keeps a little state per process (the pool of CUDA events
- *     and the copy stream of the *_host calls, the profiling hooks, cached kernel
- *     attributes per device).  Calls from several host threads must be serialised by the
- *     caller; calls on different streams from one thread are fine, but two calls that are
- *     in flight at the same time must not share a workspace.
+ *   - State the library keeps: per device, a ring of CUDA events, the copy stream of the
+ *     *_host calls, the four side streams of msa_prefill_forward_varlen, cached kernel
+ *     attributes, and ONE async status word (a device global, not part of any workspace:
+ *     two callers sharing a device cannot tell whose kernel set it; whoever reads it clears
+ *     it); per process, the profiling hooks (their events belong to the device that was
+ *     current at the first msa_profile_begin).  Calls from several host threads must be
+ *     serialised by the caller; calls on different streams from one thread are fine, but
+ *     two calls that are in flight at the same time must not share a workspace.
  *   - Beyond the four stage calls there are: whole-path calls (msa_prefill_forward,
  *     msa_prefill_forward_varlen, msa_decode_forward and their *_host forms), the fused
  *     Eq. 6 + Eq. 7 call msa_index_topk_fused (top_k <= 16), and the index branch's
@@ -121,6 +124,17 @@ msa_status_t msa_index_scores(const msa_shape_t* shape, const void* q_idx, const
  * scores [batch,H_kv,ld_scores]: columns [0, ceil(seq_lens[s]/B_k)) are written with the
  * Eq. 6 values, columns up to ceil(max_seq_len/B_k) with -inf.
  */
+/*
+ * Which kernel msa_index_scores runs for a range of q_count rows of a kv_len-token sequence on
+ * the current device (the paper has no counterpart: a query for tests and tuning).  *tensor_core
+ * is 1 for the tcgen05 kernel (d_idx in {64,128}, B_k in {64,128}, at least 32 rows), 0 for the
+ * generic kernel; *heads_per_cta is the number of index heads that share one key tile in a CTA of
+ * the tensor-core kernel (8, 4, 2 or 1: the most that divides H_kv and still leaves two CTAs per
+ * SM), 0 for the generic kernel.  Either pointer may be NULL.  Launches nothing.
+ */
+msa_status_t msa_index_scores_plan(const msa_shape_t* shape, int64_t q_count, int64_t kv_len,
+                                   int32_t* tensor_core, int32_t* heads_per_cta);
+
 msa_status_t msa_index_scores_decode(const msa_shape_t* shape, const void* q_idx,
                                      const void* k_idx_cache, const int64_t* seq_offsets,
                                      const int32_t* seq_lens, int32_t batch,
@@ -139,10 +153,15 @@ msa_status_t msa_topk_select(const msa_shape_t* shape, const float* scores, int6
                              int64_t q_begin, int64_t q_count, int64_t kv_len,
                              int32_t* block_idx, msa_stream_t stream);
 
-/* Stage 2 for batched decode: row (s, r) ranks blocks of sequence s, loc = (seq_lens[s]-1)/B_k. */
+/*
+ * Stage 2 for batched decode: row (s, r) ranks blocks of sequence s, loc = (seq_lens[s]-1)/B_k.
+ * max_seq_len bounds every seq_lens[s] (as in msa_index_scores_decode); ld_scores must hold
+ * ceil(max_seq_len/B_k) columns, else MSA_ERR_INVALID_ARG.  A device-side seq_lens[s] beyond
+ * ld_scores*B_k is not read past the row: its list is all -1 and the async status reports a bad index.
+ */
 msa_status_t msa_topk_select_decode(const msa_shape_t* shape, const float* scores,
                                     int64_t ld_scores, const int32_t* seq_lens, int32_t batch,
-                                    int32_t* block_idx, msa_stream_t stream);
+                                    int64_t max_seq_len, int32_t* block_idx, msa_stream_t stream);
 
 /* ------------------------------------------------------------------------------------
  * Stage 3, prefill - Eq. 8 (Algorithm 1, line 5): for each query of the range and each
@@ -237,8 +256,8 @@ msa_status_t msa_index_topk_fused(const msa_shape_t* shape, const void* q_idx, c
  * q_idx [q_count,H_kv,d_idx] bf16 (rows of the range), k_idx [kv_len,d_idx] bf16, block_idx
  * [q_count,H_kv,k] int32 as written by msa_topk_select (entries < 0 are padding), lse_idx
  * [q_count,H_kv] float32 (out; -inf for a row with no valid entry).  Runs after Top-k, KV-outer
- * over the (block, head) tiles like the attention, on warp-level tensor-core MMAs for
- * d_idx in {64,128} and B_k in {64,128}; any other shape takes a plain kernel that needs no
+ * over the (block, head) tiles like the attention, on tcgen05 MMAs (items of 128 queries x one
+ * key block) for d_idx in {64,128} and B_k in {64,128}; any other shape takes a plain kernel that needs no
  * workspace.  workspace >= msa_index_lse_prefill_workspace_bytes (device, 16-byte aligned).
  * Errors as msa_sparse_attn_prefill; a block index outside [-1, loc] sets the async status.
  */
@@ -343,6 +362,18 @@ msa_status_t msa_decode_forward_host(const msa_shape_t* shape, const void* q_hos
                                      void* out_host, void* workspace, size_t workspace_bytes,
                                      msa_stream_t stream);
 
+/*
+ * Test hook for the device-side bounded waits (the paper has no counterpart).  Every wait of a
+ * kernel on an mbarrier gives up after a limit of SM cycles (about two seconds by default),
+ * raises MSA_ERR_TIMEOUT in the async status and lets the kernel unwind and return.
+ * wait_limit_cycles sets that limit for the kernels launched afterwards on the current device
+ * (0 or anything above the default restores the default); producer_delay_cycles (at most 1e8)
+ * makes the warp that issues the copies of the tensor-core prefill kernels (index scoring,
+ * attention) sit out that many cycles before its first copy, so that a short limit runs out on a
+ * role that is merely late.  Both values stay until changed; production code never calls this.
+ */
+msa_status_t msa_debug_set_wait(int64_t wait_limit_cycles, int64_t producer_delay_cycles);
+
 /* Number of kernel launches the library has enqueued since the process started. */
 int64_t msa_launch_count(void);
 
@@ -354,7 +385,7 @@ int64_t msa_launch_count(void);
  * (arrays of 9: 0 index scoring, 1 top-k, 2 reverse index/schedule, 3 prefill attention,
  * 4 combine, 5 decode index scoring, 6 decode attention, 7 decode combine, 8 index-branch
  * log-sum-exp).  The first
- * msa_profile_begin() creates the event pool (8192 launches); MSA_ERR_UNSUPPORTED from
+ * msa_profile_begin() creates the event pool (16384 launches); MSA_ERR_UNSUPPORTED from
  * msa_profile_end() means the pool ran out and the sums are partial.  Not thread-safe.
  */
 msa_status_t msa_profile_begin(void);

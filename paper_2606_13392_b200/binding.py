@@ -32,7 +32,7 @@ EXPORTS = [
     "msa_prefill_forward_workspace_bytes", "msa_prefill_forward_varlen",
     "msa_prefill_forward_varlen_workspace_bytes", "msa_prefill_forward_host",
     "msa_prefill_forward_host_workspace_bytes", "msa_decode_forward", "msa_decode_forward_host",
-    "msa_launch_count", "msa_profile_begin", "msa_profile_end",
+    "msa_launch_count", "msa_profile_begin", "msa_profile_end", "msa_index_scores_plan", "msa_debug_set_wait",
 ]
 
 
@@ -170,10 +170,24 @@ def msa_topk_select(shape, scores, ld_scores, q_begin, q_count, kv_len, block_id
            "msa_topk_select")
 
 
-def msa_topk_select_decode(shape, scores, ld_scores, seq_lens, batch, block_idx, stream=None):
+def msa_topk_select_decode(shape, scores, ld_scores, seq_lens, batch, max_seq_len, block_idx, stream=None):
     _check(lib().msa_topk_select_decode(ctypes.byref(shape), _dev(scores), c_i64(ld_scores),
-                                        _dev(seq_lens), c_i32(batch), _dev(block_idx),
+                                        _dev(seq_lens), c_i32(batch), c_i64(max_seq_len), _dev(block_idx),
                                         _stream(stream)), "msa_topk_select_decode")
+
+
+def msa_index_scores_plan(shape, q_count, kv_len) -> Tuple[bool, int]:
+    """(runs on the tensor cores?, index heads per CTA) for msa_index_scores on the current device."""
+    tc, nh = c_i32(0), c_i32(0)
+    _check(lib().msa_index_scores_plan(ctypes.byref(shape), c_i64(q_count), c_i64(kv_len), ctypes.byref(tc),
+                                       ctypes.byref(nh)), "msa_index_scores_plan")
+    return bool(tc.value), int(nh.value)
+
+
+def msa_debug_set_wait(wait_limit_cycles: int = 0, producer_delay_cycles: int = 0) -> None:
+    """Test hook: shortens the device-side bounded waits (0 = the production limit) and makes the
+    copy-issuing role of the tensor-core kernels start late by the given number of SM cycles."""
+    _check(lib().msa_debug_set_wait(c_i64(wait_limit_cycles), c_i64(producer_delay_cycles)), "msa_debug_set_wait")
 
 
 def msa_sparse_attn_prefill_workspace_bytes(shape, q_count, kv_len) -> Tuple[int, int]:

@@ -213,6 +213,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const uint64_t pol_q = l2_policy_evict_last(), pol_kv = l2_policy_evict_first();
         int loaded_tile = -1, tile_seq = -1, n = 0;
         bool ok = true;
+        if (const long long late = g_debug_producer_delay; late > 0) spin_cycles(late);  // tests only
         for (int ph = 0; ph < phases && ok; ++ph) {
             int it_lo, it_hi;
             phase_items(item_off, p, ph, it_lo, it_hi);

@@ -176,6 +176,14 @@ struct DecParams {
     float scale_log2e;
 };
 
+// A register of a transposed V fragment holds one d of two consecutive keys (`key` in the low
+// half, `key + 1` in the high half).  Keys past `lim` are not part of the sequence: their P is
+// exactly 0, but the cache rows there may be uninitialised (NaN or Inf), and 0 * NaN is NaN, so
+// their V values are replaced with zeros.
+__device__ __forceinline__ uint32_t keep_visible_pair(uint32_t v, int key, int lim) {
+    return (key <= lim ? (v & 0x0000FFFFu) : 0u) | (key + 1 <= lim ? (v & 0xFFFF0000u) : 0u);
+}
+
 // 16-byte chunk `chunk` (0..15 over d) of key row `key` inside a swizzled K or V tile.
 template <int BK>
 __device__ __forceinline__ uint32_t dec_tile_addr(uint32_t tile_base, int key, int chunk) {
@@ -356,6 +364,11 @@ attn_decode_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_consta
                         const int key = w * KPW + ks * 16 + (i >> 1) * 8 + (lane & 7);
                         uint32_t r4[4];
                         ldmatrix_x4_trans(r4, dec_tile_addr<BK>(tb, key, mt * 2 + (i & 1)));
+                        if (lim < BK - 1) {  // local block: rows past the sequence's end may hold anything
+                            const int k0 = w * KPW + ks * 16 + 2 * t;
+                            r4[0] = keep_visible_pair(r4[0], k0, lim); r4[1] = keep_visible_pair(r4[1], k0, lim);
+                            r4[2] = keep_visible_pair(r4[2], k0 + 8, lim); r4[3] = keep_visible_pair(r4[3], k0 + 8, lim);
+                        }
 #pragma unroll
                         for (int hg = 0; hg < HG; ++hg)
                             mma_m16n8k16_bf16(acc[hg][mt], r4[0], r4[1], r4[2], r4[3], pb[hg][ks][0], pb[hg][ks][1]);

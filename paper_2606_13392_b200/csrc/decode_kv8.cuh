@@ -270,7 +270,12 @@ attn_decode_kv8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_co
                         ldmatrix_x4_trans(r4, dec_kv8_addr(tb, key, mp * 2 + (i >> 1)));
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
-                            const uint32_t lo = r4[half * 2], hi = r4[half * 2 + 1];  // keys 2t, 2t+1 and 8 + 2t, 8 + 2t + 1
+                            uint32_t lo = r4[half * 2], hi = r4[half * 2 + 1];  // keys 2t, 2t+1 and 8 + 2t, 8 + 2t + 1
+                            if (lim < BK - 1) {  // local block: bytes past the sequence's end may decode to NaN
+                                const int k0 = w * KPW + ks * 16 + 2 * t;
+                                lo = keep_visible_pair(lo, k0, lim);
+                                hi = keep_visible_pair(hi, k0 + 8, lim);
+                            }
                             // bytes (key 2t: d even, d odd; key 2t+1: d even, d odd) -> (d even: both keys; d odd: both keys)
                             uint32_t a0, a1, a2, a3;
                             e4m3x4_to_f16x2x2(__byte_perm(lo, 0u, 0x3120), a0, a1);

@@ -90,6 +90,7 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
     if (warp == 0) {
         if (lane == 0) {
+            if (const long long late = g_debug_producer_delay; late > 0) spin_cycles(late);  // tests only
             mbar_arrive_expect_tx(&sm.a_full, NH * DI * kIdxTileQ * 128);
             for (int h = 0; h < NH; ++h)
                 for (int a = 0; a < DI; ++a) tma_load_3d(sm.a[h][a], &tm_q, a * 64, r0 + h, (int)q0, &sm.a_full);

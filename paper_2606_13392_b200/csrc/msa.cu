@@ -172,14 +172,19 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
 // Heads sharing one key tile per CTA: the most (8, 4, 2, 1; at most 2 when d_idx = 128, for
 // shared memory) that divide H_kv and still leave at least two CTAs per SM, so that short
 // chunks keep the machine full.
+static int index_heads_per_cta(const Resolved& r, int64_t q_count) {
+    const int64_t n_qtiles = ceil_div64(q_count, kIdxTileQ);
+    const bool one_atom = r.idx_fp8 || r.d_idx == 64;  // the index vector is one 128-byte atom
+    for (int cand = one_atom ? 8 : 2; cand > 1; cand >>= 1)
+        if (r.H_kv % cand == 0 && n_qtiles * (r.H_kv / cand) >= 2 * sm_count()) return cand;
+    return 1;
+}
+
 template <int BK, int DI, bool F8 = false>
 static msa_status_t launch_index_tc_bk(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                        int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
                                        int64_t n_cols, cudaStream_t st) {
-    const int64_t n_qtiles = ceil_div64(q_count, kIdxTileQ);
-    int nh = 1;
-    for (int cand = (DI == 1 ? 8 : 2); cand > 1; cand >>= 1)
-        if (r.H_kv % cand == 0 && n_qtiles * (r.H_kv / cand) >= 2 * sm_count()) { nh = cand; break; }
+    const int nh = index_heads_per_cta(r, q_count);
     if constexpr (DI == 1) {
         if (nh == 8) return launch_index_tc<BK, 8, DI, 0, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
         if (nh == 4) return launch_index_tc<BK, 4, DI, 0, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
@@ -222,11 +227,17 @@ static msa_status_t run_index_topk_fused(const Resolved& r, const void* q_idx, c
     return launch_index_fused_bk<128, 2>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
 }
 
+// Prefill ranges of at least 32 rows run on the tensor cores; shorter ones (and decode rows of
+// shapes without a streaming kernel) take the generic kernel.
+static bool index_scores_on_tc(const Resolved& r, int64_t n_rows, int64_t kv_len) {
+    return index_tc_ok(r) && kv_len < 2147483647LL && n_rows >= 32;
+}
+
 static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const void* k_idx,
                                      const RowMap& rows, int64_t n_rows, float* scores,
                                      int64_t ld_scores, cudaStream_t st) {
     if (n_rows == 0 || rows.n_cols == 0) return MSA_OK;
-    if (rows.seq_lens == nullptr && index_tc_ok(r) && rows.kv_len < 2147483647LL && n_rows >= 32) {
+    if (rows.seq_lens == nullptr && index_scores_on_tc(r, n_rows, rows.kv_len)) {
         const int64_t qb = rows.q_begin, kl = rows.kv_len, nc = rows.n_cols;
         if (r.idx_fp8) {
             if (r.B_k == 64) return launch_index_tc_bk<64, 1, true>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
@@ -265,13 +276,15 @@ static msa_status_t run_topk(const Resolved& r, const float* scores, int64_t ld_
     const int64_t grid = ceil_div64(n_rows, kTopkWarps);
     if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
     const dim3 g((unsigned)grid), b(kTopkWarps * 32);
+    int* status = async_status_ptr();
+    if (status == nullptr) return MSA_ERR_CUDA;
     StageScope sc(kStageTopk, st);
     if (r.k <= 32)
-        topk_select_kernel<1><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx);
+        topk_select_kernel<1><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx, status);
     else if (r.k <= 64)
-        topk_select_kernel<2><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx);
+        topk_select_kernel<2><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx, status);
     else
-        topk_select_kernel<4><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx);
+        topk_select_kernel<4><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx, status);
     return launch_status();
 }
 
@@ -386,7 +399,9 @@ struct HostInHook {
     bool on = false;
     int64_t piece_rows = 0;
     int n_pieces = 0;
-    cudaEvent_t ev[256];
+    cudaEvent_t ev[256];            // the hook's own events (not drawn from the shared ring, whose
+    int created[64] = {0};          // cursor may wrap during a long call); created per device
+    cudaEvent_t own[64][256];
 };
 static cudaEvent_t next_sync_event();
 static HostInHook g_in_hook;      // Q rows, waited for by the attention of each query range
@@ -404,10 +419,15 @@ static msa_status_t upload_in_pieces(HostInHook& h, char* dst, const void* src, 
     while (ceil_div64(rows, piece) > 256) piece *= 2;
     h.piece_rows = piece;
     h.n_pieces = (int)ceil_div64(rows, piece);
+    const int dev = current_device();
     for (int i = 0; i < h.n_pieces; ++i) {
         const int64_t r0 = (int64_t)i * piece, n = (rows - r0) < piece ? (rows - r0) : piece;
-        h.ev[i] = next_sync_event();
-        if (!h.ev[i] ||
+        if (i >= h.created[dev]) {
+            if (cudaEventCreateWithFlags(&h.own[dev][i], cudaEventDisableTiming) != cudaSuccess) return MSA_ERR_CUDA;
+            h.created[dev] = i + 1;
+        }
+        h.ev[i] = h.own[dev][i];
+        if (
             cudaMemcpyAsync(dst + (size_t)r0 * row_bytes, (const char*)src + (size_t)r0 * row_bytes, (size_t)n * row_bytes,
                             cudaMemcpyHostToDevice, copy) != cudaSuccess ||
             cudaEventRecord(h.ev[i], copy) != cudaSuccess)
@@ -416,16 +436,19 @@ static msa_status_t upload_in_pieces(HostInHook& h, char* dst, const void* src, 
     return MSA_OK;
 }
 
+// A ring of events per device for orderings that are consumed at once (record on one stream, wait on
+// another, in the same call): an event may be re-recorded as soon as the wait has been enqueued.
 static cudaEvent_t next_sync_event() {
     constexpr int kPool = 2048;
-    static cudaEvent_t pool[kPool];
-    static int created = 0, cursor = 0;
-    if (created < kPool && cursor == created) {
-        if (cudaEventCreateWithFlags(&pool[created], cudaEventDisableTiming) != cudaSuccess) return nullptr;
-        ++created;
+    static cudaEvent_t pool[64][kPool];
+    static int created[64] = {0}, cursor[64] = {0};
+    const int dev = current_device();
+    if (created[dev] < kPool && cursor[dev] == created[dev]) {
+        if (cudaEventCreateWithFlags(&pool[dev][created[dev]], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        ++created[dev];
     }
-    cudaEvent_t e = pool[cursor];
-    cursor = (cursor + 1) % kPool;
+    cudaEvent_t e = pool[dev][cursor[dev]];
+    cursor[dev] = (cursor[dev] + 1) % kPool;
     return e;
 }
 
@@ -795,6 +818,32 @@ msa_status_t msa_index_scores(const msa_shape_t* shape, const void* q_idx, const
                             ld_scores, (cudaStream_t)stream);
 }
 
+msa_status_t msa_index_scores_plan(const msa_shape_t* shape, int64_t q_count, int64_t kv_len,
+                                   int32_t* tensor_core, int32_t* heads_per_cta) {
+    Resolved r;
+    msa_status_t s = resolve(shape, r);
+    if (s != MSA_OK) return s;
+    if (q_count < 0 || kv_len < 0 || q_count > kv_len) return MSA_ERR_INVALID_ARG;
+    const bool tc = q_count > 0 && index_scores_on_tc(r, q_count, kv_len);
+    if (tensor_core) *tensor_core = tc ? 1 : 0;
+    if (heads_per_cta) *heads_per_cta = tc ? index_heads_per_cta(r, q_count) : 0;
+    return MSA_OK;
+}
+
+msa_status_t msa_debug_set_wait(int64_t wait_limit_cycles, int64_t producer_delay_cycles) {
+    if (wait_limit_cycles < 0 || producer_delay_cycles < 0) return MSA_ERR_INVALID_ARG;
+    // Never longer than the production limit, and a delay well inside it: a test can shorten a
+    // wait, it cannot turn a kernel into one that runs for long.
+    const long long limit = (wait_limit_cycles == 0 || wait_limit_cycles > kWaitLimitCycles)
+                                ? kWaitLimitCycles : (long long)wait_limit_cycles;
+    if (producer_delay_cycles > 100000000LL) return MSA_ERR_INVALID_ARG;  // 50 ms
+    const long long late = (long long)producer_delay_cycles;
+    if (cudaMemcpyToSymbol(g_wait_limit_cycles, &limit, sizeof(limit)) != cudaSuccess ||
+        cudaMemcpyToSymbol(g_debug_producer_delay, &late, sizeof(late)) != cudaSuccess)
+        return MSA_ERR_CUDA;
+    return MSA_OK;
+}
+
 msa_status_t msa_index_topk_fused(const msa_shape_t* shape, const void* q_idx, const void* k_idx,
                                   int64_t q_begin, int64_t q_count, int64_t kv_len, int32_t* block_idx,
                                   msa_stream_t stream) {
@@ -843,15 +892,16 @@ msa_status_t msa_topk_select(const msa_shape_t* shape, const float* scores, int6
 }
 
 msa_status_t msa_topk_select_decode(const msa_shape_t* shape, const float* scores, int64_t ld_scores,
-                                    const int32_t* seq_lens, int32_t batch, int32_t* block_idx,
-                                    msa_stream_t stream) {
+                                    const int32_t* seq_lens, int32_t batch, int64_t max_seq_len,
+                                    int32_t* block_idx, msa_stream_t stream) {
     Resolved r;
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
-    if (batch < 0) return MSA_ERR_INVALID_ARG;
+    if (batch < 0 || max_seq_len < 0) return MSA_ERR_INVALID_ARG;
     if (batch == 0) return MSA_OK;
     if (!scores || !block_idx || !seq_lens || !aligned16(scores) || ld_scores % 4 != 0 || ld_scores <= 0)
         return MSA_ERR_INVALID_ARG;
+    if (ld_scores < ceil_div64(max_seq_len, r.B_k)) return MSA_ERR_INVALID_ARG;
     RowMap rows = decode_rows(nullptr, seq_lens, 0, r.B_k);  // offsets are not needed for ranking
     return run_topk(r, scores, ld_scores, rows, batch, block_idx, (cudaStream_t)stream);
 }
@@ -1237,7 +1287,8 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
     const size_t q_row = (size_t)r.H_q * r.d * 2, kv_row = (size_t)r.H_kv * r.d * r.kv_elt();
     const size_t qi_row = (size_t)r.H_kv * r.d_idx * r.idx_elt(), ki_row = (size_t)r.d_idx * r.idx_elt();
     cudaStream_t st = (cudaStream_t)stream;
-    static cudaStream_t lanes[kVarlenLanes] = {};
+    static cudaStream_t lanes_dev[64][kVarlenLanes] = {};
+    cudaStream_t* lanes = lanes_dev[current_device()];
     const size_t slice = (workspace_bytes / kVarlenLanes) & ~(size_t)(kAlign - 1);
     bool forked[kVarlenLanes] = {};   // lanes that hold work since the last join
     cudaEvent_t fork_ev = nullptr;    // marks the caller's stream after the last join
@@ -1321,11 +1372,37 @@ msa_status_t msa_prefill_forward_host_workspace_bytes(const msa_shape_t* shape, 
     return MSA_OK;
 }
 
+static msa_status_t prefill_forward_host_body(const msa_shape_t* shape, const void* q_host,
+                                              const void* k_host, const void* v_host,
+                                              const void* q_idx_host, const void* k_idx_host, int64_t T,
+                                              void* out_host, float* lse_host, int32_t* block_idx_host,
+                                              void* workspace, size_t workspace_bytes, msa_stream_t stream,
+                                              cudaStream_t* copy_used);
+
 msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_host,
                                       const void* k_host, const void* v_host,
                                       const void* q_idx_host, const void* k_idx_host, int64_t T,
                                       void* out_host, float* lse_host, int32_t* block_idx_host,
                                       void* workspace, size_t workspace_bytes, msa_stream_t stream) {
+    cudaStream_t copy = nullptr;
+    const msa_status_t s = prefill_forward_host_body(shape, q_host, k_host, v_host, q_idx_host, k_idx_host, T, out_host,
+                                                     lse_host, block_idx_host, workspace, workspace_bytes, stream, &copy);
+    g_in_idx_hook.on = false; g_in_hook.on = false; g_out_hook.on = false;
+    if (s != MSA_OK && copy != nullptr) {
+        // Copies from and to the caller's host buffers may be in flight: the buffers are the
+        // caller's again only once both streams have drained.
+        cudaStreamSynchronize((cudaStream_t)stream);
+        cudaStreamSynchronize(copy);
+    }
+    return s;
+}
+
+static msa_status_t prefill_forward_host_body(const msa_shape_t* shape, const void* q_host,
+                                              const void* k_host, const void* v_host,
+                                              const void* q_idx_host, const void* k_idx_host, int64_t T,
+                                              void* out_host, float* lse_host, int32_t* block_idx_host,
+                                              void* workspace, size_t workspace_bytes, msa_stream_t stream,
+                                              cudaStream_t* copy_used) {
     Resolved r;
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
@@ -1342,8 +1419,10 @@ msa_status_t msa_prefill_forward_host(const msa_shape_t* shape, const void* q_ho
     // A second stream carries the copies: the index inputs go first so that stages 1-2 start
     // while Q, K and V are still on their way; each finished query range of O is copied back
     // while the next one is computed.
-    static cudaStream_t copy = nullptr;
+    static cudaStream_t copy_dev[64] = {};
+    cudaStream_t& copy = copy_dev[current_device()];
     if (copy == nullptr && cudaStreamCreateWithFlags(&copy, cudaStreamNonBlocking) != cudaSuccess) return MSA_ERR_CUDA;
+    *copy_used = copy;
     cudaEvent_t e_in = next_sync_event(), e_idx = next_sync_event(), e_kv = next_sync_event();
     if (!e_in || !e_idx || !e_kv) return MSA_ERR_CUDA;
     if (cudaEventRecord(e_in, st) != cudaSuccess || cudaStreamWaitEvent(copy, e_in, 0) != cudaSuccess) return MSA_ERR_CUDA;
@@ -1402,7 +1481,7 @@ msa_status_t msa_decode_forward(const msa_shape_t* shape, const void* q, const v
     msa_status_t s = msa_index_scores_decode(shape, q_idx, k_idx_cache, seq_offsets, seq_lens, batch,
                                              max_seq_len, scores, ld_scores, stream);
     if (s != MSA_OK) return s;
-    s = msa_topk_select_decode(shape, scores, ld_scores, seq_lens, batch, block_idx, stream);
+    s = msa_topk_select_decode(shape, scores, ld_scores, seq_lens, batch, max_seq_len, block_idx, stream);
     if (s != MSA_OK) return s;
     return msa_sparse_attn_decode(shape, q, k_cache, v_cache, cache_tokens, seq_offsets, seq_lens,
                                   batch, block_idx, out, lse, workspace, workspace_bytes, stream);

@@ -51,15 +51,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait: gives up after ~kWaitLimitCycles SM cycles, or as soon as another role of
 // the CTA has raised *abort.  Returns false on give-up; the caller reports and unwinds.
 constexpr long long kWaitLimitCycles = 4000000000LL;  // about 2 s at 1.9 GHz
+// The limit in force (read on the slow path of a wait only) and a delay, in SM cycles, that the
+// producer role of the tensor-core kernels sits out before its first copy.  Both exist so that a
+// test can make a wait run out on a role that is merely late (msa_debug_set_wait); the defaults
+// are the production values.
+__device__ long long g_wait_limit_cycles = kWaitLimitCycles;
+__device__ long long g_debug_producer_delay = 0;
 
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
+    const long long limit = g_wait_limit_cycles;
     int spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63) == 0) {
             if (*abort != 0) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit) {
                 *abort = 1;
                 return false;
             }

@@ -323,7 +323,7 @@ struct TopkGatherStream {  // element i: block i % 8 of candidate run i / 8; blo
 template <int R>
 __global__ void __launch_bounds__(kTopkWarps * 32)
 topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap rows,
-                   int64_t n_rows, int H_kv, int B_k, int top_k, int32_t* __restrict__ block_idx) {
+                   int64_t n_rows, int H_kv, int B_k, int top_k, int32_t* __restrict__ block_idx, int* status) {
     __shared__ uint32_t stg_all[kTopkWarps][kTopkStage];
     __shared__ uint2 log_all[kTopkWarps][kTopkLog];   // (key, block) of every survivor, in index order
     __shared__ uint16_t run_all[kTopkWarps][kTopkMaxRuns + 2];
@@ -335,6 +335,11 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
     rows.get(row / H_kv, pos, len, base);
     const int64_t loc = pos / B_k;
     int32_t* orow = block_idx + row * (int64_t)top_k;
+    if (loc >= ld_scores) {  // a decode row whose length (a device value) exceeds the score pitch: nothing is read
+        if (lane == 0) report_async(status, kAsyncBadIndex, 0x201);
+        for (int e = lane; e < top_k; e += 32) orow[e] = -1;
+        return;
+    }
     if (topk_trivial_row(loc, top_k, orow, lane)) return;
     const int m = top_k - 1;  // ranked entries; candidates are blocks [0, loc), loc < 2^31
     const float* srow = scores + row * ld_scores;

@@ -324,6 +324,58 @@ def test_decode_small_batch_mixed_lengths(sharp):
     assert np.mean([r["exact"] for r in res]) >= 0.95
 
 
+@pytest.mark.parametrize("kv8,idx8,G", [(False, False, 8), (True, False, 8), (False, False, 16), (True, True, 16)])
+def test_decode_cache_slack_may_hold_anything(kv8, idx8, G):
+    # A growing cache: every sequence owns `capacity` rows of which the first seq_lens[s] are
+    # written.  The rows behind them (up to the end of the local block and beyond) hold NaN bit
+    # patterns here; the step must give exactly what it gives on a packed cache.
+    lens = (1, 100, 129, 5000, 8191, 8193, 12345)
+    cfg = CONFIGS["c5"].scaled(name="c5-slack", n_kv_heads=64 // G, seq_lens=lens, kv_fp8=kv8, idx_fp8=idx8,
+                               idx_dim=128 if idx8 else 64)
+    x = make_decode_inputs(cfg, DEV, sharp=True)
+    out, lse, I, scores = api.decode_forward(cfg, x)
+    cap = 12345 + 300
+    offs = x["seq_offsets"].cpu().numpy()
+
+    def strided(t, nan_bits):
+        wide = torch.empty((cap * len(lens),) + tuple(t.shape[1:]), dtype=t.dtype, device=DEV)
+        wide.view(torch.uint8 if t.element_size() == 1 else torch.int16).fill_(nan_bits)
+        for s_, L in enumerate(lens):
+            wide[s_ * cap: s_ * cap + L] = t[int(offs[s_]): int(offs[s_]) + L]
+        return wide
+
+    y = dict(x)
+    y["k_cache"] = strided(x["k_cache"], 0x7F if kv8 else 0x7FC0)
+    y["v_cache"] = strided(x["v_cache"], 0x7F if kv8 else 0x7FC0)
+    y["k_idx_cache"] = strided(x["k_idx_cache"], 0x7F if idx8 else 0x7FC0)
+    y["seq_offsets"] = torch.arange(len(lens), dtype=torch.int64, device=DEV) * cap
+    out2, lse2, I2, scores2 = api.decode_forward(cfg, y)
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert torch.equal(I, I2)
+    assert torch.isfinite(out2.float()).all() and torch.isfinite(lse2).all()
+    assert torch.equal(out, out2) and torch.equal(lse, lse2)
+
+
+def test_decode_topk_row_longer_than_the_score_pitch_is_reported():
+    # seq_lens is a device array: a length beyond what the score rows hold must not be read past
+    # the row.  The row's list comes back as all -1 and the status word names a bad index.
+    cfg = CONFIGS["c5"].scaled(name="c5-pitch", seq_lens=(4096, 4096))
+    shape = B.shape_of(cfg)
+    ld = B.score_ld(4096, cfg.block_size)
+    scores = torch.randn((2, cfg.n_kv_heads, ld), device=DEV)
+    lens = torch.tensor([4096, 4096 * 9], dtype=torch.int32, device=DEV)   # the second one lies
+    idx = torch.full((2, cfg.n_kv_heads, cfg.top_k), -5, dtype=torch.int32, device=DEV)
+    with pytest.raises(B.MsaError):   # the pitch cannot hold the stated maximum
+        B.msa_topk_select_decode(shape, scores, ld, lens, 2, 4096 * 9, idx)
+    B.msa_topk_select_decode(shape, scores, ld, lens, 2, 4096, idx)
+    code, _ = B.check_async_status()
+    assert code == 6  # MSA_ERR_BAD_INDEX
+    loc = 4095 // cfg.block_size   # fewer visible blocks than top_k: all of them, then padding
+    assert bool((idx[1] == -1).all()) and bool((idx[0, :, loc] == loc).all()) and bool((idx[0, :, loc + 1] == -1).all())
+    assert B.check_async_status()[0] == 0
+
+
 def test_decode_generic_shape():
     cfg = MSAConfig("dec-odd", "decode", 0, 6, 3, 16, 5, head_dim=64, idx_dim=32, seed=3,
                     seq_lens=(5, 16, 17, 400, 1000))
