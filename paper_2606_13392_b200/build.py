@@ -26,17 +26,20 @@ def _newest_source_mtime() -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compiles csrc/*.cu into libmsa_b200.so next to this file; returns its path."""
+def build_library(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
+    """Compiles csrc/*.cu into libmsa_b200.so next to this file; returns its path.
+
+    trace=True is a development build (-DMSA_TRACE): CTA 0 of the prefill attention kernel records
+    clock stamps of its roles, read back by paper_2606_13392_b200/trace.py."""
     if not force and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= _newest_source_mtime():
         return LIB_PATH
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB_PATH + ".tmp%d" % os.getpid()
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + _sources()
+    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + (["-DMSA_TRACE"] if trace else []) + ["-o", tmp] + _sources()
     subprocess.check_call(cmd)
     os.replace(tmp, LIB_PATH)
     return LIB_PATH
 
 
 if __name__ == "__main__":
-    print(build_library(force=True, verbose="-v" in sys.argv))
+    print(build_library(force=True, verbose="-v" in sys.argv, trace="--trace" in sys.argv))

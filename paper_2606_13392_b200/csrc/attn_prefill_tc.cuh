@@ -254,6 +254,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     ok = false;
                     break;
                 }
+                if (threadIdx.x == 0) MSA_STAMP(n, 12);
                 // Slot n mod 8 was last read by the epilogue of item n-8, long before S(n-2) ran.
                 AttnItemInfo& inf = sm.info[n % kAttnInfoRing];
                 if (lane < QPI && half == 0) inf.handle[lane] = h;
@@ -270,6 +271,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 if (lane >= q_lo && lane < q_hi)
                     tma_load_5d_hint(sm.q[j] + lane * Q_BYTES, &tm_q, 0, 0, 0, r * (G / 8),
                                      (int)(p.q_first + (h >> 8)), &sm.q_full[j], pol_q);
+                if (threadIdx.x == 0) MSA_STAMP(n, 13);
                 if (new_tile) {
                     // K: the buffer was the V buffer of the tile before last (or the K buffer three
                     // tiles back); V: this buffer held the previous tile's K.  One warp does all the
@@ -326,6 +328,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         break;
                     }
                     tc_fence_after();
+                    MSA_STAMP(n, 8);
                     const uint32_t ts = tmem + j * 256;
                     // Q atoms (8 rows x 64 d) of one d half are 2 KB apart; the other half sits 1 KB further.
                     const uint64_t qd0 = make_smem_desc(smem_u32(sm.q[j]), 16, 2048);
@@ -339,6 +342,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     mma_commit(&sm.q_empty[j]);
                     mma_commit(&sm.s_full[j]);
                     if (last) mma_commit(&sm.kv_empty[kb]);
+                    MSA_STAMP(n, 9);
                 }
                 if (n >= 1) {
                     const int m = n - 1, jm = m & 1;
@@ -351,6 +355,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         break;
                     }
                     tc_fence_after();
+                    MSA_STAMP(m, 10);
                     const uint32_t ts = tmem + jm * 256, to = ts + 128;
                     // V as the MN-major B operand: next 64 columns of d are BK*128 bytes away.
                     const uint64_t vd = make_smem_desc(smem_u32(sm.kv[prev_vb][0]), BK * 128, 1024);
@@ -359,6 +364,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         mma_bf16_ts(to, ts + kk * 8, vd + (uint64_t)(kk * 2048 / 16), idesc_o, kk > 0);
                     mma_commit(&sm.o_full[jm]);
                     if (prev_last) mma_commit(&sm.kv_empty[prev_vb]);
+                    MSA_STAMP(m, 11);
                 }
                 prev_vb = vb; prev_last = last; prev_new = nw;
             }
@@ -382,6 +388,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int n = j; n < n_items; n += 2) {
             if (!mbar_wait(&sm.s_full[j], (n >> 1) & 1, abort)) { report_async(status, kAsyncTimeout, 0x331); break; }
             tc_fence_after();
+            if (lane == 0 && quarter == 0) MSA_STAMP(n, 0);
             const AttnItemInfo& inf = sm.info[n % kAttnInfoRing];
             const int b = inf.block, r = inf.r, nq = inf.nq;
             const uint32_t h = inf.handle[qi];
@@ -430,6 +437,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.p_full[j]);
+            if (lane == 0 && quarter == 0) MSA_STAMP(n, 3);
 
             // ---- epilogue: O row / ell -> bf16 partial (via the staging buffer), LSE partial
             // The copies of the context's previous item have read the staging buffer long ago;
@@ -437,6 +445,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             if (lane < QPW) bulk_wait_read_all();
             if (!mbar_wait(&sm.o_full[j], (n >> 1) & 1, abort)) { report_async(status, kAsyncTimeout, 0x332); break; }
             tc_fence_after();
+            if (lane == 0 && quarter == 0) MSA_STAMP(n, 5);
             const float inv = 1.0f / ell;
             const float2 inv2 = make_float2(inv, inv);
             __syncwarp();
@@ -471,6 +480,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             }
             if (valid)
                 lse_buf[(partial_base(ql, r, p) + (h & 0xFF)) * G + g] = (mc + log2f(ell)) * 0.6931471805599453f;
+            if (lane == 0 && quarter == 0) MSA_STAMP(n, 7);
         }
         if (lane < QPW) bulk_wait_all();  // partials still on their way out
     }

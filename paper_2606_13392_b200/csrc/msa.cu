@@ -830,6 +830,13 @@ msa_status_t msa_index_scores_plan(const msa_shape_t* shape, int64_t q_count, in
     return MSA_OK;
 }
 
+#ifdef MSA_TRACE
+// Development builds only (-DMSA_TRACE): the 16 x 16 clock stamps CTA 0 of the prefill attention kernel recorded.
+extern "C" int msa_debug_read_trace(long long* host256) {
+    return cudaMemcpyFromSymbol(host256, g_trace, sizeof(long long) * 256) == cudaSuccess ? 0 : 1;
+}
+#endif
+
 msa_status_t msa_debug_set_wait(int64_t wait_limit_cycles, int64_t producer_delay_cycles) {
     if (wait_limit_cycles < 0 || producer_delay_cycles < 0) return MSA_ERR_INVALID_ARG;
     // Never longer than the production limit, and a delay well inside it: a test can shorten a

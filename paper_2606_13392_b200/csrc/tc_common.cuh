@@ -58,6 +58,20 @@ constexpr long long kWaitLimitCycles = 4000000000LL;  // about 2 s at 1.9 GHz
 __device__ long long g_wait_limit_cycles = kWaitLimitCycles;
 __device__ long long g_debug_producer_delay = 0;
 
+// Optional time stamps for kernel development (compiled in with -DMSA_TRACE only): CTA 0 records
+// clock64() of up to 16 events for 16 consecutive items starting at kTraceFirstItem.
+#ifdef MSA_TRACE
+constexpr int kTraceFirstItem = 1000;
+__device__ long long g_trace[16 * 16];
+#define MSA_STAMP(item, ev)                                                                  \
+    do {                                                                                     \
+        if (blockIdx.x == 0 && (item) >= kTraceFirstItem && (item) < kTraceFirstItem + 16)   \
+            g_trace[((item) - kTraceFirstItem) * 16 + (ev)] = clock64();                     \
+    } while (0)
+#else
+#define MSA_STAMP(item, ev) do { } while (0)
+#endif
+
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
