@@ -121,9 +121,9 @@ def index_lse(q_idx, k_idx, I, pos, block_size: int, scale: Optional[float] = No
 
 
 def sparse_attn(q, K, V, I, pos, block_size: int, scale: Optional[float] = None):
-    """Eq. 8.  q [n,H_q,d] u16, K,V [L,H_kv,d] (both u16 = bf16 or both u8 = fp8 E4M3), I [n,H_kv,k]
-    -> (O [n,H_q,d], LSE [n,H_q]) f64."""
-    q, K, V, pos = _u16(q), _idx(K), _idx(V), _pos(pos)
+    """Eq. 8.  q [n,H_q,d] (u16 = bf16 or u8 = fp8 E4M3), K,V [L,H_kv,d] (both u16 or both u8),
+    I [n,H_kv,k] -> (O [n,H_q,d], LSE [n,H_q]) f64."""
+    q, K, V, pos = _idx(q), _idx(K), _idx(V), _pos(pos)
     assert K.dtype == V.dtype
     I = np.ascontiguousarray(I, dtype=np.int32)
     n, H_q, d = q.shape
@@ -136,7 +136,8 @@ def sparse_attn(q, K, V, I, pos, block_size: int, scale: Optional[float] = None)
     LSE = np.empty((n, H_q), dtype=np.float64)
     _load().msa_oracle_sparse_attn(_p(q), _p(K), _p(V), _p(I), _p(pos), ctypes.c_int64(n),
                                    ctypes.c_int64(L), H_q, H_kv, d, block_size, k,
-                                   ctypes.c_double(scale), _p(O), _p(LSE), int(K.dtype == np.uint8))
+                                   ctypes.c_double(scale), _p(O), _p(LSE), int(K.dtype == np.uint8),
+                                   int(q.dtype == np.uint8))
     return O, LSE
 
 

@@ -201,11 +201,14 @@ void msa_oracle_topk_select(const double* M, const int64_t* pos, int64_t n, int6
  *   LSE[i,h] = log sum_j exp(z[j])   (natural log)
  * q: [n,H_q,d]; K,V: [L,H_kv,d]; I: [n,H_kv,k] (entries < 0 are padding);
  * O: [n,H_q,d]; LSE: [n,H_q].
+ * Operands stored in fp8 E4M3 (Section 4.2: the kernels also support fp8) are decoded exactly and
+ * everything after the decoding is the arithmetic above, in double: the oracle models no rounding
+ * of P or of partial results.
  */
-void msa_oracle_sparse_attn(const uint16_t* q, const void* K, const void* V,
+void msa_oracle_sparse_attn(const void* q, const void* K, const void* V,
                             const int32_t* I, const int64_t* pos, int64_t n, int64_t L,
                             int H_q, int H_kv, int d, int B_k, int k, double scale,
-                            double* O, double* LSE, int kv_fp8) {
+                            double* O, double* LSE, int kv_fp8, int q_fp8) {
     const int G = H_q / H_kv;
 #pragma omp parallel for schedule(dynamic, 1)
     for (int64_t a = 0; a < n * H_q; ++a) {
@@ -213,7 +216,7 @@ void msa_oracle_sparse_attn(const uint16_t* q, const void* K, const void* V,
         const int h = (int)(a % H_q);
         const int r = h / G;
         const int64_t i = pos[qi];
-        const uint16_t* qrow = q + a * (int64_t)d;
+        const int64_t qrow = a * (int64_t)d;  /* element offset; Q holds bf16 or fp8 E4M3 like K and V */
         const int32_t* sel = I + (qi * H_kv + r) * (int64_t)k;
         double* z = (double*)malloc(sizeof(double) * (size_t)k * (size_t)B_k);
         int64_t* tok = (int64_t*)malloc(sizeof(int64_t) * (size_t)k * (size_t)B_k);
@@ -225,7 +228,7 @@ void msa_oracle_sparse_attn(const uint16_t* q, const void* K, const void* V,
                 const int64_t krow = (j * H_kv + r) * (int64_t)d;  /* element offset; K, V hold bf16 or fp8 E4M3 */
                 double acc = 0.0;
                 for (int c = 0; c < d; ++c)
-                    acc += bf16_to_double(qrow[c]) * kv_elem(K, krow + c, kv_fp8);
+                    acc += kv_elem(q, qrow + c, q_fp8) * kv_elem(K, krow + c, kv_fp8);
                 z[nt] = acc * scale;
                 tok[nt] = j;
                 ++nt;

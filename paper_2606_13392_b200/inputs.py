@@ -45,7 +45,8 @@ class MSAConfig:
     planted_shift: float = 0.0
     seq_lens: Tuple[int, ...] = ()
     idx_fp8: bool = False  # index-branch operands (Q_idx, K_idx) rounded to fp8 E4M3 instead of bf16
-    kv_fp8: bool = False   # the K and V caches are stored in fp8 E4M3 (Q stays bf16)
+    kv_fp8: bool = False   # the K and V caches are stored in fp8 E4M3 (Q stays bf16 unless q_fp8)
+    q_fp8: bool = False    # prefill: Q is stored in fp8 E4M3 as well (needs kv_fp8)
 
     @property
     def group(self) -> int:
@@ -187,6 +188,8 @@ def make_prefill_inputs(cfg: MSAConfig, device="cpu", sharp: bool = False):
         q_idx, k_idx = q_idx.to(torch.float8_e4m3fn), k_idx.to(torch.float8_e4m3fn)
     if cfg.kv_fp8:  # prefill onto fp8 caches: K and V rounded to E4M3, Q stays bf16
         k, v = k.to(torch.float8_e4m3fn), v.to(torch.float8_e4m3fn)
+    if cfg.q_fp8:   # the same draws of Q, stored in the narrower format
+        q = q.to(torch.float8_e4m3fn)
     return {"q": q, "k": k, "v": v, "q_idx": q_idx, "k_idx": k_idx}
 
 

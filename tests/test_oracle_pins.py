@@ -463,3 +463,33 @@ def test_fp8_kv_sparse_attention_equals_bf16_of_the_same_values():
     xb = make_decode_inputs(cfg.scaled(kv_fp8=False), "cpu", sharp=True)
     Of, _ = oracle.sparse_attn(q, to_bits(xb["k_cache"][:L]), to_bits(xb["v_cache"][:L]), I, pos, cfg.block_size)
     assert 1e-4 < np.abs(Of - O8).max() < 0.2  # the rounding of K and V is there, and is small
+
+
+def test_fp8_q_sparse_attention_equals_bf16_of_the_same_values():
+    # Q stored as fp8 E4M3 as well (Section 4.2): the oracle on fp8 Q, K, V must give, bit for bit, what
+    # it gives on the bf16 tensors torch converts them to (torch's decoding is independent of the
+    # oracle's), a visibly different result from the unrounded Q, and the dense result when every block
+    # is selected (the same SDPA pin as the bf16 path, on the decoded values).
+    cfg = MSAConfig("q8", "prefill", 90, 8, 2, 16, 6, head_dim=32, idx_dim=16, seed=9, kv_fp8=True, q_fp8=True)
+    x = make_prefill_inputs(cfg, "cpu", sharp=True)
+    assert x["q"].dtype == torch.float8_e4m3fn and x["k"].dtype == torch.float8_e4m3fn
+    pos = np.array([5, 31, 32, 89])
+    I = np.tile(np.arange(6, dtype=np.int32), (len(pos), cfg.n_kv_heads, 1))
+    for a, i in enumerate(pos):
+        I[a][:, (i // cfg.block_size) + 1:] = -1
+    q8, k8, v8 = x["q"][pos], x["k"], x["v"]
+    O8, L8 = oracle.sparse_attn(to_bits(q8), to_bits(k8), to_bits(v8), I, pos, cfg.block_size)
+    bf = torch.bfloat16
+    Ob, Lb = oracle.sparse_attn(to_bits(q8.to(bf)), to_bits(k8.to(bf)), to_bits(v8.to(bf)), I, pos, cfg.block_size)
+    assert np.array_equal(O8, Ob) and np.array_equal(L8, Lb)
+    xq = make_prefill_inputs(cfg.scaled(q_fp8=False), "cpu", sharp=True)
+    Of, _ = oracle.sparse_attn(to_bits(xq["q"][pos]), to_bits(k8), to_bits(v8), I, pos, cfg.block_size)
+    assert 1e-4 < np.abs(Of - O8).max() < 0.3  # the rounding of Q is there, and is small
+    # every visible block selected: torch SDPA on the decoded values (heads repeated per group)
+    G = cfg.group
+    qf, kf, vf = q8.float(), k8.float(), v8.float()
+    for a, i in enumerate(pos):
+        kk = kf[: i + 1].repeat_interleave(G, dim=1).permute(1, 0, 2)   # [H_q, i+1, d]
+        vv = vf[: i + 1].repeat_interleave(G, dim=1).permute(1, 0, 2)
+        ref = torch.nn.functional.scaled_dot_product_attention(qf[a][:, None, :], kk, vv)[:, 0, :]
+        assert np.abs(ref.double().numpy() - O8[a]).max() < 2e-5
