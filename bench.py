@@ -54,13 +54,15 @@ def prefill_work(cfg: MSAConfig):
     tokens = (n_sel - 1) * Bk + (i % Bk) + 1          # visible tokens of the selected blocks
     pairs = int(n_sel.sum()) * cfg.n_kv_heads          # (query, group, block) pairs
     gd2 = 2 * cfg.group * cfg.head_dim                 # bytes of one (query, group) bf16 row set
+    q_el = 1.0 if cfg.q_fp8 else 2.0                   # bytes per gathered Q element
+    kv_el = 1.0 if (cfg.q_fp8 and cfg.kv_fp8) else 2.0  # (fp8 K/V with bf16 Q are widened to bf16 first)
     return {
         "index_flops": float(cfg.n_kv_heads) * cfg.idx_dim * float(sum(float(n) * (n + 1) for n in lens)),
         "attn_flops": 4.0 * cfg.n_q_heads * cfg.head_dim * float(tokens.sum()),
         "topk_bytes": 4.0 * cfg.n_kv_heads * float((loc + 1).sum()) + 4.0 * T * cfg.n_kv_heads * k,
         # KV-outer with bf16 partials: K+V once, per pair Q gather + partial write, final O
-        "attn_bytes": 2.0 * 2 * T * cfg.n_kv_heads * cfg.head_dim + pairs * (2.0 * gd2 + 4 * cfg.group)
-                      + 2.0 * T * cfg.n_q_heads * cfg.head_dim,
+        "attn_bytes": kv_el * 2 * T * cfg.n_kv_heads * cfg.head_dim
+                      + pairs * (q_el / 2.0 * gd2 + gd2 + 4 * cfg.group) + 2.0 * T * cfg.n_q_heads * cfg.head_dim,
         # combine: reads every partial (+ its LSE) once, writes O and LSE
         "combine_bytes": pairs * (gd2 + 4.0 * cfg.group) + T * cfg.n_q_heads * (2.0 * cfg.head_dim + 4),
         "pairs": pairs,
@@ -324,7 +326,8 @@ def base_line(cfg: MSAConfig, args, n_gpus: int):
 
 
 def describe(cfg: MSAConfig) -> str:
-    f8 = (", index operands fp8 E4M3" if cfg.idx_fp8 else "") + (", K/V caches fp8 E4M3" if cfg.kv_fp8 else "")
+    f8 = (", index operands fp8 E4M3" if cfg.idx_fp8 else "") + \
+        (", Q, K, V fp8 E4M3" if cfg.q_fp8 else (", K/V caches fp8 E4M3" if cfg.kv_fp8 else ""))
     if cfg.mode == "prefill" and cfg.seq_lens:
         return ("prefill fwd, %d packed sequences of %s tokens (%d in all), causal, %d q heads / %d kv heads, d_h=%d, "
                 "d_idx=%d, B_k=%d, k=%d%s"
@@ -379,7 +382,7 @@ def measure(cfg: MSAConfig, args, rank, world, dev, B, peaks, dist, e2e: bool, c
     if cfg.mode == "prefill":
         x = make_prefill_inputs(mycfg, dev)
         T = cfg.T
-        out = torch.empty_like(x["q"])
+        out = torch.empty(x["q"].shape, dtype=torch.bfloat16, device=dev)
         lse = torch.empty((T, cfg.n_q_heads), dtype=torch.float32, device=dev)
         block_idx = torch.empty((T, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32, device=dev)
         mn, pf = B.msa_prefill_forward_workspace_bytes(shape, T)

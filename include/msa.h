@@ -90,6 +90,16 @@ typedef struct {
                          /* bytes and does the same).  The allocation-free prefill */
                          /* call returns MSA_ERR_UNSUPPORTED with the flag.  Other */
                          /* values: INVALID_ARG.                                   */
+    int32_t q_fp8;       /* 0: Q is bf16.  1 (prefill only, needs kv_fp8 = 1, d_h = */
+                         /* 128, G in {8,16}, B_k in {64,128}): q holds fp8 E4M3 as */
+                         /* well (Section 4.2).  The attention kernel then reads    */
+                         /* the fp8 tensors itself: S = Q K^T on fp8 tensor-core    */
+                         /* MMAs (exact products, fp32 sums), V widened exactly to  */
+                         /* bf16 once per K/V tile, P and O = P V as with bf16      */
+                         /* operands; no bf16 copies, so no extra workspace.  out   */
+                         /* stays bf16.  Other shapes, decode calls and the         */
+                         /* allocation-free call: MSA_ERR_UNSUPPORTED.  Other       */
+                         /* values: INVALID_ARG.                                    */
 } msa_shape_t;
 
 typedef void* msa_stream_t; /* a cudaStream_t */

@@ -17,7 +17,7 @@ def prefill_forward(cfg: MSAConfig, x: Dict[str, torch.Tensor], workspace: Optio
     shape = B.shape_of(cfg)
     T = x["q"].shape[0]
     dev = x["q"].device
-    out = torch.empty_like(x["q"])
+    out = torch.empty(x["q"].shape, dtype=torch.bfloat16, device=dev)  # (Q itself may be fp8)
     lse = torch.empty((T, cfg.n_q_heads), dtype=torch.float32, device=dev) if want_lse else None
     block_idx = torch.empty((T, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32, device=dev)
     if workspace is None:
@@ -35,7 +35,7 @@ def prefill_forward_varlen(cfg: MSAConfig, x: Dict[str, torch.Tensor], cu_seqlen
     shape = B.shape_of(cfg)
     T = x["q"].shape[0]
     dev = x["q"].device
-    out = torch.empty_like(x["q"])
+    out = torch.empty(x["q"].shape, dtype=torch.bfloat16, device=dev)
     lse = torch.empty((T, cfg.n_q_heads), dtype=torch.float32, device=dev) if want_lse else None
     block_idx = torch.empty((T, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32, device=dev)
     if workspace is None:
@@ -88,7 +88,7 @@ def sparse_attn_prefill(cfg: MSAConfig, q, k, v, block_idx, q_begin: int = 0,
                         workspace_bytes: Optional[int] = None):
     shape = B.shape_of(cfg)
     q_count, kv_len = q.shape[0], k.shape[0]
-    out = torch.empty_like(q)
+    out = torch.empty(q.shape, dtype=torch.bfloat16, device=q.device)
     lse = torch.empty((q_count, cfg.n_q_heads), dtype=torch.float32, device=q.device)
     mn, pf = B.msa_sparse_attn_prefill_workspace_bytes(shape, q_count, kv_len)
     ws = B.alloc_workspace(pf if workspace_bytes is None else max(mn, workspace_bytes), q.device)

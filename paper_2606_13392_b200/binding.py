@@ -40,7 +40,7 @@ class MsaShape(ctypes.Structure):
     _fields_ = [("n_q_heads", c_i32), ("n_kv_heads", c_i32), ("head_dim", c_i32),
                 ("idx_dim", c_i32), ("block_size", c_i32), ("top_k", c_i32),
                 ("softmax_scale", ctypes.c_float), ("index_scale", ctypes.c_float),
-                ("idx_fp8", c_i32), ("kv_fp8", c_i32)]
+                ("idx_fp8", c_i32), ("kv_fp8", c_i32), ("q_fp8", c_i32)]
 
 
 class MsaError(RuntimeError):
@@ -73,7 +73,8 @@ def status_string(code: int) -> str:
 
 def shape_of(cfg: MSAConfig, softmax_scale: float = 0.0, index_scale: float = 0.0) -> MsaShape:
     return MsaShape(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.idx_dim, cfg.block_size,
-                    cfg.top_k, softmax_scale, index_scale, 1 if cfg.idx_fp8 else 0, 1 if cfg.kv_fp8 else 0)
+                    cfg.top_k, softmax_scale, index_scale, 1 if cfg.idx_fp8 else 0, 1 if cfg.kv_fp8 else 0,
+                    1 if getattr(cfg, "q_fp8", False) else 0)
 
 
 def _ptr(t) -> c_vp:
@@ -104,6 +105,14 @@ def _kv(shape, t: Optional[torch.Tensor]):
         want = 1 if shape.kv_fp8 else 2
         assert t.element_size() == want, "K/V cache element size %d, shape expects %d" % (t.element_size(), want)
     return _dev(t)
+
+
+def _q(shape, t: Optional[torch.Tensor], host: bool = False):
+    """The Q tensor: its element size must match the shape's q_fp8 flag."""
+    if t is not None:
+        want = 1 if shape.q_fp8 else 2
+        assert t.element_size() == want, "Q element size %d, shape expects %d" % (t.element_size(), want)
+    return _host(t) if host else _dev(t)
 
 
 def _host(t: Optional[torch.Tensor]):
@@ -201,7 +210,7 @@ def msa_sparse_attn_prefill_workspace_bytes(shape, q_count, kv_len) -> Tuple[int
 
 def msa_sparse_attn_prefill(shape, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse,
                             workspace, stream=None):
-    _check(lib().msa_sparse_attn_prefill(ctypes.byref(shape), _dev(q), _kv(shape, k), _kv(shape, v),
+    _check(lib().msa_sparse_attn_prefill(ctypes.byref(shape), _q(shape, q), _kv(shape, k), _kv(shape, v),
                                          _dev(block_idx), c_i64(q_begin), c_i64(q_count),
                                          c_i64(kv_len), _dev(out), _dev(lse), _dev(workspace),
                                          c_sz(workspace.numel() * workspace.element_size()),
@@ -257,7 +266,7 @@ def msa_prefill_forward_workspace_bytes(shape, T) -> Tuple[int, int]:
 
 
 def msa_prefill_forward(shape, q, k, v, q_idx, k_idx, T, out, lse, block_idx, workspace, stream=None):
-    _check(lib().msa_prefill_forward(ctypes.byref(shape), _dev(q), _kv(shape, k), _kv(shape, v), _idx(shape, q_idx),
+    _check(lib().msa_prefill_forward(ctypes.byref(shape), _q(shape, q), _kv(shape, k), _kv(shape, v), _idx(shape, q_idx),
                                      _idx(shape, k_idx), c_i64(T), _dev(out), _dev(lse), _dev(block_idx),
                                      _dev(workspace),
                                      c_sz(workspace.numel() * workspace.element_size()),
@@ -303,7 +312,7 @@ def msa_prefill_forward_varlen_workspace_bytes(shape, cu_seqlens) -> Tuple[int, 
 def msa_prefill_forward_varlen(shape, q, k, v, q_idx, k_idx, cu_seqlens, out, lse, block_idx, workspace,
                                stream=None):
     arr, n = _cu_array(cu_seqlens)
-    _check(lib().msa_prefill_forward_varlen(ctypes.byref(shape), _dev(q), _kv(shape, k), _kv(shape, v), _idx(shape, q_idx),
+    _check(lib().msa_prefill_forward_varlen(ctypes.byref(shape), _q(shape, q), _kv(shape, k), _kv(shape, v), _idx(shape, q_idx),
                                             _idx(shape, k_idx), arr, c_i32(n), _dev(out), _dev(lse),
                                             _dev(block_idx), _dev(workspace),
                                             c_sz(workspace.numel() * workspace.element_size()),
@@ -321,7 +330,7 @@ def msa_prefill_forward_host_workspace_bytes(shape, T) -> Tuple[int, int]:
 def msa_prefill_forward_host(shape, q, k, v, q_idx, k_idx, T, out, lse, block_idx, workspace,
                              stream=None):
     """q..k_idx, out, lse, block_idx are HOST tensors (pinned for full copy rate)."""
-    _check(lib().msa_prefill_forward_host(ctypes.byref(shape), _host(q), _host(k), _host(v),
+    _check(lib().msa_prefill_forward_host(ctypes.byref(shape), _q(shape, q, True), _host(k), _host(v),
                                           _idx(shape, q_idx, True), _idx(shape, k_idx, True), c_i64(T), _host(out),
                                           _host(lse), _host(block_idx), _dev(workspace),
                                           c_sz(workspace.numel() * workspace.element_size()),

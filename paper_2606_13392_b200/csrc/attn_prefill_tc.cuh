@@ -157,7 +157,17 @@ __device__ __forceinline__ int kv_v_parity(int vb) { return vb != 1 ? 1 : 0; }  
 //             of an item's time.
 constexpr int kAttnThreads = 352;
 
-template <int BK, int G>
+//
+// F8 (Section 4.2: the kernels also support fp8): Q, K and V are stored in fp8 E4M3.  A row of 128
+// fp8 is one 128-byte swizzle row, so a Q tile is 16 KB (a query's G heads are one box of G rows)
+// and a K tile BK x 128 bytes; S = Q K^T runs as kind::f8f6f4 MMAs (32 elements per step, four
+// steps), whose products and fp32 sums are those of the decoded values.  The fp8 V tile lands in
+// the half of the K buffer that an fp8 K tile leaves free and is widened once per tile (exactly:
+// every E4M3 value is a bf16 value) by the first producer warp into the V buffer, in the layout a
+// bf16 TMA load would have produced; P stays bf16 and O = P V is the bf16 path unchanged.  The
+// kernel therefore computes what the bf16 kernel computes on the decoded operands, with half the
+// bytes per gathered query and per K/V tile.
+template <int BK, int G, bool F8 = false>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, RangeParams p,
@@ -166,8 +176,9 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                        __nv_bfloat16* __restrict__ o_buf, float* __restrict__ lse_buf, int* status) {
     constexpr int QPI = 128 / G;            // queries per item
     constexpr int TMEM_COLS = 512;          // context j: S/P at j*256, O at j*256 + 128
-    constexpr uint32_t Q_BYTES = G * 256;   // one query's G heads
-    constexpr uint32_t KV_HALF = BK * 128;  // one d half of a K or V tile
+    constexpr uint32_t Q_BYTES = F8 ? G * 128 : G * 256;  // one query's G heads in the Q tile
+    constexpr uint32_t O_BYTES = G * 256;   // one query's G heads of a bf16 partial
+    constexpr uint32_t KV_HALF = BK * 128;  // one d half of a bf16 K or V tile = a whole fp8 tile
     extern __shared__ uint8_t smem_raw[];
     AttnSmem<BK>& sm =
         *reinterpret_cast<AttnSmem<BK>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -268,9 +279,14 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 __syncwarp();
                 // One box per query: its G heads x 128 d, one contiguous read of G*256 bytes, laid
                 // down as [8 heads][d half][8 heads][64 d] so that every 1 KB is one operand atom.
-                if (lane >= q_lo && lane < q_hi)
-                    tma_load_5d_hint(sm.q[j] + lane * Q_BYTES, &tm_q, 0, 0, 0, r * (G / 8),
-                                     (int)(p.q_first + (h >> 8)), &sm.q_full[j], pol_q);
+                if (lane >= q_lo && lane < q_hi) {
+                    if constexpr (F8)  // (128 bytes, the group's G heads, one query): G swizzle rows
+                        tma_load_3d_hint(sm.q[j] + lane * Q_BYTES, &tm_q, 0, r * G, (int)(p.q_first + (h >> 8)),
+                                         &sm.q_full[j], pol_q);
+                    else
+                        tma_load_5d_hint(sm.q[j] + lane * Q_BYTES, &tm_q, 0, 0, 0, r * (G / 8),
+                                         (int)(p.q_first + (h >> 8)), &sm.q_full[j], pol_q);
+                }
                 if (threadIdx.x == 0) MSA_STAMP(n, 13);
                 if (new_tile) {
                     // K: the buffer was the V buffer of the tile before last (or the K buffer three
@@ -287,15 +303,49 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     }
                     if (lane == 0 && half == 0) {
                         mbar_arrive_expect_tx(&sm.kv_full[kb], 2 * KV_HALF);
-                        tma_load_3d_hint(sm.kv[kb][0], &tm_k, 0, r, b * BK, &sm.kv_full[kb], pol_kv);
-                        tma_load_3d_hint(sm.kv[kb][1], &tm_k, 64, r, b * BK, &sm.kv_full[kb], pol_kv);
+                        if constexpr (F8) {  // the fp8 K tile, and the fp8 V tile on its way to being widened
+                            tma_load_3d_hint(sm.kv[kb][0], &tm_k, 0, r, b * BK, &sm.kv_full[kb], pol_kv);
+                            tma_load_3d_hint(sm.kv[kb][1], &tm_v, 0, r, b * BK, &sm.kv_full[kb], pol_kv);
+                        } else {
+                            tma_load_3d_hint(sm.kv[kb][0], &tm_k, 0, r, b * BK, &sm.kv_full[kb], pol_kv);
+                            tma_load_3d_hint(sm.kv[kb][1], &tm_k, 64, r, b * BK, &sm.kv_full[kb], pol_kv);
+                        }
                     }
                     if (half == 0 && v_wait && !mbar_wait(&sm.kv_empty[vb], kv_v_parity(vb) ^ 1, abort)) {
                         if (lane == 0) report_async(status, kAsyncTimeout, 0x313);
                         ok = false;
                         break;
                     }
-                    if (lane == 0 && half == 0) {
+                    if constexpr (F8) {
+                        if (half == 0) {
+                            // The fp8 V tile has landed behind the K tile: widen it into the V buffer.
+                            // Source row = key, 128 fp8 in eight 16-byte chunks, chunk c stored at
+                            // c ^ (key & 7); 16 fp8 become two chunks of the bf16 tile [d half][key][64].
+                            if (!mbar_wait(&sm.kv_full[kb], kv_k_parity(kb), abort)) {
+                                if (lane == 0) report_async(status, kAsyncTimeout, 0x314);
+                                ok = false;
+                                break;
+                            }
+                            const uint32_t src = smem_u32(sm.kv[kb][1]), dst = smem_u32(sm.kv[vb][0]);
+                            for (int i = lane; i < BK * 8; i += 32) {
+                                const int key = i >> 3, c = i & 7, sw = key & 7;
+                                uint32_t w[4], o[8];
+                                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                             : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3])
+                                             : "r"(src + key * 128 + ((c ^ sw) << 4)));
+                                e4m3x16_to_bf16x16(w, o);
+                                const uint32_t row = dst + (c >> 2) * KV_HALF + key * 128;
+                                const int cc = 2 * (c & 3);
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + ((cc ^ sw) << 4)),
+                                             "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((cc + 1) ^ sw) << 4)),
+                                             "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+                            }
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&sm.kv_full[vb]);
+                        }
+                    } else if (lane == 0 && half == 0) {
                         mbar_arrive_expect_tx(&sm.kv_full[vb], 2 * KV_HALF);
                         tma_load_3d_hint(sm.kv[vb][0], &tm_v, 0, r, b * BK, &sm.kv_full[vb], pol_kv);
                         tma_load_3d_hint(sm.kv[vb][1], &tm_v, 64, r, b * BK, &sm.kv_full[vb], pol_kv);
@@ -309,7 +359,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc_s = make_idesc_bf16(128, BK, false, false);
+            constexpr uint32_t idesc_s = F8 ? make_idesc_e4m3(128, BK) : make_idesc_bf16(128, BK, false, false);
             constexpr uint32_t idesc_o = make_idesc_bf16(128, 128, false, true);
             int prev_vb = 0, prev_last = 0, prev_new = 0;
             for (int n = 0; n <= n_items; ++n) {
@@ -330,15 +380,23 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     tc_fence_after();
                     MSA_STAMP(n, 8);
                     const uint32_t ts = tmem + j * 256;
-                    // Q atoms (8 rows x 64 d) of one d half are 2 KB apart; the other half sits 1 KB further.
-                    const uint64_t qd0 = make_smem_desc(smem_u32(sm.q[j]), 16, 2048);
-                    const uint64_t qd1 = make_smem_desc(smem_u32(sm.q[j]) + 1024, 16, 2048);
-                    const uint64_t kd0 = make_smem_desc(smem_u32(sm.kv[kb][0]), 16, 1024);
-                    const uint64_t kd1 = make_smem_desc(smem_u32(sm.kv[kb][1]), 16, 1024);
+                    if constexpr (F8) {
+                        // rows of 128 fp8: dense 1 KB atoms of 8 rows, 32 bytes (32 elements) per step
+                        const uint64_t qd = make_smem_desc(smem_u32(sm.q[j]), 16, 1024);
+                        const uint64_t kd = make_smem_desc(smem_u32(sm.kv[kb][0]), 16, 1024);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(ts, qd0 + 2 * kk, kd0 + 2 * kk, idesc_s, kk > 0);
+                        for (int kk = 0; kk < 4; ++kk) mma_e4m3_ss(ts, qd + 2 * kk, kd + 2 * kk, idesc_s, kk > 0);
+                    } else {
+                        // Q atoms (8 rows x 64 d) of one d half are 2 KB apart; the other half sits 1 KB further.
+                        const uint64_t qd0 = make_smem_desc(smem_u32(sm.q[j]), 16, 2048);
+                        const uint64_t qd1 = make_smem_desc(smem_u32(sm.q[j]) + 1024, 16, 2048);
+                        const uint64_t kd0 = make_smem_desc(smem_u32(sm.kv[kb][0]), 16, 1024);
+                        const uint64_t kd1 = make_smem_desc(smem_u32(sm.kv[kb][1]), 16, 1024);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(ts, qd1 + 2 * kk, kd1 + 2 * kk, idesc_s, true);
+                        for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(ts, qd0 + 2 * kk, kd0 + 2 * kk, idesc_s, kk > 0);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) mma_bf16_ss(ts, qd1 + 2 * kk, kd1 + 2 * kk, idesc_s, true);
+                    }
                     mma_commit(&sm.q_empty[j]);
                     mma_commit(&sm.s_full[j]);
                     if (last) mma_commit(&sm.kv_empty[kb]);
@@ -383,8 +441,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const uint32_t tmem_s = tmem + j * 256, tmem_o = tmem_s + 128;
         constexpr int QPW = 32 / G;  // queries per warp
         // staging: this thread's row goes to [query][chunk][head]; lanes < QPW copy one query each
-        uint8_t* stg_row = sm.ostage[j] + (size_t)qi * Q_BYTES + g * 16;
-        const uint8_t* stg_query = sm.ostage[j] + (size_t)(quarter * QPW + lane) * Q_BYTES;
+        uint8_t* stg_row = sm.ostage[j] + (size_t)qi * O_BYTES + g * 16;
+        const uint8_t* stg_query = sm.ostage[j] + (size_t)(quarter * QPW + lane) * O_BYTES;
         for (int n = j; n < n_items; n += 2) {
             if (!mbar_wait(&sm.s_full[j], (n >> 1) & 1, abort)) { report_async(status, kAsyncTimeout, 0x331); break; }
             tc_fence_after();
@@ -474,7 +532,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             if (lane < QPW) {
                 if (quarter * QPW + lane < nq) {
                     const int64_t pr = partial_base((int64_t)(h_copy >> 8), r, p) + (h_copy & 0xFF);
-                    bulk_store(o_buf + pr * (G * 128), stg_query, Q_BYTES);
+                    bulk_store(o_buf + pr * (G * 128), stg_query, O_BYTES);
                 }
                 bulk_commit();
             }

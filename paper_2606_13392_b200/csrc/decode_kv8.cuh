@@ -41,18 +41,6 @@ __device__ __forceinline__ void mma_m16n8k16_f16(float (&c)[4], uint32_t a0, uin
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// Four fp8 E4M3 (bytes x0 .. x3 of a register) -> two registers of two f16 each, (x0, x1) and (x2, x3);
-// exact.  (Integer bit moves instead of the conversion instruction - sign and the seven other bits
-// shifted to their f16 places, a factor 2^8 folded into the scales - were measured at the same speed.)
-__device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t four, uint32_t& lo, uint32_t& hi) {
-    asm("{\n\t.reg .b16 a, b;\n\t"
-        "mov.b32 {a, b}, %2;\n\t"
-        "cvt.rn.f16x2.e4m3x2 %0, a;\n\t"
-        "cvt.rn.f16x2.e4m3x2 %1, b;\n\t}"
-        : "=r"(lo), "=r"(hi)
-        : "r"(four));
-}
-
 // Two bf16 (lower half first) -> two f16, round to nearest.
 __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t two) {
     const float2 f = bf16x2_to_float2(two);
@@ -68,16 +56,7 @@ e4m3_to_bf16_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int6
         const uint4 in = __ldg(src + i);
         const uint32_t w[4] = {in.x, in.y, in.z, in.w};
         uint32_t o[8];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t lo, hi;
-            e4m3x4_to_f16x2x2(w[j], lo, hi);
-            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&lo));
-            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&hi));
-            const __nv_bfloat162 ab = __floats2bfloat162_rn(a.x, a.y), bb = __floats2bfloat162_rn(b.x, b.y);
-            o[2 * j] = *reinterpret_cast<const uint32_t*>(&ab);
-            o[2 * j + 1] = *reinterpret_cast<const uint32_t*>(&bb);
-        }
+        e4m3x16_to_bf16x16(w, o);
         dst[2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
         dst[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
     }

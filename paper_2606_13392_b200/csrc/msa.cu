@@ -52,6 +52,8 @@ struct Resolved {
     float softmax_scale, index_scale;
     bool kv_fp8;                                         // the K and V caches are fp8 E4M3 (else bf16)
     size_t kv_elt() const { return kv_fp8 ? 1 : 2; }    // bytes per K/V element
+    bool q_fp8;                                          // prefill: Q is fp8 E4M3 as well (needs kv_fp8)
+    size_t q_elt() const { return q_fp8 ? 1 : 2; }      // bytes per Q element
     bool idx_fp8;                                        // index-branch operands are fp8 E4M3 (else bf16)
     size_t idx_elt() const { return idx_fp8 ? 1 : 2; }  // bytes per index-branch element
 };
@@ -75,6 +77,9 @@ static msa_status_t resolve(const msa_shape_t* s, Resolved& r) {
     if (r.idx_fp8 && r.d_idx % 16 != 0) return MSA_ERR_UNSUPPORTED;  // 16-byte rows
     if (s->kv_fp8 != 0 && s->kv_fp8 != 1) return MSA_ERR_INVALID_ARG;
     r.kv_fp8 = s->kv_fp8 == 1;
+    if (s->q_fp8 != 0 && s->q_fp8 != 1) return MSA_ERR_INVALID_ARG;
+    r.q_fp8 = s->q_fp8 == 1;
+    if (r.q_fp8 && !r.kv_fp8) return MSA_ERR_UNSUPPORTED;  // fp8 Q comes with fp8 K and V
     return MSA_OK;
 }
 
@@ -470,7 +475,8 @@ static msa_status_t hook_copy_rows(const Resolved& r, const void* out, const flo
     return MSA_OK;
 }
 
-template <int BK, int G>
+// F8: Q, K and V hold fp8 E4M3; rows of 128 bytes are moved as 64 two-byte elements.
+template <int BK, int G, bool F8 = false>
 static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const void* k, const void* v,
                                         const int32_t* block_idx, int64_t q_begin, int64_t q_count,
                                         int64_t kv_len, void* out, float* lse, void* ws, size_t ws_bytes,
@@ -488,23 +494,37 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
     __nv_bfloat16* o_buf = (__nv_bfloat16*)(w + pl.off_obuf);
 
     CUtensorMap tm_q, tm_k, tm_v;
-    // Q as (64 d, 8 heads, 2 d halves, H_q/8 head groups, query): one box is a query's G heads.
-    const uint64_t qd[5] = {64, 8, 2, (uint64_t)r.H_q / 8, (uint64_t)q_count};
-    const uint64_t qs[4] = {256, 128, 2048, (uint64_t)r.H_q * 256};
-    const uint32_t qb[5] = {64, 8, 2, (uint32_t)G / 8, 1};
-    const uint64_t kd[3] = {128, (uint64_t)r.H_kv, (uint64_t)kv_len};
-    const uint64_t ks[2] = {256, (uint64_t)r.H_kv * 256};
-    const uint32_t kb[3] = {64, 1, (uint32_t)BK};
-    if (!encode_tmap_bf16(&tm_q, q, 5, qd, qs, qb) || !encode_tmap_bf16(&tm_k, k, 3, kd, ks, kb) ||
-        !encode_tmap_bf16(&tm_v, v, 3, kd, ks, kb))
-        return MSA_ERR_CUDA;
+    if constexpr (F8) {
+        // Q as (128 bytes, head, query): one box is a query's G heads, G swizzle rows.
+        const uint64_t qd[3] = {64, (uint64_t)r.H_q, (uint64_t)q_count};
+        const uint64_t qs[2] = {128, (uint64_t)r.H_q * 128};
+        const uint32_t qb[3] = {64, (uint32_t)G, 1};
+        const uint64_t kd[3] = {64, (uint64_t)r.H_kv, (uint64_t)kv_len};
+        const uint64_t ks[2] = {128, (uint64_t)r.H_kv * 128};
+        const uint32_t kb[3] = {64, 1, (uint32_t)BK};
+        // (128-byte rows whose neighbours in memory are other heads' rows: no 256-byte L2 promotion)
+        if (!encode_tmap_bf16(&tm_q, q, 3, qd, qs, qb) || !encode_tmap_bf16(&tm_k, k, 3, kd, ks, kb, true) ||
+            !encode_tmap_bf16(&tm_v, v, 3, kd, ks, kb, true))
+            return MSA_ERR_CUDA;
+    } else {
+        // Q as (64 d, 8 heads, 2 d halves, H_q/8 head groups, query): one box is a query's G heads.
+        const uint64_t qd[5] = {64, 8, 2, (uint64_t)r.H_q / 8, (uint64_t)q_count};
+        const uint64_t qs[4] = {256, 128, 2048, (uint64_t)r.H_q * 256};
+        const uint32_t qb[5] = {64, 8, 2, (uint32_t)G / 8, 1};
+        const uint64_t kd[3] = {128, (uint64_t)r.H_kv, (uint64_t)kv_len};
+        const uint64_t ks[2] = {256, (uint64_t)r.H_kv * 256};
+        const uint32_t kb[3] = {64, 1, (uint32_t)BK};
+        if (!encode_tmap_bf16(&tm_q, q, 5, qd, qs, qb) || !encode_tmap_bf16(&tm_k, k, 3, kd, ks, kb) ||
+            !encode_tmap_bf16(&tm_v, v, 3, kd, ks, kb))
+            return MSA_ERR_CUDA;
+    }
     int* status = async_status_ptr();
     if (status == nullptr) return MSA_ERR_CUDA;
     const size_t smem = sizeof(AttnSmem<BK>) + 1024;
     static bool attr_set_dev[64] = {false};  // the attribute is per device
     const int dev_id = current_device();
     if (!attr_set_dev[dev_id]) {
-        if (cudaFuncSetAttribute(attn_prefill_tc_kernel<BK, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(attn_prefill_tc_kernel<BK, G, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem) != cudaSuccess)
             return MSA_ERR_CUDA;
         attr_set_dev[dev_id] = true;
@@ -536,7 +556,7 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
             return MSA_ERR_CUDA;
         {
             StageScope sc(kStageAttn, st);
-            attn_prefill_tc_kernel<BK, G><<<grid_attn, kAttnThreads, smem, st>>>(
+            attn_prefill_tc_kernel<BK, G, F8><<<grid_attn, kAttnThreads, smem, st>>>(
                 tm_q, tm_k, tm_v, p, tile_off, item_off, handles, scale_log2e, o_buf, lse_buf, status);
         }
         {
@@ -920,6 +940,11 @@ static size_t kv_copy_bytes(const Resolved& r, int64_t kv_len) {
     return align_up((size_t)kv_len * r.H_kv * r.d * 2);
 }
 
+// Q, K and V all in fp8 on a shape of the tensor-core kernel: the kernel reads the fp8 tensors itself.
+static bool attn_fp8_direct(const Resolved& r, int64_t kv_len) {
+    return r.q_fp8 && r.kv_fp8 && attn_tc_supported(r) && kv_len < 2147483647LL;
+}
+
 msa_status_t msa_sparse_attn_prefill_workspace_bytes(const msa_shape_t* shape, int64_t q_count,
                                                      int64_t kv_len, size_t* min_bytes,
                                                      size_t* preferred_bytes) {
@@ -938,7 +963,7 @@ msa_status_t msa_sparse_attn_prefill_workspace_bytes(const msa_shape_t* shape, i
         mn = attn_plan(r, kv_len, r_min).total + 8 * kAlign;
         pf = attn_plan(r, kv_len, r_pref).total + 8 * kAlign;
     }
-    if (r.kv_fp8) {  // bf16 copies of the visible K and V rows in front
+    if (r.kv_fp8 && !attn_fp8_direct(r, kv_len)) {  // bf16 copies of the visible K and V rows in front
         mn += 2 * kv_copy_bytes(r, kv_len);
         pf += 2 * kv_copy_bytes(r, kv_len);
     }
@@ -963,6 +988,16 @@ msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, co
     msa_sparse_attn_prefill_workspace_bytes(shape, q_count, kv_len, &need, nullptr);
     if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    if (attn_fp8_direct(r, kv_len)) {
+        if (r.B_k == 64 && r.G == 8)
+            return run_attn_prefill_tc<64, 8, true>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
+        if (r.B_k == 64 && r.G == 16)
+            return run_attn_prefill_tc<64, 16, true>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
+        if (r.B_k == 128 && r.G == 8)
+            return run_attn_prefill_tc<128, 8, true>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
+        return run_attn_prefill_tc<128, 16, true>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
+    }
+    if (r.q_fp8) return MSA_ERR_UNSUPPORTED;  // fp8 Q: the tensor-core kernel's shapes only
     if (r.kv_fp8) {  // bf16 copies of the visible rows, then the bf16 path on the rest of the workspace
         if (r.d % 16 != 0) return MSA_ERR_UNSUPPORTED;  // the conversion moves 16 elements per thread
         const size_t cb = kv_copy_bytes(r, kv_len);
@@ -1128,6 +1163,7 @@ msa_status_t msa_sparse_attn_decode(const msa_shape_t* shape, const void* q, con
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
     if (batch < 0 || cache_tokens < 0) return MSA_ERR_INVALID_ARG;
+    if (r.q_fp8) return MSA_ERR_UNSUPPORTED;  // one bf16 query row per sequence: nothing to gain from fp8
     if (batch == 0) return MSA_OK;
     if (!q || !k_cache || !v_cache || !seq_offsets || !seq_lens || !block_idx || !out ||
         !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out))
@@ -1291,7 +1327,8 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
         return s;
     if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
     // Every sequence is an independent problem: the single-sequence path on row-offset pointers.
-    const size_t q_row = (size_t)r.H_q * r.d * 2, kv_row = (size_t)r.H_kv * r.d * r.kv_elt();
+    const size_t q_row = (size_t)r.H_q * r.d * r.q_elt(), o_row = (size_t)r.H_q * r.d * 2;
+    const size_t kv_row = (size_t)r.H_kv * r.d * r.kv_elt();
     const size_t qi_row = (size_t)r.H_kv * r.d_idx * r.idx_elt(), ki_row = (size_t)r.d_idx * r.idx_elt();
     cudaStream_t st = (cudaStream_t)stream;
     static cudaStream_t lanes_dev[64][kVarlenLanes] = {};
@@ -1345,7 +1382,7 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
         }
         result = msa_prefill_forward(shape, (const char*)q + o * q_row, (const char*)k + o * kv_row,
                                      (const char*)v + o * kv_row, (const char*)q_idx + o * qi_row,
-                                     (const char*)k_idx + o * ki_row, T, (char*)out + o * q_row,
+                                     (const char*)k_idx + o * ki_row, T, (char*)out + o * o_row,
                                      lse ? lse + o * r.H_q : nullptr, block_idx + o * (int64_t)r.H_kv * r.k, ws,
                                      ws_bytes, (msa_stream_t)run);
     }
@@ -1355,7 +1392,7 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
 
 static size_t host_staging_bytes(const Resolved& r, int64_t T, size_t off[8]) {
     size_t o = 0;
-    off[0] = o; o += align_up((size_t)T * r.H_q * r.d * 2);      // q
+    off[0] = o; o += align_up((size_t)T * r.H_q * r.d * r.q_elt());  // q
     off[1] = o; o += align_up((size_t)T * r.H_kv * r.d * r.kv_elt());  // k
     off[2] = o; o += align_up((size_t)T * r.H_kv * r.d * r.kv_elt());  // v
     off[3] = o; o += align_up((size_t)T * r.H_kv * r.d_idx * r.idx_elt()); // q_idx
@@ -1434,14 +1471,14 @@ static msa_status_t prefill_forward_host_body(const msa_shape_t* shape, const vo
     if (!e_in || !e_idx || !e_kv) return MSA_ERR_CUDA;
     if (cudaEventRecord(e_in, st) != cudaSuccess || cudaStreamWaitEvent(copy, e_in, 0) != cudaSuccess) return MSA_ERR_CUDA;
     const void* src[5] = {q_host, k_host, v_host, q_idx_host, k_idx_host};
-    const size_t nbytes[5] = {(size_t)T * r.H_q * r.d * 2, (size_t)T * r.H_kv * r.d * r.kv_elt(),
+    const size_t nbytes[5] = {(size_t)T * r.H_q * r.d * r.q_elt(), (size_t)T * r.H_kv * r.d * r.kv_elt(),
                               (size_t)T * r.H_kv * r.d * r.kv_elt(), (size_t)T * r.H_kv * r.d_idx * r.idx_elt(),
                               (size_t)T * r.d_idx * r.idx_elt()};
     // Order on the copy stream: K_idx, Q_idx, K, V, Q; Q_idx and Q go in pieces with an event after each,
     // so that every scoring chunk and every attention range waits only for its own rows.
     if (cudaMemcpyAsync(w + off[4], src[4], nbytes[4], cudaMemcpyHostToDevice, copy) != cudaSuccess) return MSA_ERR_CUDA;
     if (cudaEventRecord(e_idx, copy) != cudaSuccess) return MSA_ERR_CUDA;
-    const size_t qi_rb = (size_t)r.H_kv * r.d_idx * r.idx_elt(), q_rb = (size_t)r.H_q * r.d * 2;
+    const size_t qi_rb = (size_t)r.H_kv * r.d_idx * r.idx_elt(), q_rb = (size_t)r.H_q * r.d * r.q_elt();
     if (upload_in_pieces(g_in_idx_hook, w + off[3], src[3], T, qi_rb, 65536, copy) != MSA_OK) return MSA_ERR_CUDA;
     for (int i = 1; i <= 2; ++i)
         if (cudaMemcpyAsync(w + off[i], src[i], nbytes[i], cudaMemcpyHostToDevice, copy) != cudaSuccess) return MSA_ERR_CUDA;

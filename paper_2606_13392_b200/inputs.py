@@ -84,6 +84,15 @@ CONFIGS: Dict[str, MSAConfig] = {
                             idx_fp8=True, kv_fp8=True),
     "p1m-f8kv": MSAConfig("p1m-f8kv", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=7,
                           idx_fp8=True, kv_fp8=True),
+    # Q, K and V stored in fp8 E4M3 (Section 4.2), read as such by the prefill attention kernel: C3's and
+    # C4's shapes (index operands stay bf16: d_idx = 64), and the paper's regime with fp8 index operands.
+    "c3-f8qkv": MSAConfig("c3-f8qkv", "prefill", 131072, 64, 8, 128, 64, seed=2, planted_frac=0.05,
+                          planted_shift=2.0, kv_fp8=True, q_fp8=True),
+    "c4-f8qkv": MSAConfig("c4-f8qkv", "prefill", 1048576, 64, 8, 128, 64, seed=3, kv_fp8=True, q_fp8=True),
+    "p1m-f8qkv": MSAConfig("p1m-f8qkv", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=7, idx_fp8=True,
+                           kv_fp8=True, q_fp8=True),
+    "c3-16k-f8qkv": MSAConfig("c3-16k-f8qkv", "prefill", 16384, 64, 8, 128, 64, seed=2, planted_frac=0.05,
+                              planted_shift=2.0, kv_fp8=True, q_fp8=True),
     # Reduced cases of the same shapes, small enough for multi-pass profiler captures
     # (inputs still larger than L2).
     "c3-16k": MSAConfig("c3-16k", "prefill", 16384, 64, 8, 128, 64, seed=2,

@@ -846,3 +846,110 @@ def test_fp8_index_decode_d_idx_64():
                     seq_lens=(1, 130, 4096, 5000, 30000, 16384 + 64), idx_fp8=True, kv_fp8=True)
     res = run_decode_case(cfg, True)
     assert np.mean([r["exact"] for r in res]) >= 0.95
+
+
+# ---- Q, K and V in fp8 E4M3, read as such by the prefill attention kernel (Section 4.2) ----
+@pytest.mark.parametrize("name,T,Hq,Hkv,Bk,k,di,idx8", [
+    ("c3 shape", 12288 + 5, 64, 8, 128, 64, 64, False),
+    ("c3 shape, few picks", 6144 + 77, 64, 8, 128, 4, 64, False),
+    ("paper regime, fp8 index too", 20000 + 77, 64, 4, 128, 16, 128, True),
+    ("B_k 64, G 8", 4096 + 37, 16, 2, 64, 8, 64, False),
+    ("B_k 64, G 16", 3000, 32, 2, 64, 6, 64, False),
+])
+@pytest.mark.parametrize("sharp", [False, True])
+def test_fp8_qkv_prefill_matches_oracle(name, T, Hq, Hkv, Bk, k, di, idx8, sharp):
+    # The oracle is Eq. 8 on the decoded fp8 operands, in double; the kernel's products are exact and
+    # everything after S is the bf16 path, so the bf16 path's tolerances apply unchanged.
+    cfg = MSAConfig("f8qkv", "prefill", T, Hq, Hkv, Bk, k, head_dim=128, idx_dim=di, seed=T, idx_fp8=idx8,
+                    kv_fp8=True, q_fp8=True)
+    stats = run_prefill_case(cfg, sharp, n_sample=192)
+    assert stats["exact_sets"] >= 0.995
+    print(name, sharp, stats)
+
+
+def test_fp8_qkv_prefill_small_workspace_and_ranges_equal_the_whole_call():
+    cfg = CONFIGS["c3"].scaled(name="c3-f8qkv-6k", T=6144 + 77, kv_fp8=True, q_fp8=True)
+    shape = B.shape_of(cfg)
+    x = make_prefill_inputs(cfg, DEV, sharp=True)
+    mn, pf = B.msa_prefill_forward_workspace_bytes(shape, cfg.T)
+    # no bf16 copies of K and V: the workspace is that of the bf16 call
+    assert (mn, pf) == B.msa_prefill_forward_workspace_bytes(B.shape_of(cfg.scaled(kv_fp8=False, q_fp8=False)), cfg.T)
+    o1, l1, i1 = api.prefill_forward(cfg, x, workspace_bytes=pf)
+    o2, l2, i2 = api.prefill_forward(cfg, x, workspace_bytes=mn)
+    q0 = cfg.T // 2 + 3
+    o3, l3 = api.sparse_attn_prefill(cfg, x["q"][q0:], x["k"], x["v"], i1[q0:], q_begin=q0)
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert o1.dtype == torch.bfloat16
+    assert torch.equal(i1, i2) and torch.equal(o1, o2) and torch.equal(l1, l2)
+    assert torch.equal(o3, o1[q0:]) and torch.equal(l3, l1[q0:])
+    # the same values through the widening path (fp8 K/V caches, bf16 Q): S is summed in another order
+    # there, nothing else differs
+    cfg_w = cfg.scaled(q_fp8=False)
+    xw = dict(x)
+    xw["q"] = x["q"].to(torch.bfloat16)
+    ow, lw, iw = api.prefill_forward(cfg_w, xw)
+    assert torch.equal(iw, i1)
+    assert (ow.float() - o1.float()).abs().max().item() <= 4e-3 and (lw - l1).abs().max().item() <= 1e-4
+
+
+def test_fp8_qkv_varlen_and_host_calls():
+    cfg = CONFIGS["c3"].scaled(name="c3-f8qkv-var", T=0, top_k=8, kv_fp8=True, q_fp8=True)
+    lens = [1000, 37, 0, 4096 + 5, 129]
+    cu = np.concatenate([[0], np.cumsum(lens)]).tolist()
+    total = cu[-1]
+    x = make_prefill_inputs(cfg.scaled(T=total), DEV, sharp=True)
+    out, lse, I = api.prefill_forward_varlen(cfg.scaled(T=total), x, cu)
+    torch.cuda.synchronize()
+    _assert_clean()
+    for s, L in enumerate(lens):
+        if L == 0:
+            continue
+        a, b = cu[s], cu[s + 1]
+        xs = {n: t[a:b].contiguous() for n, t in x.items()}
+        o1, l1, i1 = api.prefill_forward(cfg.scaled(T=L), xs)
+        assert torch.equal(I[a:b], i1) and torch.equal(out[a:b], o1) and torch.equal(lse[a:b], l1), "sequence %d" % s
+    # host buffers: Q, K, V go up as fp8 bytes
+    T = 5000
+    cfg = CONFIGS["c3"].scaled(name="c3-f8qkv-host", T=T, kv_fp8=True, q_fp8=True)
+    shape = B.shape_of(cfg)
+    x = make_prefill_inputs(cfg, DEV, sharp=True)
+    out, lse, I = api.prefill_forward(cfg, x)
+    host = {n: t.cpu().pin_memory() for n, t in x.items()}
+    out_h = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+    lse_h = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
+    I_h = torch.empty(I.shape, dtype=torch.int32).pin_memory()
+    mn, pf = B.msa_prefill_forward_host_workspace_bytes(shape, T)
+    ws = B.alloc_workspace(pf, DEV)
+    B.msa_prefill_forward_host(shape, host["q"], host["k"], host["v"], host["q_idx"], host["k_idx"], T, out_h, lse_h, I_h, ws)
+    assert torch.equal(I_h, I.cpu()) and torch.equal(out_h, out.cpu()) and torch.equal(lse_h, lse.cpu())
+    _assert_clean()
+
+
+def test_fp8_q_is_rejected_where_it_is_not_supported():
+    x = make_prefill_inputs(CONFIGS["c1"].scaled(T=300), DEV)
+    q8 = x["q"].to(torch.float8_e4m3fn)
+    k8, v8 = x["k"].to(torch.float8_e4m3fn), x["v"].to(torch.float8_e4m3fn)
+    I = torch.zeros((300, 1, 8), dtype=torch.int32, device=DEV)
+    out = torch.empty(x["q"].shape, dtype=torch.bfloat16, device=DEV)
+    ws = B.alloc_workspace(1 << 26, DEV)
+    # fp8 Q with bf16 K/V
+    bad = B.shape_of(CONFIGS["c1"].scaled(q_fp8=True))
+    with pytest.raises(B.MsaError) as e:
+        B.msa_sparse_attn_prefill(bad, q8, x["k"], x["v"], I, 0, 300, 300, out, None, ws)
+    assert e.value.code == 2
+    # a shape outside the tensor-core kernel (d_h = 64)
+    odd = MSAConfig("odd8", "prefill", 300, 8, 1, 64, 8, head_dim=64, idx_dim=64, kv_fp8=True, q_fp8=True)
+    xo = make_prefill_inputs(odd, DEV)
+    with pytest.raises(B.MsaError) as e:
+        B.msa_sparse_attn_prefill(B.shape_of(odd), xo["q"], xo["k"], xo["v"], I, 0, 300, 300,
+                                  torch.empty(xo["q"].shape, dtype=torch.bfloat16, device=DEV), None, ws)
+    assert e.value.code == 2
+    # decode calls
+    dcfg = CONFIGS["c5"].scaled(seq_lens=(300,), kv_fp8=True, q_fp8=True, n_kv_heads=1, n_q_heads=8)
+    sh = B.shape_of(dcfg)
+    with pytest.raises(B.MsaError) as e:
+        B.msa_sparse_attn_decode(sh, x["q"][:1].contiguous(), k8, v8, 300, torch.zeros(1, dtype=torch.int64, device=DEV),
+                                 torch.tensor([300], dtype=torch.int32, device=DEV), 1, I[:1].contiguous(),
+                                 out[:1].contiguous(), None, ws)
+    assert e.value.code == 2
