@@ -28,7 +28,7 @@
  *     G in {8,16} (decode index scoring: H_kv <= 8); other shapes (d_h, d_idx multiples
  *     of 8, d_h <= 256, d_idx <= 128) run on generic kernels.  k is limited to 1..128.
  *   - State the library keeps: per device, a ring of CUDA events, the copy stream of the
- *     *_host calls, the four side streams of msa_prefill_forward_varlen, cached kernel
+ *     *_host calls, cached kernel
  *     attributes, and ONE async status word (a device global, not part of any workspace:
  *     two callers sharing a device cannot tell whose kernel set it; whoever reads it clears
  *     it); per process, the profiling hooks (their events belong to the device that was
@@ -301,15 +301,19 @@ msa_status_t msa_prefill_forward_workspace_bytes(const msa_shape_t* shape, int64
  * cu_seqlens[s] .. cu_seqlens[s+1]-1 of q, k, v, q_idx, k_idx, out, lse and block_idx;
  * cu_seqlens is a HOST array of n_seqs+1 non-decreasing row offsets (int64), cu_seqlens[0] >= 0.
  * block_idx holds block numbers relative to the row's own sequence.  Sequences of length 0 are
- * skipped.  Every sequence runs through the single-sequence path: long ones one after the other
- * on `stream` with the whole workspace; sequences of at most 8192 tokens, when a quarter of the
- * workspace holds one's preferred size, in turn on four streams owned by the library (created on
- * first use), each with its own quarter, which start behind the work `stream` holds at the call
- * and which `stream` waits for before the call returns (events only: the call may be captured
- * into a CUDA graph).  Results do not depend on which way a sequence ran.
- * workspace >= msa_prefill_forward_varlen_workspace_bytes' minimum (the largest single
- * sequence's need; its preferred size has room for the four quarters).  Errors: MSA_ERR_INVALID_ARG for a NULL or decreasing cu_seqlens or
- * n_seqs < 0, otherwise as msa_prefill_forward.
+ * skipped.  On the shapes of the tensor-core attention kernel (d_h = 128, G in {8,16}, B_k in
+ * {64,128}) a batch of two or more sequences runs as ONE problem per stage: Eq. 6 + Eq. 7 as a single
+ * launch of the fused kernel over the query tiles of all sequences (top_k <= 16; larger top_k: stages
+ * 1-2 sequence by sequence), and Eq. 8 with its blocks numbered through the batch, so that one
+ * reverse index, one attention launch and one merge serve every sequence of a query range (ranges
+ * span sequence boundaries).  Other shapes, and a batch of one, run the single-sequence call per
+ * sequence on `stream`.  Results do not depend on which way a sequence ran.  The call copies
+ * cu_seqlens and a tile list from host memory to the front of the workspace with cudaMemcpyAsync:
+ * it must not be captured into a CUDA graph.  Everything runs on `stream`; the library owns no
+ * stream here.
+ * workspace >= msa_prefill_forward_varlen_workspace_bytes' minimum (the batch's maps - 8 bytes per
+ * row, 4 per block - plus what the stages need).  Errors: MSA_ERR_INVALID_ARG for a NULL or decreasing
+ * cu_seqlens or n_seqs < 0, otherwise as msa_prefill_forward.
  */
 msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q, const void* k,
                                         const void* v, const void* q_idx, const void* k_idx,

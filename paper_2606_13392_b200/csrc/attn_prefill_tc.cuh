@@ -24,7 +24,49 @@ struct RangeParams {
     int32_t q_count;   // queries in this range
     int32_t n_blocks;  // KV blocks visible to the range: ceil((q_begin+q_first+q_count)/B_k)
     int32_t H_kv, top_k;
+    // A packed batch (several sequences token-major in one tensor, q_begin = 0): blocks are numbered
+    // through the batch, sequence after sequence, and n_blocks counts them all.  Null for one sequence.
+    const int32_t* row_pos;   // [rows]   position of a packed row inside its own sequence
+    const int32_t* row_blk0;  // [rows]   number of blocks of the sequences before the row's
+    const int32_t* blk_row0;  // [blocks] packed row of the block's first key
 };
+
+// Position of query `qrow` (a row of the call) inside its sequence, and the batch-wide number of its block 0.
+__device__ __forceinline__ int64_t query_pos(const RangeParams& p, int64_t qrow) {
+    return p.row_pos != nullptr ? (int64_t)p.row_pos[qrow] : p.q_begin + qrow;
+}
+__device__ __forceinline__ int query_blk0(const RangeParams& p, int64_t qrow) {
+    return p.row_blk0 != nullptr ? p.row_blk0[qrow] : 0;
+}
+
+// Fills the three arrays of a packed batch from the row offsets cu [n_seqs+1] and the block offsets
+// blk_cum [n_seqs+1] of its sequences (one thread per row, then per block; binary searches).
+__global__ void __launch_bounds__(256)
+packed_map_kernel(const int64_t* __restrict__ cu, const int32_t* __restrict__ blk_cum, int n_seqs, int B_k,
+                  int32_t* __restrict__ row_pos, int32_t* __restrict__ row_blk0, int32_t* __restrict__ blk_row0) {
+    const int64_t rows = cu[n_seqs] - cu[0];
+    const int64_t n_blk = blk_cum[n_seqs];
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < rows + n_blk;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        int lo = 0, hi = n_seqs;  // last sequence that starts at or before the row (the block)
+        if (i < rows) {
+            const int64_t row = cu[0] + i;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (cu[mid] <= row) lo = mid; else hi = mid;
+            }
+            row_pos[i] = (int32_t)(row - cu[lo]);
+            row_blk0[i] = blk_cum[lo];
+        } else {
+            const int32_t b = (int32_t)(i - rows);
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (blk_cum[mid] <= b) lo = mid; else hi = mid;
+            }
+            blk_row0[b] = (int32_t)(cu[lo] - cu[0]) + (b - blk_cum[lo]) * B_k;
+        }
+    }
+}
 
 // Tiles are numbered head after head: the whole grid works on one KV head at a time, so the
 // Q rows of (range, head) - gathered top_k times each - are the only hot lines in L2.
@@ -59,7 +101,8 @@ revidx_kernel(const int32_t* __restrict__ block_idx, RangeParams p, int pass, in
     const int lane = threadIdx.x & 31;
     if (row >= p.q_count * p.H_kv) return;
     const int ql = row / p.H_kv, r = row - ql * p.H_kv;
-    const int64_t loc = (p.q_begin + p.q_first + ql) / BK;
+    const int64_t loc = query_pos(p, p.q_first + ql) / BK;
+    const int blk0 = query_blk0(p, p.q_first + ql);
     const int32_t* sel = block_idx + ((p.q_first + ql) * (int64_t)p.H_kv + r) * p.top_k;
     for (int s = lane; s < p.top_k; s += 32) {
         const int32_t b = sel[s];
@@ -67,7 +110,7 @@ revidx_kernel(const int32_t* __restrict__ block_idx, RangeParams p, int pass, in
             if (b != -1 && pass == 0) report_async(status, kAsyncBadIndex, 0x301);
             continue;
         }
-        const int tile = tile_id(b, r, p);
+        const int tile = tile_id(blk0 + b, r, p);
         const int64_t e = (int64_t)row * p.top_k + s;
         if (pass == 0)
             rank[e] = (uint32_t)atomicAdd(&cnt[tile], 1);
@@ -107,7 +150,7 @@ revidx_scan_kernel(int32_t* __restrict__ cnt, int n_tiles, int qpi, int32_t* __r
 constexpr int kAttnInfoRing = 8;  // item descriptors; deeper than the furthest reader lags
 
 struct AttnItemInfo {
-    int32_t block, r, nq;
+    int32_t kv_row0, r, nq;  // row of the tile's first key in the K/V tensors; KV head; queries in the item
     int32_t kb, vb;        // K and V buffers of this item's tile
     int32_t new_tile;      // first item of its tile in this CTA: wait for the K/V loads
     int32_t last_of_tile;  // last item of its tile in this CTA: release the K/V buffers
@@ -222,7 +265,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const int handles_end = tile_off[n_tiles];
         // Q rows are gathered top_k times each, K/V tiles go by once.
         const uint64_t pol_q = l2_policy_evict_last(), pol_kv = l2_policy_evict_first();
-        int loaded_tile = -1, tile_seq = -1, n = 0;
+        int loaded_tile = -1, tile_seq = -1, n = 0, kv_row0 = 0;
         bool ok = true;
         if (const long long late = g_debug_producer_delay; late > 0) spin_cycles(late);  // tests only
         for (int ph = 0; ph < phases && ok; ++ph) {
@@ -250,6 +293,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 const int r = ph, b = tile - ph * p.n_blocks;
                 const int nq = min(QPI, p_end - first);
                 const bool new_tile = tile != loaded_tile;
+                if (new_tile) kv_row0 = p.blk_row0 != nullptr ? p.blk_row0[b] : b * BK;
                 const bool last_of_tile = (it + 1 == it_hi) || (i_next <= it + 1);
                 if (new_tile) ++tile_seq;
                 const int kb = kv_k_buf(tile_seq), vb = kv_v_buf(tile_seq);
@@ -270,7 +314,7 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 AttnItemInfo& inf = sm.info[n % kAttnInfoRing];
                 if (lane < QPI && half == 0) inf.handle[lane] = h;
                 if (lane == 0 && half == 0) {
-                    inf.block = b; inf.r = r; inf.nq = nq; inf.kb = kb; inf.vb = vb;
+                    inf.kv_row0 = kv_row0; inf.r = r; inf.nq = nq; inf.kb = kb; inf.vb = vb;
                     inf.new_tile = new_tile ? 1 : 0; inf.last_of_tile = last_of_tile ? 1 : 0;
                 }
                 __syncwarp();
@@ -304,11 +348,11 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     if (lane == 0 && half == 0) {
                         mbar_arrive_expect_tx(&sm.kv_full[kb], 2 * KV_HALF);
                         if constexpr (F8) {  // the fp8 K tile, and the fp8 V tile on its way to being widened
-                            tma_load_3d_hint(sm.kv[kb][0], &tm_k, 0, r, b * BK, &sm.kv_full[kb], pol_kv);
-                            tma_load_3d_hint(sm.kv[kb][1], &tm_v, 0, r, b * BK, &sm.kv_full[kb], pol_kv);
+                            tma_load_3d_hint(sm.kv[kb][0], &tm_k, 0, r, kv_row0, &sm.kv_full[kb], pol_kv);
+                            tma_load_3d_hint(sm.kv[kb][1], &tm_v, 0, r, kv_row0, &sm.kv_full[kb], pol_kv);
                         } else {
-                            tma_load_3d_hint(sm.kv[kb][0], &tm_k, 0, r, b * BK, &sm.kv_full[kb], pol_kv);
-                            tma_load_3d_hint(sm.kv[kb][1], &tm_k, 64, r, b * BK, &sm.kv_full[kb], pol_kv);
+                            tma_load_3d_hint(sm.kv[kb][0], &tm_k, 0, r, kv_row0, &sm.kv_full[kb], pol_kv);
+                            tma_load_3d_hint(sm.kv[kb][1], &tm_k, 64, r, kv_row0, &sm.kv_full[kb], pol_kv);
                         }
                     }
                     if (half == 0 && v_wait && !mbar_wait(&sm.kv_empty[vb], kv_v_parity(vb) ^ 1, abort)) {
@@ -347,8 +391,8 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         }
                     } else if (lane == 0 && half == 0) {
                         mbar_arrive_expect_tx(&sm.kv_full[vb], 2 * KV_HALF);
-                        tma_load_3d_hint(sm.kv[vb][0], &tm_v, 0, r, b * BK, &sm.kv_full[vb], pol_kv);
-                        tma_load_3d_hint(sm.kv[vb][1], &tm_v, 64, r, b * BK, &sm.kv_full[vb], pol_kv);
+                        tma_load_3d_hint(sm.kv[vb][0], &tm_v, 0, r, kv_row0, &sm.kv_full[vb], pol_kv);
+                        tma_load_3d_hint(sm.kv[vb][1], &tm_v, 64, r, kv_row0, &sm.kv_full[vb], pol_kv);
                     }
                     loaded_tile = tile;
                 }
@@ -448,15 +492,17 @@ attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             tc_fence_after();
             if (lane == 0 && quarter == 0) MSA_STAMP(n, 0);
             const AttnItemInfo& inf = sm.info[n % kAttnInfoRing];
-            const int b = inf.block, r = inf.r, nq = inf.nq;
+            const int kv_row0 = inf.kv_row0, r = inf.r, nq = inf.nq;
             const uint32_t h = inf.handle[qi];
             // handle of the query whose partial this lane hands to the bulk-copy engine
             const uint32_t h_copy = inf.handle[(quarter * QPW + lane) & 15];
             const bool valid = qi < nq;
             const int64_t ql = h >> 8;
+            // Row of the query in the K/V tensors (its own position for one sequence starting at row 0, its
+            // packed row in a batch); the keys of the tile at rows kv_row0.. up to that row are visible.
             const int64_t pos = p.q_begin + p.q_first + ql;
             // visible columns of this block for this query: 0..lim
-            const int64_t lim64 = pos - (int64_t)b * BK;
+            const int64_t lim64 = pos - (int64_t)kv_row0;
             const int lim = valid ? (int)(lim64 > BK - 1 ? BK - 1 : lim64) : BK - 1;
 
             uint32_t sv[BK / 32][32];
@@ -565,7 +611,7 @@ combine_kernel(const int32_t* __restrict__ block_idx, RangeParams p, const __nv_
     const int ql = blockIdx.x / p.H_kv, r = blockIdx.x % p.H_kv;
     const int t = threadIdx.x;
     const int64_t q = p.q_first + ql;
-    const int64_t loc = (p.q_begin + q) / BK;
+    const int64_t loc = query_pos(p, q) / BK;
     const int32_t* sel = block_idx + (q * p.H_kv + r) * (int64_t)p.top_k;
     const int64_t pbase = partial_base(ql, r, p);
     for (int s = t; s < p.top_k; s += G * 16) {

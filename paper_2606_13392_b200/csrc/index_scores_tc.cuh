@@ -44,6 +44,14 @@ struct IdxSmem {
 // writes, since both rank the same scaled fp32 maxima with the same tie rule.
 constexpr int kIdxFuseKeep = 15;
 
+// A packed batch (several sequences token-major in one tensor): the query tiles of all sequences in
+// the order the grid takes them (longest key prefix first).  A tile never straddles two sequences.
+struct IdxPackedTile {
+    int32_t row0;  // packed row of the sequence's first token
+    int32_t len;   // tokens of the sequence
+    int32_t qt;    // query tile inside the sequence
+};
+
 //
 // F8: the operands are fp8 E4M3 (Section 4.2), d_idx = 128 bytes = one swizzle atom (DI = 1).
 // The tiles are the same bytes in the same places as 64 bf16 per row, so the tensor maps, the
@@ -54,18 +62,25 @@ __global__ void __launch_bounds__(kIdxThreads, 1)
 index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        int64_t q_begin, int64_t q_count, int H_kv, float scale,
                        float* __restrict__ scores, int64_t ld_scores, int64_t n_cols, int* status,
-                       int32_t* __restrict__ block_idx = nullptr, int top_k = 0) {
+                       int32_t* __restrict__ block_idx = nullptr, int top_k = 0,
+                       const IdxPackedTile* __restrict__ packed = nullptr) {
     static_assert(FK == 0 || NH <= 2, "the fused form keeps its candidates in registers");
     static_assert(!F8 || DI == 1, "fp8 index vectors are one 128-byte atom");
     extern __shared__ uint8_t smem_raw[];
     IdxSmem<NH, DI, ST>& sm =
         *reinterpret_cast<IdxSmem<NH, DI, ST>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t n_qtiles = (q_count + kIdxTileQ - 1) / kIdxTileQ;
-    // Longest items first: the last query tile sees the most keys.
     const int n_hg = H_kv / NH;  // head groups
-    const int64_t qt = n_qtiles - 1 - (int64_t)(blockIdx.x / n_hg);
     const int r0 = (int)(blockIdx.x % n_hg) * NH;
+    // Longest items first: the last query tile sees the most keys.  In a packed batch the tile list
+    // says which sequence (rows row0 .. row0 + q_count of every tensor) and which of its tiles.
+    int64_t qt, row0 = 0;
+    if (packed != nullptr) {
+        const IdxPackedTile t = packed[blockIdx.x / n_hg];
+        row0 = t.row0; q_count = t.len; qt = t.qt;
+    } else {
+        qt = (q_count + kIdxTileQ - 1) / kIdxTileQ - 1 - (int64_t)(blockIdx.x / n_hg);
+    }
     const int64_t q0 = qt * kIdxTileQ;
     int64_t q_hi = q0 + kIdxTileQ - 1;
     if (q_hi > q_count - 1) q_hi = q_count - 1;
@@ -93,7 +108,7 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             if (const long long late = g_debug_producer_delay; late > 0) spin_cycles(late);  // tests only
             mbar_arrive_expect_tx(&sm.a_full, NH * DI * kIdxTileQ * 128);
             for (int h = 0; h < NH; ++h)
-                for (int a = 0; a < DI; ++a) tma_load_3d(sm.a[h][a], &tm_q, a * 64, r0 + h, (int)q0, &sm.a_full);
+                for (int a = 0; a < DI; ++a) tma_load_3d(sm.a[h][a], &tm_q, a * 64, r0 + h, (int)(row0 + q0), &sm.a_full);
             for (int t = 0; t < n_tiles; ++t) {
                 const int s = t % ST;
                 if (!mbar_wait(&sm.empty[s], ((t / ST) & 1) ^ 1, abort)) {
@@ -101,7 +116,8 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     break;
                 }
                 mbar_arrive_expect_tx(&sm.full[s], DI * kIdxTileK * 128);
-                for (int a = 0; a < DI; ++a) tma_load_2d(sm.b[s][a], &tm_k, a * 64, t * kIdxTileK, &sm.full[s]);
+                for (int a = 0; a < DI; ++a)
+                    tma_load_2d(sm.b[s][a], &tm_k, a * 64, (int)row0 + t * kIdxTileK, &sm.full[s]);
             }
             if (*abort != 0) spin_cycles(200000);  // let copies already in flight land
         }
@@ -239,7 +255,7 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         }
                     }
                 } else if (valid_row) {
-                    float* out_row = scores + (q * H_kv + r0 + h) * ld_scores;
+                    float* out_row = scores + ((row0 + q) * H_kv + r0 + h) * ld_scores;
 #pragma unroll
                     for (int i = 0; i < NB; ++i) {
                         const int64_t b = key0 / BK + i;
@@ -286,7 +302,7 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     while (j2 >= 0 && pick[j2] > v) { pick[j2 + 1] = pick[j2]; --j2; }
                     pick[j2 + 1] = v;
                 }
-                int32_t* orow = block_idx + (q * H_kv + r0 + h) * (int64_t)top_k;
+                int32_t* orow = block_idx + ((row0 + q) * H_kv + r0 + h) * (int64_t)top_k;
                 for (int i = 0; i < top_k; ++i) orow[i] = i < c ? pick[i] : (i == c ? (int32_t)loc : -1);
             }
         }
@@ -295,7 +311,7 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             const int64_t qq = q0 + rr;
             if (qq >= q_count) break;
             for (int h = 0; h < NH; ++h) {
-                float* orow = scores + (qq * H_kv + r0 + h) * ld_scores;
+                float* orow = scores + ((row0 + qq) * H_kv + r0 + h) * ld_scores;
                 for (int64_t b = (q_begin + qq) / BK + 1 + lane; b < n_cols; b += 32) orow[b] = -INFINITY;
             }
         }

@@ -139,7 +139,8 @@ bool encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64
 template <int BK, int NH, int DI, int FK = 0, bool F8 = false>
 static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                     int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
-                                    int64_t n_cols, cudaStream_t st, int32_t* block_idx = nullptr) {
+                                    int64_t n_cols, cudaStream_t st, int32_t* block_idx = nullptr,
+                                    const IdxPackedTile* packed = nullptr, int64_t n_packed = 0) {
     // key-tile stages: what fits beside the NH*DI query atoms in 227 KB of shared memory (at most 3)
     constexpr int ST = (NH * DI * 16 + 3 * DI * 32 <= 224) ? 3 : 2;
     static_assert(NH * DI * 16 + ST * DI * 32 <= 224, "shared memory budget");
@@ -164,12 +165,14 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
             return MSA_ERR_CUDA;
         attr_set_dev[dev_id] = true;
     }
-    const int64_t grid = ceil_div64(q_count, kIdxTileQ) * (r.H_kv / NH);
+    // (a packed batch: q_count and kv_len are the batch's rows, for the tensor maps; the grid follows the tile list)
+    const int64_t grid = (packed != nullptr ? n_packed : ceil_div64(q_count, kIdxTileQ)) * (r.H_kv / NH);
     if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
     {
         StageScope sc(kStageIndex, st);
         index_scores_tc_kernel<BK, NH, DI, ST, FK, F8><<<(unsigned)grid, kIdxThreads, smem, st>>>(
-            tm_q, tm_k, q_begin, q_count, r.H_kv, r.index_scale, scores, ld_scores, n_cols, status, block_idx, r.k);
+            tm_q, tm_k, q_begin, q_count, r.H_kv, r.index_scale, scores, ld_scores, n_cols, status, block_idx, r.k,
+            packed);
     }
     return launch_status();
 }
@@ -210,26 +213,29 @@ static bool index_topk_fused_ok(const Resolved& r, int64_t q_count, int64_t kv_l
 
 template <int BK, int DI, bool F8 = false>
 static msa_status_t launch_index_fused_bk(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
-                                          int64_t q_count, int64_t kv_len, int32_t* block_idx, cudaStream_t st) {
+                                          int64_t q_count, int64_t kv_len, int32_t* block_idx, cudaStream_t st,
+                                          const IdxPackedTile* packed, int64_t n_packed) {
     if (r.H_kv % 2 == 0)
         return launch_index_tc<BK, 2, DI, kIdxFuseKeep, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, nullptr, 0, 0, st,
-                                                        block_idx);
+                                                        block_idx, packed, n_packed);
     return launch_index_tc<BK, 1, DI, kIdxFuseKeep, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, nullptr, 0, 0, st,
-                                                    block_idx);
+                                                    block_idx, packed, n_packed);
 }
 
+// packed != null: a packed batch of q_count = kv_len rows in all, its query tiles listed in `packed`.
 static msa_status_t run_index_topk_fused(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
-                                         int64_t q_count, int64_t kv_len, int32_t* block_idx, cudaStream_t st) {
+                                         int64_t q_count, int64_t kv_len, int32_t* block_idx, cudaStream_t st,
+                                         const IdxPackedTile* packed = nullptr, int64_t n_packed = 0) {
     if (r.idx_fp8) {
-        if (r.B_k == 64) return launch_index_fused_bk<64, 1, true>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
-        return launch_index_fused_bk<128, 1, true>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
+        if (r.B_k == 64) return launch_index_fused_bk<64, 1, true>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st, packed, n_packed);
+        return launch_index_fused_bk<128, 1, true>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st, packed, n_packed);
     }
     if (r.d_idx == 64) {
-        if (r.B_k == 64) return launch_index_fused_bk<64, 1>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
-        return launch_index_fused_bk<128, 1>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
+        if (r.B_k == 64) return launch_index_fused_bk<64, 1>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st, packed, n_packed);
+        return launch_index_fused_bk<128, 1>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st, packed, n_packed);
     }
-    if (r.B_k == 64) return launch_index_fused_bk<64, 2>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
-    return launch_index_fused_bk<128, 2>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st);
+    if (r.B_k == 64) return launch_index_fused_bk<64, 2>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st, packed, n_packed);
+    return launch_index_fused_bk<128, 2>(r, q_idx, k_idx, q_begin, q_count, kv_len, block_idx, st, packed, n_packed);
 }
 
 // Prefill ranges of at least 32 rows run on the tensor cores; shorter ones (and decode rows of
@@ -346,10 +352,11 @@ static size_t attn_per_query_bytes(const Resolved& r) {
     return (size_t)r.H_q * r.k * r.d * 2 + (size_t)r.H_q * r.k * 4 + (size_t)r.H_kv * r.k * 8;
 }
 
-static AttnPlan attn_plan(const Resolved& r, int64_t kv_len, int64_t R) {
+// n_blocks: KV blocks of the sequence (of all sequences of a packed batch).
+static AttnPlan attn_plan_blocks(const Resolved& r, int64_t n_blocks, int64_t R) {
     AttnPlan p;
     p.R = R;
-    const size_t n_tiles = (size_t)ceil_div64(kv_len, r.B_k) * r.H_kv + 1;
+    const size_t n_tiles = (size_t)n_blocks * r.H_kv + 1;
     size_t o = 0;
     p.off_cnt = o; o += align_up(n_tiles * 4);
     p.off_tile_off = o; o += align_up(n_tiles * 4);
@@ -362,14 +369,22 @@ static AttnPlan attn_plan(const Resolved& r, int64_t kv_len, int64_t R) {
     return p;
 }
 
-static int64_t attn_range_for(const Resolved& r, int64_t q_count, int64_t kv_len, size_t ws_bytes) {
-    const size_t fixed = attn_plan(r, kv_len, 0).total + 4 * kAlign;
+static AttnPlan attn_plan(const Resolved& r, int64_t kv_len, int64_t R) {
+    return attn_plan_blocks(r, ceil_div64(kv_len, r.B_k), R);
+}
+
+static int64_t attn_range_for_blocks(const Resolved& r, int64_t q_count, int64_t n_blocks, size_t ws_bytes) {
+    const size_t fixed = attn_plan_blocks(r, n_blocks, 0).total + 4 * kAlign;
     if (ws_bytes <= fixed) return 0;
     int64_t R = (int64_t)((ws_bytes - fixed) / attn_per_query_bytes(r));
     if (R > q_count) R = q_count;
     if (R > (1 << 23)) R = 1 << 23;  // handles keep the query in 24 bits
     if (R >= 128) R = R / 128 * 128;
     return R;
+}
+
+static int64_t attn_range_for(const Resolved& r, int64_t q_count, int64_t kv_len, size_t ws_bytes) {
+    return attn_range_for_blocks(r, q_count, ceil_div64(kv_len, r.B_k), ws_bytes);
 }
 
 static int current_device() {
@@ -476,14 +491,24 @@ static msa_status_t hook_copy_rows(const Resolved& r, const void* out, const flo
 }
 
 // F8: Q, K and V hold fp8 E4M3; rows of 128 bytes are moved as 64 two-byte elements.
+// The three device arrays of a packed batch (see RangeParams) and its number of blocks; all zero for one sequence.
+struct PackedBatch {
+    const int32_t* row_pos = nullptr;
+    const int32_t* row_blk0 = nullptr;
+    const int32_t* blk_row0 = nullptr;
+    int64_t n_blocks = 0;
+};
+
 template <int BK, int G, bool F8 = false>
 static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const void* k, const void* v,
                                         const int32_t* block_idx, int64_t q_begin, int64_t q_count,
                                         int64_t kv_len, void* out, float* lse, void* ws, size_t ws_bytes,
-                                        cudaStream_t st) {
-    const int64_t R = attn_range_for(r, q_count, kv_len, ws_bytes);
+                                        cudaStream_t st, const PackedBatch& pk = PackedBatch()) {
+    const bool packed = pk.row_pos != nullptr;
+    const int64_t all_blocks = packed ? pk.n_blocks : ceil_div64(kv_len, BK);
+    const int64_t R = attn_range_for_blocks(r, q_count, all_blocks, ws_bytes);
     if (R <= 0) return MSA_ERR_WORKSPACE;
-    const AttnPlan pl = attn_plan(r, kv_len, R);
+    const AttnPlan pl = attn_plan_blocks(r, all_blocks, R);
     char* w = static_cast<char*>(ws);
     int32_t* cnt = (int32_t*)(w + pl.off_cnt);
     int32_t* tile_off = (int32_t*)(w + pl.off_tile_off);
@@ -532,11 +557,13 @@ static msa_status_t run_attn_prefill_tc(const Resolved& r, const void* q, const 
     const float scale_log2e = r.softmax_scale * 1.4426950408889634f;
     const int grid_attn = sm_count();  // one CTA per SM (all of its shared memory and TMEM)
     for (int64_t q_first = 0; q_first < q_count; q_first += R) {
-        RangeParams p;
+        RangeParams p = {};
         p.q_begin = q_begin; p.q_first = q_first;
         p.q_count = (int32_t)((q_count - q_first) < R ? (q_count - q_first) : R);
-        p.n_blocks = (int32_t)ceil_div64(q_begin + q_first + p.q_count, BK);
+        // one sequence: the blocks up to the range's last query; a packed batch: all of its blocks
+        p.n_blocks = (int32_t)(packed ? all_blocks : ceil_div64(q_begin + q_first + p.q_count, BK));
         p.H_kv = r.H_kv; p.top_k = r.k;
+        p.row_pos = pk.row_pos; p.row_blk0 = pk.row_blk0; p.blk_row0 = pk.blk_row0;
         const int n_tiles = p.n_blocks * r.H_kv;
         const unsigned eg = (unsigned)ceil_div64((int64_t)p.q_count * r.H_kv, 8);  // 8 warps (rows) per CTA
         if (cudaMemsetAsync(cnt, 0, (size_t)(n_tiles + 1) * 4, st) != cudaSuccess) return MSA_ERR_CUDA;
@@ -722,7 +749,7 @@ static msa_status_t run_index_lse(const Resolved& r, const void* q_idx, const vo
     if (per_sm > 4) per_sm = 4;
     const int grid = sm_count() * per_sm;
     for (int64_t q_first = 0; q_first < q_count; q_first += R) {
-        RangeParams p;
+        RangeParams p = {};
         p.q_begin = q_begin; p.q_first = q_first;
         p.q_count = (int32_t)((q_count - q_first) < R ? (q_count - q_first) : R);
         p.n_blocks = (int32_t)ceil_div64(q_begin + q_first + p.q_count, BK);
@@ -972,6 +999,42 @@ msa_status_t msa_sparse_attn_prefill_workspace_bytes(const msa_shape_t* shape, i
     return MSA_OK;
 }
 
+// The tensor-core attention for the shape's (B_k, G), bf16 or fp8 operands; pk: a packed batch or nothing.
+static msa_status_t attn_prefill_tc_dispatch(const Resolved& r, bool f8, const void* q, const void* k, const void* v,
+                                             const int32_t* block_idx, int64_t q_begin, int64_t q_count, int64_t kv_len,
+                                             void* out, float* lse, void* ws, size_t ws_bytes, cudaStream_t st,
+                                             const PackedBatch& pk = PackedBatch()) {
+#define MSA_ATTN_CASE(BK_, G_)                                                                                              \
+    if (r.B_k == BK_ && r.G == G_)                                                                                          \
+        return f8 ? run_attn_prefill_tc<BK_, G_, true>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, ws,      \
+                                                        ws_bytes, st, pk)                                                    \
+                  : run_attn_prefill_tc<BK_, G_, false>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, ws,     \
+                                                         ws_bytes, st, pk);
+    MSA_ATTN_CASE(64, 8)
+    MSA_ATTN_CASE(64, 16)
+    MSA_ATTN_CASE(128, 8)
+    MSA_ATTN_CASE(128, 16)
+#undef MSA_ATTN_CASE
+    return MSA_ERR_UNSUPPORTED;
+}
+
+// fp8 E4M3 -> bf16 copies of `rows` K and V rows into kb and vb (exact).
+static msa_status_t widen_kv(const Resolved& r, const void* k, const void* v, int64_t rows, char* kb, char* vb,
+                             cudaStream_t st) {
+    if (r.d % 16 != 0) return MSA_ERR_UNSUPPORTED;  // the conversion moves 16 elements per thread
+    const int64_t n16 = rows * r.H_kv * r.d / 16;
+    const unsigned grid = (unsigned)(n16 < 148 * 8 * 256 ? ceil_div64(n16 > 0 ? n16 : 1, 256) : 148 * 8);
+    {
+        StageScope sc(kStageAttn, st);
+        e4m3_to_bf16_kernel<<<grid, 256, 0, st>>>((const uint4*)k, (uint4*)kb, n16);
+    }
+    {
+        StageScope sc(kStageAttn, st);
+        e4m3_to_bf16_kernel<<<grid, 256, 0, st>>>((const uint4*)v, (uint4*)vb, n16);
+    }
+    return cudaPeekAtLastError() == cudaSuccess ? MSA_OK : MSA_ERR_CUDA;
+}
+
 msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, const void* k,
                                      const void* v, const int32_t* block_idx, int64_t q_begin,
                                      int64_t q_count, int64_t kv_len, void* out, float* lse,
@@ -988,46 +1051,23 @@ msa_status_t msa_sparse_attn_prefill(const msa_shape_t* shape, const void* q, co
     msa_sparse_attn_prefill_workspace_bytes(shape, q_count, kv_len, &need, nullptr);
     if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
-    if (attn_fp8_direct(r, kv_len)) {
-        if (r.B_k == 64 && r.G == 8)
-            return run_attn_prefill_tc<64, 8, true>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
-        if (r.B_k == 64 && r.G == 16)
-            return run_attn_prefill_tc<64, 16, true>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
-        if (r.B_k == 128 && r.G == 8)
-            return run_attn_prefill_tc<128, 8, true>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
-        return run_attn_prefill_tc<128, 16, true>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
-    }
+    if (attn_fp8_direct(r, kv_len))
+        return attn_prefill_tc_dispatch(r, true, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace,
+                                        workspace_bytes, st);
     if (r.q_fp8) return MSA_ERR_UNSUPPORTED;  // fp8 Q: the tensor-core kernel's shapes only
     if (r.kv_fp8) {  // bf16 copies of the visible rows, then the bf16 path on the rest of the workspace
-        if (r.d % 16 != 0) return MSA_ERR_UNSUPPORTED;  // the conversion moves 16 elements per thread
         const size_t cb = kv_copy_bytes(r, kv_len);
-        const int64_t n16 = kv_len * r.H_kv * r.d / 16;
         char* kb = (char*)workspace;
         char* vb = kb + cb;
-        const unsigned grid = (unsigned)(n16 < 148 * 8 * 256 ? ceil_div64(n16 > 0 ? n16 : 1, 256) : 148 * 8);
-        {
-            StageScope sc(kStageAttn, st);
-            e4m3_to_bf16_kernel<<<grid, 256, 0, st>>>((const uint4*)k, (uint4*)kb, n16);
-        }
-        {
-            StageScope sc(kStageAttn, st);
-            e4m3_to_bf16_kernel<<<grid, 256, 0, st>>>((const uint4*)v, (uint4*)vb, n16);
-        }
-        if (cudaPeekAtLastError() != cudaSuccess) return MSA_ERR_CUDA;
+        if ((s = widen_kv(r, k, v, kv_len, kb, vb, st)) != MSA_OK) return s;
         msa_shape_t wide = *shape;
         wide.kv_fp8 = 0;
         return msa_sparse_attn_prefill(&wide, q, kb, vb, block_idx, q_begin, q_count, kv_len, out, lse,
                                        (char*)workspace + 2 * cb, workspace_bytes - 2 * cb, stream);
     }
-    if (attn_tc_supported(r) && kv_len < 2147483647LL) {
-        if (r.B_k == 64 && r.G == 8)
-            return run_attn_prefill_tc<64, 8>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
-        if (r.B_k == 64 && r.G == 16)
-            return run_attn_prefill_tc<64, 16>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
-        if (r.B_k == 128 && r.G == 8)
-            return run_attn_prefill_tc<128, 8>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
-        return run_attn_prefill_tc<128, 16>(r, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace, workspace_bytes, st);
-    }
+    if (attn_tc_supported(r) && kv_len < 2147483647LL)
+        return attn_prefill_tc_dispatch(r, false, q, k, v, block_idx, q_begin, q_count, kv_len, out, lse, workspace,
+                                        workspace_bytes, st);
     return run_attn_generic(r, q, k, v, block_idx, prefill_rows(q_begin, kv_len, r.B_k), q_count, out,
                             lse, st);
 }
@@ -1283,11 +1323,68 @@ static msa_status_t check_cu_seqlens(const int64_t* cu, int32_t n_seqs) {
     return MSA_OK;
 }
 
-// Sequences of at most kVarlenSmallTokens leave much of the GPU idle at the ends of their kernels:
-// such sequences, independent problems, run on up to kVarlenLanes streams of the library's own, each
-// on its own slice of the workspace, forked from and joined to the caller's stream with events.
-constexpr int kVarlenLanes = 4;
-constexpr int64_t kVarlenSmallTokens = 8192;
+// ---------------------------------------------------------------------- packed batches
+// A batch of sequences packed token-major runs as ONE problem per stage where the kernels allow:
+// the fused index + Top-k kernel takes the query tiles of all sequences from one list (longest key
+// prefix first), and the KV-outer attention numbers its blocks through the batch, so that one
+// reverse index, one item list, one attention launch and one merge serve every sequence of a query
+// range.  What the kernels need for that sits in front of the workspace: the row offsets, the block
+// offsets, the tile list, and per row / per block the three arrays of RangeParams.
+struct VarlenPlan {
+    bool packed;            // the tensor-core attention runs once over the whole batch
+    bool fused;             // Eq. 6 + Eq. 7 in one launch over the whole batch (top_k <= 16)
+    int64_t rows, n_blocks, n_idx_tiles;
+    size_t off_cu, off_blk_cum, off_tiles, off_row_pos, off_row_blk0, off_blk_row0, meta;  // bytes
+    size_t copies;          // bf16 copies of fp8 K and V (bf16 Q), in all
+    size_t stage_min, stage_pref;
+};
+
+static msa_status_t varlen_plan(const msa_shape_t* shape, const Resolved& r, const int64_t* cu, int32_t n_seqs,
+                                VarlenPlan& vp) {
+    vp = VarlenPlan();
+    vp.rows = cu[n_seqs] - cu[0];
+    for (int32_t i = 0; i < n_seqs; ++i) {
+        const int64_t T = cu[i + 1] - cu[i];
+        vp.n_blocks += ceil_div64(T, r.B_k);
+        vp.n_idx_tiles += ceil_div64(T, kIdxTileQ);
+    }
+    vp.packed = n_seqs > 1 && attn_tc_supported(r) && vp.rows < 2147483647LL && vp.n_blocks < (1 << 24);
+    vp.fused = vp.packed && index_topk_fused_ok(r, vp.rows, vp.rows);
+    // stages 1-2 (and, unpacked, stage 3) sequence by sequence: what the largest sequence needs
+    size_t seq_min = kAlign, seq_pref = kAlign;
+    for (int32_t i = 0; i < n_seqs; ++i) {
+        size_t a = 0, b = 0;
+        const msa_status_t st = msa_prefill_forward_workspace_bytes(shape, cu[i + 1] - cu[i], &a, &b);
+        if (st != MSA_OK) return st;
+        if (a > seq_min) seq_min = a;
+        if (b > seq_pref) seq_pref = b;
+    }
+    if (!vp.packed) {
+        vp.stage_min = seq_min; vp.stage_pref = seq_pref;
+        return MSA_OK;
+    }
+    size_t o = 0;
+    vp.off_cu = o; o += align_up((size_t)(n_seqs + 1) * 8);
+    vp.off_blk_cum = o; o += align_up((size_t)(n_seqs + 1) * 4);
+    vp.off_tiles = o; o += align_up((size_t)vp.n_idx_tiles * sizeof(IdxPackedTile));
+    vp.off_row_pos = o; o += align_up((size_t)vp.rows * 4);
+    vp.off_row_blk0 = o; o += align_up((size_t)vp.rows * 4);
+    vp.off_blk_row0 = o; o += align_up((size_t)vp.n_blocks * 4);
+    vp.meta = o;
+    vp.copies = (r.kv_fp8 && !r.q_fp8) ? 2 * kv_copy_bytes(r, vp.rows) : 0;
+    const int64_t r_min = vp.rows < 256 ? vp.rows : 256;
+    int64_t r_pref = (int64_t)((32ull << 30) / attn_per_query_bytes(r));
+    if (r_pref > vp.rows) r_pref = vp.rows;
+    if (r_pref < r_min) r_pref = r_min;
+    size_t a_min = attn_plan_blocks(r, vp.n_blocks, r_min).total + 8 * kAlign;
+    size_t a_pref = attn_plan_blocks(r, vp.n_blocks, r_pref).total + 8 * kAlign;
+    if (!vp.fused) {  // score chunks of the longest sequence share the region with the attention's buffers
+        if (seq_min > a_min) a_min = seq_min;
+        if (seq_pref > a_pref) a_pref = seq_pref;
+    }
+    vp.stage_min = a_min; vp.stage_pref = a_pref;
+    return MSA_OK;
+}
 
 msa_status_t msa_prefill_forward_varlen_workspace_bytes(const msa_shape_t* shape,
                                                         const int64_t* cu_seqlens, int32_t n_seqs,
@@ -1296,18 +1393,10 @@ msa_status_t msa_prefill_forward_varlen_workspace_bytes(const msa_shape_t* shape
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
     if ((s = check_cu_seqlens(cu_seqlens, n_seqs)) != MSA_OK) return s;
-    size_t mn = kAlign, pf = kAlign, pf_small = 0;
-    for (int32_t i = 0; i < n_seqs; ++i) {
-        size_t a = 0, b = 0;
-        const int64_t T = cu_seqlens[i + 1] - cu_seqlens[i];
-        if ((s = msa_prefill_forward_workspace_bytes(shape, T, &a, &b)) != MSA_OK) return s;
-        if (a > mn) mn = a;
-        if (b > pf) pf = b;
-        if (T <= kVarlenSmallTokens && b > pf_small) pf_small = b;
-    }
-    if (n_seqs > 1 && kVarlenLanes * align_up(pf_small) > pf) pf = kVarlenLanes * align_up(pf_small);
-    if (min_bytes) *min_bytes = mn;
-    if (preferred_bytes) *preferred_bytes = pf;
+    VarlenPlan vp;
+    if ((s = varlen_plan(shape, r, cu_seqlens, n_seqs, vp)) != MSA_OK) return s;
+    if (min_bytes) *min_bytes = vp.meta + vp.copies + vp.stage_min;
+    if (preferred_bytes) *preferred_bytes = vp.meta + vp.copies + vp.stage_pref;
     return MSA_OK;
 }
 
@@ -1322,72 +1411,106 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
     if ((s = check_cu_seqlens(cu_seqlens, n_seqs)) != MSA_OK) return s;
     if (n_seqs == 0 || cu_seqlens[n_seqs] == cu_seqlens[0]) return MSA_OK;
     if (!q || !k || !v || !q_idx || !k_idx || !out || !block_idx) return MSA_ERR_INVALID_ARG;
-    size_t need = 0;
-    if ((s = msa_prefill_forward_varlen_workspace_bytes(shape, cu_seqlens, n_seqs, &need, nullptr)) != MSA_OK)
-        return s;
-    if (workspace == nullptr || workspace_bytes < need || !aligned16(workspace)) return MSA_ERR_WORKSPACE;
-    // Every sequence is an independent problem: the single-sequence path on row-offset pointers.
+    VarlenPlan vp;
+    if ((s = varlen_plan(shape, r, cu_seqlens, n_seqs, vp)) != MSA_OK) return s;
+    if (workspace == nullptr || workspace_bytes < vp.meta + vp.copies + vp.stage_min || !aligned16(workspace))
+        return MSA_ERR_WORKSPACE;
     const size_t q_row = (size_t)r.H_q * r.d * r.q_elt(), o_row = (size_t)r.H_q * r.d * 2;
     const size_t kv_row = (size_t)r.H_kv * r.d * r.kv_elt();
     const size_t qi_row = (size_t)r.H_kv * r.d_idx * r.idx_elt(), ki_row = (size_t)r.d_idx * r.idx_elt();
     cudaStream_t st = (cudaStream_t)stream;
-    static cudaStream_t lanes_dev[64][kVarlenLanes] = {};
-    cudaStream_t* lanes = lanes_dev[current_device()];
-    const size_t slice = (workspace_bytes / kVarlenLanes) & ~(size_t)(kAlign - 1);
-    bool forked[kVarlenLanes] = {};   // lanes that hold work since the last join
-    cudaEvent_t fork_ev = nullptr;    // marks the caller's stream after the last join
-    int next_lane = 0;
-    auto join = [&]() -> bool {
-        for (int l = 0; l < kVarlenLanes; ++l) {
-            if (!forked[l]) continue;
-            cudaEvent_t e = next_sync_event();
-            if (!e || cudaEventRecord(e, lanes[l]) != cudaSuccess || cudaStreamWaitEvent(st, e, 0) != cudaSuccess)
-                return false;
-            forked[l] = false;
+    const int64_t row0 = cu_seqlens[0];
+    if (!vp.packed) {  // every sequence through the single-sequence path, one after the other
+        for (int32_t i = 0; i < n_seqs; ++i) {
+            const int64_t o = cu_seqlens[i], T = cu_seqlens[i + 1] - o;
+            if (T == 0) continue;
+            s = msa_prefill_forward(shape, (const char*)q + o * q_row, (const char*)k + o * kv_row,
+                                    (const char*)v + o * kv_row, (const char*)q_idx + o * qi_row,
+                                    (const char*)k_idx + o * ki_row, T, (char*)out + o * o_row,
+                                    lse ? lse + o * r.H_q : nullptr, block_idx + o * (int64_t)r.H_kv * r.k, workspace,
+                                    workspace_bytes, stream);
+            if (s != MSA_OK) return s;
         }
-        fork_ev = nullptr;
-        return true;
-    };
-    msa_status_t result = MSA_OK;
-    for (int32_t i = 0; i < n_seqs && result == MSA_OK; ++i) {
-        const int64_t o = cu_seqlens[i], T = cu_seqlens[i + 1] - o;
-        if (T == 0) continue;
-        size_t mn = 0, pf = 0;
-        if ((result = msa_prefill_forward_workspace_bytes(shape, T, &mn, &pf)) != MSA_OK) break;
-        const bool on_lane = n_seqs > 1 && T <= kVarlenSmallTokens && pf <= slice;
-        cudaStream_t run = st;
-        char* ws = (char*)workspace;
-        size_t ws_bytes = workspace_bytes;
-        if (on_lane) {
-            const int l = next_lane;
-            next_lane = (next_lane + 1) % kVarlenLanes;
-            if (lanes[l] == nullptr && cudaStreamCreateWithFlags(&lanes[l], cudaStreamNonBlocking) != cudaSuccess) {
-                result = MSA_ERR_CUDA;
-                break;
-            }
-            if (!forked[l]) {  // the lane starts behind what the caller's stream holds now
-                if (fork_ev == nullptr) {
-                    fork_ev = next_sync_event();
-                    if (!fork_ev || cudaEventRecord(fork_ev, st) != cudaSuccess) { result = MSA_ERR_CUDA; break; }
-                }
-                if (cudaStreamWaitEvent(lanes[l], fork_ev, 0) != cudaSuccess) { result = MSA_ERR_CUDA; break; }
-                forked[l] = true;
-            }
-            run = lanes[l];
-            ws += (size_t)l * slice;
-            ws_bytes = slice;
-        } else if (!join()) {  // the whole workspace: behind every lane
-            result = MSA_ERR_CUDA;
-            break;
-        }
-        result = msa_prefill_forward(shape, (const char*)q + o * q_row, (const char*)k + o * kv_row,
-                                     (const char*)v + o * kv_row, (const char*)q_idx + o * qi_row,
-                                     (const char*)k_idx + o * ki_row, T, (char*)out + o * o_row,
-                                     lse ? lse + o * r.H_q : nullptr, block_idx + o * (int64_t)r.H_kv * r.k, ws,
-                                     ws_bytes, (msa_stream_t)run);
+        return MSA_OK;
     }
-    if (!join() && result == MSA_OK) result = MSA_ERR_CUDA;  // (also on an error: no lane is left unjoined)
-    return result;
+    // ---- the batch's maps: offsets and the tile list from the host, the per-row arrays by a kernel
+    char* w = static_cast<char*>(workspace);
+    int64_t* cu_dev = (int64_t*)(w + vp.off_cu);
+    int32_t* blk_cum_dev = (int32_t*)(w + vp.off_blk_cum);
+    IdxPackedTile* tiles_dev = (IdxPackedTile*)(w + vp.off_tiles);
+    int32_t* row_pos = (int32_t*)(w + vp.off_row_pos);
+    int32_t* row_blk0 = (int32_t*)(w + vp.off_row_blk0);
+    int32_t* blk_row0 = (int32_t*)(w + vp.off_blk_row0);
+    {
+        // (pageable host memory: the runtime has copied it out when the call returns)
+        int32_t* blk_cum = (int32_t*)malloc((size_t)(n_seqs + 1) * 4);
+        IdxPackedTile* tiles = (IdxPackedTile*)malloc((size_t)(vp.n_idx_tiles > 0 ? vp.n_idx_tiles : 1) * sizeof(IdxPackedTile));
+        if (!blk_cum || !tiles) { free(blk_cum); free(tiles); return MSA_ERR_CUDA; }
+        blk_cum[0] = 0;
+        int64_t max_qt = 0;
+        for (int32_t i = 0; i < n_seqs; ++i) {
+            const int64_t T = cu_seqlens[i + 1] - cu_seqlens[i];
+            blk_cum[i + 1] = blk_cum[i] + (int32_t)ceil_div64(T, r.B_k);
+            if (ceil_div64(T, kIdxTileQ) > max_qt) max_qt = ceil_div64(T, kIdxTileQ);
+        }
+        // longest key prefix first: by tile number inside the sequence, descending
+        int64_t n = 0;
+        for (int64_t qt = max_qt - 1; qt >= 0; --qt)
+            for (int32_t i = 0; i < n_seqs; ++i) {
+                const int64_t T = cu_seqlens[i + 1] - cu_seqlens[i];
+                if (qt < ceil_div64(T, kIdxTileQ)) {
+                    tiles[n].row0 = (int32_t)(cu_seqlens[i] - row0); tiles[n].len = (int32_t)T; tiles[n].qt = (int32_t)qt;
+                    ++n;
+                }
+            }
+        bool ok = cudaMemcpyAsync(cu_dev, cu_seqlens, (size_t)(n_seqs + 1) * 8, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+                  cudaMemcpyAsync(blk_cum_dev, blk_cum, (size_t)(n_seqs + 1) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+                  (n == 0 || cudaMemcpyAsync(tiles_dev, tiles, (size_t)n * sizeof(IdxPackedTile), cudaMemcpyHostToDevice, st) == cudaSuccess);
+        free(blk_cum);
+        free(tiles);
+        if (!ok) return MSA_ERR_CUDA;
+    }
+    {
+        const int64_t work = vp.rows + vp.n_blocks;
+        const unsigned grid = (unsigned)(ceil_div64(work, 256) < 148 * 8 ? ceil_div64(work, 256) : 148 * 8);
+        StageScope sc(kStageSchedule, st);
+        packed_map_kernel<<<grid, 256, 0, st>>>(cu_dev, blk_cum_dev, n_seqs, r.B_k, row_pos, row_blk0, blk_row0);
+    }
+    if (cudaPeekAtLastError() != cudaSuccess) return MSA_ERR_CUDA;
+    // tensors of the batch start at its first row
+    const char* qb = (const char*)q + row0 * q_row;
+    const char* kb = (const char*)k + row0 * kv_row;
+    const char* vb = (const char*)v + row0 * kv_row;
+    const char* qib = (const char*)q_idx + row0 * qi_row;
+    const char* kib = (const char*)k_idx + row0 * ki_row;
+    int32_t* bi = block_idx + row0 * (int64_t)r.H_kv * r.k;
+    char* stage = w + vp.meta + vp.copies;
+    const size_t stage_bytes = workspace_bytes - vp.meta - vp.copies;
+    // ---- stages 1-2
+    if (vp.fused) {
+        s = run_index_topk_fused(r, qib, kib, 0, vp.rows, vp.rows, bi, st, tiles_dev, vp.n_idx_tiles);
+        if (s != MSA_OK) return s;
+    } else {
+        for (int32_t i = 0; i < n_seqs; ++i) {
+            const int64_t o = cu_seqlens[i], T = cu_seqlens[i + 1] - o;
+            if (T == 0) continue;
+            s = prefill_stages_1_2(shape, r, (const char*)q_idx + o * qi_row, (const char*)k_idx + o * ki_row, T,
+                                   block_idx + o * (int64_t)r.H_kv * r.k, stage, stage_bytes, stream);
+            if (s != MSA_OK) return s;
+        }
+    }
+    // ---- stage 3, once over the batch
+    PackedBatch pk;
+    pk.row_pos = row_pos; pk.row_blk0 = row_blk0; pk.blk_row0 = blk_row0; pk.n_blocks = vp.n_blocks;
+    const bool f8 = r.q_fp8 && r.kv_fp8;
+    if (vp.copies) {  // fp8 K/V caches with bf16 Q: bf16 copies of all rows first
+        char* kw = w + vp.meta;
+        char* vw = kw + vp.copies / 2;
+        if ((s = widen_kv(r, kb, vb, vp.rows, kw, vw, st)) != MSA_OK) return s;
+        kb = kw; vb = vw;
+    }
+    return attn_prefill_tc_dispatch(r, f8, qb, kb, vb, bi, 0, vp.rows, vp.rows, (char*)out + row0 * o_row,
+                                    lse ? lse + row0 * r.H_q : nullptr, stage, stage_bytes, st, pk);
 }
 
 static size_t host_staging_bytes(const Resolved& r, int64_t T, size_t off[8]) {

@@ -138,11 +138,11 @@ def test_varlen_batch_equals_sequence_by_sequence():
 
 
 @pytest.mark.parametrize("ws", ["preferred", "minimum"])
-def test_varlen_short_sequences_side_by_side_and_long_ones_between(ws):
-    # Short sequences run on the library's own streams, each on a quarter of the workspace; a long
-    # one (more than 8192 tokens) waits for them, takes the whole workspace, and the next short ones
-    # start behind it.  With the minimum workspace everything runs on the caller's stream.  Either
-    # way every sequence must come out exactly as from its own call.
+def test_varlen_short_and_long_sequences_in_one_batch(ws):
+    # Short and long sequences mixed, an empty one, one of exactly 64 blocks: the batch runs as one
+    # problem per stage (one fused index + Top-k launch, one reverse index / attention / merge per
+    # query range, which spans sequence boundaries; many ranges with the minimum workspace).
+    # Every sequence must come out exactly as from its own call.
     cfg = CONFIGS["c3"].scaled(name="c3-varlen-mix", T=0, top_k=8)
     lens = [3000, 700, 9000, 0, 500, 64, 100, 2000, 1500, 12000, 300, 8192]
     cu = np.concatenate([[0], np.cumsum(lens)]).tolist()
@@ -714,32 +714,6 @@ def test_decode_and_prefill_calls_replay_from_a_cuda_graph():
     _assert_clean()
     assert torch.equal(want[2], pi) and torch.equal(want[0], po) and torch.equal(want[1], pl)
 
-    # the packed call: its short sequences fork onto the library's streams inside the capture
-    lens = [700, 3000, 9000, 64, 1500]
-    cu = np.concatenate([[0], np.cumsum(lens)]).tolist()
-    vcfg = CONFIGS["c3"].scaled(name="c3-graph-varlen", T=cu[-1], top_k=8)
-    vx = make_prefill_inputs(vcfg, DEV, sharp=True)
-    vshape = B.shape_of(vcfg)
-    vo = torch.empty_like(vx["q"])
-    vl = torch.empty((vcfg.T, vcfg.n_q_heads), dtype=torch.float32, device=DEV)
-    vi = torch.empty((vcfg.T, vcfg.n_kv_heads, vcfg.top_k), dtype=torch.int32, device=DEV)
-    vws = B.alloc_workspace(B.msa_prefill_forward_varlen_workspace_bytes(vshape, cu)[1], DEV)
-
-    def vstep():
-        B.msa_prefill_forward_varlen(vshape, vx["q"], vx["k"], vx["v"], vx["q_idx"], vx["k_idx"], cu, vo, vl, vi, vws)
-    with torch.cuda.stream(side):
-        vstep()
-    torch.cuda.synchronize()
-    want = (vo.clone(), vl.clone(), vi.clone())
-    vg = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(vg):
-        vstep()
-    vo.zero_(); vl.zero_(); vi.zero_()
-    vg.replay()
-    torch.cuda.synchronize()
-    _assert_clean()
-    assert torch.equal(want[2], vi) and torch.equal(want[0], vo) and torch.equal(want[1], vl)
-
 
 # ----------------------------------------------------------------- fp8 E4M3 K/V caches (decode, Section 4.2)
 @pytest.mark.parametrize("Hq,Hkv,Bk,k,lens", [
@@ -953,3 +927,36 @@ def test_fp8_q_is_rejected_where_it_is_not_supported():
                                  torch.tensor([300], dtype=torch.int32, device=DEV), 1, I[:1].contiguous(),
                                  out[:1].contiguous(), None, ws)
     assert e.value.code == 2
+
+
+def test_varlen_batch_with_larger_top_k_and_a_row_offset():
+    # top_k above the fused kernel's limit: stages 1-2 run sequence by sequence, stage 3 once over the
+    # batch; the batch starts at a row offset inside the tensors (cu_seqlens[0] > 0).
+    cfg = CONFIGS["c3"].scaled(name="c3-varlen-k64", T=0)
+    lens = [9000, 130, 2500, 1]
+    cu = (np.concatenate([[0], np.cumsum(lens)]) + 384).tolist()
+    total = cu[-1] + 77   # rows before and after the batch that the call must leave alone
+    x = make_prefill_inputs(cfg.scaled(T=total), DEV, sharp=True)
+    shape = B.shape_of(cfg)
+    out = torch.full((total, cfg.n_q_heads, 128), 7.0, dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((total, cfg.n_q_heads), 7.0, dtype=torch.float32, device=DEV)
+    I = torch.full((total, cfg.n_kv_heads, cfg.top_k), -7, dtype=torch.int32, device=DEV)
+    mn, pf = B.msa_prefill_forward_varlen_workspace_bytes(shape, cu)
+    B.msa_prefill_forward_varlen(shape, x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"], cu, out, lse, I,
+                                 B.alloc_workspace(mn, DEV))
+    torch.cuda.synchronize()
+    _assert_clean()
+    assert bool((out[:384] == 7.0).all()) and bool((out[cu[-1]:] == 7.0).all()) and bool((I[:384] == -7).all())
+    for s_, L in enumerate(lens):
+        a, b = cu[s_], cu[s_ + 1]
+        xs = {n: t[a:b].contiguous() for n, t in x.items()}
+        o1, l1, i1 = api.prefill_forward(cfg.scaled(T=L), xs)
+        assert torch.equal(I[a:b], i1) and torch.equal(out[a:b], o1) and torch.equal(lse[a:b], l1), "sequence %d" % s_
+    # oracle on the first sequence through the batch call's outputs
+    a, b, L = cu[0], cu[1], lens[0]
+    pos = sample_positions(L, cfg.block_size, cfg.top_k, 48, 5)
+    pos_t = torch.from_numpy(pos).to(DEV)
+    I_gpu = I[a:b][pos_t].cpu().numpy()
+    O_ref, LSE_ref = oracle.sparse_attn(to_bits(x["q"][a:b][pos_t]), to_bits(x["k"][a:b]), to_bits(x["v"][a:b]), I_gpu,
+                                        pos, cfg.block_size)
+    check_attn(out[a:b][pos_t].float().cpu().numpy(), lse[a:b][pos_t].cpu().numpy(), O_ref, LSE_ref, "varlen k64")
