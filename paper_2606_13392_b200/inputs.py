@@ -101,6 +101,9 @@ CONFIGS: Dict[str, MSAConfig] = {
     # eight index heads of a query tile in one CTA).
     "c3-40k": MSAConfig("c3-40k", "prefill", 40960, 64, 8, 128, 64, seed=2,
                         planted_frac=0.05, planted_shift=2.0),
+    # 296 query tiles = two full waves of the 148 one-per-SM CTAs of the full-size index kernel.
+    "c3-37k": MSAConfig("c3-37k", "prefill", 37888, 64, 8, 128, 64, seed=2,
+                        planted_frac=0.05, planted_shift=2.0),
     # Decode with the K/V caches stored in fp8 E4M3 (C5's shapes), with the cached index keys in fp8 as
     # well (c5-f8), and the paper's regime with both in fp8.
     "c5-kv8": MSAConfig("c5-kv8", "decode", 1048576, 64, 8, 128, 64, seed=4,
