@@ -182,7 +182,9 @@ NCU_TRAFFIC = {
                             "kernel": "topk_select_kernel<2>", "scale": 1.0},
     # attention: 18.5 GB read + 33.7 GB written per query range; half of the Q gathers hit L2
     ("c4", "attn_prefill"): {"bytes": 52.2e9, "captured": "c4, one query range",
-                             "kernel": "attn_prefill_tc_kernel<128,8>, one CTA per SM", "scale": 1.0},
+                             "kernel": "attn_prefill_tc_kernel<128,8>, one CTA per SM (before the packed-batch row "
+                                       "indirection and the fp8 template flag were added; same memory accesses)",
+                             "scale": 1.0},
     ("c4", "combine"): {"bytes": 34.30e9, "captured": "c4, one query range", "kernel": "combine_kernel<128,8>",
                         "scale": 1.0},
     ("c3", "attn_prefill"): {"bytes": 39.96e9, "captured": "c3, one query range",
@@ -202,7 +204,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=None,
-                    help="c1..c5 (default: c4 as the headline, plus short c3 and c5 runs reported under 'others')")
+                    help="c1..c5 (default: c4 as the headline, plus short c3, c5, c2 and c1 runs reported under 'others')")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -219,7 +221,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     primary = args.workload or "c4"
-    extras = [] if (args.workload or args.no_others) else ["c3", "c5"]
+    extras = [] if (args.workload or args.no_others) else ["c3", "c5", "c2", "c1"]
     cfg = CONFIGS[primary]
     if args.impl == "reference":
         if rank == 0:

@@ -25,6 +25,14 @@ def test_c2_full_size_sampled():
     _free()
 
 
+def test_c2_full_size_every_position():
+    # The whole sequence in the oracle: every query position, every head (a few minutes of host time).
+    stats = run_prefill_case(CONFIGS["c2"], True, n_sample=10 ** 9)
+    assert stats["rows"] == 32768 * 8 and stats["exact_sets"] >= 0.9995
+    print("c2 full", stats)
+    _free()
+
+
 def test_c3_full_size_sampled():
     stats = run_prefill_case(CONFIGS["c3"], False, n_sample=256)
     assert stats["exact_sets"] >= 0.999
@@ -55,8 +63,9 @@ def test_c5_decode_full_batch():
 
 
 # The paper's own regime at full length (bench workloads p1m, p1m-f8, pdec-f8): fused index + Top-k,
-# G = 16 attention, fp8 index operands, and prefill onto fp8 K/V caches (p1m-f8kv).
-@pytest.mark.parametrize("name", ["p1m", "p1m-f8", "p1m-f8kv"])
+# G = 16 attention, fp8 index operands, prefill onto fp8 K/V caches (p1m-f8kv) and with Q in fp8 as
+# well (p1m-f8qkv); C4's shapes with Q, K, V in fp8 (c4-f8qkv).
+@pytest.mark.parametrize("name", ["p1m", "p1m-f8", "p1m-f8kv", "p1m-f8qkv", "c4-f8qkv"])
 def test_paper_regime_1m_sampled(name):
     stats = run_prefill_case(CONFIGS[name], True, n_sample=96)
     assert stats["exact_sets"] >= 0.995
