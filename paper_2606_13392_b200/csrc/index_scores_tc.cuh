@@ -181,6 +181,14 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
                 for (int i = 0; i < FK; ++i) { ts[h][i] = -INFINITY; tb[h][i] = -1; }
         }
+        // Scores leave one unit late: a unit's maxima are stored while the next unit's accumulator is on
+        // its way to the registers, so that the store and its address arithmetic do not sit between the
+        // release of one accumulator and the wait for the next.
+        constexpr int NBP = 128 / BK;
+        float pend[NBP];
+        float* pend_ptr = nullptr;
+        int pend_n = 0;
+        float* const row_base = FK == 0 ? scores + ((row0 + q) * H_kv + r0) * ld_scores : nullptr;
         for (int t = 0; live && t < n_tiles; ++t) {
             const int64_t key0 = (int64_t)t * kIdxTileK + half * 128;
             const bool need_mask = key0 + 127 > pos;
@@ -223,6 +231,10 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     uint32_t v[4][32];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) tmem_ld_32x32(taddr + c * 32, v[c]);
+#pragma unroll
+                    for (int i = 0; i < NB; ++i)
+                        if (i < pend_n) pend_ptr[i] = pend[i];
+                    pend_n = 0;
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
@@ -255,14 +267,19 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         }
                     }
                 } else if (valid_row) {
-                    float* out_row = scores + ((row0 + q) * H_kv + r0 + h) * ld_scores;
+                    const int64_t b0 = key0 / BK;  // this thread's blocks b0 .. b0 + NB - 1; those up to loc are visible
+                    pend_ptr = row_base + h * ld_scores + b0;
 #pragma unroll
-                    for (int i = 0; i < NB; ++i) {
-                        const int64_t b = key0 / BK + i;
-                        if (b <= loc) out_row[b] = best[i] * scale;
-                    }
+                    for (int i = 0; i < NB; ++i) pend[i] = best[i] * scale;
+                    const int64_t vis = loc - b0 + 1;
+                    pend_n = vis >= NB ? NB : (vis > 0 ? (int)vis : 0);
                 }
             }
+        }
+        if constexpr (FK == 0) {
+#pragma unroll
+            for (int i = 0; i < NBP; ++i)
+                if (i < pend_n) pend_ptr[i] = pend[i];
         }
         if constexpr (FK > 0) {
             // Merge the two halves of every row.  All MMAs have completed (the last accumulator was
