@@ -127,12 +127,35 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 F8 ? make_idesc_e4m3(kIdxTileQ, kIdxTileK) : make_idesc_bf16(kIdxTileQ, kIdxTileK, false, false);
             bool ok = mbar_wait(&sm.a_full, 0, abort);
             if (!ok) report_async(status, kAsyncTimeout, 0x102);
+            // The tensor pipe takes an MMA from this thread only about as fast as it executes them, so
+            // whatever the thread does between the last MMA of one (tile, head) unit and the first of the
+            // next leaves the pipe idle: the head loop is unrolled and the operand descriptors are built
+            // once, so that a unit costs a barrier test, the MMAs and a commit.
+            uint64_t a_desc[NH][DI], b_desc[ST][DI];
+#pragma unroll
+            for (int h = 0; h < NH; ++h)
+#pragma unroll
+                for (int a = 0; a < DI; ++a) a_desc[h][a] = make_smem_desc(smem_u32(sm.a[h][a]), 16, 1024);
+#pragma unroll
+            for (int s = 0; s < ST; ++s)
+#pragma unroll
+                for (int a = 0; a < DI; ++a) b_desc[s][a] = make_smem_desc(smem_u32(sm.b[s][a]), 16, 1024);
+            int s = 0;
+            uint32_t full_par = 0;  // parity of the ring's current lap
             for (int t = 0; ok && t < n_tiles; ++t) {
-                const int s = t % ST;
-                if (!mbar_wait(&sm.full[s], (t / ST) & 1, abort)) {
+                if (!mbar_wait(&sm.full[s], full_par, abort)) {
                     report_async(status, kAsyncTimeout, 0x104);
                     break;
                 }
+                uint64_t bd[DI];
+#pragma unroll
+                for (int a = 0; a < DI; ++a) {
+                    bd[a] = b_desc[0][a];
+#pragma unroll
+                    for (int ss = 1; ss < ST; ++ss)
+                        if (ss == s) bd[a] = b_desc[ss][a];
+                }
+#pragma unroll
                 for (int h = 0; h < NH; ++h) {
                     const int u = t * NH + h, buf = u & 1;  // accumulators alternate over (tile, head)
                     if (!mbar_wait(&sm.acc_empty[buf], ((u >> 1) & 1) ^ 1, abort)) {
@@ -140,22 +163,24 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         ok = false;
                         break;
                     }
+                    MSA_STAMP(u, 10);
                     tc_fence_after();
+                    MSA_STAMP(u, 0);
 #pragma unroll
                     for (int a = 0; a < DI; ++a) {
-                        const uint64_t a_desc = make_smem_desc(smem_u32(sm.a[h][a]), 16, 1024);
-                        const uint64_t b_desc = make_smem_desc(smem_u32(sm.b[s][a]), 16, 1024);
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk) {  // 32 bytes (16 bf16 or 32 fp8) = 2 descriptor units per K step
                             if constexpr (F8)
-                                mma_e4m3_ss(tmem + buf * kIdxTileK, a_desc + 2 * kk, b_desc + 2 * kk, idesc, kk > 0);
+                                mma_e4m3_ss(tmem + buf * kIdxTileK, a_desc[h][a] + 2 * kk, bd[a] + 2 * kk, idesc, kk > 0);
                             else
-                                mma_bf16_ss(tmem + buf * kIdxTileK, a_desc + 2 * kk, b_desc + 2 * kk, idesc, (a | kk) > 0);
+                                mma_bf16_ss(tmem + buf * kIdxTileK, a_desc[h][a] + 2 * kk, bd[a] + 2 * kk, idesc, (a | kk) > 0);
                         }
                     }
                     mma_commit(&sm.acc_full[buf]);
+                    MSA_STAMP(u, 1);
                 }
                 mma_commit(&sm.empty[s]);
+                if (++s == ST) { s = 0; full_par ^= 1; }
             }
             if (*abort != 0) {  // unwinding: wait for the MMAs already issued before TMEM is freed
                 mma_commit(&sm.drain);
@@ -181,9 +206,10 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
                 for (int i = 0; i < FK; ++i) { ts[h][i] = -INFINITY; tb[h][i] = -1; }
         }
-        // Scores leave one unit late: a unit's maxima are stored while the next unit's accumulator is on
-        // its way to the registers, so that the store and its address arithmetic do not sit between the
-        // release of one accumulator and the wait for the next.
+        // Scores leave one unit late: a unit's maxima are stored right after the next unit's accumulator
+        // has been released, ahead of that unit's reductions, so that the store and its address
+        // arithmetic sit neither in front of an accumulator's release nor in front of the wait for the
+        // next one.
         constexpr int NBP = 128 / BK;
         float pend[NBP];
         float* pend_ptr = nullptr;
@@ -203,6 +229,7 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     break;
                 }
                 tc_fence_after();
+                if (lane == 0 && ew == 0) MSA_STAMP(u, 11);
                 const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + buf * kIdxTileK + half * 128;
                 constexpr int NB = 128 / BK;  // blocks in this thread's 128 columns
                 float best[NB];
@@ -231,14 +258,15 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     uint32_t v[4][32];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) tmem_ld_32x32(taddr + c * 32, v[c]);
-#pragma unroll
-                    for (int i = 0; i < NB; ++i)
-                        if (i < pend_n) pend_ptr[i] = pend[i];
-                    pend_n = 0;
                     tmem_wait_ld();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
+                    if (lane == 0) MSA_STAMP(u, 2 + ew);
+#pragma unroll
+                    for (int i = 0; i < NB; ++i)
+                        if (i < pend_n) pend_ptr[i] = pend[i];
+                    pend_n = 0;
                     if (need_mask) {
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
