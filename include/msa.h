@@ -100,6 +100,24 @@ typedef struct {
                          /* stays bf16.  Other shapes, decode calls and the         */
                          /* allocation-free call: MSA_ERR_UNSUPPORTED.  Other       */
                          /* values: INVALID_ARG.                                    */
+    int32_t score_runs;  /* Order of the blocks inside a score row, for the two     */
+                         /* calls that exchange one (msa_index_scores writes it,    */
+                         /* msa_topk_select reads it).  0: block order, column b =  */
+                         /* block b.  1 (B_k in {64,128}, ld_scores % 8 == 0): run  */
+                         /* order, the order in which the tensor-core kernel has    */
+                         /* the maxima at hand - a thread's four blocks of a run of */
+                         /* eight leave as one 16-byte store.  The eight blocks of  */
+                         /* run j stay in columns [8j, 8j+8); with n = 128 / B_k,   */
+                         /* block 8j + w sits in column 8j + 4*((w/n) mod 2) +      */
+                         /* n*(w / (2n)) + (w mod n): the columns of a run hold its */
+                         /* blocks 0 2 4 6 1 3 5 7 for B_k = 128 and 0 1 4 5 2 3 6  */
+                         /* 7 for B_k = 64.  Columns of                             */
+                         /* blocks after a query's local block are unspecified      */
+                         /* (not read by msa_topk_select).  The whole-path calls    */
+                         /* use run order in their workspace whatever this field    */
+                         /* says; decode calls take 0 only (else UNSUPPORTED).      */
+                         /* Other values: INVALID_ARG.  The paper has no            */
+                         /* counterpart: Eq. 6 fixes the values, not their place.   */
 } msa_shape_t;
 
 typedef void* msa_stream_t; /* a cudaStream_t */
@@ -121,6 +139,9 @@ msa_status_t msa_check_async_status(int32_t* detail_host);
  * q_idx  [q_count,H_kv,d_idx] bf16 (rows of the range), k_idx [kv_len,d_idx] bf16,
  * scores [q_count,H_kv,ld_scores] fp32, ld_scores >= B and a multiple of 4; columns
  * b in [0,B) of every row are written, columns [B, ld_scores) are left untouched.
+ * With shape->score_runs = 1 the columns of a row are in run order (see msa_shape_t):
+ * ld_scores >= B rounded up to 8 and a multiple of 8; the columns of blocks up to the
+ * query's local block hold the Eq. 6 values, the others are unspecified.
  */
 msa_status_t msa_index_scores(const msa_shape_t* shape, const void* q_idx, const void* k_idx,
                               int64_t q_begin, int64_t q_count, int64_t kv_len,

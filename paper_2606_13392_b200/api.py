@@ -63,11 +63,14 @@ def index_lse(cfg: MSAConfig, q_idx: torch.Tensor, k_idx: torch.Tensor, block_id
 
 
 def index_scores(cfg: MSAConfig, q_idx: torch.Tensor, k_idx: torch.Tensor, q_begin: int, q_count: int,
-                 kv_len: Optional[int] = None) -> torch.Tensor:
-    """Eq. 6 for rows [q_begin, q_begin+q_count); q_idx holds the whole sequence's rows."""
-    shape = B.shape_of(cfg)
+                 kv_len: Optional[int] = None, score_runs: int = 0) -> torch.Tensor:
+    """Eq. 6 for rows [q_begin, q_begin+q_count); q_idx holds the whole sequence's rows.
+    score_runs = 1: the columns of a row come in run order (run_order_columns gives the map)."""
+    shape = B.shape_of(cfg, score_runs=score_runs)
     kv_len = k_idx.shape[0] if kv_len is None else kv_len
     ld = B.score_ld(kv_len, cfg.block_size)
+    if score_runs:
+        ld = (ld + 7) // 8 * 8
     scores = torch.full((q_count, cfg.n_kv_heads, ld), float("nan"), dtype=torch.float32,
                         device=q_idx.device)
     B.msa_index_scores(shape, q_idx[q_begin:q_begin + q_count], k_idx, q_begin, q_count, kv_len,
@@ -75,8 +78,16 @@ def index_scores(cfg: MSAConfig, q_idx: torch.Tensor, k_idx: torch.Tensor, q_beg
     return scores
 
 
-def topk_select(cfg: MSAConfig, scores: torch.Tensor, q_begin: int, kv_len: int) -> torch.Tensor:
-    shape = B.shape_of(cfg)
+def run_order_columns(n_blocks: int, block_size: int) -> torch.Tensor:
+    """Column of block b in a score row in run order (msa_shape_t.score_runs = 1), for b < n_blocks."""
+    n = 128 // block_size
+    b = torch.arange(n_blocks, dtype=torch.int64)
+    w = b % 8
+    return (b - w) + 4 * ((w // n) % 2) + n * (w // (2 * n)) + (w % n)
+
+
+def topk_select(cfg: MSAConfig, scores: torch.Tensor, q_begin: int, kv_len: int, score_runs: int = 0) -> torch.Tensor:
+    shape = B.shape_of(cfg, score_runs=score_runs)
     q_count, _, ld = scores.shape
     block_idx = torch.empty((q_count, cfg.n_kv_heads, cfg.top_k), dtype=torch.int32,
                             device=scores.device)

@@ -40,7 +40,7 @@ class MsaShape(ctypes.Structure):
     _fields_ = [("n_q_heads", c_i32), ("n_kv_heads", c_i32), ("head_dim", c_i32),
                 ("idx_dim", c_i32), ("block_size", c_i32), ("top_k", c_i32),
                 ("softmax_scale", ctypes.c_float), ("index_scale", ctypes.c_float),
-                ("idx_fp8", c_i32), ("kv_fp8", c_i32), ("q_fp8", c_i32)]
+                ("idx_fp8", c_i32), ("kv_fp8", c_i32), ("q_fp8", c_i32), ("score_runs", c_i32)]
 
 
 class MsaError(RuntimeError):
@@ -71,10 +71,10 @@ def status_string(code: int) -> str:
     return lib().msa_status_string(code).decode()
 
 
-def shape_of(cfg: MSAConfig, softmax_scale: float = 0.0, index_scale: float = 0.0) -> MsaShape:
+def shape_of(cfg: MSAConfig, softmax_scale: float = 0.0, index_scale: float = 0.0, score_runs: int = 0) -> MsaShape:
     return MsaShape(cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.idx_dim, cfg.block_size,
                     cfg.top_k, softmax_scale, index_scale, 1 if cfg.idx_fp8 else 0, 1 if cfg.kv_fp8 else 0,
-                    1 if getattr(cfg, "q_fp8", False) else 0)
+                    1 if getattr(cfg, "q_fp8", False) else 0, score_runs)
 
 
 def _ptr(t) -> c_vp:

@@ -112,4 +112,16 @@ private:
     cudaStream_t st_;
 };
 
+// Where block b of a score row sits.  Block order (what msa_index_scores documents): at b.  Run
+// order (the tensor-core scoring kernel writes a thread's four blocks of a run of eight as one
+// 16-byte store): a run's eight blocks stay in the run's 32 bytes, those of the first half of every
+// key tile first; with nb = 2^lnb blocks per thread and tile, block w = b mod 8 is block (w mod nb)
+// of half ((w / nb) mod 2) of tile w / (2 nb) and sits at 4 half + nb tile + block.  lnb = 2 is the
+// identity (block order).
+template <class I>
+__device__ __forceinline__ I score_slot(I b, int lnb) {
+    const int w = (int)(b & 7);
+    return (b & ~(I)7) | (I)((((w >> lnb) & 1) << 2) | ((w >> (lnb + 1)) << lnb) | (w & ((1 << lnb) - 1)));
+}
+
 }  // namespace msa

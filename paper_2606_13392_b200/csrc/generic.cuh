@@ -36,7 +36,7 @@ template <int WARPS, bool F8>
 __global__ void __launch_bounds__(WARPS * 32)
 index_scores_generic_kernel(const void* __restrict__ q_idx, const void* __restrict__ k_idx, RowMap rows,
                             int64_t n_chunks, int H_kv, int d_idx, int B_k, float scale,
-                            float* __restrict__ scores, int64_t ld_scores) {
+                            float* __restrict__ scores, int64_t ld_scores, int lnb) {
     extern __shared__ float q_s[];  // [H_kv][d_idx]
     const int64_t row = blockIdx.x / n_chunks;
     const int64_t chunk = blockIdx.x % n_chunks;
@@ -51,7 +51,7 @@ index_scores_generic_kernel(const void* __restrict__ q_idx, const void* __restri
 
     const int64_t b = chunk * WARPS + warp;
     if (b >= rows.n_cols) return;
-    float* out = scores + row * (int64_t)H_kv * ld_scores + b;
+    float* out = scores + row * (int64_t)H_kv * ld_scores + score_slot(b, lnb);
     const int64_t j0 = b * B_k;
     if (pos < 0 || j0 > pos) {  // no visible token in this block
         if (lane < H_kv) out[(int64_t)lane * ld_scores] = -INFINITY;

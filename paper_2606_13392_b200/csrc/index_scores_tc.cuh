@@ -21,10 +21,12 @@ constexpr int kIdxTileK = 256;
 constexpr int kIdxThreads = 320;  // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
 
 // NH heads per CTA, DI = d_idx / 64 swizzle atoms along the contraction, ST key-tile stages.
-template <int NH, int DI, int ST>
+// RUNL: room for the block maxima of one run of eight blocks (four per epilogue thread and head).
+template <int NH, int DI, int ST, bool RUNL = false>
 struct IdxSmem {
     alignas(1024) uint8_t a[NH][DI][kIdxTileQ * 128];           // per head and atom: 128 query rows x 64 bf16
     alignas(1024) uint8_t b[ST][DI][kIdxTileK * 128];           // per stage and atom: 256 key rows x 64 bf16
+    alignas(16) float run[RUNL ? NH * 4 : 1][256];              // [head][slot of the run][epilogue thread]
     alignas(8) uint64_t full[ST];
     uint64_t empty[ST];
     uint64_t a_full;
@@ -57,7 +59,7 @@ struct IdxPackedTile {
 // The tiles are the same bytes in the same places as 64 bf16 per row, so the tensor maps, the
 // shared-memory layout and the descriptor walk are unchanged; only the MMA kind differs (32
 // contraction elements per 32-byte step instead of 16).
-template <int BK, int NH, int DI, int ST, int FK = 0, bool F8 = false>
+template <int BK, int NH, int DI, int ST, int FK = 0, bool F8 = false, bool RUNL = false>
 __global__ void __launch_bounds__(kIdxThreads, 1)
 index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        int64_t q_begin, int64_t q_count, int H_kv, float scale,
@@ -66,9 +68,10 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                        const IdxPackedTile* __restrict__ packed = nullptr) {
     static_assert(FK == 0 || NH <= 2, "the fused form keeps its candidates in registers");
     static_assert(!F8 || DI == 1, "fp8 index vectors are one 128-byte atom");
+    static_assert(!RUNL || FK == 0, "the run order is a layout of the score matrix");
     extern __shared__ uint8_t smem_raw[];
-    IdxSmem<NH, DI, ST>& sm =
-        *reinterpret_cast<IdxSmem<NH, DI, ST>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    IdxSmem<NH, DI, ST, RUNL>& sm =
+        *reinterpret_cast<IdxSmem<NH, DI, ST, RUNL>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_hg = H_kv / NH;  // head groups
     const int r0 = (int)(blockIdx.x % n_hg) * NH;
@@ -214,6 +217,13 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         float pend[NBP];
         float* pend_ptr = nullptr;
         int pend_n = 0;
+        // Run order (RUNL): the thread's maxima of one run of eight blocks - the NBP blocks of its half
+        // of every key tile, over TPR tiles - wait in shared memory (the thread's own words) and leave
+        // as one 16-byte store per head and run.
+        constexpr int TPR = 4 / NBP;
+        const int et = ew * 32 + lane;
+        float4 pend4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        bool pend4_on = false;
         float* const row_base = FK == 0 ? scores + ((row0 + q) * H_kv + r0) * ld_scores : nullptr;
         for (int t = 0; live && t < n_tiles; ++t) {
             const int64_t key0 = (int64_t)t * kIdxTileK + half * 128;
@@ -263,10 +273,15 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm.acc_empty[buf]);
                     if (lane == 0) MSA_STAMP(u, 2 + ew);
+                    if constexpr (RUNL) {
+                        if (pend4_on) *reinterpret_cast<float4*>(pend_ptr) = pend4;
+                        pend4_on = false;
+                    } else {
 #pragma unroll
-                    for (int i = 0; i < NB; ++i)
-                        if (i < pend_n) pend_ptr[i] = pend[i];
-                    pend_n = 0;
+                        for (int i = 0; i < NB; ++i)
+                            if (i < pend_n) pend_ptr[i] = pend[i];
+                        pend_n = 0;
+                    }
                     if (need_mask) {
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
@@ -294,6 +309,29 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                             }
                         }
                     }
+                } else if constexpr (RUNL) {
+                    const int ti = t % TPR;
+                    if (ti == TPR - 1 || t == n_tiles - 1) {
+                        // (the key tiles may end inside the run: its other blocks are visible to no row of the tile)
+                        float x[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            x[j] = -INFINITY;
+                            if (j / NB < ti) x[j] = sm.run[RUNL ? h * 4 + j : 0][et];
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+#pragma unroll
+                            for (int i = 0; i < NB; ++i)
+                                if (j == ti * NB + i) x[j] = best[i] * scale;
+                        const int64_t run = t / TPR;
+                        pend4 = make_float4(x[0], x[1], x[2], x[3]);
+                        pend_ptr = row_base + h * ld_scores + run * 8 + half * 4;
+                        pend4_on = valid_row && run * 8 <= loc;
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < NB; ++i) sm.run[RUNL ? h * 4 + ti * NB + i : 0][et] = best[i] * scale;
+                    }
                 } else if (valid_row) {
                     const int64_t b0 = key0 / BK;  // this thread's blocks b0 .. b0 + NB - 1; those up to loc are visible
                     pend_ptr = row_base + h * ld_scores + b0;
@@ -304,7 +342,9 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 }
             }
         }
-        if constexpr (FK == 0) {
+        if constexpr (RUNL) {
+            if (pend4_on) *reinterpret_cast<float4*>(pend_ptr) = pend4;
+        } else if constexpr (FK == 0) {
 #pragma unroll
             for (int i = 0; i < NBP; ++i)
                 if (i < pend_n) pend_ptr[i] = pend[i];
@@ -352,7 +392,7 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             }
         }
         // Blocks with no visible token: -inf (Eq. 6).  Warp ew fills rows ew, ew+8, ...
-        for (int rr = ew; FK == 0 && rr < kIdxTileQ; rr += 8) {
+        for (int rr = ew; FK == 0 && !RUNL && rr < kIdxTileQ; rr += 8) {
             const int64_t qq = q0 + rr;
             if (qq >= q_count) break;
             for (int h = 0; h < NH; ++h) {

@@ -54,6 +54,7 @@ struct Resolved {
     size_t kv_elt() const { return kv_fp8 ? 1 : 2; }    // bytes per K/V element
     bool q_fp8;                                          // prefill: Q is fp8 E4M3 as well (needs kv_fp8)
     size_t q_elt() const { return q_fp8 ? 1 : 2; }      // bytes per Q element
+    bool score_runs;                                     // score rows between the stage-1 and stage-2 calls are in run order
     bool idx_fp8;                                        // index-branch operands are fp8 E4M3 (else bf16)
     size_t idx_elt() const { return idx_fp8 ? 1 : 2; }  // bytes per index-branch element
 };
@@ -80,6 +81,9 @@ static msa_status_t resolve(const msa_shape_t* s, Resolved& r) {
     if (s->q_fp8 != 0 && s->q_fp8 != 1) return MSA_ERR_INVALID_ARG;
     r.q_fp8 = s->q_fp8 == 1;
     if (r.q_fp8 && !r.kv_fp8) return MSA_ERR_UNSUPPORTED;  // fp8 Q comes with fp8 K and V
+    if (s->score_runs != 0 && s->score_runs != 1) return MSA_ERR_INVALID_ARG;
+    r.score_runs = s->score_runs == 1;
+    if (r.score_runs && r.B_k != 64 && r.B_k != 128) return MSA_ERR_UNSUPPORTED;
     return MSA_OK;
 }
 
@@ -134,16 +138,21 @@ bool encode_tmap_bf16(CUtensorMap* map, const void* base, int rank, const uint64
 }
 
 // ---------------------------------------------------------------------- stage 1
+// log2 of the blocks one epilogue thread of the tensor-core scoring kernel holds per key tile, the
+// parameter of the run order of a score row (score_slot); 2 = block order.
+static int score_lnb(const Resolved& r, bool runs) { return !runs ? 2 : (r.B_k == 128 ? 0 : 1); }
+
 // F8: fp8 E4M3 operands with d_idx = 128; the bytes of a row are laid out like 64 bf16, so the
 // tensor maps below (bf16 element type, used only to move bytes) serve both.
-template <int BK, int NH, int DI, int FK = 0, bool F8 = false>
+template <int BK, int NH, int DI, int FK = 0, bool F8 = false, bool RUNL = false>
 static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                     int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
                                     int64_t n_cols, cudaStream_t st, int32_t* block_idx = nullptr,
                                     const IdxPackedTile* packed = nullptr, int64_t n_packed = 0) {
     // key-tile stages: what fits beside the NH*DI query atoms in 227 KB of shared memory (at most 3)
-    constexpr int ST = (NH * DI * 16 + 3 * DI * 32 <= 224) ? 3 : 2;
-    static_assert(NH * DI * 16 + ST * DI * 32 <= 224, "shared memory budget");
+    constexpr int RUN_KB = RUNL ? NH * 4 : 0;  // block maxima of a run of eight, waiting for their 16-byte store
+    constexpr int ST = (NH * DI * 16 + 3 * DI * 32 + RUN_KB <= 224) ? 3 : 2;
+    static_assert(NH * DI * 16 + ST * DI * 32 + RUN_KB <= 224, "shared memory budget");
     CUtensorMap tm_q, tm_k;
     const uint64_t row_b = (uint64_t)DI * 128;  // bytes of one index vector
     const uint64_t qd[3] = {(uint64_t)DI * 64, (uint64_t)r.H_kv, (uint64_t)q_count};
@@ -156,11 +165,11 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
         return MSA_ERR_CUDA;
     int* status = async_status_ptr();
     if (status == nullptr) return MSA_ERR_CUDA;
-    const size_t smem = sizeof(IdxSmem<NH, DI, ST>) + 1024;
+    const size_t smem = sizeof(IdxSmem<NH, DI, ST, RUNL>) + 1024;
     static bool attr_set_dev[64] = {false};  // the attribute is per device
     const int dev_id = current_device();
     if (!attr_set_dev[dev_id]) {
-        if (cudaFuncSetAttribute(index_scores_tc_kernel<BK, NH, DI, ST, FK, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(index_scores_tc_kernel<BK, NH, DI, ST, FK, F8, RUNL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem) != cudaSuccess)
             return MSA_ERR_CUDA;
         attr_set_dev[dev_id] = true;
@@ -170,7 +179,7 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
     if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
     {
         StageScope sc(kStageIndex, st);
-        index_scores_tc_kernel<BK, NH, DI, ST, FK, F8><<<(unsigned)grid, kIdxThreads, smem, st>>>(
+        index_scores_tc_kernel<BK, NH, DI, ST, FK, F8, RUNL><<<(unsigned)grid, kIdxThreads, smem, st>>>(
             tm_q, tm_k, q_begin, q_count, r.H_kv, r.index_scale, scores, ld_scores, n_cols, status, block_idx, r.k,
             packed);
     }
@@ -188,18 +197,28 @@ static int index_heads_per_cta(const Resolved& r, int64_t q_count) {
     return 1;
 }
 
-template <int BK, int DI, bool F8 = false>
-static msa_status_t launch_index_tc_bk(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
+template <int BK, int DI, bool F8, bool RUNL>
+static msa_status_t launch_index_tc_nh(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                        int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
                                        int64_t n_cols, cudaStream_t st) {
     const int nh = index_heads_per_cta(r, q_count);
     if constexpr (DI == 1) {
-        if (nh == 8) return launch_index_tc<BK, 8, DI, 0, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
-        if (nh == 4) return launch_index_tc<BK, 4, DI, 0, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+        if (nh == 8) return launch_index_tc<BK, 8, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+        if (nh == 4) return launch_index_tc<BK, 4, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
     }
-    if (nh == 2) return launch_index_tc<BK, 2, DI, 0, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
-    return launch_index_tc<BK, 1, DI, 0, F8>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    if (nh == 2) return launch_index_tc<BK, 2, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    return launch_index_tc<BK, 1, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
 }
+
+// runs: the score rows are written in run order (score_slot) instead of block order.
+template <int BK, int DI, bool F8 = false>
+static msa_status_t launch_index_tc_bk(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
+                                       int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
+                                       int64_t n_cols, cudaStream_t st, bool runs) {
+    if (runs) return launch_index_tc_nh<BK, DI, F8, true>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    return launch_index_tc_nh<BK, DI, F8, false>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+}
+
 
 // Shapes of the tensor-core index kernel: one or two 128-byte atoms per index vector.
 static bool index_tc_ok(const Resolved& r) {
@@ -246,20 +265,20 @@ static bool index_scores_on_tc(const Resolved& r, int64_t n_rows, int64_t kv_len
 
 static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const void* k_idx,
                                      const RowMap& rows, int64_t n_rows, float* scores,
-                                     int64_t ld_scores, cudaStream_t st) {
+                                     int64_t ld_scores, cudaStream_t st, bool runs = false) {
     if (n_rows == 0 || rows.n_cols == 0) return MSA_OK;
     if (rows.seq_lens == nullptr && index_scores_on_tc(r, n_rows, rows.kv_len)) {
         const int64_t qb = rows.q_begin, kl = rows.kv_len, nc = rows.n_cols;
         if (r.idx_fp8) {
-            if (r.B_k == 64) return launch_index_tc_bk<64, 1, true>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
-            return launch_index_tc_bk<128, 1, true>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
+            if (r.B_k == 64) return launch_index_tc_bk<64, 1, true>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st, runs);
+            return launch_index_tc_bk<128, 1, true>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st, runs);
         }
         if (r.d_idx == 64) {
-            if (r.B_k == 64) return launch_index_tc_bk<64, 1>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
-            return launch_index_tc_bk<128, 1>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
+            if (r.B_k == 64) return launch_index_tc_bk<64, 1>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st, runs);
+            return launch_index_tc_bk<128, 1>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st, runs);
         }
-        if (r.B_k == 64) return launch_index_tc_bk<64, 2>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
-        return launch_index_tc_bk<128, 2>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st);
+        if (r.B_k == 64) return launch_index_tc_bk<64, 2>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st, runs);
+        return launch_index_tc_bk<128, 2>(r, q_idx, k_idx, qb, n_rows, kl, scores, ld_scores, nc, st, runs);
     }
     constexpr int WARPS = 8;
     const int64_t n_chunks = ceil_div64(rows.n_cols, WARPS);
@@ -270,10 +289,10 @@ static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const
         StageScope sc(rows.seq_lens ? kStageIndexDecode : kStageIndex, st);
         if (r.idx_fp8)
             index_scores_generic_kernel<WARPS, true><<<(unsigned)grid, WARPS * 32, smem, st>>>(
-                q_idx, k_idx, rows, n_chunks, r.H_kv, r.d_idx, r.B_k, r.index_scale, scores, ld_scores);
+                q_idx, k_idx, rows, n_chunks, r.H_kv, r.d_idx, r.B_k, r.index_scale, scores, ld_scores, score_lnb(r, runs));
         else
             index_scores_generic_kernel<WARPS, false><<<(unsigned)grid, WARPS * 32, smem, st>>>(
-                q_idx, k_idx, rows, n_chunks, r.H_kv, r.d_idx, r.B_k, r.index_scale, scores, ld_scores);
+                q_idx, k_idx, rows, n_chunks, r.H_kv, r.d_idx, r.B_k, r.index_scale, scores, ld_scores, score_lnb(r, runs));
     }
     return launch_status();
 }
@@ -281,8 +300,9 @@ static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const
 // ---------------------------------------------------------------------- stage 2
 static msa_status_t run_topk(const Resolved& r, const float* scores, int64_t ld_scores,
                              const RowMap& rows, int64_t n_q, int32_t* block_idx,
-                             cudaStream_t st) {
+                             cudaStream_t st, bool runs = false) {
     const int64_t n_rows = n_q * r.H_kv;
+    const int lnb = score_lnb(r, runs);
     if (n_rows == 0) return MSA_OK;
     const int64_t grid = ceil_div64(n_rows, kTopkWarps);
     if (grid > 2147483647LL) return MSA_ERR_UNSUPPORTED;
@@ -291,11 +311,11 @@ static msa_status_t run_topk(const Resolved& r, const float* scores, int64_t ld_
     if (status == nullptr) return MSA_ERR_CUDA;
     StageScope sc(kStageTopk, st);
     if (r.k <= 32)
-        topk_select_kernel<1><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx, status);
+        topk_select_kernel<1><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx, status, lnb);
     else if (r.k <= 64)
-        topk_select_kernel<2><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx, status);
+        topk_select_kernel<2><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx, status, lnb);
     else
-        topk_select_kernel<4><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx, status);
+        topk_select_kernel<4><<<g, b, 0, st>>>(scores, ld_scores, rows, n_rows, r.H_kv, r.B_k, r.k, block_idx, status, lnb);
     return launch_status();
 }
 
@@ -861,8 +881,9 @@ msa_status_t msa_index_scores(const msa_shape_t* shape, const void* q_idx, const
         return MSA_ERR_INVALID_ARG;
     const int64_t B = ceil_div64(kv_len, r.B_k);
     if (ld_scores < B || ld_scores % 4 != 0) return MSA_ERR_INVALID_ARG;
+    if (r.score_runs && (ld_scores < (B + 7) / 8 * 8 || ld_scores % 8 != 0)) return MSA_ERR_INVALID_ARG;
     return run_index_scores(r, q_idx, k_idx, prefill_rows(q_begin, kv_len, r.B_k), q_count, scores,
-                            ld_scores, (cudaStream_t)stream);
+                            ld_scores, (cudaStream_t)stream, r.score_runs);
 }
 
 msa_status_t msa_index_scores_plan(const msa_shape_t* shape, int64_t q_count, int64_t kv_len,
@@ -918,6 +939,7 @@ msa_status_t msa_index_scores_decode(const msa_shape_t* shape, const void* q_idx
     Resolved r;
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
+    if (r.score_runs) return MSA_ERR_UNSUPPORTED;  // decode rows are in block order
     if (batch < 0 || max_seq_len < 0) return MSA_ERR_INVALID_ARG;
     if (batch == 0) return MSA_OK;
     if (!q_idx || !k_idx_cache || !seq_offsets || !seq_lens || !scores || !aligned16(q_idx) ||
@@ -941,8 +963,10 @@ msa_status_t msa_topk_select(const msa_shape_t* shape, const float* scores, int6
     if (q_count == 0) return MSA_OK;
     if (!scores || !block_idx || !aligned16(scores)) return MSA_ERR_INVALID_ARG;
     if (ld_scores < ceil_div64(kv_len, r.B_k) || ld_scores % 4 != 0) return MSA_ERR_INVALID_ARG;
+    if (r.score_runs && (ld_scores < (ceil_div64(kv_len, r.B_k) + 7) / 8 * 8 || ld_scores % 8 != 0))
+        return MSA_ERR_INVALID_ARG;
     return run_topk(r, scores, ld_scores, prefill_rows(q_begin, kv_len, r.B_k), q_count, block_idx,
-                    (cudaStream_t)stream);
+                    (cudaStream_t)stream, r.score_runs);
 }
 
 msa_status_t msa_topk_select_decode(const msa_shape_t* shape, const float* scores, int64_t ld_scores,
@@ -951,6 +975,7 @@ msa_status_t msa_topk_select_decode(const msa_shape_t* shape, const float* score
     Resolved r;
     msa_status_t s = resolve(shape, r);
     if (s != MSA_OK) return s;
+    if (r.score_runs) return MSA_ERR_UNSUPPORTED;  // decode rows are in block order
     if (batch < 0 || max_seq_len < 0) return MSA_ERR_INVALID_ARG;
     if (batch == 0) return MSA_OK;
     if (!scores || !block_idx || !seq_lens || !aligned16(scores) || ld_scores % 4 != 0 || ld_scores <= 0)
@@ -1237,7 +1262,7 @@ msa_status_t msa_sparse_attn_decode(const msa_shape_t* shape, const void* q, con
 }
 
 // ---------------------------------------------------------------------- whole path
-static int64_t score_ld(int64_t T, int B_k) { return (ceil_div64(T, B_k) + 3) / 4 * 4; }
+static int64_t score_ld(int64_t T, int B_k) { return (ceil_div64(T, B_k) + 7) / 8 * 8; }  // whole runs of eight blocks
 
 static int64_t pick_score_chunk(const Resolved& r, int64_t T, size_t bytes_for_scores) {
     const size_t row_bytes = sizeof(float) * (size_t)r.H_kv * (size_t)score_ld(T, r.B_k);
@@ -1302,15 +1327,17 @@ static msa_status_t prefill_stages_1_2(const msa_shape_t* shape, const Resolved&
     const int64_t chunk = pick_score_chunk(r, T, workspace_bytes);
     if (chunk <= 0) return MSA_ERR_WORKSPACE;
     float* scores = static_cast<float*>(workspace);
+    const bool runs = r.B_k == 64 || r.B_k == 128;  // the workspace's score rows are in run order where one exists
     for (int64_t q0 = 0; q0 < T; q0 += chunk) {
         const int64_t qc = (T - q0) < chunk ? (T - q0) : chunk;
         const char* qi = static_cast<const char*>(q_idx) + (size_t)q0 * r.H_kv * r.d_idx * r.idx_elt();
         // Only keys up to the chunk's last query are visible, so score that prefix.
         const int64_t kv_vis = q0 + qc;
         if (wait_rows(g_in_idx_hook, q0 + qc - 1, (cudaStream_t)stream) != MSA_OK) return MSA_ERR_CUDA;
-        s = msa_index_scores(shape, qi, k_idx, q0, qc, kv_vis, scores, ld, stream);
+        s = run_index_scores(r, qi, k_idx, prefill_rows(q0, kv_vis, r.B_k), qc, scores, ld, (cudaStream_t)stream, runs);
         if (s != MSA_OK) return s;
-        s = msa_topk_select(shape, scores, ld, q0, qc, kv_vis, block_idx + (size_t)q0 * r.H_kv * r.k, stream);
+        s = run_topk(r, scores, ld, prefill_rows(q0, kv_vis, r.B_k), qc, block_idx + (size_t)q0 * r.H_kv * r.k,
+                     (cudaStream_t)stream, runs);
         if (s != MSA_OK) return s;
     }
     return MSA_OK;

@@ -115,7 +115,8 @@ constexpr int kTopkLog = 512;    // survivors remembered per row for the index p
 struct TopkPlainStream {            // blocks [0, n) of a score row
     const float* srow;
     int n;
-    __device__ __forceinline__ float score(int i) const { return i < n ? __ldg(srow + i) : -INFINITY; }
+    int lnb;
+    __device__ __forceinline__ float score(int i) const { return i < n ? __ldg(srow + score_slot(i, lnb)) : -INFINITY; }
     __device__ __forceinline__ bool in(int i) const { return i < n; }
     __device__ __forceinline__ uint32_t block(int i) const { return (uint32_t)i; }
 };
@@ -295,7 +296,7 @@ __device__ __forceinline__ bool topk_trivial_row(int64_t loc, int top_k, int32_t
 constexpr int kTopkRunBlocks = 8;
 constexpr int kTopkMaxRuns = 1024;     // candidate list capacity (rows of up to 8192 blocks)
 
-struct TopkRunMaxStream {  // element i: maximum of blocks [8i, 8i+8); rows are 16-byte aligned
+struct TopkRunMaxStream {  // element i: maximum of blocks [8i, 8i+8), in either order of a run; rows are 16-byte aligned
     const float* srow;
     int n;
     __device__ __forceinline__ float score(int i) const {
@@ -313,17 +314,19 @@ struct TopkGatherStream {  // element i: block i % 8 of candidate run i / 8; blo
     const uint16_t* run;   // candidate runs, ascending
     int n;                 // 8 * number of candidate runs
     int loc;
+    int lnb;
     __device__ __forceinline__ uint32_t block(int i) const {
         return (uint32_t)run[i >> 3] * kTopkRunBlocks + (uint32_t)(i & 7);
     }
     __device__ __forceinline__ bool in(int i) const { return i < n && (int)block(i) < loc; }
-    __device__ __forceinline__ float score(int i) const { return in(i) ? __ldg(srow + block(i)) : -INFINITY; }
+    __device__ __forceinline__ float score(int i) const { return in(i) ? __ldg(srow + score_slot((int)block(i), lnb)) : -INFINITY; }
 };
 
 template <int R>
 __global__ void __launch_bounds__(kTopkWarps * 32)
 topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap rows,
-                   int64_t n_rows, int H_kv, int B_k, int top_k, int32_t* __restrict__ block_idx, int* status) {
+                   int64_t n_rows, int H_kv, int B_k, int top_k, int32_t* __restrict__ block_idx, int* status,
+                   int lnb) {
     __shared__ uint32_t stg_all[kTopkWarps][kTopkStage];
     __shared__ uint2 log_all[kTopkWarps][kTopkLog];   // (key, block) of every survivor, in index order
     __shared__ uint16_t run_all[kTopkWarps][kTopkMaxRuns + 2];
@@ -350,7 +353,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
     bool log_ok;
     const int64_t n_full = loc / kTopkRunBlocks;  // runs wholly before the local block
     if (n_full < 2 * m || n_full > kTopkMaxRuns) {  // short row (or one beyond the list): one level
-        const TopkPlainStream st{srow, (int)loc};
+        const TopkPlainStream st{srow, (int)loc, lnb};
         topk_pass1<R>(st, m, -INFINITY, sc, kept, n_log, log_ok, lane);
         topk_pass2<R>(st, m, sc, kept, n_log, log_ok, outb, lane);
     } else {
@@ -416,7 +419,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         // 3. select among the candidates' blocks; scores below tau0 cannot be selected.  The floor
         // only has to lie below tau0: a hair below it, whatever its sign or size.
         const float floor_f = tau0 - fmaxf(fabsf(tau0) * 1e-6f, 1e-30f);
-        const TopkGatherStream gs{srow, run, n_run * kTopkRunBlocks, (int)loc};
+        const TopkGatherStream gs{srow, run, n_run * kTopkRunBlocks, (int)loc, lnb};
         topk_pass1<R>(gs, m, floor_f, sc, kept, n_log, log_ok, lane);
         topk_pass2<R>(gs, m, sc, kept, n_log, log_ok, outb, lane);
     }

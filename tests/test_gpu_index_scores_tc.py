@@ -2,7 +2,8 @@
 kernel takes at full size: ranges long enough that eight (or four, two, one) index heads share a
 CTA, deep key prefixes (the key-tile ring wraps many times), a range that starts inside the
 sequence, the tile that crosses the diagonal at a large position, both block sizes, both index
-widths and fp8 operands.  Every case asserts, through msa_index_scores_plan, that the call it
+widths and fp8 operands, in block order and in run order (the order msa_prefill_forward uses in its
+workspace; msa_topk_select must pick the same lists from either).  Every case asserts, through msa_index_scores_plan, that the call it
 compares ran on the tensor-core kernel with the expected number of heads per CTA, so that the
 comparison cannot silently fall on the generic kernel."""
 
@@ -41,28 +42,42 @@ def _index_only_inputs(cfg: MSAConfig, sharp: bool):
     return x["q_idx"], x["k_idx"]
 
 
-def check_range(cfg: MSAConfig, q_idx, k_idx, q0: int, qc: int, want_nh: int, n_rows: int = 128, seed: int = 0):
-    shape = B.shape_of(cfg)
+def check_range(cfg: MSAConfig, q_idx, k_idx, q0: int, qc: int, want_nh: int, n_rows: int = 128, seed: int = 0,
+                score_runs: int = 0):
+    shape = B.shape_of(cfg, score_runs=score_runs)
     tc, nh = B.msa_index_scores_plan(shape, qc, cfg.T)
     assert tc and nh == want_nh, "expected the tensor-core kernel with %d heads per CTA, got tc=%s nh=%d" % (
         want_nh, tc, nh)
     n0 = B.launch_count()
-    M = api.index_scores(cfg, q_idx, k_idx, q0, qc)   # NaN-filled before the call
+    M = api.index_scores(cfg, q_idx, k_idx, q0, qc, score_runs=score_runs)   # NaN-filled before the call
     torch.cuda.synchronize()
     assert B.launch_count() == n0 + 1
     code, detail = B.check_async_status()
     assert code == 0, (code, detail)
     nb = cfg.n_blocks
     # columns the call must not touch keep their fill
-    assert torch.isnan(M[:, :, nb:]).all()
-    assert not torch.isnan(M[:, :, :nb]).any()
+    nb_written = (nb + 7) // 8 * 8 if score_runs else nb
+    assert torch.isnan(M[:, :, nb_written:]).all()
+    if not score_runs:
+        assert not torch.isnan(M[:, :, :nb]).any()
+    cols = api.run_order_columns(nb, cfg.block_size).to(DEV) if score_runs else torch.arange(nb, device=DEV)
     kib = to_bits(k_idx)
     worst = 0.0
     for pos in _runs(q0, qc, cfg.T, n_rows, seed):
         pos_t = torch.from_numpy(pos).to(DEV)
         M_ref = oracle.index_scores(to_bits(q_idx[pos_t]), kib, pos, cfg.block_size)
-        M_gpu = M[pos_t - q0][:, :, :nb].cpu().numpy()
+        M_gpu = M[pos_t - q0][:, :, cols].cpu().numpy()
+        if score_runs:  # columns of blocks after the local block are unspecified in run order
+            hidden = np.arange(nb)[None, :] > (pos // cfg.block_size)[:, None]
+            M_gpu[np.broadcast_to(hidden[:, None, :], M_gpu.shape)] = -np.inf
         worst = max(worst, check_scores(M_gpu, M_ref, pos, cfg.block_size))
+    if score_runs:
+        # Stage 2 on the run-ordered rows picks, bit for bit, the lists it picks from block-ordered ones.
+        M0 = api.index_scores(cfg, q_idx, k_idx, q0, qc)
+        I1 = api.topk_select(cfg, M, q0, cfg.T, score_runs=1)
+        I0 = api.topk_select(cfg, M0, q0, cfg.T)
+        torch.cuda.synchronize()
+        assert torch.equal(I0, I1)
     return worst
 
 
@@ -80,22 +95,25 @@ def check_range(cfg: MSAConfig, q_idx, k_idx, q0: int, qc: int, want_nh: int, n_
     ("fp8 operands, NH8", 41000, 8, 64, 128, True, 41000 - 37900, 37900, 8),
 ])
 @pytest.mark.parametrize("sharp", [False, True])
-def test_tensor_core_scores_match_oracle(name, T, Hkv, Bk, di, fp8, q0, qc, nh, sharp):
-    cfg = MSAConfig("idx-tc", "prefill", T, Hkv, Hkv, Bk, 8, head_dim=8, idx_dim=di, seed=T + Hkv, idx_fp8=fp8)
+@pytest.mark.parametrize("score_runs", [0, 1])
+def test_tensor_core_scores_match_oracle(name, T, Hkv, Bk, di, fp8, q0, qc, nh, sharp, score_runs):
+    top_k = 8 if not score_runs else (64 if Hkv == 8 else 24)  # run order: stage 2 on the rows as well
+    cfg = MSAConfig("idx-tc", "prefill", T, Hkv, Hkv, Bk, top_k, head_dim=8, idx_dim=di, seed=T + Hkv, idx_fp8=fp8)
     q_idx, k_idx = _index_only_inputs(cfg, sharp)
-    worst = check_range(cfg, q_idx, k_idx, q0, qc, nh, n_rows=96, seed=T)
-    print(name, sharp, "max score error %.3g" % worst)
+    worst = check_range(cfg, q_idx, k_idx, q0, qc, nh, n_rows=96, seed=T, score_runs=score_runs)
+    print(name, sharp, score_runs, "max score error %.3g" % worst)
 
 
+@pytest.mark.parametrize("score_runs", [0, 1])
 @pytest.mark.parametrize("name,rows", [("c3", 128), ("c4", 64)])
-def test_full_size_chunk_scores_match_oracle(name, rows):
+def test_full_size_chunk_scores_match_oracle(name, rows, score_runs):
     # The last query chunk of the full-size configurations as msa_prefill_forward scores it: 32 768
     # rows (40 960 at c3, where the chunk is the whole tail) against the whole key prefix, eight heads
     # per CTA; thousands of key tiles per CTA at c4.
     cfg = CONFIGS[name]
     q_idx, k_idx = _index_only_inputs(cfg, False)
     qc = 40960
-    worst = check_range(cfg, q_idx, k_idx, cfg.T - qc, qc, 8, n_rows=rows, seed=1)
-    print(name, "max score error %.3g" % worst)
+    worst = check_range(cfg, q_idx, k_idx, cfg.T - qc, qc, 8, n_rows=rows, seed=1, score_runs=score_runs)
+    print(name, score_runs, "max score error %.3g" % worst)
     del q_idx, k_idx
     torch.cuda.empty_cache()
