@@ -112,6 +112,13 @@ private:
     cudaStream_t st_;
 };
 
+// Three-input maximum (one instruction on sm_100).
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // Where block b of a score row sits.  Block order (what msa_index_scores documents): at b.  Run
 // order (the tensor-core scoring kernel writes a thread's four blocks of a run of eight as one
 // 16-byte store): a run's eight blocks stay in the run's 32 bytes, those of the first half of every

@@ -292,13 +292,8 @@ __device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, ui
         : "memory");
 }
 
-// Three-input maximum (one instruction on sm_100) and a depth-4 reduction tree over 32 values:
-// keeps the reduction off a 32-long dependency chain.
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
+// A depth-4 reduction tree of three-input maxima over 32 values: keeps the reduction off a 32-long
+// dependency chain.
 
 __device__ __forceinline__ float tree_max32(const uint32_t (&v)[32]) {
     float a[11];

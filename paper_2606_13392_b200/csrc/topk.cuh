@@ -103,12 +103,14 @@ __device__ __forceinline__ int warp_excl_scan(int v, int lane) {
 
 constexpr int kTopkWarps = 4;
 #ifndef MSA_TOPK_LOADS
-#define MSA_TOPK_LOADS 8
+#define MSA_TOPK_LOADS 4
 #endif
 constexpr int kTopkLoads = MSA_TOPK_LOADS;            // coalesced 32-wide loads per round
 constexpr int kTopkRound = 32 * kTopkLoads;           // blocks covered by one round
 constexpr int kTopkStage = 32 + kTopkRound;           // flush threshold (32) + one round of pushes
 constexpr int kTopkLog = 512;    // survivors remembered per row for the index pass
+constexpr int kTopkRunBlocks = 8;       // two-level selection: blocks per run
+constexpr int kTopkMaxRuns = 1024;     // two-level selection: candidate list capacity (rows of up to 8192 blocks)
 
 // A row as the selection sees it: element i of n has a score and a block index; the elements come
 // in ascending block order.
@@ -268,6 +270,108 @@ __device__ __forceinline__ void topk_pass2(const Stream& st, int m, const TopkSc
     __syncwarp();
 }
 
+// The selection once the threshold key is known: from a list of (key, block) in block order that
+// holds every block that can be selected, the blocks above the threshold and the first need_ties
+// blocks that equal it, written ascending to outb[0..m).
+__device__ __forceinline__ void topk_take_listed(const uint2* lst, int n_lst, uint32_t tau, int need_ties, int m,
+                                                 int32_t* outb, int lane) {
+    const unsigned lt_mask = (1u << lane) - 1u;
+    int out_cnt = 0, ties_seen = 0;
+    for (int e0 = 0; e0 < n_lst && out_cnt < m; e0 += 32) {
+        const int e = e0 + lane;
+        uint2 kv = make_uint2(0u, 0u);
+        if (e < n_lst) kv = lst[e];
+        const bool gt = e < n_lst && kv.x > tau, eq = e < n_lst && kv.x == tau;
+        const unsigned eqm = __ballot_sync(0xffffffffu, eq);
+        bool take = gt;
+        if (eqm != 0u) {
+            take = take || (eq && (ties_seen + __popc(eqm & lt_mask)) < need_ties);
+            ties_seen += __popc(eqm);
+        }
+        const unsigned tm = __ballot_sync(0xffffffffu, take);
+        if (take) {
+            const int w = out_cnt + __popc(tm & lt_mask);
+            if (w < m) outb[w] = (int32_t)kv.y;
+        }
+        out_cnt += __popc(tm);
+    }
+    __syncwarp();
+}
+
+// Step 3 of the two-level selection when few blocks reach tau0 (the usual case: the m run maxima
+// that define tau0 and a handful of second-best blocks).  Every lane loads whole candidate runs
+// (32 bytes each), the blocks that reach tau0 are listed in block order, and the threshold - the
+// m-th largest of the n listed keys - is found by taking away the n - m smallest, one warp-wide
+// minimum at a time.  Returns false (nothing written) when more than kTopkListMax blocks reach
+// tau0 or more than kTopkDropMax would have to go; the caller then ranks the candidates' blocks
+// with the two general passes.  LNB: the order of the blocks inside a run (score_slot).
+constexpr int kTopkListMax = 128;
+constexpr int kTopkDropMax = 32;
+
+template <int LNB>
+__device__ __forceinline__ bool topk_few_above(const float* srow, const uint16_t* run, int n_run, int loc, float tau0,
+                                               int m, uint2* lst, int32_t* outb, int lane) {
+    int n_lst = 0;
+    for (int c0 = 0; c0 < n_run; c0 += 32) {
+        const int c = c0 + lane;
+        const bool have = c < n_run;
+        const int g = have ? (int)run[c] : 0;
+        float x[8];
+        {
+            const float4* p = reinterpret_cast<const float4*>(srow) + 2 * g;
+            const float4 a = have ? __ldg(p) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 b = have ? __ldg(p + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float y[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int w = 0; w < 8; ++w) x[w] = y[score_slot(w, LNB)];  // block order
+        }
+        unsigned mine = 0u;  // bit w: block 8 g + w reaches tau0 and may rank (it lies before the local block)
+#pragma unroll
+        for (int w = 0; w < 8; ++w)
+            if (have && g * kTopkRunBlocks + w < loc && x[w] >= tau0) mine |= 1u << w;
+        const int cnt = __popc(mine);
+        const int before = warp_excl_scan(cnt, lane);
+        const int total = __shfl_sync(0xffffffffu, before + cnt, 31);
+        if (n_lst + total > kTopkListMax) return false;
+        int at = n_lst + before;
+#pragma unroll
+        for (int w = 0; w < 8; ++w)
+            if (mine & (1u << w)) lst[at++] = make_uint2(topk_key(x[w]), (uint32_t)(g * kTopkRunBlocks + w));
+        n_lst += total;
+    }
+    const int drop = n_lst - m;  // >= 0: m different runs reach tau0
+    if (drop > kTopkDropMax || drop < 0) return false;
+    __syncwarp();
+    uint32_t sv[kTopkListMax / 32];
+#pragma unroll
+    for (int j = 0; j < kTopkListMax / 32; ++j) sv[j] = (j * 32 + lane < n_lst) ? lst[j * 32 + lane].x : 0xFFFFFFFFu;
+    uint32_t tau = 0u;
+    for (int it = 0; it <= drop; ++it) {
+        uint32_t lmin = sv[0];
+#pragma unroll
+        for (int j = 1; j < kTopkListMax / 32; ++j) lmin = min(lmin, sv[j]);
+        uint32_t wmin = lmin;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) wmin = min(wmin, __shfl_xor_sync(0xffffffffu, wmin, o));
+        tau = wmin;
+        if (it == drop) break;
+        const unsigned holders = __ballot_sync(0xffffffffu, lmin == wmin);
+        if (lane == __ffs(holders) - 1) {  // one copy of the minimum goes
+            bool gone = false;
+#pragma unroll
+            for (int j = 0; j < kTopkListMax / 32; ++j)
+                if (!gone && sv[j] == wmin) { sv[j] = 0xFFFFFFFFu; gone = true; }
+        }
+    }
+    // tau is the m-th largest key; what is left in sv besides the removed ones is >= tau
+    int n_gt = 0;
+#pragma unroll
+    for (int j = 0; j < kTopkListMax / 32; ++j)
+        n_gt += __popc(__ballot_sync(0xffffffffu, sv[j] != 0xFFFFFFFFu && sv[j] > tau));
+    topk_take_listed(lst, n_lst, tau, m - n_gt, m, outb, lane);
+    return true;
+}
+
 // Rows with at most top_k visible blocks, or top_k = 1: no ranking.  Returns true if the row is done.
 __device__ __forceinline__ bool topk_trivial_row(int64_t loc, int top_k, int32_t* orow, int lane) {
     if (loc <= top_k - 1) {  // every visible block is selected
@@ -293,8 +397,6 @@ __device__ __forceinline__ bool topk_trivial_row(int64_t loc, int top_k, int32_t
 //      select from it exactly what they would select from the whole row, ties included.
 // The merge networks, which dominate a one-level selection, then run on about a third of the
 // survivors (run maxima first, then the few blocks above tau0).
-constexpr int kTopkRunBlocks = 8;
-constexpr int kTopkMaxRuns = 1024;     // candidate list capacity (rows of up to 8192 blocks)
 
 struct TopkRunMaxStream {  // element i: maximum of blocks [8i, 8i+8), in either order of a run; rows are 16-byte aligned
     const float* srow;
@@ -303,7 +405,7 @@ struct TopkRunMaxStream {  // element i: maximum of blocks [8i, 8i+8), in either
         if (i >= n) return -INFINITY;
         const float4* p = reinterpret_cast<const float4*>(srow) + 2 * i;
         const float4 a = __ldg(p), b = __ldg(p + 1);
-        return fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w)));
+        return max3(max3(a.x, a.y, a.z), max3(a.w, b.x, b.y), fmaxf(b.z, b.w));
     }
     __device__ __forceinline__ bool in(int i) const { return i < n; }
     __device__ __forceinline__ uint32_t block(int i) const { return (uint32_t)i; }
@@ -418,10 +520,16 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         __syncwarp();
         // 3. select among the candidates' blocks; scores below tau0 cannot be selected.  The floor
         // only has to lie below tau0: a hair below it, whatever its sign or size.
-        const float floor_f = tau0 - fmaxf(fabsf(tau0) * 1e-6f, 1e-30f);
-        const TopkGatherStream gs{srow, run, n_run * kTopkRunBlocks, (int)loc, lnb};
-        topk_pass1<R>(gs, m, floor_f, sc, kept, n_log, log_ok, lane);
-        topk_pass2<R>(gs, m, sc, kept, n_log, log_ok, outb, lane);
+        const bool few = lnb == 0   ? topk_few_above<0>(srow, run, n_run, (int)loc, tau0, m, log_all[warp], outb, lane)
+                         : lnb == 1 ? topk_few_above<1>(srow, run, n_run, (int)loc, tau0, m, log_all[warp], outb, lane)
+                                    : topk_few_above<2>(srow, run, n_run, (int)loc, tau0, m, log_all[warp], outb, lane);
+        if (!few) {
+            __syncwarp();
+            const float floor_f = tau0 - fmaxf(fabsf(tau0) * 1e-6f, 1e-30f);
+            const TopkGatherStream gs{srow, run, n_run * kTopkRunBlocks, (int)loc, lnb};
+            topk_pass1<R>(gs, m, floor_f, sc, kept, n_log, log_ok, lane);
+            topk_pass2<R>(gs, m, sc, kept, n_log, log_ok, outb, lane);
+        }
     }
     // Block order makes the list ascending with no final sort; the local block is appended by
     // construction (never ranked).

@@ -628,11 +628,13 @@ def test_two_level_topk_long_rows_bit_exact(T, Hq, Hkv, k, di, ties, sharp):
 
 
 @pytest.mark.parametrize("n_blocks,k,levels", [(3000, 20, 0), (8192, 64, 0), (8192, 64, 5), (5000, 33, 3),
-                                               (9000, 17, 0)])
+                                               (9000, 17, 0), (8192, 64, -64), (4100, 32, -24), (6000, 128, -16)])
 def test_two_level_topk_on_arbitrary_long_score_rows(n_blocks, k, levels):
-    # Top-k alone on synthetic score rows: continuous values, and values from a handful of levels
-    # (whole runs tie, the threshold is shared by hundreds of blocks); rows at many positions,
-    # including ones beyond the candidate list's capacity (n_blocks 9000), which take one level.
+    # Top-k alone on synthetic score rows: continuous values, values from a handful of levels
+    # (whole runs tie, the threshold is shared by hundreds of blocks) and normal values rounded to
+    # multiples of 1/|levels| (a few blocks tie with the threshold: the short list of blocks above the
+    # run-maxima threshold still decides them by block order); rows at many positions, including
+    # ones beyond the candidate list's capacity (n_blocks 9000), which take one level.
     Bk = 16
     T = n_blocks * Bk
     cfg = MSAConfig("top2-raw", "prefill", T, 4, 2, Bk, k, head_dim=64, idx_dim=32, seed=n_blocks)
@@ -643,8 +645,10 @@ def test_two_level_topk_on_arbitrary_long_score_rows(n_blocks, k, levels):
     for run in runs:
         q0, qc = int(run[0]), len(run)
         M = torch.randn((qc, 2, ld), generator=g)
-        if levels:
+        if levels > 0:
             M = torch.randint(0, levels, (qc, 2, ld), generator=g).float() * 0.5 - 1.0
+        elif levels < 0:
+            M = torch.round(M * float(-levels)) / float(-levels)
         I = api.topk_select(cfg, M.to(DEV), q0, T).cpu().numpy()
         I_ref = oracle.topk_select(M[:, :, :n_blocks].double().numpy(), np.arange(q0, q0 + qc), T, Bk, k)
         assert np.array_equal(I, I_ref), (q0, qc)
