@@ -176,9 +176,9 @@ def oracle_sample_size(cfg: MSAConfig) -> int:
 # of the units the two launches process (traffic grows in proportion to them).  An entry goes
 # stale when its kernel changes; `kernel` names the form that was captured so that this shows.
 NCU_TRAFFIC = {
-    ("c4", "index_scores"): {"bytes": 38.85e9, "captured": "c4, one 32768-query chunk",
-                             "kernel": "index_scores_tc_kernel<128,8,1,3>", "scale": 1.0},
-    ("c4", "topk_select"): {"bytes": 17.89e9, "captured": "c4, one 32768-query chunk",
+    ("c4", "index_scores"): {"bytes": 17.79e9, "captured": "c4, one 131072-query chunk",
+                             "kernel": "index_scores_tc_kernel<128,8,1,2,0,0,1> (scores in run order)", "scale": 1.0},
+    ("c4", "topk_select"): {"bytes": 18.06e9, "captured": "c4, one 131072-query chunk",
                             "kernel": "topk_select_kernel<2>", "scale": 1.0},
     # attention: 18.5 GB read + 33.7 GB written per query range; half of the Q gathers hit L2
     ("c4", "attn_prefill"): {"bytes": 52.2e9, "captured": "c4, one query range",
