@@ -110,6 +110,11 @@ constexpr int kTopkRound = 32 * kTopkLoads;           // blocks covered by one r
 constexpr int kTopkStage = 32 + kTopkRound;           // flush threshold (32) + one round of pushes
 constexpr int kTopkLog = 512;    // survivors remembered per row for the index pass
 constexpr int kTopkRunBlocks = 8;       // two-level selection: blocks per run
+#ifndef MSA_TOPK_RUNLOADS
+#define MSA_TOPK_RUNLOADS 4
+#endif
+constexpr int kTopkRunLoads = MSA_TOPK_RUNLOADS;  // two-level selection: runs per lane and round of the run-maxima pass
+constexpr int kTopkTau0Slack = 4;       // two-level selection: candidate runs accepted beyond the m needed
 constexpr int kTopkMaxRuns = 1024;     // two-level selection: candidate list capacity (rows of up to 8192 blocks)
 
 // A row as the selection sees it: element i of n has a score and a block index; the elements come
@@ -350,9 +355,7 @@ __device__ __forceinline__ bool topk_few_above(const float* srow, const uint16_t
         uint32_t lmin = sv[0];
 #pragma unroll
         for (int j = 1; j < kTopkListMax / 32; ++j) lmin = min(lmin, sv[j]);
-        uint32_t wmin = lmin;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) wmin = min(wmin, __shfl_xor_sync(0xffffffffu, wmin, o));
+        const uint32_t wmin = __reduce_min_sync(0xffffffffu, lmin);
         tau = wmin;
         if (it == drop) break;
         const unsigned holders = __ballot_sync(0xffffffffu, lmin == wmin);
@@ -461,9 +464,9 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
     } else {
         // 1. A threshold from the run maxima.  Any value that m run maxima reach will do, so no exact
         // selection: every lane keeps the S = 2R largest of the maxima it sees (sorted registers, no
-        // branches), the 32 S kept values - maxima of different runs - are sorted once, and tau0 is
-        // the m-th largest of them (the exact m-th largest run maximum unless one lane saw more than S
-        // of the m largest, and then a little lower).
+        // branches), and tau0 is a value that m to m + kTopkTau0Slack of the 32 S kept values - maxima
+        // of different runs - reach, found by bisection (close to the m-th largest run maximum unless
+        // one lane saw more than S of the m largest, and then a little lower).
         const TopkRunMaxStream rs{srow, (int)n_full};
         constexpr int S = 2 * R;
         float top[S];
@@ -471,17 +474,17 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         for (int i = 0; i < S; ++i) top[i] = -INFINITY;
         float* runmax = reinterpret_cast<float*>(log_all[warp]);  // the log is not in use before step 3
         static_assert(kTopkLog * sizeof(uint2) >= kTopkMaxRuns * sizeof(float), "run maxima share the log");
-        float nx[4];
+        float nx[kTopkRunLoads];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) nx[u] = rs.score(u * 32 + lane);  // -inf beyond n_full
-        for (int g0 = 0; g0 < (int)n_full; g0 += 32 * 4) {
-            float x[4];
+        for (int u = 0; u < kTopkRunLoads; ++u) nx[u] = rs.score(u * 32 + lane);  // -inf beyond n_full
+        for (int g0 = 0; g0 < (int)n_full; g0 += 32 * kTopkRunLoads) {
+            float x[kTopkRunLoads];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) x[u] = nx[u];
+            for (int u = 0; u < kTopkRunLoads; ++u) x[u] = nx[u];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) nx[u] = rs.score(g0 + 128 + u * 32 + lane);  // in flight during the inserts
+            for (int u = 0; u < kTopkRunLoads; ++u) nx[u] = rs.score(g0 + 32 * kTopkRunLoads + u * 32 + lane);  // in flight during the inserts
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < kTopkRunLoads; ++u) {
                 float v = x[u];
                 if (g0 + u * 32 + lane < (int)n_full) runmax[g0 + u * 32 + lane] = v;
 #pragma unroll
@@ -495,12 +498,24 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         uint32_t tk[S];
 #pragma unroll
         for (int i = 0; i < S; ++i) tk[i] = topk_key(top[i]);
+        // Bisection on the key: the largest value found that at least m of the 32 S kept maxima reach
+        // (there are at least 2 m real ones), stopping as soon as no more than m + kTopkTau0Slack do.
+        uint32_t lo = __reduce_min_sync(0xffffffffu, tk[S - 1]);      // every kept maximum reaches it
+        uint32_t hi = __reduce_max_sync(0xffffffffu, tk[0]) + 1u;     // none reaches it (keys stay below 2^32 - 1)
+        for (int it = 0; it < 32 && hi - lo > 1u; ++it) {
+            const uint32_t mid = lo + ((hi - lo) >> 1);
+            int c = 0;
 #pragma unroll
-        for (int size = 2; size <= 32 * S; size <<= 1) {
-#pragma unroll
-            for (int stride = size >> 1; stride > 0; stride >>= 1) bitonic_stage<S>(tk, lane, size, stride);
+            for (int i = 0; i < S; ++i) c += tk[i] >= mid ? 1 : 0;
+            c = __reduce_add_sync(0xffffffffu, c);
+            if (c >= m) {
+                lo = mid;
+                if (c <= m + kTopkTau0Slack) break;
+            } else {
+                hi = mid;
+            }
         }
-        const float tau0 = topk_key_score(element_at<S>(tk, m - 1));  // 32 S >= 2 m values
+        const float tau0 = topk_key_score(lo);  // finite: lo lies between two kept maxima
         // 2. candidate runs, ascending (their maxima wait in shared memory)
         uint16_t* run = run_all[warp];
         const unsigned lt_mask = (1u << lane) - 1u;
@@ -508,7 +523,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         __syncwarp();
         for (int g0 = 0; g0 < (int)n_full; g0 += 32) {
             const int g = g0 + lane;
-            const bool c = g < (int)n_full && runmax[g] >= tau0;  // tau0 is a real score
+            const bool c = g < (int)n_full && runmax[g] >= tau0;
             const unsigned cm = __ballot_sync(0xffffffffu, c);
             if (c) run[n_run + __popc(cm & lt_mask)] = (uint16_t)g;
             n_run += __popc(cm);
