@@ -14,10 +14,16 @@ struct RowMap {
     const int64_t* seq_offsets;  // decode: token offset of each sequence (nullptr => prefill)
     const int32_t* seq_lens;     // decode: length of each sequence
     int64_t n_cols;              // score columns to write per row (>= this row's block count)
+    const int32_t* row_pos = nullptr;  // packed prefill batch: position of every packed row in its own sequence;
+                                       // row r of the call is packed row q_begin + r (stage 2 only)
 
     __device__ __forceinline__ void get(int64_t row, int64_t& pos, int64_t& len,
                                         int64_t& base) const {
-        if (seq_lens != nullptr) {
+        if (row_pos != nullptr) {
+            pos = row_pos[q_begin + row];
+            len = pos + 1;
+            base = 0;
+        } else if (seq_lens != nullptr) {
             len = seq_lens[row];
             pos = len - 1;
             base = seq_offsets != nullptr ? seq_offsets[row] : 0;

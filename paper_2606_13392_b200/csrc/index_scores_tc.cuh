@@ -65,7 +65,7 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                        int64_t q_begin, int64_t q_count, int H_kv, float scale,
                        float* __restrict__ scores, int64_t ld_scores, int64_t n_cols, int* status,
                        int32_t* __restrict__ block_idx = nullptr, int top_k = 0,
-                       const IdxPackedTile* __restrict__ packed = nullptr) {
+                       const IdxPackedTile* __restrict__ packed = nullptr, int64_t score_row0 = 0) {
     static_assert(FK == 0 || NH <= 2, "the fused form keeps its candidates in registers");
     static_assert(!F8 || DI == 1, "fp8 index vectors are one 128-byte atom");
     static_assert(!RUNL || FK == 0, "the run order is a layout of the score matrix");
@@ -224,7 +224,8 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const int et = ew * 32 + lane;
         float4 pend4 = make_float4(0.f, 0.f, 0.f, 0.f);
         bool pend4_on = false;
-        float* const row_base = FK == 0 ? scores + ((row0 + q) * H_kv + r0) * ld_scores : nullptr;
+        // (a packed batch scored group by group: the score matrix starts at packed row score_row0)
+        float* const row_base = FK == 0 ? scores + ((row0 + q - score_row0) * H_kv + r0) * ld_scores : nullptr;
         for (int t = 0; live && t < n_tiles; ++t) {
             const int64_t key0 = (int64_t)t * kIdxTileK + half * 128;
             const bool need_mask = key0 + 127 > pos;
@@ -396,7 +397,7 @@ index_scores_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             const int64_t qq = q0 + rr;
             if (qq >= q_count) break;
             for (int h = 0; h < NH; ++h) {
-                float* orow = scores + ((row0 + qq) * H_kv + r0 + h) * ld_scores;
+                float* orow = scores + ((row0 + qq - score_row0) * H_kv + r0 + h) * ld_scores;
                 for (int64_t b = (q_begin + qq) / BK + 1 + lane; b < n_cols; b += 32) orow[b] = -INFINITY;
             }
         }

@@ -148,7 +148,8 @@ template <int BK, int NH, int DI, int FK = 0, bool F8 = false, bool RUNL = false
 static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                     int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
                                     int64_t n_cols, cudaStream_t st, int32_t* block_idx = nullptr,
-                                    const IdxPackedTile* packed = nullptr, int64_t n_packed = 0) {
+                                    const IdxPackedTile* packed = nullptr, int64_t n_packed = 0,
+                                    int64_t score_row0 = 0) {
     // key-tile stages: what fits beside the NH*DI query atoms in 227 KB of shared memory (at most 3)
     constexpr int RUN_KB = RUNL ? NH * 4 : 0;  // block maxima of a run of eight, waiting for their 16-byte store
     constexpr int ST = (NH * DI * 16 + 3 * DI * 32 + RUN_KB <= 224) ? 3 : 2;
@@ -181,7 +182,7 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
         StageScope sc(kStageIndex, st);
         index_scores_tc_kernel<BK, NH, DI, ST, FK, F8, RUNL><<<(unsigned)grid, kIdxThreads, smem, st>>>(
             tm_q, tm_k, q_begin, q_count, r.H_kv, r.index_scale, scores, ld_scores, n_cols, status, block_idx, r.k,
-            packed);
+            packed, score_row0);
     }
     return launch_status();
 }
@@ -189,25 +190,31 @@ static msa_status_t launch_index_tc(const Resolved& r, const void* q_idx, const 
 // Heads sharing one key tile per CTA: the most (8, 4, 2, 1; at most 2 when d_idx = 128, for
 // shared memory) that divide H_kv and still leave at least two CTAs per SM, so that short
 // chunks keep the machine full.
+static int index_heads_for_tiles(const Resolved& r, int64_t n_qtiles);
 static int index_heads_per_cta(const Resolved& r, int64_t q_count) {
-    const int64_t n_qtiles = ceil_div64(q_count, kIdxTileQ);
+    return index_heads_for_tiles(r, ceil_div64(q_count, kIdxTileQ));
+}
+static int index_heads_for_tiles(const Resolved& r, int64_t n_qtiles) {
     const bool one_atom = r.idx_fp8 || r.d_idx == 64;  // the index vector is one 128-byte atom
     for (int cand = one_atom ? 8 : 2; cand > 1; cand >>= 1)
         if (r.H_kv % cand == 0 && n_qtiles * (r.H_kv / cand) >= 2 * sm_count()) return cand;
     return 1;
 }
 
+// packed != null: a group of sequences of a packed batch (q_count = kv_len = the batch's rows), its query
+// tiles listed in `packed`; the score matrix starts at packed row score_row0.
 template <int BK, int DI, bool F8, bool RUNL>
 static msa_status_t launch_index_tc_nh(const Resolved& r, const void* q_idx, const void* k_idx, int64_t q_begin,
                                        int64_t q_count, int64_t kv_len, float* scores, int64_t ld_scores,
-                                       int64_t n_cols, cudaStream_t st) {
-    const int nh = index_heads_per_cta(r, q_count);
+                                       int64_t n_cols, cudaStream_t st, const IdxPackedTile* packed = nullptr,
+                                       int64_t n_packed = 0, int64_t score_row0 = 0) {
+    const int nh = packed != nullptr ? index_heads_for_tiles(r, n_packed) : index_heads_per_cta(r, q_count);
     if constexpr (DI == 1) {
-        if (nh == 8) return launch_index_tc<BK, 8, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
-        if (nh == 4) return launch_index_tc<BK, 4, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+        if (nh == 8) return launch_index_tc<BK, 8, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st, nullptr, packed, n_packed, score_row0);
+        if (nh == 4) return launch_index_tc<BK, 4, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st, nullptr, packed, n_packed, score_row0);
     }
-    if (nh == 2) return launch_index_tc<BK, 2, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
-    return launch_index_tc<BK, 1, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st);
+    if (nh == 2) return launch_index_tc<BK, 2, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st, nullptr, packed, n_packed, score_row0);
+    return launch_index_tc<BK, 1, DI, 0, F8, RUNL>(r, q_idx, k_idx, q_begin, q_count, kv_len, scores, ld_scores, n_cols, st, nullptr, packed, n_packed, score_row0);
 }
 
 // runs: the score rows are written in run order (score_slot) instead of block order.
@@ -295,6 +302,25 @@ static msa_status_t run_index_scores(const Resolved& r, const void* q_idx, const
                 q_idx, k_idx, rows, n_chunks, r.H_kv, r.d_idx, r.B_k, r.index_scale, scores, ld_scores, score_lnb(r, runs));
     }
     return launch_status();
+}
+
+// Eq. 6 for a group of sequences of a packed batch in one launch (tensor-core shapes only): the
+// group's query tiles are listed in `tiles`; scores [group rows, H_kv, ld] in run order, row 0 =
+// packed row score_row0.
+static msa_status_t run_index_scores_packed(const Resolved& r, const void* q_idx, const void* k_idx, int64_t batch_rows,
+                                            float* scores, int64_t ld, cudaStream_t st, const IdxPackedTile* tiles,
+                                            int64_t n_tiles, int64_t score_row0) {
+    if (n_tiles == 0) return MSA_OK;
+    if (r.idx_fp8) {
+        if (r.B_k == 64) return launch_index_tc_nh<64, 1, true, true>(r, q_idx, k_idx, 0, batch_rows, batch_rows, scores, ld, ld, st, tiles, n_tiles, score_row0);
+        return launch_index_tc_nh<128, 1, true, true>(r, q_idx, k_idx, 0, batch_rows, batch_rows, scores, ld, ld, st, tiles, n_tiles, score_row0);
+    }
+    if (r.d_idx == 64) {
+        if (r.B_k == 64) return launch_index_tc_nh<64, 1, false, true>(r, q_idx, k_idx, 0, batch_rows, batch_rows, scores, ld, ld, st, tiles, n_tiles, score_row0);
+        return launch_index_tc_nh<128, 1, false, true>(r, q_idx, k_idx, 0, batch_rows, batch_rows, scores, ld, ld, st, tiles, n_tiles, score_row0);
+    }
+    if (r.B_k == 64) return launch_index_tc_nh<64, 2, false, true>(r, q_idx, k_idx, 0, batch_rows, batch_rows, scores, ld, ld, st, tiles, n_tiles, score_row0);
+    return launch_index_tc_nh<128, 2, false, true>(r, q_idx, k_idx, 0, batch_rows, batch_rows, scores, ld, ld, st, tiles, n_tiles, score_row0);
 }
 
 // ---------------------------------------------------------------------- stage 2
@@ -1468,6 +1494,16 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
     int32_t* row_pos = (int32_t*)(w + vp.off_row_pos);
     int32_t* row_blk0 = (int32_t*)(w + vp.off_row_blk0);
     int32_t* blk_row0 = (int32_t*)(w + vp.off_blk_row0);
+    char* stage = w + vp.meta + vp.copies;
+    const size_t stage_bytes = workspace_bytes - vp.meta - vp.copies;
+    // top_k > 16 on the tensor-core shapes: stages 1-2 run on groups of consecutive sequences, as many
+    // as the score matrix of the stage region holds rows for; one scoring launch and one Top-k launch
+    // per group.  A sequence too long for the region alone takes the single-sequence path (in chunks).
+    struct SeqGroup { int32_t seq_a, seq_b; int64_t row_a, row_b, tile_off, n_tiles; };
+    const bool grouped = !vp.fused && index_tc_ok(r) && vp.rows >= 32;
+    SeqGroup* groups = nullptr;
+    int32_t n_groups = 0;
+    int64_t group_ld = 0;
     {
         // (pageable host memory: the runtime has copied it out when the call returns)
         int32_t* blk_cum = (int32_t*)malloc((size_t)(n_seqs + 1) * 4);
@@ -1482,20 +1518,55 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
         }
         // longest key prefix first: by tile number inside the sequence, descending
         int64_t n = 0;
-        for (int64_t qt = max_qt - 1; qt >= 0; --qt)
-            for (int32_t i = 0; i < n_seqs; ++i) {
-                const int64_t T = cu_seqlens[i + 1] - cu_seqlens[i];
-                if (qt < ceil_div64(T, kIdxTileQ)) {
-                    tiles[n].row0 = (int32_t)(cu_seqlens[i] - row0); tiles[n].len = (int32_t)T; tiles[n].qt = (int32_t)qt;
-                    ++n;
+        auto list_tiles = [&](int32_t seq_a, int32_t seq_b) {
+            int64_t top_qt = 0;
+            for (int32_t i = seq_a; i < seq_b; ++i)
+                if (ceil_div64(cu_seqlens[i + 1] - cu_seqlens[i], kIdxTileQ) > top_qt)
+                    top_qt = ceil_div64(cu_seqlens[i + 1] - cu_seqlens[i], kIdxTileQ);
+            for (int64_t qt = top_qt - 1; qt >= 0; --qt)
+                for (int32_t i = seq_a; i < seq_b; ++i) {
+                    const int64_t T = cu_seqlens[i + 1] - cu_seqlens[i];
+                    if (qt < ceil_div64(T, kIdxTileQ)) {
+                        tiles[n].row0 = (int32_t)(cu_seqlens[i] - row0); tiles[n].len = (int32_t)T; tiles[n].qt = (int32_t)qt;
+                        ++n;
+                    }
                 }
+        };
+        if (!grouped) {
+            list_tiles(0, n_seqs);
+        } else {
+            groups = (SeqGroup*)malloc((size_t)n_seqs * sizeof(SeqGroup));
+            if (!groups) { free(blk_cum); free(tiles); return MSA_ERR_CUDA; }
+            group_ld = score_ld(max_qt * kIdxTileQ, r.B_k);
+            const int64_t rows_cap = (int64_t)(stage_bytes / (sizeof(float) * (size_t)r.H_kv * (size_t)group_ld));
+            int32_t a = 0;
+            while (a < n_seqs) {
+                int32_t b = a;
+                int64_t rows_in = 0;
+                while (b < n_seqs && rows_in + (cu_seqlens[b + 1] - cu_seqlens[b]) <= rows_cap) {
+                    rows_in += cu_seqlens[b + 1] - cu_seqlens[b];
+                    ++b;
+                }
+                SeqGroup g;
+                g.seq_a = a; g.row_a = cu_seqlens[a] - row0; g.tile_off = n;
+                if (b == a) {  // this sequence alone does not fit: n_tiles = -1 marks the single-sequence path
+                    b = a + 1;
+                    g.n_tiles = -1;
+                } else {
+                    list_tiles(a, b);
+                    g.n_tiles = n - g.tile_off;
+                }
+                g.seq_b = b; g.row_b = cu_seqlens[b] - row0;
+                groups[n_groups++] = g;
+                a = b;
             }
+        }
         bool ok = cudaMemcpyAsync(cu_dev, cu_seqlens, (size_t)(n_seqs + 1) * 8, cudaMemcpyHostToDevice, st) == cudaSuccess &&
                   cudaMemcpyAsync(blk_cum_dev, blk_cum, (size_t)(n_seqs + 1) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
                   (n == 0 || cudaMemcpyAsync(tiles_dev, tiles, (size_t)n * sizeof(IdxPackedTile), cudaMemcpyHostToDevice, st) == cudaSuccess);
         free(blk_cum);
         free(tiles);
-        if (!ok) return MSA_ERR_CUDA;
+        if (!ok) { free(groups); return MSA_ERR_CUDA; }
     }
     {
         const int64_t work = vp.rows + vp.n_blocks;
@@ -1503,7 +1574,7 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
         StageScope sc(kStageSchedule, st);
         packed_map_kernel<<<grid, 256, 0, st>>>(cu_dev, blk_cum_dev, n_seqs, r.B_k, row_pos, row_blk0, blk_row0);
     }
-    if (cudaPeekAtLastError() != cudaSuccess) return MSA_ERR_CUDA;
+    if (cudaPeekAtLastError() != cudaSuccess) { free(groups); return MSA_ERR_CUDA; }
     // tensors of the batch start at its first row
     const char* qb = (const char*)q + row0 * q_row;
     const char* kb = (const char*)k + row0 * kv_row;
@@ -1511,11 +1582,30 @@ msa_status_t msa_prefill_forward_varlen(const msa_shape_t* shape, const void* q,
     const char* qib = (const char*)q_idx + row0 * qi_row;
     const char* kib = (const char*)k_idx + row0 * ki_row;
     int32_t* bi = block_idx + row0 * (int64_t)r.H_kv * r.k;
-    char* stage = w + vp.meta + vp.copies;
-    const size_t stage_bytes = workspace_bytes - vp.meta - vp.copies;
     // ---- stages 1-2
     if (vp.fused) {
         s = run_index_topk_fused(r, qib, kib, 0, vp.rows, vp.rows, bi, st, tiles_dev, vp.n_idx_tiles);
+        if (s != MSA_OK) return s;
+    } else if (grouped) {
+        float* scores = reinterpret_cast<float*>(stage);
+        for (int32_t gi = 0; gi < n_groups && s == MSA_OK; ++gi) {
+            const SeqGroup& g = groups[gi];
+            if (g.row_b == g.row_a) continue;
+            if (g.n_tiles < 0) {
+                const int64_t o = cu_seqlens[g.seq_a];
+                s = prefill_stages_1_2(shape, r, (const char*)q_idx + o * qi_row, (const char*)k_idx + o * ki_row,
+                                       cu_seqlens[g.seq_a + 1] - o, block_idx + o * (int64_t)r.H_kv * r.k, stage,
+                                       stage_bytes, stream);
+                continue;
+            }
+            s = run_index_scores_packed(r, qib, kib, vp.rows, scores, group_ld, st, tiles_dev + g.tile_off, g.n_tiles,
+                                        g.row_a);
+            if (s != MSA_OK) break;
+            RowMap rows = prefill_rows(g.row_a, 0, r.B_k);
+            rows.row_pos = row_pos;
+            s = run_topk(r, scores, group_ld, rows, g.row_b - g.row_a, bi + g.row_a * (int64_t)r.H_kv * r.k, st, true);
+        }
+        free(groups);
         if (s != MSA_OK) return s;
     } else {
         for (int32_t i = 0; i < n_seqs; ++i) {

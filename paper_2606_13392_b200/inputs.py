@@ -123,6 +123,9 @@ CONFIGS: Dict[str, MSAConfig] = {
                          seq_lens=(8192,) * 128),
     "pvar-2k": MSAConfig("pvar-2k", "prefill", 1048576, 64, 4, 128, 16, idx_dim=128, seed=11,
                          seq_lens=(2048,) * 512),
+    # The C2 shape (B_k = 64, top_k = 32: above the fused kernel's limit) as 256 packed sequences of
+    # 4096 tokens: stages 1-2 run on groups of sequences, one launch each.
+    "c2var-4k": MSAConfig("c2var-4k", "prefill", 1048576, 64, 8, 64, 32, seed=12, seq_lens=(4096,) * 256),
     # A light decode step (8 sequences of 32K): launch gaps weigh as much as the kernels.
     "c5-light": MSAConfig("c5-light", "decode", 32768, 64, 8, 128, 64, seed=4, seq_lens=(32768,) * 8),
     "c5-small": MSAConfig("c5-small", "decode", 131072, 64, 8, 128, 64, seed=4,

@@ -933,11 +933,18 @@ def test_fp8_q_is_rejected_where_it_is_not_supported():
     assert e.value.code == 2
 
 
-def test_varlen_batch_with_larger_top_k_and_a_row_offset():
-    # top_k above the fused kernel's limit: stages 1-2 run sequence by sequence, stage 3 once over the
-    # batch; the batch starts at a row offset inside the tensors (cu_seqlens[0] > 0).
-    cfg = CONFIGS["c3"].scaled(name="c3-varlen-k64", T=0)
-    lens = [9000, 130, 2500, 1]
+@pytest.mark.parametrize("base,lens,ws", [
+    ("c3", [9000, 130, 2500, 1], "minimum"),
+    ("c3", [9000, 130, 2500, 1], "preferred"),
+    ("c2", [700, 5000, 0, 64, 3000, 8192 + 9, 31, 1500], "preferred"),
+    ("c2", [700, 5000, 0, 64, 3000, 8192 + 9, 31, 1500], "minimum"),
+])
+def test_varlen_batch_with_larger_top_k_and_a_row_offset(base, lens, ws):
+    # top_k above the fused kernel's limit: stages 1-2 run on groups of consecutive sequences (one
+    # scoring launch and one Top-k launch per group: one group with the preferred workspace, several
+    # - and the single-sequence path for a sequence that does not fit - with the minimum), stage 3
+    # once over the batch; the batch starts at a row offset inside the tensors (cu_seqlens[0] > 0).
+    cfg = CONFIGS[base].scaled(name=base + "-varlen-k", T=0)
     cu = (np.concatenate([[0], np.cumsum(lens)]) + 384).tolist()
     total = cu[-1] + 77   # rows before and after the batch that the call must leave alone
     x = make_prefill_inputs(cfg.scaled(T=total), DEV, sharp=True)
@@ -946,18 +953,28 @@ def test_varlen_batch_with_larger_top_k_and_a_row_offset():
     lse = torch.full((total, cfg.n_q_heads), 7.0, dtype=torch.float32, device=DEV)
     I = torch.full((total, cfg.n_kv_heads, cfg.top_k), -7, dtype=torch.int32, device=DEV)
     mn, pf = B.msa_prefill_forward_varlen_workspace_bytes(shape, cu)
+    n0 = B.launch_count()
     B.msa_prefill_forward_varlen(shape, x["q"], x["k"], x["v"], x["q_idx"], x["k_idx"], cu, out, lse, I,
-                                 B.alloc_workspace(mn, DEV))
+                                 B.alloc_workspace(mn if ws == "minimum" else pf, DEV))
+    n_batch = B.launch_count() - n0
+    if ws == "preferred":  # as many launches as ONE sequence of the batch's size takes, plus the one that builds the maps
+        one = cfg.scaled(T=sum(lens))
+        n0 = B.launch_count()
+        api.prefill_forward(one, {n: t[:sum(lens)].contiguous() for n, t in x.items()})
+        assert n_batch <= B.launch_count() - n0 + 1, (n_batch, B.launch_count() - n0)
     torch.cuda.synchronize()
     _assert_clean()
     assert bool((out[:384] == 7.0).all()) and bool((out[cu[-1]:] == 7.0).all()) and bool((I[:384] == -7).all())
     for s_, L in enumerate(lens):
+        if L == 0:
+            continue
         a, b = cu[s_], cu[s_ + 1]
         xs = {n: t[a:b].contiguous() for n, t in x.items()}
         o1, l1, i1 = api.prefill_forward(cfg.scaled(T=L), xs)
         assert torch.equal(I[a:b], i1) and torch.equal(out[a:b], o1) and torch.equal(lse[a:b], l1), "sequence %d" % s_
-    # oracle on the first sequence through the batch call's outputs
-    a, b, L = cu[0], cu[1], lens[0]
+    # oracle on the longest sequence through the batch call's outputs
+    s_ = int(np.argmax(lens))
+    a, b, L = cu[s_], cu[s_ + 1], lens[s_]
     pos = sample_positions(L, cfg.block_size, cfg.top_k, 48, 5)
     pos_t = torch.from_numpy(pos).to(DEV)
     I_gpu = I[a:b][pos_t].cpu().numpy()
