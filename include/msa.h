@@ -326,9 +326,9 @@ msa_status_t msa_prefill_forward_workspace_bytes(const msa_shape_t* shape, int64
  * {64,128}) a batch of two or more sequences runs as ONE problem per stage: Eq. 6 + Eq. 7 as a single
  * launch of the fused kernel over the query tiles of all sequences (top_k <= 16), or (larger top_k)
  * one scoring launch and one Top-k launch per group of consecutive sequences - as many sequences as
- * the workspace holds score rows for, all of them with the preferred workspace unless the batch is
- * larger than 32768 rows of its longest sequence's pitch; a sequence too long for the region alone
- * is scored by the single-sequence path in chunks - and Eq. 8 with its blocks numbered through the batch, so that one
+ * the workspace holds score rows for (a row takes 4 * H_kv * the block count of the batch's longest
+ * sequence, rounded up to 8, bytes); a sequence too long for the region alone is scored by the
+ * single-sequence path in chunks - and Eq. 8 with its blocks numbered through the batch, so that one
  * reverse index, one attention launch and one merge serve every sequence of a query range (ranges
  * span sequence boundaries).  Other shapes, and a batch of one, run the single-sequence call per
  * sequence on `stream`.  Results do not depend on which way a sequence ran.  The call copies
