@@ -68,6 +68,28 @@ def test_argument_validation_without_launch(lib):
     bad = B.shape_of(CONFIGS["c1"].scaled(head_dim=100))
     assert lib.msa_topk_select(ctypes.byref(bad), null, i64(4), i64(0), i64(0), i64(0), null, null) == 2
     assert lib.msa_index_scores(None, null, null, i64(0), i64(0), i64(0), null, i64(4), null) == 1
+    # order of the blocks inside a score row: 0 or 1; run order exists for B_k 64 and 128 only,
+    # and the decode calls take block order only
+    bad = B.shape_of(CONFIGS["c1"], score_runs=2)
+    assert lib.msa_topk_select(ctypes.byref(bad), null, i64(8), i64(0), i64(0), i64(0), null, null) == 1
+    bad = B.shape_of(CONFIGS["c1"].scaled(block_size=16), score_runs=1)
+    assert lib.msa_topk_select(ctypes.byref(bad), null, i64(8), i64(0), i64(0), i64(0), null, null) == 2
+    runs = B.shape_of(CONFIGS["c1"], score_runs=1)
+    assert lib.msa_topk_select(ctypes.byref(runs), null, i64(8), i64(0), i64(0), i64(0), null, null) == 0
+    assert lib.msa_topk_select_decode(ctypes.byref(runs), null, i64(8), null, ctypes.c_int32(0), i64(0), null,
+                                      null) == 2
+
+
+def test_run_order_columns_are_a_permutation_inside_every_run():
+    # msa_shape_t.score_runs = 1: the columns of a run of eight hold its blocks 0 2 4 6 1 3 5 7
+    # (B_k = 128: one block per epilogue thread and key tile) or 0 1 4 5 2 3 6 7 (B_k = 64: two).
+    from paper_2606_13392_b200 import api
+    for bk, holds in ((128, [0, 2, 4, 6, 1, 3, 5, 7]), (64, [0, 1, 4, 5, 2, 3, 6, 7])):
+        cols = api.run_order_columns(24, bk).tolist()
+        assert sorted(cols) == list(range(24))
+        for run in range(3):
+            assert [cols.index(8 * run + c) - 8 * run for c in range(8)] == holds
+        assert api.run_order_columns(13, bk).tolist() == cols[:13]
 
 
 def test_workspace_queries(lib):
