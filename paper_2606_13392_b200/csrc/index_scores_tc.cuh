@@ -9,7 +9,10 @@
 // runs.  Sharing one key tile among NH heads matters: with one head per CTA every 512 MMA
 // cycles need a fresh 32 KB tile from L2, about 9 TB/s over the chip, and the kernel is
 // L2-bound at 60 % tensor duty.  Only the tile that crosses the diagonal applies the causal
-// mask.  Blocks beyond a query's local block are filled with -inf at the end.
+// mask.  In block order (RUNL = false) every thread stores its maxima one (tile, head) unit late
+// and blocks beyond a query's local block are filled with -inf at the end; in run order (RUNL = true,
+// see score_slot) a thread's maxima of a run of eight blocks wait in shared memory and leave as one
+// 16-byte store, and nothing is written beyond the run of the local block.
 #pragma once
 
 #include "tc_common.cuh"
