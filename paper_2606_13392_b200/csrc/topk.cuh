@@ -457,7 +457,10 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
     int n_log;
     bool log_ok;
     const int64_t n_full = loc / kTopkRunBlocks;  // runs wholly before the local block
-    if (n_full < 2 * m || n_full > kTopkMaxRuns) {  // short row (or one beyond the list): one level
+    // Rows of fewer than 2 m runs can still take two levels when their runs are split into halves or
+    // quarters for the threshold (4 or 2 blocks each): 2 m such groups make the threshold tight enough.
+    const int sub = n_full >= 2 * m ? 1 : (2 * n_full >= 2 * m ? 2 : (4 * n_full >= 2 * m ? 4 : 0));
+    if (sub == 0 || n_full > kTopkMaxRuns) {  // short row (or one beyond the list): one level
         const TopkPlainStream st{srow, (int)loc, lnb};
         topk_pass1<R>(st, m, -INFINITY, sc, kept, n_log, log_ok, lane);
         topk_pass2<R>(st, m, sc, kept, n_log, log_ok, outb, lane);
@@ -474,10 +477,42 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         for (int i = 0; i < S; ++i) top[i] = -INFINITY;
         float* runmax = reinterpret_cast<float*>(log_all[warp]);  // the log is not in use before step 3
         static_assert(kTopkLog * sizeof(uint2) >= kTopkMaxRuns * sizeof(float), "run maxima share the log");
+        auto keep = [&](float v) {  // top[] <- the S largest of top[] and v, sorted
+#pragma unroll
+            for (int i = 0; i < S; ++i) {
+                const float hi = fmaxf(top[i], v);
+                v = fminf(top[i], v);
+                top[i] = hi;
+            }
+        };
+        if (sub != 1) {
+            // fewer than 2 m <= 64 R runs, i.e. at most 2 R per lane: all loads first, then the maxima of the
+            // runs (for step 2) and of their halves or quarters (for the threshold)
+            float4 a[2 * R], b[2 * R];
+#pragma unroll
+            for (int u = 0; u < 2 * R; ++u) {
+                const int g = u * 32 + lane;
+                const float4* pr = reinterpret_cast<const float4*>(srow) + 2 * g;
+                a[u] = g < (int)n_full ? __ldg(pr) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                b[u] = g < (int)n_full ? __ldg(pr + 1) : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            }
+#pragma unroll
+            for (int u = 0; u < 2 * R; ++u) {
+                const int g = u * 32 + lane;
+                const float a0 = fmaxf(a[u].x, a[u].y), a1 = fmaxf(a[u].z, a[u].w);
+                const float b0 = fmaxf(b[u].x, b[u].y), b1 = fmaxf(b[u].z, b[u].w);
+                if (g < (int)n_full) runmax[g] = fmaxf(fmaxf(a0, a1), fmaxf(b0, b1));
+                if (sub == 2) {
+                    keep(fmaxf(a0, a1)); keep(fmaxf(b0, b1));
+                } else {
+                    keep(a0); keep(a1); keep(b0); keep(b1);
+                }
+            }
+        }
         float nx[kTopkRunLoads];
 #pragma unroll
-        for (int u = 0; u < kTopkRunLoads; ++u) nx[u] = rs.score(u * 32 + lane);  // -inf beyond n_full
-        for (int g0 = 0; g0 < (int)n_full; g0 += 32 * kTopkRunLoads) {
+        for (int u = 0; u < kTopkRunLoads; ++u) nx[u] = sub == 1 ? rs.score(u * 32 + lane) : -INFINITY;  // -inf beyond n_full
+        for (int g0 = 0; sub == 1 && g0 < (int)n_full; g0 += 32 * kTopkRunLoads) {
             float x[kTopkRunLoads];
 #pragma unroll
             for (int u = 0; u < kTopkRunLoads; ++u) x[u] = nx[u];
@@ -485,14 +520,8 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
             for (int u = 0; u < kTopkRunLoads; ++u) nx[u] = rs.score(g0 + 32 * kTopkRunLoads + u * 32 + lane);  // in flight during the inserts
 #pragma unroll
             for (int u = 0; u < kTopkRunLoads; ++u) {
-                float v = x[u];
-                if (g0 + u * 32 + lane < (int)n_full) runmax[g0 + u * 32 + lane] = v;
-#pragma unroll
-                for (int i = 0; i < S; ++i) {
-                    const float hi = fmaxf(top[i], v);
-                    v = fminf(top[i], v);
-                    top[i] = hi;
-                }
+                if (g0 + u * 32 + lane < (int)n_full) runmax[g0 + u * 32 + lane] = x[u];
+                keep(x[u]);
             }
         }
         uint32_t tk[S];
