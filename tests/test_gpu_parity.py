@@ -654,6 +654,36 @@ def test_two_level_topk_on_arbitrary_long_score_rows(n_blocks, k, levels):
         assert np.array_equal(I, I_ref), (q0, qc)
 
 
+@pytest.mark.parametrize("Bk,n_blocks,k,levels", [(128, 700, 64, 0), (128, 700, 64, 6), (64, 1100, 32, 4),
+                                                 (128, 2600, 64, -48), (64, 300, 64, 3), (128, 4200, 16, -16)])
+def test_topk_reads_run_ordered_rows_like_block_ordered_ones(Bk, n_blocks, k, levels):
+    # Stage 2 alone on synthetic score rows handed over in run order (msa_shape_t.score_runs = 1):
+    # the lists must be those of the same rows in block order and the oracle's, with continuous
+    # values, with a handful of levels (whole runs tie) and with values rounded to multiples of
+    # 1/|levels| (a few ties at the threshold); rows of every length class (one level, two levels with
+    # quarters, halves and whole runs as threshold groups).
+    T = n_blocks * Bk
+    cfg = MSAConfig("top-runs", "prefill", T, 4, 2, Bk, k, head_dim=64, idx_dim=64, seed=n_blocks)
+    g = torch.Generator().manual_seed(n_blocks + k)
+    ld = (n_blocks + 7) // 8 * 8
+    cols = api.run_order_columns(n_blocks, Bk)
+    pos = np.unique(np.concatenate([np.arange(T - 24, T), np.linspace(Bk * (k - 1), T - 1, 120).astype(np.int64)]))
+    for run in np.split(pos, np.where(np.diff(pos) != 1)[0] + 1):
+        q0, qc = int(run[0]), len(run)
+        M = torch.randn((qc, 2, ld), generator=g)
+        if levels > 0:
+            M = torch.randint(0, levels, (qc, 2, ld), generator=g).float() * 0.5 - 1.0
+        elif levels < 0:
+            M = torch.round(M * float(-levels)) / float(-levels)
+        M_runs = torch.full_like(M, float("nan"))   # columns of blocks that do not exist stay NaN
+        M_runs[:, :, cols] = M[:, :, :n_blocks]
+        I_blk = api.topk_select(cfg, M.to(DEV), q0, T).cpu().numpy()
+        I_run = api.topk_select(cfg, M_runs.to(DEV), q0, T, score_runs=1).cpu().numpy()
+        I_ref = oracle.topk_select(M[:, :, :n_blocks].double().numpy(), np.arange(q0, q0 + qc), T, Bk, k)
+        assert np.array_equal(I_blk, I_ref), (q0, qc)
+        assert np.array_equal(I_run, I_ref), (q0, qc)
+
+
 # ----------------------------------------------------------------- CUDA graphs
 def test_decode_and_prefill_calls_replay_from_a_cuda_graph():
     # A decode step is a handful of short kernels: serving loops capture it once and replay it.
