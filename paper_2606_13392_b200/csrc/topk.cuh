@@ -115,7 +115,11 @@ constexpr int kTopkRunBlocks = 8;       // two-level selection: blocks per run
 #endif
 constexpr int kTopkRunLoads = MSA_TOPK_RUNLOADS;  // two-level selection: runs per lane and round of the run-maxima pass
 constexpr int kTopkTau0Slack = 4;       // two-level selection: candidate runs accepted beyond the m needed
-constexpr int kTopkMaxRuns = 1024;     // two-level selection: candidate list capacity (rows of up to 8192 blocks)
+constexpr int kTopkMaxRuns = 1024;     // two-level selection: rows of up to 8192 blocks (their run maxima wait in shared memory)
+// Candidate runs listed per row (a row with more - ties by the hundred - takes one level).  The list is kept
+// short on purpose: with room for all kTopkMaxRuns runs (28 KB of shared memory per CTA instead of 22, so less
+// of the SM's array left as L1) the kernel took 0.280 instead of 0.219 ms on 8192 rows of up to 8192 scores.
+constexpr int kTopkMaxCand = 254;
 
 // A row as the selection sees it: element i of n has a score and a block index; the elements come
 // in ascending block order.
@@ -434,7 +438,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
                    int lnb) {
     __shared__ uint32_t stg_all[kTopkWarps][kTopkStage];
     __shared__ uint2 log_all[kTopkWarps][kTopkLog];   // (key, block) of every survivor, in index order
-    __shared__ uint16_t run_all[kTopkWarps][kTopkMaxRuns + 2];
+    __shared__ uint16_t run_all[kTopkWarps][kTopkMaxCand + 2];
     __shared__ int32_t out_all[kTopkWarps][32 * R];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * kTopkWarps + warp;
@@ -460,10 +464,13 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
     // Rows of fewer than 2 m runs can still take two levels when their runs are split into halves or
     // quarters for the threshold (4 or 2 blocks each): 2 m such groups make the threshold tight enough.
     const int sub = n_full >= 2 * m ? 1 : (2 * n_full >= 2 * m ? 2 : (4 * n_full >= 2 * m ? 4 : 0));
-    if (sub == 0 || n_full > kTopkMaxRuns) {  // short row (or one beyond the list): one level
+    auto one_level = [&]() {
         const TopkPlainStream st{srow, (int)loc, lnb};
         topk_pass1<R>(st, m, -INFINITY, sc, kept, n_log, log_ok, lane);
         topk_pass2<R>(st, m, sc, kept, n_log, log_ok, outb, lane);
+    };
+    if (sub == 0 || n_full > kTopkMaxRuns) {  // short row (or one beyond the run-maxima array): one level
+        one_level();
     } else {
         // 1. A threshold from the run maxima.  Any value that m run maxima reach will do, so no exact
         // selection: every lane keeps the S = 2R largest of the maxima it sees (sorted registers, no
@@ -554,14 +561,17 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
             const int g = g0 + lane;
             const bool c = g < (int)n_full && runmax[g] >= tau0;
             const unsigned cm = __ballot_sync(0xffffffffu, c);
-            if (c) run[n_run + __popc(cm & lt_mask)] = (uint16_t)g;
+            if (c && n_run + __popc(cm & lt_mask) < kTopkMaxCand) run[n_run + __popc(cm & lt_mask)] = (uint16_t)g;
             n_run += __popc(cm);
         }
         if (n_full * kTopkRunBlocks < loc) {  // the run that holds the local block
-            if (lane == 0) run[n_run] = (uint16_t)n_full;
+            if (lane == 0 && n_run < kTopkMaxCand + 1) run[n_run] = (uint16_t)n_full;
             ++n_run;
         }
         __syncwarp();
+        if (n_run > kTopkMaxCand + 1) {  // ties by the hundred: the list does not hold the candidates
+            one_level();
+        } else {
         // 3. select among the candidates' blocks; scores below tau0 cannot be selected.  The floor
         // only has to lie below tau0: a hair below it, whatever its sign or size.
         const bool few = lnb == 0   ? topk_few_above<0>(srow, run, n_run, (int)loc, tau0, m, log_all[warp], outb, lane)
@@ -573,6 +583,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
             const TopkGatherStream gs{srow, run, n_run * kTopkRunBlocks, (int)loc, lnb};
             topk_pass1<R>(gs, m, floor_f, sc, kept, n_log, log_ok, lane);
             topk_pass2<R>(gs, m, sc, kept, n_log, log_ok, outb, lane);
+        }
         }
     }
     // Block order makes the list ascending with no final sort; the local block is appended by
