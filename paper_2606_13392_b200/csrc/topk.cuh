@@ -117,8 +117,9 @@ constexpr int kTopkRunLoads = MSA_TOPK_RUNLOADS;  // two-level selection: runs p
 constexpr int kTopkTau0Slack = 4;       // two-level selection: candidate runs accepted beyond the m needed
 constexpr int kTopkMaxRuns = 1024;     // two-level selection: rows of up to 8192 blocks (their run maxima wait in shared memory)
 // Candidate runs listed per row (a row with more - ties by the hundred - takes one level).  The list is kept
-// short on purpose: with room for all kTopkMaxRuns runs (28 KB of shared memory per CTA instead of 22, so less
-// of the SM's array left as L1) the kernel took 0.280 instead of 0.219 ms on 8192 rows of up to 8192 scores.
+// short on purpose: with room for all kTopkMaxRuns runs the kernel needed 28 KB of shared memory per CTA and 71
+// registers, seven CTAs per SM; with this list it is 22 KB and 64 registers, eight CTAs, and 0.219 instead of
+// 0.280 ms on 8192 rows of up to 8192 scores.
 constexpr int kTopkMaxCand = 254;
 
 // A row as the selection sees it: element i of n has a score and a block index; the elements come
