@@ -102,13 +102,16 @@ __device__ __forceinline__ int warp_excl_scan(int v, int lane) {
 }
 
 constexpr int kTopkWarps = 4;
+// The kernel waits for memory more than for anything else: nine CTAs per SM (56 registers, 14 KB of shared
+// memory each, which also leaves the SM most of its array as L1 for the second look at the candidate runs).
+constexpr int kTopkMinCtas = 9;
 #ifndef MSA_TOPK_LOADS
 #define MSA_TOPK_LOADS 4
 #endif
 constexpr int kTopkLoads = MSA_TOPK_LOADS;            // coalesced 32-wide loads per round
 constexpr int kTopkRound = 32 * kTopkLoads;           // blocks covered by one round
 constexpr int kTopkStage = 32 + kTopkRound;           // flush threshold (32) + one round of pushes
-constexpr int kTopkLog = 512;    // survivors remembered per row for the index pass
+constexpr int kTopkLog = 256;    // survivors remembered per row for the index pass (a row with more is walked a second time)    // survivors remembered per row for the index pass
 constexpr int kTopkRunBlocks = 8;       // two-level selection: blocks per run
 #ifndef MSA_TOPK_RUNLOADS
 #define MSA_TOPK_RUNLOADS 4
@@ -433,7 +436,7 @@ struct TopkGatherStream {  // element i: block i % 8 of candidate run i / 8; blo
 };
 
 template <int R>
-__global__ void __launch_bounds__(kTopkWarps * 32)
+__global__ void __launch_bounds__(kTopkWarps * 32, kTopkMinCtas)
 topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap rows,
                    int64_t n_rows, int H_kv, int B_k, int top_k, int32_t* __restrict__ block_idx, int* status,
                    int lnb) {
@@ -483,8 +486,10 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         float top[S];
 #pragma unroll
         for (int i = 0; i < S; ++i) top[i] = -INFINITY;
-        float* runmax = reinterpret_cast<float*>(log_all[warp]);  // the log is not in use before step 3
-        static_assert(kTopkLog * sizeof(uint2) >= kTopkMaxRuns * sizeof(float), "run maxima share the log");
+        // The run maxima wait for step 2 in shared memory rounded UP to bf16 (half the room): step 2 only asks
+        // whether a run can hold a block that reaches tau0, and a run listed in vain adds no block to step 3.
+        __nv_bfloat16* runmax = reinterpret_cast<__nv_bfloat16*>(log_all[warp]);  // the log is not in use before step 3
+        static_assert(kTopkLog * sizeof(uint2) >= kTopkMaxRuns * sizeof(__nv_bfloat16), "run maxima share the log");
         auto keep = [&](float v) {  // top[] <- the S largest of top[] and v, sorted
 #pragma unroll
             for (int i = 0; i < S; ++i) {
@@ -509,7 +514,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
                 const int g = u * 32 + lane;
                 const float a0 = fmaxf(a[u].x, a[u].y), a1 = fmaxf(a[u].z, a[u].w);
                 const float b0 = fmaxf(b[u].x, b[u].y), b1 = fmaxf(b[u].z, b[u].w);
-                if (g < (int)n_full) runmax[g] = fmaxf(fmaxf(a0, a1), fmaxf(b0, b1));
+                if (g < (int)n_full) runmax[g] = __float2bfloat16_ru(fmaxf(fmaxf(a0, a1), fmaxf(b0, b1)));
                 if (sub == 2) {
                     keep(fmaxf(a0, a1)); keep(fmaxf(b0, b1));
                 } else {
@@ -528,7 +533,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
             for (int u = 0; u < kTopkRunLoads; ++u) nx[u] = rs.score(g0 + 32 * kTopkRunLoads + u * 32 + lane);  // in flight during the inserts
 #pragma unroll
             for (int u = 0; u < kTopkRunLoads; ++u) {
-                if (g0 + u * 32 + lane < (int)n_full) runmax[g0 + u * 32 + lane] = x[u];
+                if (g0 + u * 32 + lane < (int)n_full) runmax[g0 + u * 32 + lane] = __float2bfloat16_ru(x[u]);
                 keep(x[u]);
             }
         }
@@ -560,7 +565,7 @@ topk_select_kernel(const float* __restrict__ scores, int64_t ld_scores, RowMap r
         __syncwarp();
         for (int g0 = 0; g0 < (int)n_full; g0 += 32) {
             const int g = g0 + lane;
-            const bool c = g < (int)n_full && runmax[g] >= tau0;
+            const bool c = g < (int)n_full && __bfloat162float(runmax[g]) >= tau0;
             const unsigned cm = __ballot_sync(0xffffffffu, c);
             if (c && n_run + __popc(cm & lt_mask) < kTopkMaxCand) run[n_run + __popc(cm & lt_mask)] = (uint16_t)g;
             n_run += __popc(cm);
